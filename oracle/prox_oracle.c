@@ -1,0 +1,280 @@
+/*
+ * prox_oracle.c -- TEST INFRASTRUCTURE, not part of the product.
+ *
+ * A plain, slow, fp64 CPU statement of what the approximate query cache
+ * computes, written from the paper so that the CUDA library can be checked
+ * against it.  It shares no code with the CUDA path and must never be called
+ * by it: only the tests, the smoke check and the CPU-baseline leg of the
+ * benchmark may use it.
+ *
+ * What it follows:
+ *   - Algorithm 1 ("Cache lookup in PROXIMITY-FLAT"), one query at a time, in
+ *     stream order: distances from the query to every cached key, the nearest
+ *     key, the test min_dist <= tau (inclusive, as Algorithm 1 and Section 3
+ *     state it), the database call on a miss, eviction when |C| >= c, insert.
+ *   - Section 3.3.2 (eviction policy): FIFO evicts the oldest inserted entry
+ *     whatever its use; LRU evicts the entry unused for the longest time.
+ *   - Section 2.1 / Section 3 (retrieveDocumentIndices): the database call is
+ *     the exact k nearest rows of the corpus, returned as a list sorted by
+ *     increasing distance (the FAISS-Flat case of Section 4.2.1).
+ *
+ * Readings where the paper is silent (the same readings are listed in the
+ * design notes of the repository):
+ *   - distance = squared Euclidean distance, for the cache keys and for the
+ *     corpus alike (Section 3.1: the cache uses the database's distance);
+ *   - ties between keys at equal distance go to the lowest slot; ties between
+ *     corpus rows go to the lowest row id;
+ *   - slots fill in index order 0..c-1, afterwards the victim's slot is reused;
+ *   - every query owns one logical time stamp; an insert counts as a use;
+ *   - a hit returns the stored list (and the stored distances of the key's own
+ *     query) unchanged and alters nothing but the LRU stamp;
+ *   - an empty cache is a miss; capacity 0 is rejected.
+ *
+ * All sums are taken in double precision over the float inputs, one term
+ * after the other in index order.  OpenMP only splits independent rows over
+ * threads; the order inside a row and the selection pass stay sequential, so
+ * the result does not depend on the thread count.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ORACLE_LRU = 0, ORACLE_FIFO = 1 };
+
+typedef struct {
+    /* stored state of Algorithm 1: tau, c, the database D and the dict C */
+    const float *corpus;   /* N x d, borrowed; NULL = trace-only (no database) */
+    int64_t N;
+    int32_t d, k;
+    int64_t capacity;
+    double tau;
+    int32_t policy;
+    /* the dict C: slot s holds a key (copy of the query), its value list */
+    float *keys;           /* capacity x d */
+    int64_t *val_ids;      /* capacity x k */
+    double *val_dists;     /* capacity x k */
+    int64_t *stamp;        /* capacity: LRU = last use, FIFO = insertion time */
+    int64_t *origin;       /* capacity: stream index of the query that made the key */
+    uint8_t *valid;        /* capacity */
+    int64_t count;         /* |C| */
+    int64_t clock;         /* logical time = number of queries seen */
+    /* counters */
+    int64_t probe_madds;   /* multiply-adds spent in key distances (Section 3.2: c*d per query) */
+    int64_t n_hits, n_misses, n_evictions;
+    double *scratch;       /* N distances for the database call */
+} oracle_t;
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* Squared Euclidean distance, Algorithm 1 "distance(q, k)": sum_j (a_j - b_j)^2 in fp64. */
+double oracle_sqdist(const float *a, const float *b, int32_t d) {
+    double acc = 0.0;
+    for (int32_t j = 0; j < d; ++j) {
+        double diff = (double)a[j] - (double)b[j];
+        acc += diff * diff;
+    }
+    return acc;
+}
+
+/*
+ * One pass of the selection behind retrieveDocumentIndices(q) over rows
+ * [base_id, base_id + n) of the corpus (chunk points at row base_id).  The k
+ * best rows seen so far are kept in out_ids / out_dists, sorted by (distance
+ * ascending, row id ascending); *have is how many are filled.  Chunks must be
+ * fed in ascending row order so that equal distances keep the lower id first.
+ */
+void oracle_topk_update(const float *chunk, int64_t n, int32_t d, int64_t base_id, const float *q,
+                        int32_t k, double *scratch, int64_t *out_ids, double *out_dists,
+                        int32_t *have_io) {
+    double *dist = scratch;
+    int own = 0;
+    if (!dist) { dist = (double *)malloc(sizeof(double) * (size_t)n); own = 1; }
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i) dist[i] = oracle_sqdist(q, chunk + i * (int64_t)d, d);
+
+    int32_t have = *have_io;
+    for (int64_t i = 0; i < n; ++i) {
+        double v = dist[i];
+        if (have == k && !(v < out_dists[k - 1])) continue;   /* equal to the worst: the earlier id stays */
+        int32_t pos = (have < k) ? have : k - 1;
+        while (pos > 0 && out_dists[pos - 1] > v) {            /* strictly greater: earlier ids stay in front */
+            out_dists[pos] = out_dists[pos - 1];
+            out_ids[pos] = out_ids[pos - 1];
+            --pos;
+        }
+        out_dists[pos] = v;
+        out_ids[pos] = base_id + i;
+        if (have < k) ++have;
+    }
+    *have_io = have;
+    if (own) free(dist);
+}
+
+/*
+ * retrieveDocumentIndices(q): the k rows of the corpus closest to q, as a list
+ * sorted by (distance ascending, row id ascending).  Every row is measured.
+ */
+void oracle_exact_topk(const float *corpus, int64_t N, int32_t d, const float *q, int32_t k,
+                       double *scratch, int64_t *out_ids, double *out_dists) {
+    int32_t have = 0;
+    oracle_topk_update(corpus, N, d, 0, q, k, scratch, out_ids, out_dists, &have);
+    for (int32_t r = have; r < k; ++r) { out_ids[r] = -1; out_dists[r] = INFINITY; }
+}
+
+oracle_t *oracle_create(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
+                        double tau, int32_t policy) {
+    if (d < 1 || k < 1 || capacity < 1 || !(tau >= 0.0)) return NULL;
+    if (policy != ORACLE_LRU && policy != ORACLE_FIFO) return NULL;
+    if (corpus && (N < 1 || k > N)) return NULL;
+    oracle_t *o = (oracle_t *)calloc(1, sizeof(oracle_t));
+    if (!o) return NULL;
+    o->corpus = corpus; o->N = N; o->d = d; o->k = k;
+    o->capacity = capacity; o->tau = tau; o->policy = policy;
+    o->keys = (float *)calloc((size_t)capacity * d, sizeof(float));
+    o->val_ids = (int64_t *)calloc((size_t)capacity * k, sizeof(int64_t));
+    o->val_dists = (double *)calloc((size_t)capacity * k, sizeof(double));
+    o->stamp = (int64_t *)calloc((size_t)capacity, sizeof(int64_t));
+    o->origin = (int64_t *)calloc((size_t)capacity, sizeof(int64_t));
+    o->valid = (uint8_t *)calloc((size_t)capacity, 1);
+    o->scratch = corpus ? (double *)malloc(sizeof(double) * (size_t)N) : NULL;
+    return o;
+}
+
+void oracle_destroy(oracle_t *o) {
+    if (!o) return;
+    free(o->keys); free(o->val_ids); free(o->val_dists); free(o->stamp);
+    free(o->origin); free(o->valid); free(o->scratch); free(o);
+}
+
+void oracle_reset(oracle_t *o) {
+    memset(o->valid, 0, (size_t)o->capacity);
+    o->count = 0; o->clock = 0;
+    o->probe_madds = 0; o->n_hits = o->n_misses = o->n_evictions = 0;
+}
+
+void oracle_counters(const oracle_t *o, int64_t *out5) {
+    out5[0] = o->probe_madds; out5[1] = o->n_hits; out5[2] = o->n_misses;
+    out5[3] = o->n_evictions; out5[4] = o->count;
+}
+
+/* Load n keys into slots 0..n-1 with stamps 0..n-1 and empty value lists (test/bench set-up). */
+int oracle_cache_load(oracle_t *o, const float *keys, int64_t n) {
+    if (n < 0 || n > o->capacity) return 1;
+    oracle_reset(o);
+    memcpy(o->keys, keys, sizeof(float) * (size_t)n * o->d);
+    for (int64_t s = 0; s < n; ++s) {
+        o->valid[s] = 1; o->stamp[s] = s; o->origin[s] = -1 - s;
+        for (int32_t r = 0; r < o->k; ++r) { o->val_ids[s * o->k + r] = -1; o->val_dists[s * o->k + r] = 0.0; }
+    }
+    o->count = n; o->clock = n;
+    return 0;
+}
+
+/*
+ * One LOOKUP(q) of Algorithm 1.
+ *   force: -1 = decide by the threshold test; 0 / 1 = take "miss" / "hit"
+ *          instead (used by a harness to keep two state machines in step on a
+ *          query whose distance ties with tau to rounding; never by default).
+ * Outputs (any may be NULL):
+ *   out_ids[k], out_dists[k]  the returned list (dists: those stored with the key on a hit)
+ *   trace[0] hit (0/1)
+ *   trace[1] slot: the matched slot on a hit, the slot written on a miss
+ *   trace[2] stream index of the query whose miss created the matched key (hit), else own index
+ *   trace[3] slot evicted by this query, or -1
+ *   dtrace[0] distance to the nearest key (+inf if the cache is empty)
+ *   dtrace[1] distance to the second nearest key (+inf if fewer than two)
+ */
+void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids, double *out_dists,
+                   int64_t *trace, double *dtrace) {
+    const int32_t d = o->d, k = o->k;
+    const int64_t t = o->clock++;                 /* this query's time stamp */
+
+    /* lines 2-3 of Algorithm 1: all key distances, then the minimum (first minimum in slot order) */
+    double best = INFINITY, second = INFINITY;
+    int64_t best_slot = -1;
+    for (int64_t s = 0; s < o->capacity; ++s) {
+        if (!o->valid[s]) continue;
+        double dist = oracle_sqdist(q, o->keys + s * d, d);
+        o->probe_madds += d;
+        if (dist < best) { second = best; best = dist; best_slot = s; }
+        else if (dist < second) second = dist;
+    }
+    if (dtrace) { dtrace[0] = best; dtrace[1] = second; }
+
+    int hit = (best_slot >= 0 && best <= o->tau);  /* line 4: min_dist <= tau */
+    if (force == 0) hit = 0;
+    if (force == 1 && best_slot >= 0) hit = 1;
+
+    if (hit) {                                     /* line 5: return C[key] */
+        if (o->policy == ORACLE_LRU) o->stamp[best_slot] = t;   /* a hit is a use (LRU only) */
+        if (out_ids) memcpy(out_ids, o->val_ids + best_slot * k, sizeof(int64_t) * k);
+        if (out_dists) memcpy(out_dists, o->val_dists + best_slot * k, sizeof(double) * k);
+        if (trace) { trace[0] = 1; trace[1] = best_slot; trace[2] = o->origin[best_slot]; trace[3] = -1; }
+        o->n_hits++;
+        return;
+    }
+
+    /* line 6: I <- D.retrieveDocumentIndices(q) */
+    int64_t *ids = (int64_t *)malloc(sizeof(int64_t) * k);
+    double *dists = (double *)malloc(sizeof(double) * k);
+    if (o->corpus) oracle_exact_topk(o->corpus, o->N, d, q, k, o->scratch, ids, dists);
+    else for (int32_t r = 0; r < k; ++r) { ids[r] = -1; dists[r] = 0.0; }
+
+    /* lines 7-8: if |C| >= c evict one entry (the smallest stamp; stamps are unique) */
+    int64_t slot, evicted = -1;
+    if (o->count >= o->capacity) {
+        slot = -1;
+        for (int64_t s = 0; s < o->capacity; ++s)
+            if (o->valid[s] && (slot < 0 || o->stamp[s] < o->stamp[slot])) slot = s;
+        o->valid[slot] = 0; o->count--; o->n_evictions++;
+        evicted = slot;
+    } else {
+        slot = o->count;                           /* slots fill in index order */
+    }
+
+    /* line 9: C[q] <- I */
+    memcpy(o->keys + slot * d, q, sizeof(float) * d);
+    memcpy(o->val_ids + slot * k, ids, sizeof(int64_t) * k);
+    memcpy(o->val_dists + slot * k, dists, sizeof(double) * k);
+    o->valid[slot] = 1; o->stamp[slot] = t; o->origin[slot] = t; o->count++;
+    o->n_misses++;
+
+    /* line 10: return I */
+    if (out_ids) memcpy(out_ids, ids, sizeof(int64_t) * k);
+    if (out_dists) memcpy(out_dists, dists, sizeof(double) * k);
+    if (trace) { trace[0] = 0; trace[1] = slot; trace[2] = t; trace[3] = evicted; }
+    free(ids); free(dists);
+}
+
+/* A stream of n queries, strictly one after the other.  force may be NULL. */
+void oracle_query_stream(oracle_t *o, const float *queries, int64_t n, const int32_t *force,
+                         int64_t *out_ids, double *out_dists, int64_t *trace, double *dtrace) {
+    for (int64_t i = 0; i < n; ++i)
+        oracle_lookup(o, queries + i * o->d, force ? force[i] : -1,
+                      out_ids ? out_ids + i * o->k : NULL,
+                      out_dists ? out_dists + i * o->k : NULL,
+                      trace ? trace + i * 4 : NULL, dtrace ? dtrace + i * 2 : NULL);
+}
+
+/* The database call alone for a set of queries (used to check sampled misses at large N). */
+void oracle_knn_batch(const float *corpus, int64_t N, int32_t d, const float *queries, int64_t n,
+                      int32_t k, int64_t *out_ids, double *out_dists) {
+    double *scratch = (double *)malloc(sizeof(double) * (size_t)N);
+    for (int64_t i = 0; i < n; ++i)
+        oracle_exact_topk(corpus, N, d, queries + i * d, k, scratch, out_ids + i * k, out_dists + i * k);
+    free(scratch);
+}
+
+/* Read-only views for tests. */
+int64_t oracle_slot_stamp(const oracle_t *o, int64_t s) { return o->valid[s] ? o->stamp[s] : -1; }
+int64_t oracle_slot_origin(const oracle_t *o, int64_t s) { return o->valid[s] ? o->origin[s] : -1; }

@@ -1,0 +1,227 @@
+"""Pins of the CPU oracle against things other than itself: closed forms, an independent
+numpy brute force, the invariants that Algorithm 1 and Section 3.3 of the paper imply,
+hand-traced eviction sequences, and the paper's own operation count (Section 3.2)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2503_05530_b200 import workloads as W
+from golden_traces import all_traces
+
+POL = {"lru": oracle.LRU, "fifo": oracle.FIFO}
+
+
+def unit_rows(n, d, seed):
+    r = np.random.default_rng(seed).standard_normal((n, d))
+    return (r / np.linalg.norm(r, axis=1, keepdims=True)).astype(np.float32)
+
+
+# ---------------------------------------------------------------- distance (Algorithm 1, line 2)
+def test_sqdist_closed_forms():
+    assert oracle.sqdist([1, 2, 3], [4, 6, 8]) == 50.0           # 9 + 16 + 25
+    e = np.eye(8, dtype=np.float32)
+    for i in range(8):
+        for j in range(8):
+            assert oracle.sqdist(e[i], e[j]) == (0.0 if i == j else 2.0)   # orthonormal basis
+    a = unit_rows(5, 768, 0)
+    for i in range(5):
+        assert oracle.sqdist(a[i], a[i]) == 0.0                   # duplicates: exactly zero
+        for j in range(5):                                        # |a-b|^2 = |a|^2 + |b|^2 - 2 a.b
+            a64, b64 = a[i].astype(np.float64), a[j].astype(np.float64)
+            closed = a64 @ a64 + b64 @ b64 - 2 * (a64 @ b64)
+            assert abs(oracle.sqdist(a[i], a[j]) - closed) < 1e-12
+            assert oracle.sqdist(a[i], a[j]) == oracle.sqdist(a[j], a[i])
+    # not a dot product, not an unsquared norm, not a difference without the square
+    assert oracle.sqdist([3, 0], [0, 4]) == 25.0
+    assert oracle.sqdist([-1, -1], [1, 1]) == 8.0
+
+
+# ---------------------------------------------------------------- database call (Algorithm 1, line 6)
+@pytest.mark.parametrize("n,d,k,seed", [(50, 3, 5, 0), (1000, 16, 10, 1), (777, 128, 32, 2), (64, 768, 64, 3)])
+def test_exact_topk_vs_numpy_bruteforce(n, d, k, seed):
+    X = unit_rows(n, d, seed)
+    Q = unit_rows(7, d, seed + 100)
+    ids, dists = oracle.exact_topk(X, Q, k)
+    X64, Q64 = X.astype(np.float64), Q.astype(np.float64)
+    for i in range(Q.shape[0]):
+        full = ((X64 - Q64[i]) ** 2).sum(1)
+        order = np.lexsort((np.arange(n), full))[:k]              # by distance, then id
+        assert np.array_equal(ids[i], order)
+        assert np.allclose(dists[i], full[order], rtol=1e-13, atol=0)
+        assert np.all(np.diff(dists[i]) >= 0)                     # "sorted list" (Section 3)
+
+
+def test_exact_topk_planted_ties_and_permutation():
+    X = unit_rows(300, 32, 5)
+    q = unit_rows(1, 32, 6)[0]
+    X[17] = q                                                     # planted exact neighbour
+    X[250] = X[40]                                                # duplicate rows: equal distance
+    ids, dists = oracle.exact_topk(X, q, 300)
+    assert ids[0, 0] == 17 and dists[0, 0] == 0.0
+    p40, p250 = np.where(ids[0] == 40)[0][0], np.where(ids[0] == 250)[0][0]
+    assert p250 == p40 + 1                                        # tie: lower id first
+    perm = np.random.default_rng(0).permutation(300)
+    ids_p, dists_p = oracle.exact_topk(X[perm], q, 20)
+    ids_s, dists_s = oracle.exact_topk(X, q, 20)
+    assert np.array_equal(dists_p, dists_s)                       # same multiset of rows
+    assert set(perm[ids_p[0]]) == set(ids_s[0])
+
+
+def test_chunked_topk_equals_whole():
+    X, q = unit_rows(1000, 24, 7), unit_rows(1, 24, 8)[0]
+    X[900] = X[3]
+    whole_ids, whole_d = oracle.exact_topk(X, q, 1000)
+    ch = oracle.ChunkedTopK(q, 1000)
+    for a, b in [(0, 1), (1, 333), (333, 334), (334, 1000)]:
+        ch.feed(X[a:b])
+    assert np.array_equal(ch.ids, whole_ids[0]) and np.array_equal(ch.dists, whole_d[0])
+
+
+# ---------------------------------------------------------------- invariants of Algorithm 1
+def small_workload(seed=0, N=400, d=32, nq=120, topics=15):
+    torch.manual_seed(0)
+    X = W.make_corpus(N, d, 8, seed)
+    q, ranks, rows = W.make_query_stream(X, nq, topics, 1.1, 0.02, seed)
+    return X.numpy(), q.numpy(), ranks.numpy()
+
+
+@pytest.mark.parametrize("policy", ["lru", "fifo"])
+def test_tau_zero_without_duplicates_is_plain_knn(policy):
+    X, Q, _ = small_workload()
+    o = oracle.Oracle(X, X.shape[1], 5, 10, 0.0, POL[policy])
+    r = o.query(Q)
+    assert r["hit"].sum() == 0                                    # tau = 0: exact matching only (Section 3.3.3)
+    ids, dists = oracle.exact_topk(X, Q, 5)
+    assert np.array_equal(r["ids"], ids) and np.array_equal(r["dists"], dists)
+    c = o.counters()
+    assert c["misses"] == len(Q) and c["evictions"] == len(Q) - 10 and c["count"] == 10
+
+
+@pytest.mark.parametrize("tau", [0.0, 0.3])
+def test_exact_duplicate_of_resident_key_hits(tau):
+    X, Q, _ = small_workload(1)
+    Q = Q.copy()
+    Q[50] = Q[47]                                                 # 47 is still resident (capacity 10 > 3)
+    o = oracle.Oracle(X, X.shape[1], 4, 10, tau, oracle.LRU)
+    r = o.query(Q)
+    if tau == 0.0:
+        assert r["hit"].sum() == 1
+    assert r["hit"][50] == 1
+    assert np.array_equal(r["ids"][50], r["ids"][r["origin"][50]])
+    if r["hit"][47] == 0:                                         # 47 became a key: its copy is at distance 0
+        assert r["best"][50] == 0.0 and r["origin"][50] == 47
+    else:                                                         # 47 hit a key that LRU kept: the copy sees the same
+        assert r["best"][50] <= r["best"][47] and r["best"][50] <= tau
+
+
+def test_huge_tau_every_later_query_hits_first_key():
+    X, Q, _ = small_workload(2)
+    o = oracle.Oracle(X, X.shape[1], 6, 10, 4.0 + 1e-6, oracle.FIFO)   # unit vectors: distance <= 4
+    r = o.query(Q)
+    assert r["hit"][0] == 0 and r["hit"][1:].all()
+    assert (r["slot"] == 0).all() and (r["origin"] == 0).all()
+    assert (r["ids"] == r["ids"][0]).all() and (r["dists"] == r["dists"][0]).all()
+    assert o.counters()["count"] == 1 and o.counters()["evictions"] == 0
+    ids0, _ = oracle.exact_topk(X, Q[0], 6)
+    assert np.array_equal(r["ids"][0], ids0[0])
+
+
+@pytest.mark.parametrize("policy", ["lru", "fifo"])
+def test_capacity_one(policy):
+    X, Q, _ = small_workload(3)
+    tau = 0.2
+    o = oracle.Oracle(X, X.shape[1], 3, 1, tau, POL[policy])
+    r = o.query(Q)
+    last_miss = -1
+    for i in range(len(Q)):
+        if last_miss >= 0:
+            dist = float(((Q[i].astype(np.float64) - Q[last_miss].astype(np.float64)) ** 2).sum())
+            assert r["hit"][i] == (dist <= tau)                   # only the most recent miss is resident
+            assert abs(r["best"][i] - dist) < 1e-12
+        else:
+            assert r["hit"][i] == 0 and np.isinf(r["best"][i])     # empty cache: a miss
+        if r["hit"][i]:
+            assert r["origin"][i] == last_miss and np.array_equal(r["ids"][i], r["ids"][last_miss])
+        else:
+            assert r["slot"][i] == 0 and r["evicted"][i] == (0 if last_miss >= 0 else -1)
+            last_miss = i
+    assert 0 < r["hit"].sum() < len(Q)
+
+
+def test_hit_returns_nearest_key_and_eviction_only_when_full():
+    X, Q, _ = small_workload(4, nq=200)
+    cap, tau = 12, 0.15
+    o = oracle.Oracle(X, X.shape[1], 3, cap, tau, oracle.LRU)
+    r = o.query(Q)
+    # replay with an independent dict-based model written straight from Algorithm 1
+    keys, stamp = {}, {}
+    Q64 = Q.astype(np.float64)
+    for i in range(len(Q)):
+        dist = {s: float(((Q64[i] - Q64[j]) ** 2).sum()) for s, j in keys.items()}
+        best = min(dist, key=lambda s: (dist[s], s)) if dist else None
+        if best is not None and dist[best] <= tau:
+            assert r["hit"][i] == 1 and r["slot"][i] == best and r["origin"][i] == keys[best]
+            stamp[best] = i
+        else:
+            assert r["hit"][i] == 0
+            if len(keys) >= cap:                                  # evict only when |C| >= c
+                victim = min(stamp, key=stamp.get)
+                assert r["evicted"][i] == victim
+                del keys[victim], stamp[victim]
+                slot = victim
+            else:
+                assert r["evicted"][i] == -1
+                slot = len(keys)
+            assert r["slot"][i] == slot
+            keys[slot], stamp[slot] = i, i
+    assert 0 < r["hit"].sum() < len(Q) and o.counters()["evictions"] > 0
+
+
+def test_hit_rate_grows_with_tau_on_the_synthetic_stream():
+    X, Q, _ = small_workload(5, nq=300)
+    rates = []
+    for tau in [0.0, 0.02, 0.1, 0.5, 2.0, 4.1]:
+        o = oracle.Oracle(None, X.shape[1], 1, 20, tau, oracle.LRU)
+        rates.append(o.query(Q)["hit"].mean())
+    assert rates[0] == 0.0 and rates[-1] == (len(Q) - 1) / len(Q)
+    assert all(b >= a for a, b in zip(rates, rates[1:]))
+
+
+# ---------------------------------------------------------------- hand-traced eviction orders
+@pytest.mark.parametrize("tr", all_traces(), ids=lambda t: t["name"])
+def test_golden_traces(tr):
+    o = oracle.Oracle(tr["corpus"], tr["corpus"].shape[1], tr["k"], tr["capacity"], tr["tau"], POL[tr["policy"]])
+    r = o.query(tr["queries"])
+    assert np.array_equal(r["hit"], tr["hit"])
+    assert np.array_equal(r["slot"], tr["slot"])
+    assert np.array_equal(r["evicted"], tr["evicted"])
+    assert np.array_equal(r["ids"], tr["ids"])
+
+
+def test_fifo_and_lru_traces_differ():
+    by = {t["name"]: t for t in all_traces()}
+    a, b = by["trace_c2_fifo.txt"], by["trace_c2_lru.txt"]
+    assert np.array_equal(a["queries"], b["queries"]) and not np.array_equal(a["hit"], b["hit"])
+
+
+# ---------------------------------------------------------------- the paper's operation count
+def test_flat_probe_operation_count():
+    """Section 3.2: with c = 10 000 entries and d = 768 one FLAT lookup performs
+    10 000 x 768 = 7.68 million operations."""
+    keys = unit_rows(10_000, 768, 11)
+    o = oracle.Oracle(None, 768, 1, 10_000, 0.0, oracle.LRU)
+    o.cache_load(keys)
+    o.query(unit_rows(1, 768, 12))
+    assert o.counters()["probe_madds"] == 7_680_000
+
+
+# ---------------------------------------------------------------- forcing a decision
+def test_forced_decisions_follow_the_branch():
+    X, Q, _ = small_workload(6, nq=40)
+    o = oracle.Oracle(X, X.shape[1], 2, 8, 0.0, oracle.LRU)
+    force = np.full(40, -1, np.int32)
+    force[5] = 1                                                  # a forced hit returns the nearest key's list
+    r = o.query(Q, force)
+    assert r["hit"][5] == 1 and np.array_equal(r["ids"][5], r["ids"][r["origin"][5]])
+    assert r["hit"].sum() == 1
