@@ -1,0 +1,156 @@
+/*
+ * prox.h -- C ABI of the B200 approximate query cache with exact top-k corpus scan.
+ *
+ * The library keeps, on one GPU, the state of Algorithm 1 of the paper ("Cache
+ * lookup in PROXIMITY-FLAT"): the tolerance tau, the capacity c, the database D
+ * (a corpus of N embeddings of dimension d) and the key-value store C whose keys
+ * are earlier query embeddings and whose values are their top-k lists.  One call
+ * of prox_query_batch performs LOOKUP(q) for a batch of queries with exactly the
+ * outcome of running Algorithm 1 on them one after the other in index order.
+ *
+ * Conventions
+ *  - Distances are squared Euclidean distances, for keys and corpus alike
+ *    (Section 3.1: the cache uses the distance function of the database).
+ *  - Every pointer marked DEVICE is a device pointer valid on the GPU that was
+ *    current when prox_create ran; HOST pointers are ordinary host memory.
+ *  - Calls on one handle must be ordered on one stream at a time: the cache is
+ *    state.  prox_query_batch only enqueues work; its outputs are valid once
+ *    the stream has reached the end of that work.
+ *  - Functions returning int32_t return PROX_OK or an error code; a text for the
+ *    last error of the calling thread is available from prox_last_error().
+ *  - Inputs must be finite; this is not checked on the device.
+ */
+#ifndef PROX_H_
+#define PROX_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct prox_handle prox_handle;      /* opaque, owned by the library */
+
+enum { PROX_LRU = 0, PROX_FIFO = 1 };        /* Section 3.3.2: eviction policy */
+
+enum {
+    PROX_OK = 0,
+    PROX_ERR_INVALID_ARG = 1,   /* nothing was launched */
+    PROX_ERR_OOM = 2,
+    PROX_ERR_CUDA = 3,
+    PROX_ERR_UNSUPPORTED = 4,   /* shape outside what the kernels are built for */
+    PROX_ERR_TIMEOUT = 5,       /* a bounded device-side wait ran out (latched) */
+    PROX_ERR_INTERNAL = 6       /* a device-side capacity or bounds check failed (latched) */
+};
+
+enum {
+    PROX_MAX_K = 64,            /* largest k */
+    PROX_MAX_BATCH = 1024,      /* largest B of one call */
+    PROX_SCAN_AUTO = 0,         /* prox_set_scan_mode: tensor-core scan (default) */
+    PROX_SCAN_CUDA_CORE = 1     /* prox_set_scan_mode: plain CUDA-core scan of the same bf16 scores */
+};
+
+/*
+ * prox_create -- set up the stored state of Algorithm 1 (tau, c, D, C = {}).
+ *   corpus   DEVICE, N x d fp32 row-major, BORROWED: the caller keeps it alive and
+ *            unchanged until prox_destroy.  The library makes its own bf16 copy
+ *            (round to nearest even) and per-row norms for the scan.
+ *   N        number of corpus rows, 1 <= N < 2^31.
+ *   d        embedding dimension, a multiple of 16, 16 <= d <= 4096.
+ *   k        neighbours per query, 1 <= k <= min(N, PROX_MAX_K).
+ *   capacity c of Section 3.3.1, >= 1 (c = 0 is rejected: Algorithm 1 would evict from an empty store).
+ *   tau      tolerance of Section 3.3.3 on the squared distance, >= 0 and not NaN;
+ *            a key matches when distance <= tau (Algorithm 1, line 4).
+ *   policy   PROX_LRU or PROX_FIFO.
+ * Returns NULL on failure (see prox_last_error).  Allocates with cudaMalloc on
+ * the current device and synchronises that device before returning.
+ */
+prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
+                         float tau, int32_t policy);
+
+/*
+ * prox_query_batch -- LOOKUP(q) of Algorithm 1 for queries 0..B-1, with the
+ * outcome of processing them strictly in index order: query i sees the inserts,
+ * evictions and LRU touches of queries 0..i-1 of the same batch.
+ *   queries   DEVICE, B x d fp32 row-major, borrowed until the enqueued work is done.
+ *   B         1 <= B <= PROX_MAX_BATCH.
+ *   out_ids   DEVICE, B x k int64: the returned list I (corpus row ids, nearest first;
+ *             ties by lower id).  On a hit: the list stored with the matched key.
+ *   out_dists DEVICE, B x k fp32: squared distances belonging to out_ids.  On a hit these
+ *             are the distances stored with the key, i.e. those of the key's own query.
+ *   out_hit   DEVICE, B bytes: 1 = cache hit (Algorithm 1, line 5), 0 = miss (lines 6-10).
+ *   stream    a cudaStream_t (NULL = the default stream).
+ * Misses are answered by an exact k-nearest-neighbour search over the whole corpus
+ * (Algorithm 1, line 6, with a flat exact index as in Section 4.2.1).
+ * Asynchronous; no device-to-host copy and no synchronisation happens inside.
+ * Errors found on the device are latched and reported by prox_status.
+ */
+int32_t prox_query_batch(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
+                         float *out_dists, uint8_t *out_hit, void *stream);
+
+/*
+ * prox_query_batch_host -- the same call for HOST buffers (queries, out_ids, out_dists,
+ * out_hit are host pointers, ideally pinned).  Copies the queries to the device, runs
+ * prox_query_batch, copies the three outputs back and synchronises the stream.
+ */
+int32_t prox_query_batch_host(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
+                              float *out_dists, uint8_t *out_hit, void *stream);
+
+/* prox_reset_cache -- C = {} (count and clock to zero); the corpus stays.  Asynchronous on stream. */
+int32_t prox_reset_cache(prox_handle *h, void *stream);
+
+/* prox_destroy -- synchronise the device and free everything the library owns.  NULL is a no-op. */
+void prox_destroy(prox_handle *h);
+
+/* prox_last_error -- text of the calling thread's last error ("" if none); static storage. */
+const char *prox_last_error(void);
+
+/* ---- diagnostics and benchmark hooks (outside Algorithm 1) ------------------------------- */
+
+/*
+ * prox_cache_load -- fill slots 0..n-1 with the given keys (DEVICE, n x d fp32), stamps
+ * 0..n-1 and empty value lists (ids -1, distances 0); count = clock = n.  Stands in for
+ * n earlier misses when only the probe is measured (the lookup-time experiment of
+ * Section 4.4.1).  n <= capacity.  Asynchronous on stream.
+ */
+int32_t prox_cache_load(prox_handle *h, const float *keys, int64_t n, void *stream);
+
+/*
+ * prox_probe_batch -- lines 2-4 and 7-9 of Algorithm 1 only: probe, threshold test,
+ * LRU touch, eviction and insertion of the query as a key, with an empty value list in
+ * place of the database call.
+ *   out_hit      DEVICE, B bytes.
+ *   out_slot     DEVICE, B int32: the matched slot on a hit, the written slot on a miss.
+ *   out_min_dist DEVICE, B fp32: distance to the nearest key at the time of the lookup
+ *                (+inf when the cache was empty).
+ */
+int32_t prox_probe_batch(prox_handle *h, const float *queries, int32_t B, uint8_t *out_hit,
+                         int32_t *out_slot, float *out_min_dist, void *stream);
+
+typedef struct prox_stats {
+    int64_t queries, hits, misses;      /* since create / reset */
+    int64_t intra_batch_hits;           /* hits on a key inserted earlier in the same batch */
+    int64_t evictions;
+    int64_t scan_batches;               /* batches in which the corpus was scanned */
+    int64_t uncertified;                /* misses whose bf16 candidate set was not proven complete */
+    int64_t fallback_rows;              /* rows collected by the exact fp32 pass for those misses */
+    int64_t unresolved;                 /* misses whose exact pass overflowed (result best effort) */
+    int64_t count;                      /* |C| now */
+} prox_stats;
+
+/* prox_get_stats -- synchronises the stream, then copies the device counters to *out (HOST). */
+int32_t prox_get_stats(prox_handle *h, prox_stats *out, void *stream);
+
+/* prox_status -- synchronises the stream and returns the latched device error (PROX_OK if none). */
+int32_t prox_status(prox_handle *h, void *stream);
+
+/* prox_set_scan_mode -- PROX_SCAN_AUTO or PROX_SCAN_CUDA_CORE (for cross-checks and timing). */
+int32_t prox_set_scan_mode(prox_handle *h, int32_t mode);
+
+/* prox_kernel_launches -- kernels launched by this handle so far (host-side count). */
+int64_t prox_kernel_launches(const prox_handle *h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PROX_H_ */

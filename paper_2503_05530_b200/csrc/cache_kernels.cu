@@ -1,0 +1,655 @@
+// Cache-side kernels: the probe (lines 2-3 of Algorithm 1 for a whole batch), the
+// sequential-order resolve (lines 4-9), and the copies that read and write the value slots.
+//
+// How a batch is made to behave like B sequential lookups.  During one batch the only
+// pre-batch entries that can be evicted are the R = min(B, |C|) entries that come first in
+// eviction order (every query causes at most one touch or one eviction, so fewer than B
+// entries can leave or be refreshed before the last query).  The probe therefore reduces
+// the distances to all other ("safe") slots to one minimum per query, and keeps full rows
+// only for the R at-risk slots and for the earlier queries of the same batch.  The resolve
+// then replays the batch in index order on those rows alone.
+#include <cfloat>
+#include <cmath>
+
+#include "prox_internal.h"
+#include "topk_device.cuh"
+
+namespace prox {
+
+
+// ------------------------------------------------------------------------------------------
+// At-risk list: the R entries with the smallest stamps, in stamp order (Section 3.3.2: the
+// victim is always the entry with the oldest insertion (FIFO) or oldest use (LRU)).
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+risk_select_kernel(DevState *st, const u64 *__restrict__ stamp, int32_t *risk_pos,
+                   int32_t *risk_slot, u64 *risk_stamp, int B, long long C) {
+    __shared__ unsigned hist[256];
+    __shared__ u64 s_key[1024];
+    __shared__ int s_val[1024];
+    __shared__ u64 s_prefix, s_mask;
+    __shared__ int s_remaining, s_n;
+    const int tid = threadIdx.x;
+
+    const int prev = st->n_risk;
+    for (int r = tid; r < prev; r += blockDim.x) risk_pos[risk_slot[r]] = -1;
+    const long long count = st->count;
+    const long long clock = st->clock;
+    __syncthreads();
+
+    int R = 0;
+    if (count + B > C) R = (int)(count < (long long)B ? count : (long long)B);
+    if (R == 0) {
+        if (tid == 0) st->n_risk = 0;
+        return;
+    }
+
+    u64 T = ~0ull;                       // R-th smallest stamp
+    if ((long long)R < count) {
+        int nd = 1;
+        while (nd < 8 && (clock >> (8 * nd)) != 0) ++nd;
+        if (tid == 0) { s_prefix = 0; s_mask = 0; s_remaining = R; }
+        for (int p = nd - 1; p >= 0; --p) {
+            if (tid < 256) hist[tid] = 0;
+            __syncthreads();
+            const u64 prefix = s_prefix, mask = s_mask;
+            for (long long s = tid; s < count; s += blockDim.x) {
+                const u64 v = stamp[s];
+                if ((v & mask) == prefix) atomicAdd(&hist[(unsigned)(v >> (8 * p)) & 255u], 1u);
+            }
+            __syncthreads();
+            if (tid == 0) {
+                int rem = s_remaining, b = 0;
+                while (b < 255 && (int)hist[b] < rem) { rem -= (int)hist[b]; ++b; }
+                s_remaining = rem;
+                s_prefix = prefix | ((u64)b << (8 * p));
+                s_mask = mask | (0xffull << (8 * p));
+            }
+            __syncthreads();
+        }
+        T = s_prefix;
+    }
+
+    if (tid == 0) s_n = 0;
+    s_key[tid] = ~0ull;
+    s_val[tid] = 0x7fffffff;
+    __syncthreads();
+    for (long long s = tid; s < count; s += blockDim.x) {
+        const u64 v = stamp[s];
+        if (v <= T) {
+            const int pos = atomicAdd(&s_n, 1);
+            if (pos < 1024) { s_key[pos] = v; s_val[pos] = (int)s; }
+        }
+    }
+    __syncthreads();
+    if (s_n != R) {                      // stamps must be unique; anything else is a broken state
+        if (tid == 0) { atomicCAS(&st->error, 0, PROX_ERR_INTERNAL); st->n_risk = 0; }
+        return;
+    }
+    int n2 = 1;
+    while (n2 < R) n2 <<= 1;
+    block_sort_asc(s_key, s_val, n2);
+    if (tid < R) {
+        risk_slot[tid] = s_val[tid];
+        risk_stamp[tid] = s_key[tid];
+        risk_pos[s_val[tid]] = tid;
+    }
+    if (tid == 0) st->n_risk = R;
+}
+
+// ------------------------------------------------------------------------------------------
+// Probe: squared distances, in fp64 over the fp32 values and in difference form (so that a
+// bitwise duplicate is at distance exactly 0), from each query to every valid key and to
+// every earlier query of the batch.  Columns are [0, count) = slots, then [count, count+B) =
+// the batch itself.  Tile: 32 queries x 64 columns per block, d in chunks of 32.
+// ------------------------------------------------------------------------------------------
+constexpr int PQ = 32, PC = 64, PD = 32;
+
+__global__ void __launch_bounds__(256)
+probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
+             const float *__restrict__ queries, const int32_t *__restrict__ risk_pos, int B, int d,
+             double *__restrict__ part_min, int32_t *__restrict__ part_arg,
+             double *__restrict__ d_risk, double *__restrict__ d_intra) {
+    __shared__ double qs[PQ][PD + 1];
+    __shared__ double ks[PC][PD + 1];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const long long count = st->count;
+    const long long ncols = count + B;
+    const long long ntiles = (ncols + PC - 1) / PC;
+    const int S = gridDim.y, sp = blockIdx.y;
+    const long long per = (ntiles + S - 1) / S;
+    const long long t_begin = sp * per;
+    const long long t_end = (t_begin + per < ntiles) ? t_begin + per : ntiles;
+    const int q0 = blockIdx.x * PQ;
+
+    double best_d[2] = {INFINITY, INFINITY};
+    int best_s[2] = {0x7fffffff, 0x7fffffff};
+
+    for (long long t = t_begin; t < t_end; ++t) {
+        const long long c0 = t * PC;
+        double acc[2][4];
+#pragma unroll
+        for (int a = 0; a < 2; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+
+        for (int kc = 0; kc < d; kc += PD) {
+            __syncthreads();
+#pragma unroll
+            for (int it = 0; it < (PQ * PD) / 256; ++it) {
+                const int idx = it * 256 + tid, r = idx / PD, c = idx % PD;
+                const int qi = q0 + r;
+                qs[r][c] = (qi < B && kc + c < d) ? (double)queries[(size_t)qi * d + kc + c] : 0.0;
+            }
+#pragma unroll
+            for (int it = 0; it < (PC * PD) / 256; ++it) {
+                const int idx = it * 256 + tid, r = idx / PD, c = idx % PD;
+                const long long col = c0 + r;
+                double v = 0.0;
+                if (col < ncols && kc + c < d) {
+                    const float *src = (col < count) ? keys + (size_t)col * d
+                                                     : queries + (size_t)(col - count) * d;
+                    v = (double)src[kc + c];
+                }
+                ks[r][c] = v;
+            }
+            __syncthreads();
+#pragma unroll 8
+            for (int j = 0; j < PD; ++j) {
+                const double qa = qs[ty * 2][j], qb2 = qs[ty * 2 + 1][j];
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const double kv = ks[tx + 16 * b][j];
+                    const double d0 = qa - kv, d1 = qb2 - kv;
+                    acc[0][b] = fma(d0, d0, acc[0][b]);
+                    acc[1][b] = fma(d1, d1, acc[1][b]);
+                }
+            }
+        }
+#pragma unroll
+        for (int a = 0; a < 2; ++a) {
+            const int i = q0 + ty * 2 + a;
+            if (i >= B) continue;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const long long col = c0 + tx + 16 * b;
+                if (col >= ncols) continue;
+                const double v = acc[a][b];
+                if (col < count) {
+                    const int rp = risk_pos[col];
+                    if (rp >= 0) {
+                        d_risk[(size_t)i * kMaxBatch + rp] = v;
+                    } else if (v < best_d[a] || (v == best_d[a] && (int)col < best_s[a])) {
+                        best_d[a] = v;
+                        best_s[a] = (int)col;
+                    }
+                } else {
+                    const int j = (int)(col - count);
+                    if (j < i) d_intra[(size_t)i * kMaxBatch + j] = v;
+                }
+            }
+        }
+    }
+    // minimum over the 16 threads that share a query (lanes of one half warp)
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+#pragma unroll
+        for (int m = 1; m < 16; m <<= 1) {
+            const double od = __shfl_xor_sync(0xffffffffu, best_d[a], m);
+            const int os = __shfl_xor_sync(0xffffffffu, best_s[a], m);
+            if (od < best_d[a] || (od == best_d[a] && os < best_s[a])) { best_d[a] = od; best_s[a] = os; }
+        }
+        const int i = q0 + ty * 2 + a;
+        if (tx == 0 && i < B) {
+            part_min[(size_t)i * kProbeSplitMax + sp] = best_d[a];
+            part_arg[(size_t)i * kProbeSplitMax + sp] = best_s[a];
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Per query: reduce the partial safe minima; list the at-risk and in-batch keys within tau
+// (Algorithm 1, line 4, inclusive).  code < kMaxBatch: at-risk position; else kMaxBatch + j.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+build_candidates_kernel(const DevState *__restrict__ st, int B, int S, double tau,
+                        const double *__restrict__ part_min, const int32_t *__restrict__ part_arg,
+                        const double *__restrict__ d_risk, const double *__restrict__ d_intra,
+                        double *safe_min, int32_t *safe_arg, double *cand_d, int32_t *cand_code,
+                        int32_t *n_cand) {
+    __shared__ int s_n;
+    const int i = blockIdx.x, tid = threadIdx.x;
+    if (i >= B) return;
+    if (tid == 0) s_n = 0;
+    __syncthreads();
+    if (tid < 32) {
+        double bd = INFINITY;
+        int bs = 0x7fffffff;
+        for (int s = tid; s < S; s += 32) {
+            const double v = part_min[(size_t)i * kProbeSplitMax + s];
+            const int a = part_arg[(size_t)i * kProbeSplitMax + s];
+            if (v < bd || (v == bd && a < bs)) { bd = v; bs = a; }
+        }
+#pragma unroll
+        for (int m = 1; m < 32; m <<= 1) {
+            const double od = __shfl_xor_sync(0xffffffffu, bd, m);
+            const int os = __shfl_xor_sync(0xffffffffu, bs, m);
+            if (od < bd || (od == bd && os < bs)) { bd = od; bs = os; }
+        }
+        if (tid == 0) {
+            safe_min[i] = bd;
+            safe_arg[i] = (bs == 0x7fffffff) ? -1 : bs;
+        }
+    }
+    const int R = st->n_risk;
+    const size_t base = (size_t)i * (2 * kMaxBatch);
+    for (int e = tid; e < R + i; e += blockDim.x) {
+        double v;
+        int code;
+        if (e < R) { v = d_risk[(size_t)i * kMaxBatch + e]; code = e; }
+        else { v = d_intra[(size_t)i * kMaxBatch + (e - R)]; code = kMaxBatch + (e - R); }
+        if (v <= tau) {
+            const int pos = atomicAdd(&s_n, 1);
+            cand_d[base + pos] = v;
+            cand_code[base + pos] = code;
+        }
+    }
+    __syncthreads();
+    if (tid == 0) n_cand[i] = s_n;
+}
+
+// ------------------------------------------------------------------------------------------
+// Resolve: replay queries 0..B-1 in order (Algorithm 1, lines 4-9) on the candidate lists.
+// One block; warp 0 walks the batch, the other warps only help to load and store.
+// ------------------------------------------------------------------------------------------
+constexpr int kCsrCap = 8192;
+
+struct ResolveSmem {
+    u64 r_stamp[kMaxBatch];
+    u64 b_stamp[kMaxBatch];
+    double safe_min[kMaxBatch];
+    double csr_d[kCsrCap];
+    int csr_code[kCsrCap];
+    int r_slot[kMaxBatch];
+    int b_slot[kMaxBatch];
+    int safe_arg[kMaxBatch];
+    int ncand[kMaxBatch];
+    int off[kMaxBatch + 1];
+    int warp_tot[32];
+    unsigned char r_alive[kMaxBatch];
+    unsigned char r_touched[kMaxBatch];
+};
+
+__device__ __forceinline__ void lexmin_shfl(double &d, int &slot, int &code) {
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const double od = __shfl_xor_sync(0xffffffffu, d, m);
+        const int os = __shfl_xor_sync(0xffffffffu, slot, m);
+        const int oc = __shfl_xor_sync(0xffffffffu, code, m);
+        if (od < d || (od == d && os < slot)) { d = od; slot = os; code = oc; }
+    }
+}
+
+__global__ void __launch_bounds__(1024)
+resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *stamp,
+               const int32_t *__restrict__ risk_slot, const u64 *__restrict__ risk_stamp,
+               const double *__restrict__ g_safe_min, const int32_t *__restrict__ g_safe_arg,
+               const double *__restrict__ cand_d, const int32_t *__restrict__ cand_code,
+               const int32_t *__restrict__ n_cand, uint8_t *out_hit, int32_t *src, int32_t *src_kind,
+               int32_t *ins_slot, int32_t *evt_slot, float *evt_dist, int32_t *miss_list,
+               int32_t *miss_rank) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    ResolveSmem &sm = *reinterpret_cast<ResolveSmem *>(smem_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int R = st->n_risk;
+    const long long count0 = st->count, clock0 = st->clock;
+
+    // ---- load
+    {
+        const int i = tid;
+        int n = 0;
+        if (i < B) {
+            n = n_cand[i];
+            sm.safe_min[i] = g_safe_min[i];
+            sm.safe_arg[i] = g_safe_arg[i];
+            sm.b_slot[i] = -1;
+            sm.b_stamp[i] = 0;
+        }
+        if (i < R) {
+            sm.r_slot[i] = risk_slot[i];
+            sm.r_stamp[i] = risk_stamp[i];
+            sm.r_alive[i] = 1;
+            sm.r_touched[i] = 0;
+        }
+        if (i < kMaxBatch) sm.ncand[i] = n;
+        // exclusive prefix sum of n over the block
+        int x = n;
+#pragma unroll
+        for (int m = 1; m < 32; m <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, x, m);
+            if (lane >= m) x += y;
+        }
+        if (lane == 31) sm.warp_tot[warp] = x;
+        __syncthreads();
+        if (warp == 0) {
+            int w = sm.warp_tot[lane];
+#pragma unroll
+            for (int m = 1; m < 32; m <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, w, m);
+                if (lane >= m) w += y;
+            }
+            sm.warp_tot[lane] = w;
+        }
+        __syncthreads();
+        const int incl = x + (warp > 0 ? sm.warp_tot[warp - 1] : 0);
+        if (i < kMaxBatch) sm.off[i] = incl - n;
+        if (i == kMaxBatch - 1) sm.off[kMaxBatch] = incl;
+        __syncthreads();
+        for (int row = warp; row < B; row += 32) {
+            const int o = sm.off[row], nn = sm.ncand[row];
+            if (o + nn <= kCsrCap)
+                for (int e = lane; e < nn; e += 32) {
+                    sm.csr_d[o + e] = cand_d[(size_t)row * (2 * kMaxBatch) + e];
+                    sm.csr_code[o + e] = cand_code[(size_t)row * (2 * kMaxBatch) + e];
+                }
+        }
+        __syncthreads();
+    }
+
+    // ---- sequential replay by warp 0
+    if (warp == 0) {
+        long long cnt = count0;
+        int p = 0, n_miss = 0, n_hit = 0, n_intra = 0, n_evict = 0;
+        for (int i = 0; i < B; ++i) {
+            const u64 t = (u64)(clock0 + i);
+            const int n = sm.ncand[i], o = sm.off[i];
+            const bool in_smem = (o + n <= kCsrCap);
+            double bd = INFINITY;
+            int bslot = 0x7fffffff, bcode = -1;
+            for (int e = lane; e < n; e += 32) {
+                double v;
+                int code;
+                if (in_smem) { v = sm.csr_d[o + e]; code = sm.csr_code[o + e]; }
+                else { v = cand_d[(size_t)i * (2 * kMaxBatch) + e]; code = cand_code[(size_t)i * (2 * kMaxBatch) + e]; }
+                int slot;
+                bool valid;
+                if (code < kMaxBatch) { valid = sm.r_alive[code] != 0; slot = sm.r_slot[code]; }
+                else { slot = sm.b_slot[code - kMaxBatch]; valid = slot >= 0; }
+                if (valid && (v < bd || (v == bd && slot < bslot))) { bd = v; bslot = slot; bcode = code; }
+            }
+            if (lane == 0) {
+                const double sd = sm.safe_min[i];
+                const int sa = sm.safe_arg[i];
+                if (sa >= 0 && sd <= tau && (sd < bd || (sd == bd && sa < bslot))) { bd = sd; bslot = sa; bcode = -2; }
+            }
+            lexmin_shfl(bd, bslot, bcode);
+            const bool hit = (bcode != -1);
+            if (hit) {
+                ++n_hit;
+                if (lane == 0) {
+                    out_hit[i] = 1;
+                    evt_slot[i] = bslot;
+                    evt_dist[i] = (float)bd;
+                    miss_rank[i] = -1;
+                    if (bcode == -2) {
+                        src_kind[i] = 1; src[i] = bslot;
+                        if (policy == PROX_LRU) stamp[bslot] = t;
+                    } else if (bcode < kMaxBatch) {
+                        src_kind[i] = 1; src[i] = bslot;
+                        if (policy == PROX_LRU) { sm.r_stamp[bcode] = t; sm.r_touched[bcode] = 1; }
+                    } else {
+                        src_kind[i] = 2; src[i] = bcode - kMaxBatch;
+                        if (policy == PROX_LRU) sm.b_stamp[bcode - kMaxBatch] = t;
+                    }
+                }
+                if (bcode >= kMaxBatch) ++n_intra;
+            } else {
+                int slot;
+                if (cnt < C) {
+                    slot = (int)cnt;
+                    ++cnt;
+                } else {
+                    // victim: the first at-risk entry in stamp order that is still there and untouched
+                    while (p < R && (sm.r_touched[p] || !sm.r_alive[p])) ++p;
+                    __syncwarp();                           // every lane has read before lane 0 writes
+                    if (p < R) {
+                        slot = sm.r_slot[p];
+                        if (lane == 0) sm.r_alive[p] = 0;
+                        ++p;
+                    } else {
+                        // only refreshed entries and entries of this batch are left: smallest stamp
+                        u64 bs = ~0ull;
+                        int bc = -1;
+                        for (int e = lane; e < R + i; e += 32) {
+                            u64 v;
+                            bool ok;
+                            if (e < R) { ok = sm.r_alive[e] != 0; v = sm.r_stamp[e]; }
+                            else { ok = sm.b_slot[e - R] >= 0; v = sm.b_stamp[e - R]; }
+                            if (ok && v < bs) { bs = v; bc = e; }
+                        }
+#pragma unroll
+                        for (int m = 1; m < 32; m <<= 1) {
+                            const u64 ov = __shfl_xor_sync(0xffffffffu, bs, m);
+                            const int oc = __shfl_xor_sync(0xffffffffu, bc, m);
+                            if (ov < bs) { bs = ov; bc = oc; }
+                        }
+                        if (bc < 0) {                       // cannot happen with capacity >= 1
+                            if (lane == 0) atomicCAS(&st->error, 0, PROX_ERR_INTERNAL);
+                            slot = 0;
+                        } else if (bc < R) {
+                            slot = sm.r_slot[bc];
+                            if (lane == 0) sm.r_alive[bc] = 0;
+                        } else {
+                            slot = sm.b_slot[bc - R];
+                            if (lane == 0) sm.b_slot[bc - R] = -1;
+                        }
+                    }
+                    ++n_evict;
+                }
+                if (lane == 0) {
+                    out_hit[i] = 0;
+                    src_kind[i] = 0; src[i] = -1;
+                    evt_slot[i] = slot;
+                    evt_dist[i] = INFINITY;
+                    sm.b_slot[i] = slot;
+                    sm.b_stamp[i] = t;
+                    miss_list[n_miss] = i;
+                    miss_rank[i] = n_miss;
+                }
+                ++n_miss;
+            }
+            __syncwarp();
+        }
+        if (lane == 0) {
+            st->count = cnt;
+            st->clock = clock0 + B;
+            st->n_miss = n_miss;
+            st->queries += B;
+            st->hits += n_hit;
+            st->misses += n_miss;
+            st->intra_hits += n_intra;
+            st->evictions += n_evict;
+        }
+    }
+    __syncthreads();
+
+    // ---- write back stamps and the slots that entries of this batch own at batch end
+    for (int r = tid; r < R; r += blockDim.x)
+        if (sm.r_alive[r]) stamp[sm.r_slot[r]] = sm.r_stamp[r];
+    for (int j = tid; j < B; j += blockDim.x) {
+        const int s = sm.b_slot[j];
+        ins_slot[j] = s;
+        if (s >= 0) stamp[s] = sm.b_stamp[j];
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Value-slot traffic.
+// ------------------------------------------------------------------------------------------
+// Hits on a key that was resident before the batch: copy its stored list (Algorithm 1, line 5).
+// Runs before any slot is overwritten by this batch.
+__global__ void gather_hits_kernel(int B, int k, const int32_t *__restrict__ src,
+                                   const int32_t *__restrict__ src_kind,
+                                   const int32_t *__restrict__ val_ids,
+                                   const float *__restrict__ val_dists, int64_t *out_ids,
+                                   float *out_dists) {
+    const int i = blockIdx.x;
+    if (i >= B || src_kind[i] != 1) return;
+    const int s = src[i];
+    for (int r = threadIdx.x; r < k; r += blockDim.x) {
+        out_ids[(size_t)i * k + r] = (int64_t)val_ids[(size_t)s * k + r];
+        out_dists[(size_t)i * k + r] = val_dists[(size_t)s * k + r];
+    }
+}
+
+// Misses return their fresh list (line 10); hits on a key inserted earlier in the batch return
+// that query's list; entries that own a slot at batch end are written (line 9).
+__global__ void scatter_kernel(int B, int d, int k, int with_values, const float *__restrict__ queries,
+                               const int32_t *__restrict__ src, const int32_t *__restrict__ src_kind,
+                               const int32_t *__restrict__ ins_slot,
+                               const int32_t *__restrict__ miss_rank,
+                               const int32_t *__restrict__ res_ids,
+                               const double *__restrict__ res_dists, float *keys, int32_t *val_ids,
+                               float *val_dists, int64_t *out_ids, float *out_dists) {
+    const int i = blockIdx.x;
+    if (i >= B) return;
+    const int kind = src_kind[i];
+    const int owner = (kind == 0) ? i : (kind == 2 ? src[i] : -1);
+    const int m = (owner >= 0) ? miss_rank[owner] : -1;
+    if (with_values && m >= 0) {
+        for (int r = threadIdx.x; r < k; r += blockDim.x) {
+            out_ids[(size_t)i * k + r] = (int64_t)res_ids[(size_t)m * k + r];
+            out_dists[(size_t)i * k + r] = (float)res_dists[(size_t)m * k + r];
+        }
+    }
+    const int slot = ins_slot[i];
+    if (slot >= 0) {
+        for (int j = threadIdx.x; j < d; j += blockDim.x)
+            keys[(size_t)slot * d + j] = queries[(size_t)i * d + j];
+        for (int r = threadIdx.x; r < k; r += blockDim.x) {
+            val_ids[(size_t)slot * k + r] = with_values ? res_ids[(size_t)m * k + r] : -1;
+            val_dists[(size_t)slot * k + r] = with_values ? (float)res_dists[(size_t)m * k + r] : 0.f;
+        }
+    }
+}
+
+__global__ void copy_probe_outputs_kernel(int B, const int32_t *__restrict__ evt_slot,
+                                          const float *__restrict__ evt_dist, int32_t *out_slot,
+                                          float *out_min_dist) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= B) return;
+    if (out_slot) out_slot[i] = evt_slot[i];
+    if (out_min_dist) out_min_dist[i] = evt_dist[i];
+}
+
+__global__ void reset_kernel(DevState *st, int32_t *risk_pos, long long C, long long n_loaded) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < C) risk_pos[i] = -1;
+    if (i == 0) {
+        const float e_max = st->e_max;
+        const int err = st->error;
+        *st = DevState{};
+        st->e_max = e_max;
+        st->error = err;
+        st->count = n_loaded;
+        st->clock = n_loaded;
+    }
+}
+
+__global__ void cache_load_kernel(long long n, int d, int k, const float *__restrict__ src, float *keys,
+                                  int32_t *val_ids, float *val_dists, u64 *stamp) {
+    const long long s = blockIdx.x;
+    if (s >= n) return;
+    for (int j = threadIdx.x; j < d; j += blockDim.x) keys[(size_t)s * d + j] = src[(size_t)s * d + j];
+    for (int r = threadIdx.x; r < k; r += blockDim.x) {
+        val_ids[(size_t)s * k + r] = -1;
+        val_dists[(size_t)s * k + r] = 0.f;
+    }
+    if (threadIdx.x == 0) stamp[s] = (u64)s;
+}
+
+// ------------------------------------------------------------------------------------------
+// Launchers
+// ------------------------------------------------------------------------------------------
+static int probe_splits(const prox_handle *h, int B) {
+    const long long ntiles = (h->C + B + PC - 1) / PC;
+    const int qtiles = (B + PQ - 1) / PQ;
+    long long want = (4LL * h->num_sms + qtiles - 1) / qtiles;     // about four blocks per SM
+    if (want > ntiles) want = ntiles;
+    if (want > kProbeSplitMax) want = kProbeSplitMax;
+    if (want < 1) want = 1;
+    return (int)want;
+}
+
+void launch_risk_select(prox_handle *h, int B, cudaStream_t s) {
+    risk_select_kernel<<<1, 1024, 0, s>>>(h->st, h->stamp, h->risk_pos, h->risk_slot, h->risk_stamp, B,
+                                          (long long)h->C);
+    h->launches++;
+}
+
+void launch_probe(prox_handle *h, const float *q, int B, cudaStream_t s) {
+    dim3 grid((B + PQ - 1) / PQ, probe_splits(h, B));
+    probe_kernel<<<grid, 256, 0, s>>>(h->st, h->keys, q, h->risk_pos, B, h->d, h->part_min, h->part_arg,
+                                      h->d_risk, h->d_intra);
+    h->launches++;
+}
+
+void launch_build_candidates(prox_handle *h, int B, cudaStream_t s) {
+    build_candidates_kernel<<<B, 128, 0, s>>>(h->st, B, probe_splits(h, B), (double)h->tau, h->part_min,
+                                              h->part_arg, h->d_risk, h->d_intra, h->safe_min,
+                                              h->safe_arg, h->cand_d, h->cand_code, h->n_cand);
+    h->launches++;
+}
+
+void launch_resolve(prox_handle *h, int B, uint8_t *out_hit, cudaStream_t s) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)sizeof(ResolveSmem));
+        attr_set = true;
+    }
+    resolve_kernel<<<1, 1024, sizeof(ResolveSmem), s>>>(
+        h->st, B, (long long)h->C, (double)h->tau, h->policy, h->stamp, h->risk_slot, h->risk_stamp,
+        h->safe_min, h->safe_arg, h->cand_d, h->cand_code, h->n_cand, out_hit, h->src, h->src_kind,
+        h->ins_slot, h->evt_slot, h->evt_dist, h->miss_list, h->miss_rank);
+    h->launches++;
+}
+
+void launch_gather_hits(prox_handle *h, int B, int64_t *out_ids, float *out_dists, cudaStream_t s) {
+    gather_hits_kernel<<<B, 64, 0, s>>>(B, h->k, h->src, h->src_kind, h->val_ids, h->val_dists, out_ids,
+                                        out_dists);
+    h->launches++;
+}
+
+void launch_scatter(prox_handle *h, const float *q, int B, int64_t *out_ids, float *out_dists,
+                    int with_values, cudaStream_t s) {
+    scatter_kernel<<<B, 128, 0, s>>>(B, h->d, h->k, with_values, q, h->src, h->src_kind, h->ins_slot,
+                                     h->miss_rank, h->res_ids, h->res_dists, h->keys, h->val_ids,
+                                     h->val_dists, out_ids, out_dists);
+    h->launches++;
+}
+
+void launch_probe_outputs(prox_handle *h, int B, int32_t *out_slot, float *out_min_dist, cudaStream_t s) {
+    copy_probe_outputs_kernel<<<(B + 255) / 256, 256, 0, s>>>(B, h->evt_slot, h->evt_dist, out_slot,
+                                                             out_min_dist);
+    h->launches++;
+}
+
+void launch_reset(prox_handle *h, cudaStream_t s) {
+    const long long C = h->C;
+    reset_kernel<<<(unsigned)((C + 255) / 256), 256, 0, s>>>(h->st, h->risk_pos, C, 0);
+    h->launches++;
+}
+
+void launch_cache_load(prox_handle *h, const float *keys, int64_t n, cudaStream_t s) {
+    const long long C = h->C;
+    reset_kernel<<<(unsigned)((C + 255) / 256), 256, 0, s>>>(h->st, h->risk_pos, C, (long long)n);
+    h->launches++;
+    if (n > 0) {
+        cache_load_kernel<<<(unsigned)n, 128, 0, s>>>((long long)n, h->d, h->k, keys, h->keys, h->val_ids,
+                                                      h->val_dists, h->stamp);
+        h->launches++;
+    }
+}
+
+}  // namespace prox

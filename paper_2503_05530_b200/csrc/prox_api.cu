@@ -1,0 +1,263 @@
+// C ABI of the library: argument checks, memory, and the order of the kernels of one batch.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "prox_internal.h"
+
+using namespace prox;
+
+static thread_local char g_err[256] = "";
+
+static void set_err(const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
+extern "C" const char *prox_last_error(void) { return g_err; }
+
+template <typename T>
+static bool dev_alloc(T *&p, size_t n) {
+    void *q = nullptr;
+    if (cudaMalloc(&q, n * sizeof(T)) != cudaSuccess) {
+        cudaGetLastError();
+        p = nullptr;
+        return false;
+    }
+    p = static_cast<T *>(q);
+    return true;
+}
+
+static void free_all(prox_handle *h) {
+    void *ptrs[] = {h->xb, h->xh, h->keys, h->val_ids, h->val_dists, h->stamp, h->risk_pos, h->st,
+                    h->risk_slot, h->risk_stamp, h->part_min, h->part_arg, h->d_risk, h->d_intra,
+                    h->safe_min, h->safe_arg, h->cand_d, h->cand_code, h->n_cand, h->src, h->src_kind,
+                    h->ins_slot, h->evt_slot, h->evt_dist, h->miss_list, h->miss_rank, h->qb, h->qbn,
+                    h->qerr, h->thr_g, h->buf, h->buf_cnt, h->cand_id, h->cand_score, h->cand_n,
+                    h->cand_sk, h->res_ids, h->res_dists, h->fail_list, h->fail_radius, h->coll_id,
+                    h->coll_n, h->stage_q, h->stage_ids, h->stage_dists, h->stage_hit};
+    for (void *p : ptrs)
+        if (p) cudaFree(p);
+}
+
+static int check_launch(const char *what) {
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        set_err("%s: %s", what, cudaGetErrorString(e));
+        return PROX_ERR_CUDA;
+    }
+    return PROX_OK;
+}
+
+extern "C" prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, int32_t k,
+                                    int64_t capacity, float tau, int32_t policy) {
+    g_err[0] = 0;
+    if (!corpus) { set_err("corpus is NULL"); return nullptr; }
+    if (N < 1 || N >= (1LL << 31)) { set_err("N must be in [1, 2^31)"); return nullptr; }
+    if (d < 16 || d > 4096 || d % 16) { set_err("d must be a multiple of 16 in [16, 4096]"); return nullptr; }
+    if (k < 1 || k > kMaxK || k > N) { set_err("k must be in [1, min(N, %d)]", kMaxK); return nullptr; }
+    if (capacity < 1 || capacity >= (1LL << 31)) { set_err("capacity must be in [1, 2^31)"); return nullptr; }
+    if (!(tau >= 0.f) || std::isinf(tau)) { set_err("tau must be finite and >= 0"); return nullptr; }
+    if (policy != PROX_LRU && policy != PROX_FIFO) { set_err("policy must be PROX_LRU or PROX_FIFO"); return nullptr; }
+
+    prox_handle *h = new (std::nothrow) prox_handle();
+    if (!h) { set_err("out of host memory"); return nullptr; }
+    std::memset(h, 0, sizeof(*h));
+    h->corpus = corpus; h->N = N; h->d = d; h->k = k; h->C = capacity; h->tau = tau; h->policy = policy;
+    h->kp = 4 * k < 64 ? 64 : (4 * k > kMaxKp ? kMaxKp : 4 * k);
+    h->scan_mode = PROX_SCAN_AUTO;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&h->device) != cudaSuccess ||
+        cudaGetDeviceProperties(&prop, h->device) != cudaSuccess) {
+        set_err("no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
+        delete h;
+        return nullptr;
+    }
+    if (prop.major != 10) {
+        set_err("this library is built for sm_100a (B200); found compute capability %d.%d", prop.major, prop.minor);
+        delete h;
+        return nullptr;
+    }
+    h->num_sms = prop.multiProcessorCount;
+    h->scan_ctas = h->num_sms;
+
+    const size_t MB = kMaxBatch, C = (size_t)capacity, P = (size_t)h->scan_ctas;
+    bool ok = true;
+    ok = ok && dev_alloc(h->xb, (size_t)N * d) && dev_alloc(h->xh, (size_t)N);
+    ok = ok && dev_alloc(h->keys, C * d) && dev_alloc(h->val_ids, C * k) && dev_alloc(h->val_dists, C * k);
+    ok = ok && dev_alloc(h->stamp, C) && dev_alloc(h->risk_pos, C) && dev_alloc(h->st, 1);
+    ok = ok && dev_alloc(h->risk_slot, MB) && dev_alloc(h->risk_stamp, MB);
+    ok = ok && dev_alloc(h->part_min, MB * kProbeSplitMax) && dev_alloc(h->part_arg, MB * kProbeSplitMax);
+    ok = ok && dev_alloc(h->d_risk, MB * MB) && dev_alloc(h->d_intra, MB * MB);
+    ok = ok && dev_alloc(h->safe_min, MB) && dev_alloc(h->safe_arg, MB);
+    ok = ok && dev_alloc(h->cand_d, MB * 2 * MB) && dev_alloc(h->cand_code, MB * 2 * MB) && dev_alloc(h->n_cand, MB);
+    ok = ok && dev_alloc(h->src, MB) && dev_alloc(h->src_kind, MB) && dev_alloc(h->ins_slot, MB);
+    ok = ok && dev_alloc(h->evt_slot, MB) && dev_alloc(h->evt_dist, MB);
+    ok = ok && dev_alloc(h->miss_list, MB) && dev_alloc(h->miss_rank, MB);
+    ok = ok && dev_alloc(h->qb, MB * d) && dev_alloc(h->qbn, MB) && dev_alloc(h->qerr, MB) && dev_alloc(h->thr_g, MB);
+    ok = ok && dev_alloc(h->buf, P * kScanQ * kBufCap) && dev_alloc(h->buf_cnt, P * kScanQ);
+    ok = ok && dev_alloc(h->cand_id, MB * kMaxKp) && dev_alloc(h->cand_score, MB * kMaxKp);
+    ok = ok && dev_alloc(h->cand_n, MB) && dev_alloc(h->cand_sk, MB);
+    ok = ok && dev_alloc(h->res_ids, MB * k) && dev_alloc(h->res_dists, MB * k);
+    ok = ok && dev_alloc(h->fail_list, MB) && dev_alloc(h->fail_radius, MB);
+    ok = ok && dev_alloc(h->coll_id, MB * kCollectCap) && dev_alloc(h->coll_n, MB);
+    ok = ok && dev_alloc(h->stage_q, MB * d) && dev_alloc(h->stage_ids, MB * k);
+    ok = ok && dev_alloc(h->stage_dists, MB * k) && dev_alloc(h->stage_hit, MB);
+    if (!ok) {
+        set_err("out of device memory");
+        free_all(h);
+        delete h;
+        return nullptr;
+    }
+    cudaMemset(h->st, 0, sizeof(DevState));
+    cudaMemset(h->qb, 0, MB * d * sizeof(__nv_bfloat16));
+    cudaMemset(h->buf_cnt, 0, P * kScanQ * sizeof(int32_t));
+    launch_convert_corpus(h, 0);
+    launch_reset(h, 0);
+    const cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        set_err("set-up kernels failed: %s", cudaGetErrorString(e));
+        free_all(h);
+        delete h;
+        return nullptr;
+    }
+    return h;
+}
+
+extern "C" void prox_destroy(prox_handle *h) {
+    if (!h) return;
+    cudaDeviceSynchronize();
+    free_all(h);
+    delete h;
+}
+
+static int check_batch_args(prox_handle *h, const void *queries, int32_t B) {
+    g_err[0] = 0;
+    if (!h) { set_err("handle is NULL"); return PROX_ERR_INVALID_ARG; }
+    if (!queries) { set_err("queries is NULL"); return PROX_ERR_INVALID_ARG; }
+    if (B < 1 || B > kMaxBatch) { set_err("B must be in [1, %d]", kMaxBatch); return PROX_ERR_INVALID_ARG; }
+    return PROX_OK;
+}
+
+static void enqueue_probe_and_resolve(prox_handle *h, const float *queries, int32_t B, uint8_t *out_hit,
+                                      cudaStream_t s) {
+    launch_risk_select(h, B, s);
+    launch_probe(h, queries, B, s);
+    launch_build_candidates(h, B, s);
+    launch_resolve(h, B, out_hit, s);
+}
+
+extern "C" int32_t prox_query_batch(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
+                                    float *out_dists, uint8_t *out_hit, void *stream) {
+    int rc = check_batch_args(h, queries, B);
+    if (rc) return rc;
+    if (!out_ids || !out_dists || !out_hit) { set_err("an output pointer is NULL"); return PROX_ERR_INVALID_ARG; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    enqueue_probe_and_resolve(h, queries, B, out_hit, s);
+    launch_gather_hits(h, B, out_ids, out_dists, s);
+    launch_prep_miss(h, queries, B, s);
+    const int passes = (B + kScanQ - 1) / kScanQ;
+    for (int p = 0; p < passes; ++p) {
+        if (h->scan_mode == PROX_SCAN_CUDA_CORE || launch_scan_pass_tc(h, p, s) != 0) launch_scan_pass(h, p, s);
+        launch_merge_select(h, p, B, s);
+    }
+    launch_rerank(h, queries, B, s);
+    launch_fallback(h, queries, B, s);
+    launch_scatter(h, queries, B, out_ids, out_dists, 1, s);
+    return check_launch("prox_query_batch");
+}
+
+extern "C" int32_t prox_query_batch_host(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
+                                         float *out_dists, uint8_t *out_hit, void *stream) {
+    int rc = check_batch_args(h, queries, B);
+    if (rc) return rc;
+    if (!out_ids || !out_dists || !out_hit) { set_err("an output pointer is NULL"); return PROX_ERR_INVALID_ARG; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t k = h->k;
+    if (cudaMemcpyAsync(h->stage_q, queries, (size_t)B * h->d * sizeof(float), cudaMemcpyHostToDevice, s) !=
+        cudaSuccess)
+        return check_launch("copy of the queries");
+    rc = prox_query_batch(h, h->stage_q, B, h->stage_ids, h->stage_dists, h->stage_hit, stream);
+    if (rc) return rc;
+    cudaMemcpyAsync(out_ids, h->stage_ids, (size_t)B * k * sizeof(int64_t), cudaMemcpyDeviceToHost, s);
+    cudaMemcpyAsync(out_dists, h->stage_dists, (size_t)B * k * sizeof(float), cudaMemcpyDeviceToHost, s);
+    cudaMemcpyAsync(out_hit, h->stage_hit, (size_t)B, cudaMemcpyDeviceToHost, s);
+    const cudaError_t e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) {
+        set_err("prox_query_batch_host: %s", cudaGetErrorString(e));
+        return PROX_ERR_CUDA;
+    }
+    return PROX_OK;
+}
+
+extern "C" int32_t prox_probe_batch(prox_handle *h, const float *queries, int32_t B, uint8_t *out_hit,
+                                    int32_t *out_slot, float *out_min_dist, void *stream) {
+    int rc = check_batch_args(h, queries, B);
+    if (rc) return rc;
+    if (!out_hit) { set_err("out_hit is NULL"); return PROX_ERR_INVALID_ARG; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    enqueue_probe_and_resolve(h, queries, B, out_hit, s);
+    if (out_slot || out_min_dist) launch_probe_outputs(h, B, out_slot, out_min_dist, s);
+    launch_scatter(h, queries, B, nullptr, nullptr, 0, s);
+    return check_launch("prox_probe_batch");
+}
+
+extern "C" int32_t prox_reset_cache(prox_handle *h, void *stream) {
+    g_err[0] = 0;
+    if (!h) { set_err("handle is NULL"); return PROX_ERR_INVALID_ARG; }
+    launch_reset(h, static_cast<cudaStream_t>(stream));
+    return check_launch("prox_reset_cache");
+}
+
+extern "C" int32_t prox_cache_load(prox_handle *h, const float *keys, int64_t n, void *stream) {
+    g_err[0] = 0;
+    if (!h) { set_err("handle is NULL"); return PROX_ERR_INVALID_ARG; }
+    if (n < 0 || n > h->C) { set_err("n must be in [0, capacity]"); return PROX_ERR_INVALID_ARG; }
+    if (n > 0 && !keys) { set_err("keys is NULL"); return PROX_ERR_INVALID_ARG; }
+    launch_cache_load(h, keys, n, static_cast<cudaStream_t>(stream));
+    return check_launch("prox_cache_load");
+}
+
+extern "C" int32_t prox_get_stats(prox_handle *h, prox_stats *out, void *stream) {
+    g_err[0] = 0;
+    if (!h || !out) { set_err("NULL argument"); return PROX_ERR_INVALID_ARG; }
+    DevState st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(&st, h->st, sizeof(st), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) { set_err("prox_get_stats: %s", cudaGetErrorString(e)); return PROX_ERR_CUDA; }
+    out->queries = st.queries; out->hits = st.hits; out->misses = st.misses;
+    out->intra_batch_hits = st.intra_hits; out->evictions = st.evictions;
+    out->scan_batches = st.scan_batches; out->uncertified = st.uncertified;
+    out->fallback_rows = st.fallback_rows; out->unresolved = st.unresolved; out->count = st.count;
+    return PROX_OK;
+}
+
+extern "C" int32_t prox_status(prox_handle *h, void *stream) {
+    g_err[0] = 0;
+    if (!h) { set_err("handle is NULL"); return PROX_ERR_INVALID_ARG; }
+    DevState st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(&st, h->st, sizeof(st), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) { set_err("prox_status: %s", cudaGetErrorString(e)); return PROX_ERR_CUDA; }
+    if (st.error) set_err("device-side error %d latched", st.error);
+    return st.error;
+}
+
+extern "C" int32_t prox_set_scan_mode(prox_handle *h, int32_t mode) {
+    g_err[0] = 0;
+    if (!h || (mode != PROX_SCAN_AUTO && mode != PROX_SCAN_CUDA_CORE)) {
+        set_err("bad handle or mode");
+        return PROX_ERR_INVALID_ARG;
+    }
+    h->scan_mode = mode;
+    return PROX_OK;
+}
+
+extern "C" int64_t prox_kernel_launches(const prox_handle *h) { return h ? h->launches : 0; }

@@ -1,0 +1,127 @@
+// Internal layout of a handle and the host-side launchers of every kernel.
+#pragma once
+#include <cstdint>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "../../include/prox.h"
+
+namespace prox {
+
+constexpr int kMaxK = PROX_MAX_K;            // largest k
+constexpr int kMaxKp = 256;                  // largest k' (candidates kept by the coarse scan)
+constexpr int kMaxBatch = PROX_MAX_BATCH;    // largest B
+constexpr int kScanQ = 256;                  // queries per scan pass (MMA N dimension)
+constexpr int kTileRows = 128;               // corpus rows per scan tile (MMA M dimension)
+constexpr int kBufCap = 512;                 // entries of one (CTA, query) candidate buffer
+constexpr int kCollectCap = 2048;            // rows the exact pass may collect per query
+constexpr int kProbeSplitMax = 64;           // column splits of the probe grid
+
+// Device-resident scalars of a handle.
+struct DevState {
+    long long count;          // |C|
+    long long clock;          // logical time = queries seen (plus loaded keys)
+    int n_risk;               // at-risk slots of the current batch
+    int n_miss;               // misses of the current batch
+    int n_fail;               // misses whose candidate set was not certified
+    int error;                // latched PROX_ERR_* found on the device
+    float e_max;              // upper bound of |x - bf16(x)| over corpus rows
+    float xn_max;             // upper bound of |bf16(x)| over corpus rows
+    // statistics
+    long long queries, hits, misses, intra_hits, evictions, scan_batches, uncertified,
+        fallback_rows, unresolved;
+};
+
+}  // namespace prox
+
+struct prox_handle {
+    // stored state of Algorithm 1
+    const float *corpus;      // N x d fp32, borrowed
+    int64_t N;
+    int32_t d, k, kp;
+    int64_t C;
+    float tau;
+    int32_t policy;
+    int device, num_sms;
+    int scan_mode;
+    int64_t launches;
+
+    // corpus copies for the scan
+    __nv_bfloat16 *xb;        // N x d
+    float *xh;                // N: 0.5 * |bf16(x)|^2
+
+    // key-value store
+    float *keys;              // C x d
+    int32_t *val_ids;         // C x k
+    float *val_dists;         // C x k
+    unsigned long long *stamp;  // C
+    int32_t *risk_pos;        // C: position in the at-risk list or -1
+    prox::DevState *st;
+
+    // per-batch scratch
+    int32_t *risk_slot;               // kMaxBatch
+    unsigned long long *risk_stamp;   // kMaxBatch
+    double *part_min;                 // kMaxBatch x kProbeSplitMax
+    int32_t *part_arg;                // kMaxBatch x kProbeSplitMax
+    double *d_risk;                   // kMaxBatch x kMaxBatch
+    double *d_intra;                  // kMaxBatch x kMaxBatch
+    double *safe_min;                 // kMaxBatch
+    int32_t *safe_arg;                // kMaxBatch
+    double *cand_d;                   // kMaxBatch x 2 kMaxBatch   (probe candidates <= tau)
+    int32_t *cand_code;               // kMaxBatch x 2 kMaxBatch
+    int32_t *n_cand;                  // kMaxBatch
+    int32_t *src;                     // kMaxBatch: hit source (slot, or batch index), -1 on a miss
+    int32_t *src_kind;                // kMaxBatch: 0 miss, 1 pre-batch slot, 2 batch entry
+    int32_t *ins_slot;                // kMaxBatch: slot written at batch end or -1
+    int32_t *evt_slot;                // kMaxBatch: matched / written slot at the time of the lookup
+    float *evt_dist;                  // kMaxBatch: distance to the matched key (+inf on a miss)
+    int32_t *miss_list;               // kMaxBatch
+    int32_t *miss_rank;               // kMaxBatch
+
+    __nv_bfloat16 *qb;                // kMaxBatch x d: bf16 copies of the miss queries
+    float *qbn;                       // kMaxBatch: |bf16(q)|^2
+    float *qerr;                      // kMaxBatch: upper bound of |q - bf16(q)|
+    uint32_t *thr_g;                  // kMaxBatch: shared score thresholds (ordered-uint form)
+    unsigned long long *buf;          // P x kScanQ x kBufCap candidate entries
+    int32_t *buf_cnt;                 // P x kScanQ
+    int32_t scan_ctas;                // P
+    int32_t *cand_id;                 // kMaxBatch x kMaxKp
+    float *cand_score;                // kMaxBatch x kMaxKp
+    int32_t *cand_n;                  // kMaxBatch
+    float *cand_sk;                   // kMaxBatch: k'-th best coarse score (-inf if fewer rows)
+    int32_t *res_ids;                 // kMaxBatch x k
+    double *res_dists;                // kMaxBatch x k
+    int32_t *fail_list;               // kMaxBatch
+    float *fail_radius;               // kMaxBatch: exact k-th distance among the candidates
+    int32_t *coll_id;                 // kMaxBatch x kCollectCap (indexed by position in fail_list)
+    int32_t *coll_n;                  // kMaxBatch
+
+    // staging for the host-buffer entry point
+    float *stage_q;
+    int64_t *stage_ids;
+    float *stage_dists;
+    uint8_t *stage_hit;
+};
+
+namespace prox {
+// create-time kernels
+void launch_convert_corpus(prox_handle *h, cudaStream_t s);
+// cache kernels
+void launch_risk_select(prox_handle *h, int B, cudaStream_t s);
+void launch_probe(prox_handle *h, const float *q, int B, cudaStream_t s);
+void launch_build_candidates(prox_handle *h, int B, cudaStream_t s);
+void launch_resolve(prox_handle *h, int B, uint8_t *out_hit, cudaStream_t s);
+void launch_gather_hits(prox_handle *h, int B, int64_t *out_ids, float *out_dists, cudaStream_t s);
+void launch_scatter(prox_handle *h, const float *q, int B, int64_t *out_ids, float *out_dists,
+                    int with_values, cudaStream_t s);
+void launch_probe_outputs(prox_handle *h, int B, int32_t *out_slot, float *out_min_dist, cudaStream_t s);
+void launch_cache_load(prox_handle *h, const float *keys, int64_t n, cudaStream_t s);
+void launch_reset(prox_handle *h, cudaStream_t s);
+// scan kernels
+void launch_prep_miss(prox_handle *h, const float *q, int B, cudaStream_t s);
+void launch_scan_pass(prox_handle *h, int pass, cudaStream_t s);       // CUDA-core scan
+int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s);     // tcgen05 scan; nonzero = not available
+void launch_merge_select(prox_handle *h, int pass, int B, cudaStream_t s);
+void launch_rerank(prox_handle *h, const float *q, int B, cudaStream_t s);
+void launch_fallback(prox_handle *h, const float *q, int B, cudaStream_t s);
+}  // namespace prox

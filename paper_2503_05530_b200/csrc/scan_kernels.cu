@@ -1,0 +1,549 @@
+// Miss path: exact k nearest corpus rows for the queries that missed (Algorithm 1, line 6,
+// with an exact flat index as in Section 4.2.1).
+//
+// Route to the exact answer:
+//   1. coarse scores  s(q, x) = bf16(q).bf16(x) - |bf16(x)|^2 / 2   for every corpus row, so that
+//      |bf16(q) - bf16(x)|^2 = |bf16(q)|^2 - 2 s; the k' rows with the largest s are kept per
+//      query (this file: the CUDA-core version of that scan; scan_tcgen05.cu: tensor cores);
+//   2. the k' candidates are measured exactly, sum_j (q_j - x_j)^2 in fp64 over the fp32 rows,
+//      and sorted by (distance, row id): the first k are the answer if the certificate holds;
+//   3. certificate: with a = |q - bf16(q)| and e >= |x - bf16(x)| for every row, a row outside
+//      the candidate set has coarse distance >= c' (the k'-th best), hence true distance
+//      >= (sqrt(c') - a - e)^2.  If the exact k-th candidate distance is below that bound, no
+//      outside row can belong to the top k;
+//   4. otherwise (rare) the query takes an exact fp32 pass over the whole corpus that collects
+//      every row within the k-th candidate distance (plus the fp32 rounding margin), and those
+//      rows are measured in fp64 like the candidates.
+#include <cfloat>
+#include <cmath>
+
+#include "prox_internal.h"
+#include "topk_device.cuh"
+
+namespace prox {
+
+
+// ------------------------------------------------------------------------------------------
+// Create time: bf16 copy (round to nearest even), half squared norms of the rounded rows and
+// the largest rounding error norm.  One warp per row.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+convert_corpus_kernel(const float *__restrict__ x, long long N, int d, __nv_bfloat16 *__restrict__ xb,
+                      float *__restrict__ xh, DevState *st) {
+    const int lane = threadIdx.x & 31;
+    const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+    float emax = 0.f, nmax = 0.f;
+    for (long long r = warp; r < N; r += nwarps) {
+        const float *src = x + (size_t)r * d;
+        __nv_bfloat16 *dst = xb + (size_t)r * d;
+        float nn = 0.f, ee = 0.f;
+        for (int j = lane * 4; j < d; j += 128) {
+            const float4 v = *reinterpret_cast<const float4 *>(src + j);
+            const __nv_bfloat16 b0 = __float2bfloat16_rn(v.x), b1 = __float2bfloat16_rn(v.y),
+                                b2 = __float2bfloat16_rn(v.z), b3 = __float2bfloat16_rn(v.w);
+            const float f0 = __bfloat162float(b0), f1 = __bfloat162float(b1), f2 = __bfloat162float(b2),
+                        f3 = __bfloat162float(b3);
+            nn += f0 * f0 + f1 * f1 + f2 * f2 + f3 * f3;
+            ee += (v.x - f0) * (v.x - f0) + (v.y - f1) * (v.y - f1) + (v.z - f2) * (v.z - f2) +
+                  (v.w - f3) * (v.w - f3);
+            __nv_bfloat162 p0, p1;
+            p0.x = b0; p0.y = b1; p1.x = b2; p1.y = b3;
+            *reinterpret_cast<__nv_bfloat162 *>(dst + j) = p0;
+            *reinterpret_cast<__nv_bfloat162 *>(dst + j + 2) = p1;
+        }
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1) {
+            nn += __shfl_xor_sync(0xffffffffu, nn, m);
+            ee += __shfl_xor_sync(0xffffffffu, ee, m);
+        }
+        if (lane == 0) xh[r] = 0.5f * nn;
+        emax = fmaxf(emax, ee);
+        nmax = fmaxf(nmax, nn);
+    }
+    if (lane == 0) {                                       // positive floats order as ints
+        atomicMax(reinterpret_cast<int *>(&st->e_max), __float_as_int(sqrtf(emax) * 1.0001f));
+        atomicMax(reinterpret_cast<int *>(&st->xn_max), __float_as_int(sqrtf(nmax) * 1.0001f));
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Per batch: bf16 copies of the miss queries in miss order, their norms and rounding errors;
+// resets of the per-batch scan state.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+prep_miss_kernel(DevState *st, const float *__restrict__ queries, int B, int d,
+                 const int32_t *__restrict__ miss_list, __nv_bfloat16 *qb, float *qbn, float *qerr,
+                 uint32_t *thr_g, int32_t *coll_n) {
+    __shared__ float red[2][4];
+    const int m = blockIdx.x, tid = threadIdx.x;
+    const int n_miss = st->n_miss;
+    if (m == 0) {
+        for (int i = tid; i < kMaxBatch; i += blockDim.x) {
+            thr_g[i] = f2o(-INFINITY);
+            coll_n[i] = 0;
+        }
+        if (tid == 0) {
+            st->n_fail = 0;
+            if (n_miss > 0) st->scan_batches++;
+        }
+    }
+    if (m >= n_miss) {
+        for (int j = tid; j < d; j += blockDim.x) qb[(size_t)m * d + j] = __float2bfloat16_rn(0.f);
+        return;
+    }
+    const float *src = queries + (size_t)miss_list[m] * d;
+    float nn = 0.f, ee = 0.f;
+    for (int j = tid; j < d; j += blockDim.x) {
+        const float v = src[j];
+        const __nv_bfloat16 b = __float2bfloat16_rn(v);
+        const float f = __bfloat162float(b);
+        qb[(size_t)m * d + j] = b;
+        nn += f * f;
+        ee += (v - f) * (v - f);
+    }
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) {
+        nn += __shfl_xor_sync(0xffffffffu, nn, s);
+        ee += __shfl_xor_sync(0xffffffffu, ee, s);
+    }
+    if ((tid & 31) == 0) { red[0][tid >> 5] = nn; red[1][tid >> 5] = ee; }
+    __syncthreads();
+    if (tid == 0) {
+        qbn[m] = red[0][0] + red[0][1] + red[0][2] + red[0][3];
+        qerr[m] = sqrtf(red[1][0] + red[1][1] + red[1][2] + red[1][3]) * 1.0001f;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Candidate buffers.  Each scanning block owns, per query of the pass, kBufCap entries in
+// global memory.  A score enters the buffer if it beats the query's threshold; when a
+// buffer could overflow during the next tile, a warp sorts it, keeps the best k' and raises
+// the threshold to the k'-th score.  Thresholds are shared between blocks through thr_g (a
+// block's k'-th best is a lower bound of the global k'-th best).
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void warp_compact(u64 *qbuf, int *cnt, float *thr, uint32_t *thr_g_q, int kp) {
+    const int lane = threadIdx.x & 31;
+    const int n = *cnt < kBufCap ? *cnt : kBufCap;
+    u64 v[kBufCap / 32];
+#pragma unroll
+    for (int it = 0; it < kBufCap / 32; ++it) {
+        const int e = it * 32 + lane;
+        v[it] = (e < n) ? qbuf[e] : 0ull;
+    }
+    warp_sort_desc<kBufCap / 32>(v);
+    const int keep = n < kp ? n : kp;
+    u64 kth = 0ull;
+#pragma unroll
+    for (int it = 0; it < kBufCap / 32; ++it) {
+        const int e = it * 32 + lane;
+        if (e < keep) qbuf[e] = v[it];
+        if (it == ((kp - 1) >> 5)) kth = v[it];
+    }
+    kth = __shfl_sync(0xffffffffu, kth, (kp - 1) & 31);
+    __syncwarp();
+    if (lane == 0) {
+        *cnt = keep;
+        if (n >= kp) {
+            const float s = entry_score(kth);
+            if (s > *thr) *thr = s;
+            atomicMax(thr_g_q, (uint32_t)(kth >> 32));
+        }
+    }
+}
+
+// CUDA-core scan of one pass (up to kScanQ miss queries): tile = 128 rows x 64 queries,
+// d in chunks of 32, fp32 accumulation of bf16 products.
+__global__ void __launch_bounds__(256)
+scan_cc_kernel(const DevState *__restrict__ st, const __nv_bfloat16 *__restrict__ xb,
+               const float *__restrict__ xh, const __nv_bfloat16 *__restrict__ qb, long long N, int d,
+               int pass, int kp, uint32_t *thr_g, u64 *buf, int32_t *buf_cnt) {
+    __shared__ float xs[kTileRows][33];
+    __shared__ float qs[64][33];
+    __shared__ float thr[kScanQ];
+    __shared__ int cnt[kScanQ];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4, lane = tid & 31, warp = tid >> 5;
+    const int q0 = pass * kScanQ;
+    int nq = st->n_miss - q0;
+    if (nq > kScanQ) nq = kScanQ;
+    if (nq <= 0) return;
+    thr_g += q0;
+    u64 *mybuf = buf + (size_t)blockIdx.x * kScanQ * kBufCap;
+    for (int q = tid; q < kScanQ; q += blockDim.x) { thr[q] = -INFINITY; cnt[q] = 0; }
+    __syncthreads();
+
+    const long long ntiles = (N + kTileRows - 1) / kTileRows;
+    for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const long long row0 = tile * kTileRows;
+        for (int q = tid; q < nq; q += blockDim.x) thr[q] = fmaxf(thr[q], o2f(thr_g[q]));
+        for (int qg = 0; qg < nq; qg += 64) {
+            float acc[8][4];
+#pragma unroll
+            for (int a = 0; a < 8; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+            for (int kc = 0; kc < d; kc += 32) {
+                __syncthreads();
+#pragma unroll
+                for (int it = 0; it < 16; ++it) {
+                    const int idx = it * 256 + tid, r = idx >> 5, c = idx & 31;
+                    const long long row = row0 + r;
+                    xs[r][c] = (row < N && kc + c < d) ? __bfloat162float(xb[(size_t)row * d + kc + c]) : 0.f;
+                }
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const int idx = it * 256 + tid, r = idx >> 5, c = idx & 31;
+                    const int q = qg + r;
+                    qs[r][c] = (q < nq && kc + c < d) ? __bfloat162float(qb[(size_t)(q0 + q) * d + kc + c]) : 0.f;
+                }
+                __syncthreads();
+#pragma unroll 4
+                for (int j = 0; j < 32; ++j) {
+                    float xv[8], qv[4];
+#pragma unroll
+                    for (int a = 0; a < 8; ++a) xv[a] = xs[ty + 16 * a][j];
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) qv[b] = qs[tx + 16 * b][j];
+#pragma unroll
+                    for (int a = 0; a < 8; ++a)
+#pragma unroll
+                        for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(xv[a], qv[b], acc[a][b]);
+                }
+            }
+#pragma unroll
+            for (int a = 0; a < 8; ++a) {
+                const long long row = row0 + ty + 16 * a;
+                if (row >= N) continue;
+                const float hn = xh[row];
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const int q = qg + tx + 16 * b;
+                    if (q >= nq) continue;
+                    const float s = acc[a][b] - hn;
+                    if (s > thr[q]) {
+                        const int pos = atomicAdd(&cnt[q], 1);
+                        if (pos < kBufCap) mybuf[(size_t)q * kBufCap + pos] = pack_entry(s, (int32_t)row);
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        for (int q = warp; q < nq; q += 8)
+            if (cnt[q] > kBufCap - kTileRows)
+                warp_compact(mybuf + (size_t)q * kBufCap, &cnt[q], &thr[q], &thr_g[q], kp);
+        __syncthreads();
+    }
+    for (int q = warp; q < nq; q += 8)
+        warp_compact(mybuf + (size_t)q * kBufCap, &cnt[q], &thr[q], &thr_g[q], kp);
+    __syncthreads();
+    for (int q = tid; q < nq; q += blockDim.x) buf_cnt[(size_t)blockIdx.x * kScanQ + q] = cnt[q];
+}
+
+// ------------------------------------------------------------------------------------------
+// Merge: per query, the k' best entries over all blocks' buffers (each already cut to k').
+// Radix select on the 32-bit ordered score, then a collection pass.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+merge_select_kernel(const DevState *__restrict__ st, int pass, int P, int kp, const u64 *__restrict__ buf,
+                    const int32_t *__restrict__ buf_cnt, int32_t *cand_id, float *cand_score,
+                    int32_t *cand_n, float *cand_sk) {
+    __shared__ unsigned hist[256];
+    __shared__ uint32_t s_prefix, s_mask;
+    __shared__ int s_remaining, s_total, s_gt, s_eq;
+    const int q = blockIdx.x, tid = threadIdx.x;
+    const int m = pass * kScanQ + q;
+    if (m >= st->n_miss) return;
+
+    if (tid == 0) { s_total = 0; s_gt = 0; s_eq = 0; }
+    __syncthreads();
+    int local = 0;
+    for (int p = tid; p < P; p += blockDim.x) local += buf_cnt[(size_t)p * kScanQ + q];
+    if (local) atomicAdd(&s_total, local);
+    __syncthreads();
+    const int total = s_total;
+    const int span = P * kp;                       // entry (p, e) <-> idx = p * kp + e, e < cnt[p]
+
+    uint32_t T = 0;                                // ordered score of the k'-th best (0: keep all)
+    if (total >= kp) {
+        if (tid == 0) { s_prefix = 0; s_mask = 0; s_remaining = kp; }
+        for (int dg = 3; dg >= 0; --dg) {
+            if (tid < 256) hist[tid] = 0;
+            __syncthreads();
+            const uint32_t prefix = s_prefix, mask = s_mask;
+            for (int idx = tid; idx < span; idx += blockDim.x) {
+                const int p = idx / kp, e = idx - p * kp;
+                if (e < buf_cnt[(size_t)p * kScanQ + q]) {
+                    const uint32_t o = (uint32_t)(buf[((size_t)p * kScanQ + q) * kBufCap + e] >> 32);
+                    if ((o & mask) == prefix) atomicAdd(&hist[(o >> (8 * dg)) & 255u], 1u);
+                }
+            }
+            __syncthreads();
+            if (tid == 0) {                        // walk the digits from the top: largest scores first
+                int rem = s_remaining, b = 255;
+                while (b > 0 && (int)hist[b] < rem) { rem -= (int)hist[b]; --b; }
+                s_remaining = rem;
+                s_prefix = prefix | ((uint32_t)b << (8 * dg));
+                s_mask = mask | (0xffu << (8 * dg));
+            }
+            __syncthreads();
+        }
+        T = s_prefix;
+    }
+    // entries above T all go in; entries equal to T fill what is left
+    const int keep = total < kp ? total : kp;
+    for (int idx = tid; idx < span; idx += blockDim.x) {
+        const int p = idx / kp, e = idx - p * kp;
+        if (e < buf_cnt[(size_t)p * kScanQ + q]) {
+            const u64 ent = buf[((size_t)p * kScanQ + q) * kBufCap + e];
+            const uint32_t o = (uint32_t)(ent >> 32);
+            if (o > T || total < kp) {
+                const int pos = atomicAdd(&s_gt, 1);
+                cand_id[(size_t)m * kMaxKp + pos] = entry_row(ent);
+                cand_score[(size_t)m * kMaxKp + pos] = o2f(o);
+            }
+        }
+    }
+    __syncthreads();
+    const int n_gt = s_gt;
+    if (total >= kp) {
+        for (int idx = tid; idx < span; idx += blockDim.x) {
+            const int p = idx / kp, e = idx - p * kp;
+            if (e < buf_cnt[(size_t)p * kScanQ + q]) {
+                const u64 ent = buf[((size_t)p * kScanQ + q) * kBufCap + e];
+                if ((uint32_t)(ent >> 32) == T) {
+                    const int pos = n_gt + atomicAdd(&s_eq, 1);
+                    if (pos < kp) {
+                        cand_id[(size_t)m * kMaxKp + pos] = entry_row(ent);
+                        cand_score[(size_t)m * kMaxKp + pos] = o2f(T);
+                    }
+                }
+            }
+        }
+    }
+    if (tid == 0) {
+        cand_n[m] = keep;
+        cand_sk[m] = (total >= kp) ? o2f(T) : -INFINITY;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Exact distances of a query's candidates and the final order.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ double exact_sqdist_warp(const float *__restrict__ q_sm,
+                                                    const float *__restrict__ x, int d) {
+    const int lane = threadIdx.x & 31;
+    double acc = 0.0;
+    for (int j = lane; j < d; j += 32) {
+        const double df = (double)q_sm[j] - (double)x[j];
+        acc = fma(df, df, acc);
+    }
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, m);
+    return acc;
+}
+
+constexpr int kRerankMax = kCollectCap;            // entries the sort buffers hold
+
+// mode 0: candidates of the coarse scan (+ certificate); mode 1: rows collected by the exact pass
+__global__ void __launch_bounds__(256)
+rerank_kernel(DevState *st, int mode, const float *__restrict__ corpus, const float *__restrict__ queries,
+              int d, int k, long long N, const int32_t *__restrict__ miss_list,
+              const int32_t *__restrict__ cand_id, const int32_t *__restrict__ cand_n,
+              const float *__restrict__ cand_sk, const float *__restrict__ qbn,
+              const float *__restrict__ qerr, int32_t *res_ids, double *res_dists, int32_t *fail_list,
+              float *fail_radius, const int32_t *__restrict__ coll_id, const int32_t *__restrict__ coll_n) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *sd = reinterpret_cast<double *>(smem_raw);                 // kRerankMax
+    int *sid = reinterpret_cast<int *>(sd + kRerankMax);               // kRerankMax
+    float *q_sm = reinterpret_cast<float *>(sid + kRerankMax);         // d
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    int m, n;
+    const int32_t *ids;
+    if (mode == 0) {
+        m = blockIdx.x;
+        if (m >= st->n_miss) return;
+        n = cand_n[m];
+        ids = cand_id + (size_t)m * kMaxKp;
+    } else {
+        const int f = blockIdx.x;
+        if (f >= st->n_fail) return;
+        m = fail_list[f];
+        n = coll_n[f];
+        if (n > kCollectCap) {
+            n = kCollectCap;
+            if (tid == 0) atomicAdd((u64 *)&st->unresolved, 1ull);
+        }
+        if (tid == 0) atomicAdd((u64 *)&st->fallback_rows, (u64)n);
+        ids = coll_id + (size_t)f * kCollectCap;
+    }
+    const float *q = queries + (size_t)miss_list[m] * d;
+    for (int j = tid; j < d; j += blockDim.x) q_sm[j] = q[j];
+    int n2 = 1;
+    while (n2 < n) n2 <<= 1;
+    for (int e = tid; e < n2; e += blockDim.x) { sd[e] = INFINITY; sid[e] = 0x7fffffff; }
+    __syncthreads();
+    for (int c = warp; c < n; c += 8) {
+        const int row = ids[c];
+        const double v = exact_sqdist_warp(q_sm, corpus + (size_t)row * d, d);
+        if (lane == 0) { sd[c] = v; sid[c] = row; }
+    }
+    block_sort_asc(sd, sid, n2);
+    if (n < k) {                                    // cannot happen: k <= N and the sets hold >= k rows
+        if (tid == 0) atomicCAS(&st->error, 0, PROX_ERR_INTERNAL);
+        return;
+    }
+    for (int r = tid; r < k; r += blockDim.x) {
+        res_ids[(size_t)m * k + r] = sid[r];
+        res_dists[(size_t)m * k + r] = sd[r];
+    }
+    if (mode == 0 && tid == 0) {
+        const float sk = cand_sk[m];
+        bool certified = true;
+        if ((long long)n < N) {                     // rows outside the candidate set exist
+            // coarse distance of any outside row >= |bf16 q|^2 - 2 sk, less the fp32 slack of the
+            // accumulated dot product and of the stored norms
+            const double qn = sqrt((double)qbn[m]), xn = (double)st->xn_max;
+            const double slack = 4.0 * (double)(d + 16) * 5.9604644775390625e-08 *
+                                 (2.0 * qn * xn + xn * xn + qn * qn);
+            const double cprime = (double)qbn[m] - 2.0 * (double)sk - slack;
+            const double g = (double)qerr[m] + (double)st->e_max;
+            const double root = cprime > 0.0 ? sqrt(cprime) : 0.0;
+            const double lower = root > g ? (root - g) * (root - g) : 0.0;
+            certified = sd[k - 1] < lower;
+        }
+        if (!certified) {
+            const int f = atomicAdd(&st->n_fail, 1);
+            fail_list[f] = m;
+            fail_radius[f] = (float)sd[k - 1] * (1.f + 1e-6f) + 1e-30f;   // rounded up
+            atomicAdd((u64 *)&st->uncertified, 1ull);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Exact pass for uncertified queries: every corpus row within the radius (the exact k-th
+// candidate distance) in fp32 difference form, with the fp32 rounding margin on top.
+// Eight queries per sweep of the corpus; one warp per row.
+// ------------------------------------------------------------------------------------------
+constexpr int kFallbackGroup = 8;
+
+__global__ void __launch_bounds__(256)
+fallback_collect_kernel(DevState *st, const float *__restrict__ corpus, const float *__restrict__ queries,
+                        long long N, int d, const int32_t *__restrict__ miss_list,
+                        const int32_t *__restrict__ fail_list, const float *__restrict__ fail_radius,
+                        int32_t *coll_id, int32_t *coll_n) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *q_sm = reinterpret_cast<float *>(smem_raw);                  // kFallbackGroup x d
+    __shared__ float radius[kFallbackGroup];
+    const int n_fail = st->n_fail;
+    if (n_fail == 0) return;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const long long warp = ((long long)blockIdx.x * blockDim.x + tid) >> 5;
+    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+    const float margin = (float)(d + 8) * 1.1920929e-07f;              // (d + 8) * 2^-23, relative
+
+    for (int g0 = 0; g0 < n_fail; g0 += kFallbackGroup) {
+        const int ng = (n_fail - g0 < kFallbackGroup) ? n_fail - g0 : kFallbackGroup;
+        __syncthreads();
+        for (int idx = tid; idx < kFallbackGroup * d; idx += blockDim.x) {
+            const int f = idx / d, j = idx - f * d;
+            q_sm[idx] = (f < ng) ? queries[(size_t)miss_list[fail_list[g0 + f]] * d + j] : 0.f;
+        }
+        if (tid < kFallbackGroup) radius[tid] = (tid < ng) ? fail_radius[g0 + tid] : -1.f;
+        __syncthreads();
+        for (long long r = warp; r < N; r += nwarps) {
+            const float *x = corpus + (size_t)r * d;
+            float acc[kFallbackGroup];
+#pragma unroll
+            for (int f = 0; f < kFallbackGroup; ++f) acc[f] = 0.f;
+            for (int j = lane; j < d; j += 32) {
+                const float xv = x[j];
+#pragma unroll
+                for (int f = 0; f < kFallbackGroup; ++f) {
+                    const float df = q_sm[f * d + j] - xv;
+                    acc[f] = fmaf(df, df, acc[f]);
+                }
+            }
+#pragma unroll
+            for (int f = 0; f < kFallbackGroup; ++f)
+#pragma unroll
+                for (int s = 16; s > 0; s >>= 1) acc[f] += __shfl_xor_sync(0xffffffffu, acc[f], s);
+            if (lane < ng) {
+                float mine = 0.f;
+#pragma unroll
+                for (int f = 0; f < kFallbackGroup; ++f)
+                    if (f == lane) mine = acc[f];
+                const float rad = radius[lane];
+                if (mine <= rad * (1.f + margin) + 1e-30f) {
+                    const int pos = atomicAdd(&coll_n[g0 + lane], 1);
+                    if (pos < kCollectCap) coll_id[(size_t)(g0 + lane) * kCollectCap + pos] = (int32_t)r;
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Launchers
+// ------------------------------------------------------------------------------------------
+void launch_convert_corpus(prox_handle *h, cudaStream_t s) {
+    convert_corpus_kernel<<<h->num_sms * 8, 256, 0, s>>>(h->corpus, (long long)h->N, h->d, h->xb, h->xh,
+                                                         h->st);
+    h->launches++;
+}
+
+void launch_prep_miss(prox_handle *h, const float *q, int B, cudaStream_t s) {
+    int rows = ((B + kScanQ - 1) / kScanQ) * kScanQ;      // zero the padding rows of the last pass too
+    if (rows > kMaxBatch) rows = kMaxBatch;
+    prep_miss_kernel<<<rows, 128, 0, s>>>(h->st, q, B, h->d, h->miss_list, h->qb, h->qbn, h->qerr, h->thr_g,
+                                          h->coll_n);
+    h->launches++;
+}
+
+void launch_scan_pass(prox_handle *h, int pass, cudaStream_t s) {
+    scan_cc_kernel<<<h->scan_ctas, 256, 0, s>>>(h->st, h->xb, h->xh, h->qb, (long long)h->N, h->d, pass,
+                                                h->kp, h->thr_g, h->buf, h->buf_cnt);
+    h->launches++;
+}
+
+void launch_merge_select(prox_handle *h, int pass, int B, cudaStream_t s) {
+    int nq = B - pass * kScanQ;
+    if (nq > kScanQ) nq = kScanQ;
+    if (nq <= 0) return;
+    merge_select_kernel<<<nq, 1024, 0, s>>>(h->st, pass, h->scan_ctas, h->kp, h->buf, h->buf_cnt, h->cand_id,
+                                            h->cand_score, h->cand_n, h->cand_sk);
+    h->launches++;
+}
+
+static size_t rerank_smem(int d) { return (size_t)kRerankMax * 12 + (size_t)d * 4; }
+
+void launch_rerank(prox_handle *h, const float *q, int B, cudaStream_t s) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(rerank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)rerank_smem(4096));
+        cudaFuncSetAttribute(fallback_collect_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kFallbackGroup * 4096 * 4);
+        attr_set = true;
+    }
+    rerank_kernel<<<B, 256, rerank_smem(h->d), s>>>(h->st, 0, h->corpus, q, h->d, h->k, (long long)h->N,
+                                                    h->miss_list, h->cand_id, h->cand_n, h->cand_sk, h->qbn,
+                                                    h->qerr, h->res_ids, h->res_dists, h->fail_list,
+                                                    h->fail_radius, h->coll_id, h->coll_n);
+    h->launches++;
+}
+
+void launch_fallback(prox_handle *h, const float *q, int B, cudaStream_t s) {
+    fallback_collect_kernel<<<h->num_sms * 4, 256, (size_t)kFallbackGroup * h->d * 4, s>>>(
+        h->st, h->corpus, q, (long long)h->N, h->d, h->miss_list, h->fail_list, h->fail_radius, h->coll_id,
+        h->coll_n);
+    h->launches++;
+    rerank_kernel<<<B, 256, rerank_smem(h->d), s>>>(h->st, 1, h->corpus, q, h->d, h->k, (long long)h->N,
+                                                    h->miss_list, h->cand_id, h->cand_n, h->cand_sk, h->qbn,
+                                                    h->qerr, h->res_ids, h->res_dists, h->fail_list,
+                                                    h->fail_radius, h->coll_id, h->coll_n);
+    h->launches++;
+}
+
+}  // namespace prox

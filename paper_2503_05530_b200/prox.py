@@ -1,0 +1,188 @@
+"""ctypes binding of the CUDA library (``libprox.so``): argument marshalling only.
+
+Every step of a lookup runs in the library's kernels; this module converts
+tensors to pointers and sizes.  It raises if the library has not been built:
+there is no CPU path.  PyTorch is used for device memory and streams.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libprox.so")
+
+LRU, FIFO = 0, 1
+OK, ERR_INVALID_ARG, ERR_OOM, ERR_CUDA, ERR_UNSUPPORTED, ERR_TIMEOUT, ERR_INTERNAL = range(7)
+MAX_K, MAX_BATCH = 64, 1024
+SCAN_AUTO, SCAN_CUDA_CORE = 0, 1
+_POLICY = {"lru": LRU, "fifo": FIFO, LRU: LRU, FIFO: FIFO}
+
+
+class ProxError(RuntimeError):
+    pass
+
+
+class Stats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("queries", "hits", "misses", "intra_batch_hits", "evictions",
+                                          "scan_batches", "uncertified", "fallback_rows", "unresolved",
+                                          "count")]
+
+    def as_dict(self) -> dict:
+        return {n: int(getattr(self, n)) for n, _ in self._fields_}
+
+
+_lib = None
+
+
+def load_library():
+    """dlopen the CUDA library; fails loudly if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ProxError(f"{LIB_PATH} is not built: run `python -c 'import __graft_entry__ as g; g.build()'` "
+                        "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, i32, i64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
+    L.prox_create.restype = vp
+    L.prox_create.argtypes = [vp, i64, i32, i32, i64, f32, i32]
+    L.prox_query_batch.restype = i32
+    L.prox_query_batch.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    L.prox_query_batch_host.restype = i32
+    L.prox_query_batch_host.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    L.prox_reset_cache.restype = i32
+    L.prox_reset_cache.argtypes = [vp, vp]
+    L.prox_destroy.restype = None
+    L.prox_destroy.argtypes = [vp]
+    L.prox_last_error.restype = C.c_char_p
+    L.prox_cache_load.restype = i32
+    L.prox_cache_load.argtypes = [vp, vp, i64, vp]
+    L.prox_probe_batch.restype = i32
+    L.prox_probe_batch.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    L.prox_get_stats.restype = i32
+    L.prox_get_stats.argtypes = [vp, C.POINTER(Stats), vp]
+    L.prox_status.restype = i32
+    L.prox_status.argtypes = [vp, vp]
+    L.prox_set_scan_mode.restype = i32
+    L.prox_set_scan_mode.argtypes = [vp, i32]
+    L.prox_kernel_launches.restype = i64
+    L.prox_kernel_launches.argtypes = [vp]
+    _lib = L
+    return L
+
+
+def last_error() -> str:
+    return load_library().prox_last_error().decode()
+
+
+def _check(rc: int):
+    if rc != OK:
+        raise ProxError(f"prox error {rc}: {last_error()}")
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dev_f32(t: torch.Tensor, what: str) -> torch.Tensor:
+    if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and t.dim() == 2):
+        raise ProxError(f"{what} must be a contiguous 2-d float32 CUDA tensor")
+    return t
+
+
+class Prox:
+    """prox_create / prox_query_batch / prox_reset_cache / prox_destroy with tensors."""
+
+    def __init__(self, corpus: torch.Tensor, k: int, capacity: int, tau: float, policy="lru"):
+        self._lib = load_library()
+        self._corpus = _dev_f32(corpus, "corpus")      # borrowed by the library: keep it alive
+        self.N, self.d = corpus.shape
+        self.k, self.capacity, self.tau = int(k), int(capacity), float(tau)
+        self.policy = _POLICY[policy]
+        with torch.cuda.device(corpus.device):
+            self._h = self._lib.prox_create(corpus.data_ptr(), self.N, self.d, self.k, self.capacity,
+                                            self.tau, self.policy)
+        if not self._h:
+            raise ProxError(f"prox_create failed: {last_error()}")
+        self.device = corpus.device
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.prox_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
+
+    def query_batch(self, queries: torch.Tensor, out_ids=None, out_dists=None, out_hit=None, stream=None):
+        q = _dev_f32(queries, "queries")
+        B = q.shape[0]
+        if q.shape[1] != self.d:
+            raise ProxError("queries have the wrong dimension")
+        if out_ids is None:
+            out_ids = torch.empty(B, self.k, dtype=torch.int64, device=self.device)
+        if out_dists is None:
+            out_dists = torch.empty(B, self.k, dtype=torch.float32, device=self.device)
+        if out_hit is None:
+            out_hit = torch.empty(B, dtype=torch.uint8, device=self.device)
+        _check(self._lib.prox_query_batch(self._h, q.data_ptr(), B, out_ids.data_ptr(), out_dists.data_ptr(),
+                                          out_hit.data_ptr(), _stream_ptr(stream)))
+        return out_ids, out_dists, out_hit
+
+    def query_batch_host(self, queries: torch.Tensor, out_ids: torch.Tensor, out_dists: torch.Tensor,
+                         out_hit: torch.Tensor, stream=None):
+        """Host tensors in and out (pinned for speed); synchronises the stream."""
+        B = queries.shape[0]
+        for t in (queries, out_ids, out_dists, out_hit):
+            if t.is_cuda or not t.is_contiguous():
+                raise ProxError("query_batch_host takes contiguous host tensors")
+        _check(self._lib.prox_query_batch_host(self._h, queries.data_ptr(), B, out_ids.data_ptr(),
+                                               out_dists.data_ptr(), out_hit.data_ptr(), _stream_ptr(stream)))
+        return out_ids, out_dists, out_hit
+
+    def probe_batch(self, queries: torch.Tensor, stream=None):
+        q = _dev_f32(queries, "queries")
+        B = q.shape[0]
+        hit = torch.empty(B, dtype=torch.uint8, device=self.device)
+        slot = torch.empty(B, dtype=torch.int32, device=self.device)
+        dist = torch.empty(B, dtype=torch.float32, device=self.device)
+        _check(self._lib.prox_probe_batch(self._h, q.data_ptr(), B, hit.data_ptr(), slot.data_ptr(),
+                                          dist.data_ptr(), _stream_ptr(stream)))
+        return hit, slot, dist
+
+    def cache_load(self, keys: torch.Tensor, stream=None):
+        kk = _dev_f32(keys, "keys")
+        if kk.shape[1] != self.d:
+            raise ProxError("keys have the wrong dimension")
+        _check(self._lib.prox_cache_load(self._h, kk.data_ptr(), kk.shape[0], _stream_ptr(stream)))
+
+    def reset_cache(self, stream=None):
+        _check(self._lib.prox_reset_cache(self._h, _stream_ptr(stream)))
+
+    def stats(self, stream=None) -> dict:
+        st = Stats()
+        _check(self._lib.prox_get_stats(self._h, C.byref(st), _stream_ptr(stream)))
+        return st.as_dict()
+
+    def status(self, stream=None) -> int:
+        return int(self._lib.prox_status(self._h, _stream_ptr(stream)))
+
+    def set_scan_mode(self, mode: int):
+        _check(self._lib.prox_set_scan_mode(self._h, mode))
+
+    def kernel_launches(self) -> int:
+        return int(self._lib.prox_kernel_launches(self._h))

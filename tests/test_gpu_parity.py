@@ -1,0 +1,204 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 oracle on the same
+seeded bytes, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2503_05530_b200 import prox, workloads as W
+from golden_traces import all_traces
+from parity import compare, run_gpu, run_oracle
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def stream(N, d, comps, nq, topics, s, sigma, seed=0):
+    X = W.make_corpus(N, d, comps, seed)
+    Q, _, _ = W.make_query_stream(X, nq, topics, s, sigma, seed)
+    return X, Q
+
+
+def check(X, Q, k, cap, tau, policy, batch, **kw):
+    gpu = run_gpu(X.to(DEV), Q.to(DEV), k, cap, tau, policy, batch, **kw)
+    return compare(X.numpy(), Q.numpy(), k, cap, tau, policy, gpu), gpu
+
+
+# ------------------------------------------------------------------ hand-traced sequences
+@pytest.mark.parametrize("tr", all_traces(), ids=lambda t: t["name"])
+@pytest.mark.parametrize("batch", [1, 3, 64])
+def test_golden_traces_on_gpu(tr, batch):
+    X, Q = torch.from_numpy(tr["corpus"]), torch.from_numpy(tr["queries"])
+    ids, dists, hit, stats = run_gpu(X.to(DEV), Q.to(DEV), tr["k"], tr["capacity"], tr["tau"], tr["policy"], batch)
+    assert np.array_equal(hit, tr["hit"])
+    assert np.array_equal(ids, tr["ids"])
+    assert stats["evictions"] == int((tr["evicted"] >= 0).sum())
+
+
+def test_golden_trace_slots_via_probe():
+    for tr in all_traces():
+        X = torch.from_numpy(tr["corpus"]).to(DEV)
+        p = prox.Prox(X, tr["k"], tr["capacity"], tr["tau"], tr["policy"])
+        hit, slot, dist = p.probe_batch(torch.from_numpy(tr["queries"]).to(DEV))
+        torch.cuda.synchronize()
+        assert np.array_equal(hit.cpu().numpy(), tr["hit"]) and np.array_equal(slot.cpu().numpy(), tr["slot"])
+        p.close()
+
+
+# ------------------------------------------------------------------ the small sequential configuration
+def test_tiny_sequential_config():
+    c = W.CONFIGS["tiny"]
+    X, Q, _, _ = W.build_workload(c, seed=0)
+    res, _ = check(X, Q, c.k, c.capacity, c.taus[0], c.policy, c.batch)
+    assert 0.0 < res["hit_rate"] < 1.0
+
+
+# ------------------------------------------------------------------ batching must be unobservable
+@pytest.mark.parametrize("policy", ["lru", "fifo"])
+def test_batch_size_is_unobservable(policy):
+    X, Q = stream(5003, 128, 16, 700, 60, 1.1, 0.02, seed=3)
+    outs = []
+    for batch in [1, 7, 64, 256, 1024]:
+        res, gpu = check(X, Q, 10, 50, 0.5, policy, batch)
+        outs.append(gpu)
+    for g in outs[1:]:
+        assert np.array_equal(g[0], outs[0][0]) and np.array_equal(g[2], outs[0][2])
+        assert np.array_equal(g[1], outs[0][1])
+    assert 0.05 < res["hit_rate"] < 0.99
+
+
+# ------------------------------------------------------------------ tau sweep on a cut-down 1M-style stream
+@pytest.mark.parametrize("tau", [0.0, 0.25, 0.5, 1.0, 2.0])
+def test_tau_sweep_lru_batch64(tau):
+    X, Q = stream(20011, 768, 32, 2500, 300, 1.1, 0.02, seed=1)
+    res, gpu = check(X, Q, 10, 100, tau, "lru", 64)
+    if tau == 0.0:
+        assert res["hit_rate"] == 0.0
+        ids, dists = oracle.exact_topk(X.numpy(), Q.numpy()[:50], 10)
+        assert np.array_equal(gpu[0][:50], ids)              # tau = 0: plain kNN
+    if tau == 2.0:
+        assert res["hit_rate"] > 0.9
+
+
+def test_k32_batch256_lru():
+    X, Q = stream(30001, 768, 24, 1500, 200, 1.0, 0.03, seed=2)
+    res, _ = check(X, Q, 32, 300, 1.0, "lru", 256)
+    assert 0.0 < res["hit_rate"] < 1.0
+
+
+def test_d128_batch1024_fifo_ragged_tail():
+    X, Q = stream(50007, 128, 64, 2500, 700, 0.6, 0.05, seed=4)
+    check(X, Q, 10, 500, 0.3, "fifo", 1024)
+
+
+# ------------------------------------------------------------------ degenerate cases
+def test_exact_duplicates_hit_at_tau_zero_in_and_across_batches():
+    X, Q = stream(3000, 64, 8, 200, 200, 0.0, 0.05, seed=5)
+    Q = Q.clone()
+    Q[10] = Q[3]            # same batch (B = 64)
+    Q[130] = Q[100]         # across batches
+    Q[131] = Q[100]
+    res, gpu = check(X, Q, 5, 150, 0.0, "lru", 64)
+    hit = gpu[2]
+    assert hit.sum() == 3 and hit[10] == 1 and hit[130] == 1 and hit[131] == 1
+    assert np.array_equal(gpu[0][10], gpu[0][3]) and np.array_equal(gpu[0][131], gpu[0][100])
+
+
+def test_huge_tau_everything_hits_the_first_key():
+    X, Q = stream(2000, 64, 8, 300, 50, 1.0, 0.05, seed=6)
+    res, gpu = check(X, Q, 8, 20, 4.5, "fifo", 128)
+    assert gpu[2][0] == 0 and gpu[2][1:].all() and (gpu[0] == gpu[0][0]).all()
+    assert gpu[3]["count"] == 1
+
+
+@pytest.mark.parametrize("policy", ["lru", "fifo"])
+@pytest.mark.parametrize("cap", [1, 5])
+def test_capacity_smaller_than_batch(policy, cap):
+    X, Q = stream(4000, 64, 8, 600, 40, 1.1, 0.03, seed=7)
+    res, gpu = check(X, Q, 4, cap, 0.35, policy, 64)
+    assert gpu[3]["evictions"] > 64 and 0.0 < res["hit_rate"] < 1.0
+
+
+def test_corpus_smaller_than_candidate_count():
+    for N, k in [(10, 10), (37, 5), (64, 64), (129, 3)]:
+        X, Q = stream(N, 16, 2, 40, 10, 1.0, 0.05, seed=N)
+        check(X, Q, k, 8, 0.01, "lru", 16)
+
+
+def test_uncertified_queries_take_the_exact_pass():
+    # rows packed so tightly around one point that the bf16 scores cannot separate them
+    g = torch.Generator().manual_seed(11)
+    c = torch.randn(256, generator=g)
+    X = c + 2e-4 * torch.randn(6000, 256, generator=g)
+    X = X / X.norm(dim=1, keepdim=True)
+    Q = X[:40] + 1e-4 * torch.randn(40, 256, generator=g)
+    Q = (Q / Q.norm(dim=1, keepdim=True)).contiguous()
+    X = X.contiguous()
+    gpu = run_gpu(X.to(DEV), Q.to(DEV), 10, 16, 0.0, "lru", 8)
+    assert gpu[3]["uncertified"] > 0 and gpu[3]["unresolved"] == 0
+    ids, dists = oracle.exact_topk(X.numpy(), Q.numpy(), 10)
+    assert np.array_equal(gpu[0], ids)
+    assert np.allclose(gpu[1], dists, rtol=1e-4, atol=1e-12)
+
+
+# ------------------------------------------------------------------ probe only, pre-filled cache
+@pytest.mark.parametrize("policy", ["lru", "fifo"])
+def test_probe_only_prefilled_cache(policy):
+    keys, centres = W.make_probe_keys(3000, 768, 64, seed=8)
+    p = prox.Prox(keys[:64].contiguous().to(DEV), 1, 3000, 0.5, policy)
+    p.cache_load(keys.to(DEV))
+    o = oracle.Oracle(None, 768, 1, 3000, float(np.float32(0.5)), oracle.LRU if policy == "lru" else oracle.FIFO)
+    o.cache_load(keys.numpy())
+    for b in range(3):
+        Q = W.make_probe_batch(keys, centres, 1024, 0.02, 8, b)
+        hit, slot, dist = p.probe_batch(Q.to(DEV))
+        torch.cuda.synchronize()
+        r = o.query(Q.numpy())
+        assert np.array_equal(hit.cpu().numpy(), r["hit"])
+        assert np.array_equal(slot.cpu().numpy(), r["slot"])
+        h = r["hit"] == 1
+        assert np.allclose(dist.cpu().numpy()[h], r["best"][h], rtol=1e-6)
+        assert 0.3 < r["hit"].mean() < 0.9
+    assert p.status() == prox.OK
+    p.close()
+
+
+# ------------------------------------------------------------------ API behaviour
+def test_host_buffer_entry_point_equals_device_entry_point():
+    X, Q = stream(6001, 128, 8, 300, 40, 1.1, 0.02, seed=9)
+    a = run_gpu(X.to(DEV), Q.to(DEV), 10, 30, 0.5, "lru", 64)
+    b = run_gpu(X.to(DEV), Q.to(DEV), 10, 30, 0.5, "lru", 64, host_api=True)
+    for x, y in zip(a[:3], b[:3]):
+        assert np.array_equal(x, y)
+
+
+def test_cuda_core_scan_equals_default_scan():
+    X, Q = stream(9001, 768, 8, 200, 40, 1.1, 0.02, seed=10)
+    a = run_gpu(X.to(DEV), Q.to(DEV), 10, 30, 0.25, "lru", 64)
+    b = run_gpu(X.to(DEV), Q.to(DEV), 10, 30, 0.25, "lru", 64, scan_mode=prox.SCAN_CUDA_CORE)
+    for x, y in zip(a[:3], b[:3]):
+        assert np.array_equal(x, y)
+
+
+def test_reset_cache_and_argument_checks():
+    X, Q = stream(2000, 64, 4, 128, 20, 1.0, 0.02, seed=12)
+    Xd, Qd = X.to(DEV), Q.to(DEV)
+    p = prox.Prox(Xd, 5, 32, 0.5, "lru")
+    a = [t.clone() for t in p.query_batch(Qd)]
+    p.reset_cache()
+    b = p.query_batch(Qd)
+    torch.cuda.synchronize()
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+    assert p.stats()["queries"] == 128
+    lib = prox.load_library()
+    assert lib.prox_query_batch(p._h, Qd.data_ptr(), 0, b[0].data_ptr(), b[1].data_ptr(), b[2].data_ptr(), None) == prox.ERR_INVALID_ARG
+    assert lib.prox_query_batch(p._h, Qd.data_ptr(), 1025, b[0].data_ptr(), b[1].data_ptr(), b[2].data_ptr(), None) == prox.ERR_INVALID_ARG
+    assert lib.prox_query_batch(p._h, None, 4, b[0].data_ptr(), b[1].data_ptr(), b[2].data_ptr(), None) == prox.ERR_INVALID_ARG
+    p.close()
+    for bad in [dict(k=0), dict(k=65), dict(capacity=0), dict(tau=-1.0), dict(tau=float("nan")), dict(policy=2)]:
+        args = dict(k=5, capacity=8, tau=0.5, policy=0)
+        args.update(bad)
+        assert not lib.prox_create(Xd.data_ptr(), 2000, 64, args["k"], args["capacity"], args["tau"], args["policy"])
+        assert prox.last_error() != ""
+    assert not lib.prox_create(Xd.data_ptr(), 2000, 60, 5, 8, 0.5, 0)      # d not a multiple of 16
