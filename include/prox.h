@@ -121,8 +121,7 @@ int32_t prox_cache_load(prox_handle *h, const float *keys, int64_t n, void *stre
  * place of the database call.
  *   out_hit      DEVICE, B bytes.
  *   out_slot     DEVICE, B int32: the matched slot on a hit, the written slot on a miss.
- *   out_min_dist DEVICE, B fp32: distance to the nearest key at the time of the lookup
- *                (+inf when the cache was empty).
+ *   out_min_dist DEVICE, B fp32: on a hit the distance to the matched (nearest) key, on a miss +inf.
  */
 int32_t prox_probe_batch(prox_handle *h, const float *queries, int32_t B, uint8_t *out_hit,
                          int32_t *out_slot, float *out_min_dist, void *stream);
@@ -149,6 +148,28 @@ int32_t prox_set_scan_mode(prox_handle *h, int32_t mode);
 
 /* prox_kernel_launches -- kernels launched by this handle so far (host-side count). */
 int64_t prox_kernel_launches(const prox_handle *h);
+
+/* Stages of one batch, in launch order (indices of the arrays of prox_profile_read). */
+enum {
+    PROX_STAGE_RISK_SELECT = 0, PROX_STAGE_PROBE = 1, PROX_STAGE_CANDIDATES = 2, PROX_STAGE_RESOLVE = 3,
+    PROX_STAGE_GATHER = 4, PROX_STAGE_PREP_MISS = 5, PROX_STAGE_SCAN = 6, PROX_STAGE_MERGE = 7,
+    PROX_STAGE_RERANK = 8, PROX_STAGE_EXACT_PASS = 9, PROX_STAGE_SCATTER = 10, PROX_N_STAGES = 11
+};
+
+/*
+ * prox_profile -- stage_mask bit s set: record a pair of CUDA events on the caller's stream
+ * around every launch of stage s from now on (0 switches recording off and drops what was
+ * recorded).  For measurement only: each pair costs about a microsecond of stream time.
+ */
+int32_t prox_profile(prox_handle *h, uint32_t stage_mask);
+
+/*
+ * prox_profile_read -- synchronises the stream, adds up the recorded intervals per stage into
+ * ms_by_stage[PROX_N_STAGES] and their number into launches_by_stage[PROX_N_STAGES] (both HOST),
+ * and clears the records.  A stage launched for a batch without misses still counts: its
+ * kernels return at once.
+ */
+int32_t prox_profile_read(prox_handle *h, double *ms_by_stage, int64_t *launches_by_stage, void *stream);
 
 #ifdef __cplusplus
 }

@@ -4,12 +4,53 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "prox_internal.h"
 
 using namespace prox;
 
 static thread_local char g_err[256] = "";
+
+namespace prox {
+// Event pairs recorded around stage launches while prox_profile is on.
+struct Profiler {
+    struct Rec { cudaEvent_t a, b; int stage; };
+    uint32_t mask = 0;
+    std::vector<Rec> recs;      // used records
+    std::vector<Rec> pool;      // events ready for reuse
+    bool open_rec = false;
+    void begin(int stage, cudaStream_t s) {
+        if (!(mask >> stage & 1u)) return;
+        Rec r;
+        if (!pool.empty()) { r = pool.back(); pool.pop_back(); }
+        else if (cudaEventCreate(&r.a) != cudaSuccess || cudaEventCreate(&r.b) != cudaSuccess) return;
+        r.stage = stage;
+        cudaEventRecord(r.a, s);
+        recs.push_back(r);
+        open_rec = true;
+    }
+    void end(cudaStream_t s) {
+        if (open_rec) cudaEventRecord(recs.back().b, s);
+        open_rec = false;
+    }
+    void drop() {
+        for (auto &r : recs) pool.push_back(r);
+        recs.clear();
+    }
+    ~Profiler() {
+        drop();
+        for (auto &r : pool) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    }
+};
+}  // namespace prox
+
+struct StageScope {
+    Profiler *p;
+    cudaStream_t s;
+    StageScope(prox_handle *h, int stage, cudaStream_t st) : p(h->prof), s(st) { if (p) p->begin(stage, s); }
+    ~StageScope() { if (p) p->end(s); }
+};
 
 static void set_err(const char *fmt, ...) {
     va_list ap;
@@ -131,6 +172,8 @@ extern "C" prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, i
 extern "C" void prox_destroy(prox_handle *h) {
     if (!h) return;
     cudaDeviceSynchronize();
+    delete h->prof;
+    free_scan_tc(h);
     free_all(h);
     delete h;
 }
@@ -145,10 +188,10 @@ static int check_batch_args(prox_handle *h, const void *queries, int32_t B) {
 
 static void enqueue_probe_and_resolve(prox_handle *h, const float *queries, int32_t B, uint8_t *out_hit,
                                       cudaStream_t s) {
-    launch_risk_select(h, B, s);
-    launch_probe(h, queries, B, s);
-    launch_build_candidates(h, B, s);
-    launch_resolve(h, B, out_hit, s);
+    { StageScope t(h, PROX_STAGE_RISK_SELECT, s); launch_risk_select(h, B, s); }
+    { StageScope t(h, PROX_STAGE_PROBE, s); launch_probe(h, queries, B, s); }
+    { StageScope t(h, PROX_STAGE_CANDIDATES, s); launch_build_candidates(h, B, s); }
+    { StageScope t(h, PROX_STAGE_RESOLVE, s); launch_resolve(h, B, out_hit, s); }
 }
 
 extern "C" int32_t prox_query_batch(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
@@ -159,16 +202,19 @@ extern "C" int32_t prox_query_batch(prox_handle *h, const float *queries, int32_
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
     enqueue_probe_and_resolve(h, queries, B, out_hit, s);
-    launch_gather_hits(h, B, out_ids, out_dists, s);
-    launch_prep_miss(h, queries, B, s);
+    { StageScope t(h, PROX_STAGE_GATHER, s); launch_gather_hits(h, B, out_ids, out_dists, s); }
+    { StageScope t(h, PROX_STAGE_PREP_MISS, s); launch_prep_miss(h, queries, B, s); }
     const int passes = (B + kScanQ - 1) / kScanQ;
     for (int p = 0; p < passes; ++p) {
-        if (h->scan_mode == PROX_SCAN_CUDA_CORE || launch_scan_pass_tc(h, p, s) != 0) launch_scan_pass(h, p, s);
-        launch_merge_select(h, p, B, s);
+        {
+            StageScope t(h, PROX_STAGE_SCAN, s);
+            if (h->scan_mode == PROX_SCAN_CUDA_CORE || launch_scan_pass_tc(h, p, s) != 0) launch_scan_pass(h, p, s);
+        }
+        { StageScope t(h, PROX_STAGE_MERGE, s); launch_merge_select(h, p, B, s); }
     }
-    launch_rerank(h, queries, B, s);
-    launch_fallback(h, queries, B, s);
-    launch_scatter(h, queries, B, out_ids, out_dists, 1, s);
+    { StageScope t(h, PROX_STAGE_RERANK, s); launch_rerank(h, queries, B, s); }
+    { StageScope t(h, PROX_STAGE_EXACT_PASS, s); launch_fallback(h, queries, B, s); }
+    { StageScope t(h, PROX_STAGE_SCATTER, s); launch_scatter(h, queries, B, out_ids, out_dists, 1, s); }
     return check_launch("prox_query_batch");
 }
 
@@ -203,7 +249,7 @@ extern "C" int32_t prox_probe_batch(prox_handle *h, const float *queries, int32_
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     enqueue_probe_and_resolve(h, queries, B, out_hit, s);
     if (out_slot || out_min_dist) launch_probe_outputs(h, B, out_slot, out_min_dist, s);
-    launch_scatter(h, queries, B, nullptr, nullptr, 0, s);
+    { StageScope t(h, PROX_STAGE_SCATTER, s); launch_scatter(h, queries, B, nullptr, nullptr, 0, s); }
     return check_launch("prox_probe_batch");
 }
 
@@ -261,3 +307,38 @@ extern "C" int32_t prox_set_scan_mode(prox_handle *h, int32_t mode) {
 }
 
 extern "C" int64_t prox_kernel_launches(const prox_handle *h) { return h ? h->launches : 0; }
+
+extern "C" int32_t prox_profile(prox_handle *h, uint32_t stage_mask) {
+    g_err[0] = 0;
+    if (!h) { set_err("handle is NULL"); return PROX_ERR_INVALID_ARG; }
+    if (stage_mask == 0) {
+        delete h->prof;
+        h->prof = nullptr;
+        return PROX_OK;
+    }
+    if (!h->prof) h->prof = new (std::nothrow) Profiler();
+    if (!h->prof) { set_err("out of host memory"); return PROX_ERR_OOM; }
+    h->prof->mask = stage_mask;
+    return PROX_OK;
+}
+
+extern "C" int32_t prox_profile_read(prox_handle *h, double *ms_by_stage, int64_t *launches_by_stage,
+                                     void *stream) {
+    g_err[0] = 0;
+    if (!h || !ms_by_stage || !launches_by_stage) { set_err("NULL argument"); return PROX_ERR_INVALID_ARG; }
+    for (int i = 0; i < PROX_N_STAGES; ++i) { ms_by_stage[i] = 0.0; launches_by_stage[i] = 0; }
+    const cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { set_err("prox_profile_read: %s", cudaGetErrorString(e)); return PROX_ERR_CUDA; }
+    if (!h->prof) return PROX_OK;
+    for (auto &r : h->prof->recs) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) {
+            ms_by_stage[r.stage] += ms;
+            launches_by_stage[r.stage] += 1;
+        } else {
+            cudaGetLastError();
+        }
+    }
+    h->prof->drop();
+    return PROX_OK;
+}

@@ -32,6 +32,8 @@ struct DevState {
         fallback_rows, unresolved;
 };
 
+struct Profiler;
+
 }  // namespace prox
 
 struct prox_handle {
@@ -45,6 +47,8 @@ struct prox_handle {
     int device, num_sms;
     int scan_mode;
     int64_t launches;
+    prox::Profiler *prof;     // event records of prox_profile (NULL when off)
+    void *tc_state;           // tensor maps of the tensor-core scan (made on first use)
 
     // corpus copies for the scan
     __nv_bfloat16 *xb;        // N x d
@@ -121,6 +125,7 @@ void launch_reset(prox_handle *h, cudaStream_t s);
 void launch_prep_miss(prox_handle *h, const float *q, int B, cudaStream_t s);
 void launch_scan_pass(prox_handle *h, int pass, cudaStream_t s);       // CUDA-core scan
 int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s);     // tcgen05 scan; nonzero = not available
+void free_scan_tc(prox_handle *h);
 void launch_merge_select(prox_handle *h, int pass, int B, cudaStream_t s);
 void launch_rerank(prox_handle *h, const float *q, int B, cudaStream_t s);
 void launch_fallback(prox_handle *h, const float *q, int B, cudaStream_t s);

@@ -122,36 +122,6 @@ prep_miss_kernel(DevState *st, const float *__restrict__ queries, int B, int d,
 // the threshold to the k'-th score.  Thresholds are shared between blocks through thr_g (a
 // block's k'-th best is a lower bound of the global k'-th best).
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ void warp_compact(u64 *qbuf, int *cnt, float *thr, uint32_t *thr_g_q, int kp) {
-    const int lane = threadIdx.x & 31;
-    const int n = *cnt < kBufCap ? *cnt : kBufCap;
-    u64 v[kBufCap / 32];
-#pragma unroll
-    for (int it = 0; it < kBufCap / 32; ++it) {
-        const int e = it * 32 + lane;
-        v[it] = (e < n) ? qbuf[e] : 0ull;
-    }
-    warp_sort_desc<kBufCap / 32>(v);
-    const int keep = n < kp ? n : kp;
-    u64 kth = 0ull;
-#pragma unroll
-    for (int it = 0; it < kBufCap / 32; ++it) {
-        const int e = it * 32 + lane;
-        if (e < keep) qbuf[e] = v[it];
-        if (it == ((kp - 1) >> 5)) kth = v[it];
-    }
-    kth = __shfl_sync(0xffffffffu, kth, (kp - 1) & 31);
-    __syncwarp();
-    if (lane == 0) {
-        *cnt = keep;
-        if (n >= kp) {
-            const float s = entry_score(kth);
-            if (s > *thr) *thr = s;
-            atomicMax(thr_g_q, (uint32_t)(kth >> 32));
-        }
-    }
-}
-
 // CUDA-core scan of one pass (up to kScanQ miss queries): tile = 128 rows x 64 queries,
 // d in chunks of 32, fp32 accumulation of bf16 products.
 __global__ void __launch_bounds__(256)
@@ -230,11 +200,11 @@ scan_cc_kernel(const DevState *__restrict__ st, const __nv_bfloat16 *__restrict_
         __syncthreads();
         for (int q = warp; q < nq; q += 8)
             if (cnt[q] > kBufCap - kTileRows)
-                warp_compact(mybuf + (size_t)q * kBufCap, &cnt[q], &thr[q], &thr_g[q], kp);
+                warp_compact<kBufCap>(mybuf + (size_t)q * kBufCap, &cnt[q], &thr[q], &thr_g[q], kp);
         __syncthreads();
     }
     for (int q = warp; q < nq; q += 8)
-        warp_compact(mybuf + (size_t)q * kBufCap, &cnt[q], &thr[q], &thr_g[q], kp);
+        warp_compact<kBufCap>(mybuf + (size_t)q * kBufCap, &cnt[q], &thr[q], &thr_g[q], kp);
     __syncthreads();
     for (int q = tid; q < nq; q += blockDim.x) buf_cnt[(size_t)blockIdx.x * kScanQ + q] = cnt[q];
 }

@@ -1,5 +1,414 @@
-// Tensor-core scan (placeholder until the tcgen05 kernel lands): reports "not available".
+// Tensor-core corpus scan for sm_100a: coarse scores s = bf16(q).bf16(x) - |bf16(x)|^2 / 2 for
+// every corpus row and up to 256 miss queries per pass, with the per-query best-k' selection
+// fused into the accumulator read-out (Algorithm 1, line 6: the database call of the misses).
+//
+// One persistent block per SM, 6 warps:
+//   warp 0   one lane issues TMA loads (cp.async.bulk.tensor, no multicast) of 128-row x 64-col
+//            bf16 corpus tiles, and of the matching query tile unless the whole query block
+//            fits in shared memory and is loaded once, into a ring of mbarrier-guarded stages;
+//   warp 1   allocates tensor memory; one lane issues tcgen05.mma (M = 128 corpus rows,
+//            N = padded query count, K = 16 per instruction, fp32 accumulators in tensor memory,
+//            two accumulator buffers so that the read-out of tile t overlaps the products of t+1);
+//   warps 2-5  read the accumulators (tcgen05.ld, one corpus row per thread), subtract the row's
+//            half norm, compare with the query's threshold and append survivors to the block's
+//            candidate buffers; they sort and cut a buffer when it could overflow.
+// Every wait on an mbarrier is bounded in time; on expiry the block latches PROX_ERR_TIMEOUT,
+// stops issuing work, lets copies in flight land, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include <new>
+
 #include "prox_internal.h"
+#include "topk_device.cuh"
+
 namespace prox {
-int launch_scan_pass_tc(prox_handle *, int, cudaStream_t) { return 1; }
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kMaxStages = 8;
+constexpr int kChunkK = 64;                          // bf16 elements per 128-byte swizzle row
+constexpr int kATileBytes = kTileRows * 128;         // 16 KB
+constexpr int kTileRegion = 220 * 1024;              // shared memory for operand tiles
+constexpr int kQResidentMax = 128 * 1024;            // query block kept resident up to this size
+constexpr int kTmemCols = 512;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: false if the limit ran out or another thread of the block gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+#pragma unroll 1
+    for (int i = 0; i < 128; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+#pragma unroll 1
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_ns() - t0 > kWaitLimitNs) {
+            *abort_flag = 1;
+            return false;
+        }
+        __nanosleep(32);
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major operand tile whose rows are 128 bytes
+// (64 bf16) written by TMA with the 128-byte swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t desc = 0;
+    desc |= (uint64_t)((addr & 0x3ffffu) >> 4);          // start address, 16-byte units
+    desc |= (uint64_t)(1024u >> 4) << 32;                // stride between 8-row groups
+    desc |= 1ull << 46;                                  // descriptor version of sm_100
+    desc |= 2ull << 61;                                  // 128-byte swizzle
+    return desc;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
+}
+
+struct ScanArgs {
+    DevState *st;
+    const float *xh;
+    uint32_t *thr_g;
+    u64 *buf;
+    int32_t *buf_cnt;
+    long long N;
+    int d, pass, kp;
+};
+
+struct Control {
+    unsigned long long full[kMaxStages], empty[kMaxStages], tmem_full[2], tmem_empty[2], q_full;
+    float thr[kScanQ];
+    int cnt[kScanQ];
+    uint32_t tmem_base;
+    int abort_flag;        // set by any role whose wait ran out
+    int abort_epi;         // written by read-out threads only, read after their barrier
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_q32,
+               const __grid_constant__ CUtensorMap tm_q64, const __grid_constant__ CUtensorMap tm_q128,
+               const __grid_constant__ CUtensorMap tm_q256, const ScanArgs a) {
+    extern __shared__ unsigned char smem_dyn[];
+    __shared__ Control ctl;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    const int q0 = a.pass * kScanQ;
+    int nq = a.st->n_miss - q0;
+    if (nq > kScanQ) nq = kScanQ;
+    if (nq <= 0) return;                                  // nothing missed in this pass
+    const int n_pad = nq <= 32 ? 32 : (nq <= 64 ? 64 : (nq <= 128 ? 128 : 256));
+    const CUtensorMap *tm_q = n_pad == 32 ? &tm_q32 : (n_pad == 64 ? &tm_q64 : (n_pad == 128 ? &tm_q128 : &tm_q256));
+    const int nk = a.d / kChunkK;
+    const int b_tile_bytes = n_pad * 128;
+    const int q_block_bytes = b_tile_bytes * nk;
+    const bool resident = q_block_bytes <= kQResidentMax;
+    const int stage_bytes = resident ? kATileBytes : kATileBytes + b_tile_bytes;
+    int stages = (kTileRegion - (resident ? q_block_bytes : 0)) / stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+
+    const uint32_t tiles0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;       // 1024-byte aligned
+    const uint32_t q_res0 = tiles0;
+    const uint32_t stage0 = tiles0 + (resident ? (uint32_t)q_block_bytes : 0u);
+    volatile int *abort_flag = &ctl.abort_flag;
+    uint32_t *thr_g = a.thr_g + q0;
+    u64 *mybuf = a.buf + (size_t)blockIdx.x * kScanQ * kBufCap;
+    const long long ntiles = (a.N + kTileRows - 1) / kTileRows;
+
+    if (tid == 0) {
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(smem_u32(&ctl.full[s]), 1);
+            mbar_init(smem_u32(&ctl.empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&ctl.tmem_full[b]), 1);
+            mbar_init(smem_u32(&ctl.tmem_empty[b]), 4);
+        }
+        mbar_init(smem_u32(&ctl.q_full), 1);
+        ctl.abort_flag = 0;
+        ctl.abort_epi = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    for (int q = tid; q < kScanQ; q += kThreads) { ctl.thr[q] = -INFINITY; ctl.cnt[q] = 0; }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&ctl.tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl.tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            if (resident) {
+                mbar_expect_tx(smem_u32(&ctl.q_full), (uint32_t)q_block_bytes);
+                for (int kc = 0; kc < nk; ++kc)
+                    tma_load_2d(q_res0 + kc * b_tile_bytes, tm_q, kc * kChunkK, q0, smem_u32(&ctl.q_full));
+            }
+            uint32_t g = 0;
+            bool ok = true;
+            for (long long tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
+                const int row0 = (int)(tile * kTileRows);
+                for (int kc = 0; kc < nk; ++kc, ++g) {
+                    const int s = g % stages;
+                    const uint32_t ph = (g / stages) & 1u;
+                    if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t fb = smem_u32(&ctl.full[s]);
+                    const uint32_t dst = stage0 + s * stage_bytes;
+                    mbar_expect_tx(fb, (uint32_t)stage_bytes);
+                    tma_load_2d(dst, &tm_x, kc * kChunkK, row0, fb);
+                    if (!resident) tma_load_2d(dst + kATileBytes, tm_q, kc * kChunkK, q0, fb);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc_bf16(n_pad);
+            bool ok = true;
+            if (resident) ok = mbar_wait(smem_u32(&ctl.q_full), 0, abort_flag);
+            uint32_t g = 0, it = 0;
+            for (long long tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x, ++it) {
+                const uint32_t b = it & 1u, bph = (it >> 1) & 1u;
+                if (!mbar_wait(smem_u32(&ctl.tmem_empty[b]), bph ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + b * (uint32_t)kScanQ;
+                for (int kc = 0; kc < nk; ++kc, ++g) {
+                    const int s = g % stages;
+                    const uint32_t ph = (g / stages) & 1u;
+                    if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = stage0 + s * stage_bytes;
+                    const uint32_t b_addr = resident ? q_res0 + kc * b_tile_bytes : a_addr + kATileBytes;
+                    const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(b_addr);
+#pragma unroll
+                    for (int k4 = 0; k4 < kChunkK / 16; ++k4)     // 16 bf16 = 32 bytes = 2 descriptor units
+                        tc_mma_bf16(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (kc | k4) ? 1u : 0u);
+                    tc_commit(smem_u32(&ctl.empty[s]));           // the stage is free once these are done
+                }
+                if (ok) tc_commit(smem_u32(&ctl.tmem_full[b]));   // accumulator complete
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ accumulator read-out
+        const int e = warp - 2;                                   // 0..3
+        const int quarter = warp & 3;                             // tensor-memory lanes this warp may read
+        const int et = e * 32 + lane;                             // 0..127
+        uint32_t it = 0;
+        for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
+            const uint32_t b = it & 1u, bph = (it >> 1) & 1u;
+            const long long row = tile * kTileRows + quarter * 32 + lane;
+            bool ok = mbar_wait(smem_u32(&ctl.tmem_full[b]), bph, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+                tc_fence_after();
+                const bool row_ok = row < a.N;
+                const float hn = row_ok ? a.xh[row] : 0.f;
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)kScanQ;
+                for (int c0 = 0; c0 < n_pad; c0 += 32) {
+                    uint32_t v[32];
+                    tc_ld32(taddr + c0, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int q = c0 + j;
+                        const float s = __uint_as_float(v[j]) - hn;
+                        if (row_ok && q < nq && s > ctl.thr[q]) {
+                            const int pos = atomicAdd(&ctl.cnt[q], 1);
+                            if (pos < kBufCap) mybuf[(size_t)q * kBufCap + pos] = pack_entry(s, (int32_t)row);
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[b]));
+            } else if (lane == 0) {
+                ctl.abort_epi = 1;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (ctl.abort_epi) break;
+            // thresholds and buffers of the queries this warp owns (q = e mod 4)
+            for (int qb = e; qb < nq; qb += 128) {
+                const int q = qb + 4 * lane;
+                bool need = false;
+                if (q < nq) {
+                    const float g = o2f(__ldcg(&thr_g[q]));
+                    if (g > ctl.thr[q]) ctl.thr[q] = g;
+                    need = ctl.cnt[q] > kBufCap - kTileRows;
+                }
+                unsigned m = __ballot_sync(0xffffffffu, need);
+                while (m) {
+                    const int l = __ffs(m) - 1;
+                    m &= m - 1;
+                    const int qq = qb + 4 * l;
+                    warp_compact<kBufCap>(mybuf + (size_t)qq * kBufCap, &ctl.cnt[qq], &ctl.thr[qq], &thr_g[qq], a.kp);
+                }
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+        if (!ctl.abort_epi) {
+            for (int q = e; q < nq; q += 4)
+                warp_compact<kBufCap>(mybuf + (size_t)q * kBufCap, &ctl.cnt[q], &ctl.thr[q], &thr_g[q], a.kp);
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            for (int q = et; q < nq; q += 128) a.buf_cnt[(size_t)blockIdx.x * kScanQ + q] = ctl.cnt[q];
+        } else {
+            for (int q = et; q < nq; q += 128) a.buf_cnt[(size_t)blockIdx.x * kScanQ + q] = 0;
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (ctl.abort_flag) {
+        if (tid == 0) atomicCAS(&a.st->error, 0, PROX_ERR_TIMEOUT);
+        // let copies and products that were already issued finish before memory is handed back
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {kChunkK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct Maps {
+    CUtensorMap x, q32, q64, q128, q256;
+    bool ok = false;
+};
+
+}  // namespace
+
+// Returns nonzero when the tensor-core path cannot take this handle (d not a multiple of 64,
+// fewer corpus rows than one tile, or no tensor-map encoder in the driver); the caller then
+// runs the CUDA-core scan.
+int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s) {
+    if (h->d % kChunkK || h->N < kTileRows) return 1;
+    if (!h->tc_state) {
+        Maps *m = new (std::nothrow) Maps();
+        if (!m) return 1;
+        h->tc_state = m;
+        m->ok = make_map(&m->x, h->xb, (uint64_t)h->N, (uint64_t)h->d, kTileRows) &&
+                make_map(&m->q32, h->qb, kMaxBatch, (uint64_t)h->d, 32) &&
+                make_map(&m->q64, h->qb, kMaxBatch, (uint64_t)h->d, 64) &&
+                make_map(&m->q128, h->qb, kMaxBatch, (uint64_t)h->d, 128) &&
+                make_map(&m->q256, h->qb, kMaxBatch, (uint64_t)h->d, 256);
+        cudaFuncSetAttribute(scan_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
+    }
+    Maps &maps = *static_cast<Maps *>(h->tc_state);
+    if (!maps.ok) return 1;
+    ScanArgs a;
+    a.st = h->st; a.xh = h->xh; a.thr_g = h->thr_g; a.buf = h->buf; a.buf_cnt = h->buf_cnt;
+    a.N = (long long)h->N; a.d = h->d; a.pass = pass; a.kp = h->kp;
+    scan_tc_kernel<<<h->scan_ctas, kThreads, kTileRegion + 1024, s>>>(maps.x, maps.q32, maps.q64, maps.q128,
+                                                                     maps.q256, a);
+    h->launches++;
+    return 0;
+}
+
+void free_scan_tc(prox_handle *h) {
+    delete static_cast<Maps *>(h->tc_state);
+    h->tc_state = nullptr;
+}
+
 }  // namespace prox

@@ -35,11 +35,15 @@ __device__ __forceinline__ u64 shfl_xor_u64(u64 v, int m) {
 // v[0] of lane 1 the next, ... v[1] of lane 0 the 33rd, and so on.
 template <int ITEMS>
 __device__ __forceinline__ void warp_sort_desc(u64 (&v)[ITEMS]) {
+    constexpr int LOG = (ITEMS == 1 ? 5 : ITEMS == 2 ? 6 : ITEMS == 4 ? 7 : ITEMS == 8 ? 8 : ITEMS == 16 ? 9 : 10);
+    static_assert((32 << (LOG - 5)) == ITEMS * 32, "ITEMS must be a power of two up to 32");
     const int lane = threadIdx.x & 31;
 #pragma unroll
-    for (int k = 2; k <= ITEMS * 32; k <<= 1) {
+    for (int lk = 1; lk <= LOG; ++lk) {
+        const int k = 1 << lk;
 #pragma unroll
-        for (int j = k >> 1; j > 0; j >>= 1) {
+        for (int lj = lk - 1; lj >= 0; --lj) {
+            const int j = 1 << lj;
             if (j >= 32) {
                 const int dj = j >> 5;
 #pragma unroll
@@ -48,7 +52,7 @@ __device__ __forceinline__ void warp_sort_desc(u64 (&v)[ITEMS]) {
                     if (partner > it) {
                         const int e = it * 32 + lane;
                         const bool desc = ((e & k) == 0);
-                        u64 a = v[it], b = v[partner];
+                        const u64 a = v[it], b = v[partner];
                         const bool swap = desc ? (a < b) : (a > b);
                         v[it] = swap ? b : a;
                         v[partner] = swap ? a : b;
@@ -60,13 +64,48 @@ __device__ __forceinline__ void warp_sort_desc(u64 (&v)[ITEMS]) {
                     const int e = it * 32 + lane;
                     const bool desc = ((e & k) == 0);
                     const bool lower = ((lane & j) == 0);       // this lane holds the lower index of the pair
-                    u64 mine = v[it];
-                    u64 other = shfl_xor_u64(mine, j);
+                    const u64 mine = v[it];
+                    const u64 other = shfl_xor_u64(mine, j);
                     // descending block: lower index keeps the max; ascending block: lower keeps the min
                     const bool keep_max = (desc == lower);
                     v[it] = keep_max ? (mine > other ? mine : other) : (mine < other ? mine : other);
                 }
             }
+        }
+    }
+}
+
+// One (block, query) candidate buffer: sort its *cnt entries (at most CAP), keep the best kp,
+// raise the block's threshold to the kp-th score and publish it (atomic max on the ordered
+// form) for the other blocks.  Called by a whole warp; the entries were written by threads
+// of the same block before a barrier.
+template <int CAP>
+__device__ __forceinline__ void warp_compact(u64 *qbuf, int *cnt, float *thr, uint32_t *thr_g_q, int kp) {
+    const int lane = threadIdx.x & 31;
+    const int n = *cnt < CAP ? *cnt : CAP;
+    u64 v[CAP / 32];
+#pragma unroll
+    for (int it = 0; it < CAP / 32; ++it) {
+        const int e = it * 32 + lane;
+        v[it] = (e < n) ? qbuf[e] : 0ull;
+    }
+    warp_sort_desc<CAP / 32>(v);
+    const int keep = n < kp ? n : kp;
+    u64 kth = 0ull;
+#pragma unroll
+    for (int it = 0; it < CAP / 32; ++it) {
+        const int e = it * 32 + lane;
+        if (e < keep) qbuf[e] = v[it];
+        kth |= (e == kp - 1) ? v[it] : 0ull;             // only the owning lane picks it up
+    }
+    kth = __shfl_sync(0xffffffffu, kth, (kp - 1) & 31);
+    __syncwarp();
+    if (lane == 0) {
+        *cnt = keep;
+        if (n >= kp) {
+            const float s = entry_score(kth);
+            if (s > *thr) *thr = s;
+            atomicMax(thr_g_q, (uint32_t)(kth >> 32));
         }
     }
 }

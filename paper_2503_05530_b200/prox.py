@@ -18,6 +18,8 @@ LRU, FIFO = 0, 1
 OK, ERR_INVALID_ARG, ERR_OOM, ERR_CUDA, ERR_UNSUPPORTED, ERR_TIMEOUT, ERR_INTERNAL = range(7)
 MAX_K, MAX_BATCH = 64, 1024
 SCAN_AUTO, SCAN_CUDA_CORE = 0, 1
+STAGES = ("risk_select", "probe", "candidates", "resolve", "gather", "prep_miss", "scan", "merge",
+          "rerank", "exact_pass", "scatter")
 _POLICY = {"lru": LRU, "fifo": FIFO, LRU: LRU, FIFO: FIFO}
 
 
@@ -70,6 +72,10 @@ def load_library():
     L.prox_set_scan_mode.argtypes = [vp, i32]
     L.prox_kernel_launches.restype = i64
     L.prox_kernel_launches.argtypes = [vp]
+    L.prox_profile.restype = i32
+    L.prox_profile.argtypes = [vp, C.c_uint32]
+    L.prox_profile_read.restype = i32
+    L.prox_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64), vp]
     _lib = L
     return L
 
@@ -186,3 +192,20 @@ class Prox:
 
     def kernel_launches(self) -> int:
         return int(self._lib.prox_kernel_launches(self._h))
+
+    def profile(self, stages=None):
+        """Record CUDA events around the named stages (None = all, () = off)."""
+        if stages is None:
+            mask = (1 << len(STAGES)) - 1
+        else:
+            mask = 0
+            for name in stages:
+                mask |= 1 << STAGES.index(name)
+        _check(self._lib.prox_profile(self._h, mask))
+
+    def profile_read(self, stream=None) -> dict:
+        """{stage: (milliseconds, launches)} since the last read; synchronises the stream."""
+        ms = (C.c_double * len(STAGES))()
+        n = (C.c_int64 * len(STAGES))()
+        _check(self._lib.prox_profile_read(self._h, ms, n, _stream_ptr(stream)))
+        return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(STAGES)}

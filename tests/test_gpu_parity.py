@@ -144,7 +144,7 @@ def test_uncertified_queries_take_the_exact_pass():
 # ------------------------------------------------------------------ probe only, pre-filled cache
 @pytest.mark.parametrize("policy", ["lru", "fifo"])
 def test_probe_only_prefilled_cache(policy):
-    keys, centres = W.make_probe_keys(3000, 768, 64, seed=8)
+    keys, centres = W.make_probe_keys(3000, 768, 4096, seed=8)
     p = prox.Prox(keys[:64].contiguous().to(DEV), 1, 3000, 0.5, policy)
     p.cache_load(keys.to(DEV))
     o = oracle.Oracle(None, 768, 1, 3000, float(np.float32(0.5)), oracle.LRU if policy == "lru" else oracle.FIFO)
