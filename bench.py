@@ -233,6 +233,16 @@ def run_ours(args):
             r["d2h"] = B * k * 12 + B
             handle_args = dict(ids=ids[: 64].cpu().numpy(), dists=dists[:64].cpu().numpy(), hit=hit[:64].cpu().numpy(),
                                q=qs[:64].cpu().numpy())
+        if args.stages and rank == 0:
+            p.reset_cache()
+            p.profile(None)
+            p.profile_read()
+            for q, i_, d_, h_ in batches:
+                p.query_batch(q, i_, d_, h_)
+            prof = p.profile_read()
+            p.profile(())
+            print(json.dumps(dict(stage_ms_per_step={kk: round(v[0] / K, 4) for kk, v in prof.items()}, tau=tau)),
+                  file=sys.stderr, flush=True)
         results[tau] = r
         p.close()
         del p
@@ -385,6 +395,7 @@ def main():
     ap.add_argument("--default-steps", type=int, default=200)
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stages", action="store_true", help="also print the time of every stage (one extra run)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -140,7 +140,7 @@ struct ScanArgs {
 
 struct Control {
     unsigned long long full[kMaxStages], empty[kMaxStages], tmem_full[2], tmem_empty[2], q_full;
-    float thr[kScanQ];
+    alignas(16) float thr[kScanQ];
     int cnt[kScanQ];
     uint32_t tmem_base;
     int abort_flag;        // set by any role whose wait ran out
@@ -192,7 +192,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    for (int q = tid; q < kScanQ; q += kThreads) { ctl.thr[q] = -INFINITY; ctl.cnt[q] = 0; }
+    for (int q = tid; q < kScanQ; q += kThreads) { ctl.thr[q] = q < nq ? -INFINITY : INFINITY; ctl.cnt[q] = 0; }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&ctl.tmem_base)), "r"(kTmemCols) : "memory");
@@ -268,20 +268,33 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 tc_fence_after();
-                const bool row_ok = row < a.N;
-                const float hn = row_ok ? a.xh[row] : 0.f;
+                // rows past the end get an infinite half norm, columns past nq an infinite threshold:
+                // neither can pass, so the compare loop needs no bounds tests
+                const float hn = row < a.N ? a.xh[row] : INFINITY;
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)kScanQ;
                 for (int c0 = 0; c0 < n_pad; c0 += 32) {
                     uint32_t v[32];
                     tc_ld32(taddr + c0, v);
-                    tc_wait_ld();
+                    float t[32];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int q = c0 + j;
-                        const float s = __uint_as_float(v[j]) - hn;
-                        if (row_ok && q < nq && s > ctl.thr[q]) {
-                            const int pos = atomicAdd(&ctl.cnt[q], 1);
-                            if (pos < kBufCap) mybuf[(size_t)q * kBufCap + pos] = pack_entry(s, (int32_t)row);
+                    for (int j4 = 0; j4 < 8; ++j4) {
+                        const float4 t4 = *reinterpret_cast<const float4 *>(&ctl.thr[c0 + 4 * j4]);
+                        t[4 * j4] = t4.x; t[4 * j4 + 1] = t4.y; t[4 * j4 + 2] = t4.z; t[4 * j4 + 3] = t4.w;
+                    }
+                    tc_wait_ld();
+                    uint32_t pass = 0;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        pass |= (__uint_as_float(v[j]) - hn > t[j]) ? (1u << j) : 0u;
+                    if (pass) {                                   // rare once the thresholds have settled
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (pass & (1u << j)) {
+                                const int q = c0 + j;
+                                const int pos = atomicAdd(&ctl.cnt[q], 1);
+                                if (pos < kBufCap)
+                                    mybuf[(size_t)q * kBufCap + pos] = pack_entry(__uint_as_float(v[j]) - hn, (int32_t)row);
+                            }
                         }
                     }
                 }
