@@ -2,16 +2,17 @@
 // every corpus row and up to 256 miss queries per pass, with the per-query best-k' selection
 // fused into the accumulator read-out (Algorithm 1, line 6: the database call of the misses).
 //
-// One persistent block per SM, 6 warps:
+// One persistent block per SM, 10 warps:
 //   warp 0   one lane issues TMA loads (cp.async.bulk.tensor, no multicast) of 128-row x 64-col
 //            bf16 corpus tiles, and of the matching query tile unless the whole query block
 //            fits in shared memory and is loaded once, into a ring of mbarrier-guarded stages;
 //   warp 1   allocates tensor memory; one lane issues tcgen05.mma (M = 128 corpus rows,
 //            N = padded query count, K = 16 per instruction, fp32 accumulators in tensor memory,
 //            two accumulator buffers so that the read-out of tile t overlaps the products of t+1);
-//   warps 2-5  read the accumulators (tcgen05.ld, one corpus row per thread), subtract the row's
-//            half norm, compare with the query's threshold and append survivors to the block's
-//            candidate buffers; they sort and cut a buffer when it could overflow.
+//   warps 2-9  read the accumulators (tcgen05.ld, one corpus row per thread, two warps per
+//            tensor-memory lane quarter splitting the columns), subtract the row's half norm,
+//            compare with the query's threshold and append survivors to the block's candidate
+//            buffers; they sort and cut a buffer when it could overflow.
 // Every wait on an mbarrier is bounded in time; on expiry the block latches PROX_ERR_TIMEOUT,
 // stops issuing work, lets copies in flight land, frees its tensor memory and returns.
 #include <cuda.h>
@@ -25,7 +26,7 @@ namespace prox {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;                        // 2 control warps + 8 read-out warps
 constexpr int kMaxStages = 8;
 constexpr int kChunkK = 64;                          // bf16 elements per 128-byte swizzle row
 constexpr int kATileBytes = kTileRows * 128;         // 16 KB
@@ -128,6 +129,31 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
 }
 
+// Thresholds and survivors of 32 accumulator columns (queries c0 .. c0+31) of one corpus row.
+__device__ __forceinline__ void readout32(const uint32_t (&v)[32], int c0, float hn, int32_t row,
+                                          const float *thr, int *cnt, int *need, u64 *mybuf) {
+    uint32_t pass = 0;
+#pragma unroll
+    for (int j4 = 0; j4 < 8; ++j4) {
+        const float4 t4 = *reinterpret_cast<const float4 *>(&thr[c0 + 4 * j4]);
+        pass |= (__uint_as_float(v[4 * j4]) - hn > t4.x) ? (1u << (4 * j4)) : 0u;
+        pass |= (__uint_as_float(v[4 * j4 + 1]) - hn > t4.y) ? (2u << (4 * j4)) : 0u;
+        pass |= (__uint_as_float(v[4 * j4 + 2]) - hn > t4.z) ? (4u << (4 * j4)) : 0u;
+        pass |= (__uint_as_float(v[4 * j4 + 3]) - hn > t4.w) ? (8u << (4 * j4)) : 0u;
+    }
+    if (pass) {                                                   // rare once the thresholds have settled
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            if (pass & (1u << j)) {
+                const int q = c0 + j;
+                const int pos = atomicAdd(&cnt[q], 1);
+                if (pos < kBufCap) mybuf[(size_t)q * kBufCap + pos] = pack_entry(__uint_as_float(v[j]) - hn, row);
+                if (pos >= kBufCap - kTileRows) *need = 1;        // this buffer must be cut before the next tile
+            }
+        }
+    }
+}
+
 struct ScanArgs {
     DevState *st;
     const float *xh;
@@ -145,6 +171,7 @@ struct Control {
     uint32_t tmem_base;
     int abort_flag;        // set by any role whose wait ran out
     int abort_epi;         // written by read-out threads only, read after their barrier
+    int need[3];           // per tile (mod 3): some candidate buffer must be cut before the next tile
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -184,11 +211,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl.tmem_full[b]), 1);
-            mbar_init(smem_u32(&ctl.tmem_empty[b]), 4);
+            mbar_init(smem_u32(&ctl.tmem_empty[b]), 8);
         }
         mbar_init(smem_u32(&ctl.q_full), 1);
         ctl.abort_flag = 0;
         ctl.abort_epi = 0;
+        ctl.need[0] = ctl.need[1] = ctl.need[2] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -257,45 +285,42 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         }
     } else {
         // ------------------------------------------------------------ accumulator read-out
-        const int e = warp - 2;                                   // 0..3
-        const int quarter = warp & 3;                             // tensor-memory lanes this warp may read
-        const int et = e * 32 + lane;                             // 0..127
+        // Eight warps: warp w may read tensor-memory lanes 32 (w mod 4) .. +31; the two warps that
+        // share a lane quarter split the columns.  Thread et owns query et for threshold upkeep.
+        const int e = warp - 2;                                   // 0..7
+        const int quarter = warp & 3;
+        const int half = e >> 2;
+        const int et = e * 32 + lane;                             // 0..255
+        const int cw = n_pad >= 64 ? n_pad / 2 : 32;              // columns per warp
+        const int col_begin = half * cw;
+        const bool active = col_begin < n_pad;
         uint32_t it = 0;
+        long long row = (long long)blockIdx.x * kTileRows + quarter * 32 + lane;
+        float hn = (blockIdx.x < ntiles && row < a.N) ? a.xh[row] : INFINITY;
         for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
             const uint32_t b = it & 1u, bph = (it >> 1) & 1u;
-            const long long row = tile * kTileRows + quarter * 32 + lane;
+            const int flag_now = it % 3, flag_next = (it + 1) % 3;
+            // loads whose latency should hide behind the wait and the read-out
+            const long long row_next = row + (long long)gridDim.x * kTileRows;
+            const float hn_next = (tile + gridDim.x < ntiles && row_next < a.N) ? a.xh[row_next] : INFINITY;
+            const uint32_t g_thr = et < nq ? __ldcg(&thr_g[et]) : 0u;
+            if (et == 0) ctl.need[flag_next] = 0;                 // last read two tiles ago
             bool ok = mbar_wait(smem_u32(&ctl.tmem_full[b]), bph, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 tc_fence_after();
-                // rows past the end get an infinite half norm, columns past nq an infinite threshold:
-                // neither can pass, so the compare loop needs no bounds tests
-                const float hn = row < a.N ? a.xh[row] : INFINITY;
+                // rows past the end carry an infinite half norm, columns past nq an infinite
+                // threshold: neither can pass, so the compare loop needs no bounds tests
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)kScanQ;
-                for (int c0 = 0; c0 < n_pad; c0 += 32) {
-                    uint32_t v[32];
-                    tc_ld32(taddr + c0, v);
-                    float t[32];
-#pragma unroll
-                    for (int j4 = 0; j4 < 8; ++j4) {
-                        const float4 t4 = *reinterpret_cast<const float4 *>(&ctl.thr[c0 + 4 * j4]);
-                        t[4 * j4] = t4.x; t[4 * j4 + 1] = t4.y; t[4 * j4 + 2] = t4.z; t[4 * j4 + 3] = t4.w;
-                    }
-                    tc_wait_ld();
-                    uint32_t pass = 0;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        pass |= (__uint_as_float(v[j]) - hn > t[j]) ? (1u << j) : 0u;
-                    if (pass) {                                   // rare once the thresholds have settled
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (pass & (1u << j)) {
-                                const int q = c0 + j;
-                                const int pos = atomicAdd(&ctl.cnt[q], 1);
-                                if (pos < kBufCap)
-                                    mybuf[(size_t)q * kBufCap + pos] = pack_entry(__uint_as_float(v[j]) - hn, (int32_t)row);
-                            }
-                        }
+                if (active) {
+                    for (int c0 = col_begin; c0 < col_begin + cw; c0 += 64) {
+                        const bool two = c0 + 32 < col_begin + cw;
+                        uint32_t v0[32], v1[32];
+                        tc_ld32(taddr + c0, v0);
+                        if (two) tc_ld32(taddr + c0 + 32, v1);
+                        tc_wait_ld();
+                        readout32(v0, c0, hn, (int32_t)row, ctl.thr, ctl.cnt, &ctl.need[flag_now], mybuf);
+                        if (two) readout32(v1, c0 + 32, hn, (int32_t)row, ctl.thr, ctl.cnt, &ctl.need[flag_now], mybuf);
                     }
                 }
                 tc_fence_before();
@@ -304,34 +329,36 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             } else if (lane == 0) {
                 ctl.abort_epi = 1;
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             if (ctl.abort_epi) break;
-            // thresholds and buffers of the queries this warp owns (q = e mod 4)
-            for (int qb = e; qb < nq; qb += 128) {
-                const int q = qb + 4 * lane;
-                bool need = false;
-                if (q < nq) {
-                    const float g = o2f(__ldcg(&thr_g[q]));
-                    if (g > ctl.thr[q]) ctl.thr[q] = g;
-                    need = ctl.cnt[q] > kBufCap - kTileRows;
-                }
-                unsigned m = __ballot_sync(0xffffffffu, need);
+            // threshold upkeep: a stale (lower) threshold only lets more rows through, so no
+            // barrier is needed unless some buffer has to be cut before the next tile
+            if (et < nq) {
+                const float g = o2f(g_thr);
+                if (g > ctl.thr[et]) ctl.thr[et] = g;
+            }
+            if (ctl.need[flag_now]) {
+                const bool mine = et < nq && ctl.cnt[et] > kBufCap - kTileRows;
+                unsigned m = __ballot_sync(0xffffffffu, mine);
                 while (m) {
                     const int l = __ffs(m) - 1;
                     m &= m - 1;
-                    const int qq = qb + 4 * l;
+                    const int qq = e * 32 + l;
                     warp_compact<kBufCap>(mybuf + (size_t)qq * kBufCap, &ctl.cnt[qq], &ctl.thr[qq], &thr_g[qq], a.kp);
                 }
+                asm volatile("bar.sync 1, 256;" ::: "memory");
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            row = row_next;
+            hn = hn_next;
         }
         if (!ctl.abort_epi) {
-            for (int q = e; q < nq; q += 4)
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            for (int q = e; q < nq; q += 8)
                 warp_compact<kBufCap>(mybuf + (size_t)q * kBufCap, &ctl.cnt[q], &ctl.thr[q], &thr_g[q], a.kp);
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            for (int q = et; q < nq; q += 128) a.buf_cnt[(size_t)blockIdx.x * kScanQ + q] = ctl.cnt[q];
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            for (int q = et; q < nq; q += 256) a.buf_cnt[(size_t)blockIdx.x * kScanQ + q] = ctl.cnt[q];
         } else {
-            for (int q = et; q < nq; q += 128) a.buf_cnt[(size_t)blockIdx.x * kScanQ + q] = 0;
+            for (int q = et; q < nq; q += 256) a.buf_cnt[(size_t)blockIdx.x * kScanQ + q] = 0;
         }
     }
 
