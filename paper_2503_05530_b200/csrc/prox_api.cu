@@ -78,7 +78,7 @@ static void free_all(prox_handle *h) {
                     h->risk_slot, h->risk_stamp, h->part_min, h->part_arg, h->d_risk, h->d_intra,
                     h->safe_min, h->safe_arg, h->cand_d, h->cand_code, h->n_cand, h->src, h->src_kind,
                     h->ins_slot, h->evt_slot, h->evt_dist, h->miss_list, h->miss_rank, h->qb, h->qbn,
-                    h->qerr, h->thr_g, h->buf, h->buf_cnt, h->cand_id, h->cand_score, h->cand_n,
+                    h->qerr, h->thr_g, h->top1, h->buf, h->buf_cnt, h->cand_id, h->cand_score, h->cand_n,
                     h->cand_sk, h->res_ids, h->res_dists, h->fail_list, h->fail_radius, h->coll_id,
                     h->coll_n, h->stage_q, h->stage_ids, h->stage_dists, h->stage_hit};
     for (void *p : ptrs)
@@ -140,6 +140,7 @@ extern "C" prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, i
     ok = ok && dev_alloc(h->evt_slot, MB) && dev_alloc(h->evt_dist, MB);
     ok = ok && dev_alloc(h->miss_list, MB) && dev_alloc(h->miss_rank, MB);
     ok = ok && dev_alloc(h->qb, MB * d) && dev_alloc(h->qbn, MB) && dev_alloc(h->qerr, MB) && dev_alloc(h->thr_g, MB);
+    ok = ok && dev_alloc(h->top1, MB * P);
     ok = ok && dev_alloc(h->buf, P * kScanQ * kBufCap) && dev_alloc(h->buf_cnt, P * kScanQ);
     ok = ok && dev_alloc(h->cand_id, MB * kMaxKp) && dev_alloc(h->cand_score, MB * kMaxKp);
     ok = ok && dev_alloc(h->cand_n, MB) && dev_alloc(h->cand_sk, MB);

@@ -86,6 +86,7 @@ struct prox_handle {
     float *qbn;                       // kMaxBatch: |bf16(q)|^2
     float *qerr;                      // kMaxBatch: upper bound of |q - bf16(q)|
     uint32_t *thr_g;                  // kMaxBatch: shared score thresholds (ordered-uint form)
+    uint32_t *top1;                   // kMaxBatch x P: each block's best score per miss query (ordered-uint form)
     unsigned long long *buf;          // P x kScanQ x kBufCap candidate entries
     int32_t *buf_cnt;                 // P x kScanQ
     int32_t scan_ctas;                // P

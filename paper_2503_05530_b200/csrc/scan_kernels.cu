@@ -74,10 +74,11 @@ convert_corpus_kernel(const float *__restrict__ x, long long N, int d, __nv_bflo
 __global__ void __launch_bounds__(128)
 prep_miss_kernel(DevState *st, const float *__restrict__ queries, int B, int d,
                  const int32_t *__restrict__ miss_list, __nv_bfloat16 *qb, float *qbn, float *qerr,
-                 uint32_t *thr_g, int32_t *coll_n) {
+                 uint32_t *thr_g, int32_t *coll_n, uint32_t *top1, int n_blocks) {
     __shared__ float red[2][4];
     const int m = blockIdx.x, tid = threadIdx.x;
     const int n_miss = st->n_miss;
+    for (int i = tid; i < n_blocks; i += blockDim.x) top1[(size_t)m * n_blocks + i] = 0u;
     if (m == 0) {
         for (int i = tid; i < kMaxBatch; i += blockDim.x) {
             thr_g[i] = f2o(-INFINITY);
@@ -127,7 +128,7 @@ prep_miss_kernel(DevState *st, const float *__restrict__ queries, int B, int d,
 __global__ void __launch_bounds__(256)
 scan_cc_kernel(const DevState *__restrict__ st, const __nv_bfloat16 *__restrict__ xb,
                const float *__restrict__ xh, const __nv_bfloat16 *__restrict__ qb, long long N, int d,
-               int pass, int kp, uint32_t *thr_g, u64 *buf, int32_t *buf_cnt) {
+               int pass, int kp, uint32_t *thr_g, uint32_t *top1, u64 *buf, int32_t *buf_cnt) {
     __shared__ float xs[kTileRows][33];
     __shared__ float qs[64][33];
     __shared__ float thr[kScanQ];
@@ -138,6 +139,7 @@ scan_cc_kernel(const DevState *__restrict__ st, const __nv_bfloat16 *__restrict_
     if (nq > kScanQ) nq = kScanQ;
     if (nq <= 0) return;
     thr_g += q0;
+    top1 += (size_t)q0 * gridDim.x;
     u64 *mybuf = buf + (size_t)blockIdx.x * kScanQ * kBufCap;
     for (int q = tid; q < kScanQ; q += blockDim.x) { thr[q] = -INFINITY; cnt[q] = 0; }
     __syncthreads();
@@ -200,11 +202,13 @@ scan_cc_kernel(const DevState *__restrict__ st, const __nv_bfloat16 *__restrict_
         __syncthreads();
         for (int q = warp; q < nq; q += 8)
             if (cnt[q] > kBufCap - kTileRows)
-                warp_compact<kBufCap>(mybuf + (size_t)q * kBufCap, &cnt[q], &thr[q], &thr_g[q], kp);
+                warp_compact<kBufCap>(mybuf + (size_t)q * kBufCap, &cnt[q], &thr[q], &thr_g[q], kp,
+                                      top1 + (size_t)q * gridDim.x, blockIdx.x, gridDim.x, false);
         __syncthreads();
     }
     for (int q = warp; q < nq; q += 8)
-        warp_compact<kBufCap>(mybuf + (size_t)q * kBufCap, &cnt[q], &thr[q], &thr_g[q], kp);
+        warp_compact<kBufCap>(mybuf + (size_t)q * kBufCap, &cnt[q], &thr[q], &thr_g[q], kp,
+                              top1 + (size_t)q * gridDim.x, blockIdx.x, gridDim.x, true);
     __syncthreads();
     for (int q = tid; q < nq; q += blockDim.x) buf_cnt[(size_t)blockIdx.x * kScanQ + q] = cnt[q];
 }
@@ -467,13 +471,13 @@ void launch_prep_miss(prox_handle *h, const float *q, int B, cudaStream_t s) {
     int rows = ((B + kScanQ - 1) / kScanQ) * kScanQ;      // zero the padding rows of the last pass too
     if (rows > kMaxBatch) rows = kMaxBatch;
     prep_miss_kernel<<<rows, 128, 0, s>>>(h->st, q, B, h->d, h->miss_list, h->qb, h->qbn, h->qerr, h->thr_g,
-                                          h->coll_n);
+                                          h->coll_n, h->top1, h->scan_ctas);
     h->launches++;
 }
 
 void launch_scan_pass(prox_handle *h, int pass, cudaStream_t s) {
     scan_cc_kernel<<<h->scan_ctas, 256, 0, s>>>(h->st, h->xb, h->xh, h->qb, (long long)h->N, h->d, pass,
-                                                h->kp, h->thr_g, h->buf, h->buf_cnt);
+                                                h->kp, h->thr_g, h->top1, h->buf, h->buf_cnt);
     h->launches++;
 }
 

@@ -158,6 +158,7 @@ struct ScanArgs {
     DevState *st;
     const float *xh;
     uint32_t *thr_g;
+    uint32_t *top1;
     u64 *buf;
     int32_t *buf_cnt;
     long long N;
@@ -201,6 +202,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     const uint32_t stage0 = tiles0 + (resident ? (uint32_t)q_block_bytes : 0u);
     volatile int *abort_flag = &ctl.abort_flag;
     uint32_t *thr_g = a.thr_g + q0;
+    uint32_t *top1 = a.top1 + (size_t)q0 * gridDim.x;
     u64 *mybuf = a.buf + (size_t)blockIdx.x * kScanQ * kBufCap;
     const long long ntiles = (a.N + kTileRows - 1) / kTileRows;
 
@@ -344,7 +346,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     const int l = __ffs(m) - 1;
                     m &= m - 1;
                     const int qq = e * 32 + l;
-                    warp_compact<kBufCap>(mybuf + (size_t)qq * kBufCap, &ctl.cnt[qq], &ctl.thr[qq], &thr_g[qq], a.kp);
+                    warp_compact<kBufCap>(mybuf + (size_t)qq * kBufCap, &ctl.cnt[qq], &ctl.thr[qq], &thr_g[qq], a.kp,
+                                          top1 + (size_t)qq * gridDim.x, blockIdx.x, gridDim.x, false);
                 }
                 asm volatile("bar.sync 1, 256;" ::: "memory");
             }
@@ -354,7 +357,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         if (!ctl.abort_epi) {
             asm volatile("bar.sync 1, 256;" ::: "memory");
             for (int q = e; q < nq; q += 8)
-                warp_compact<kBufCap>(mybuf + (size_t)q * kBufCap, &ctl.cnt[q], &ctl.thr[q], &thr_g[q], a.kp);
+                warp_compact<kBufCap>(mybuf + (size_t)q * kBufCap, &ctl.cnt[q], &ctl.thr[q], &thr_g[q], a.kp,
+                                      top1 + (size_t)q * gridDim.x, blockIdx.x, gridDim.x, true);
             asm volatile("bar.sync 1, 256;" ::: "memory");
             for (int q = et; q < nq; q += 256) a.buf_cnt[(size_t)blockIdx.x * kScanQ + q] = ctl.cnt[q];
         } else {
@@ -438,7 +442,7 @@ int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s) {
     Maps &maps = *static_cast<Maps *>(h->tc_state);
     if (!maps.ok) return 1;
     ScanArgs a;
-    a.st = h->st; a.xh = h->xh; a.thr_g = h->thr_g; a.buf = h->buf; a.buf_cnt = h->buf_cnt;
+    a.st = h->st; a.xh = h->xh; a.thr_g = h->thr_g; a.top1 = h->top1; a.buf = h->buf; a.buf_cnt = h->buf_cnt;
     a.N = (long long)h->N; a.d = h->d; a.pass = pass; a.kp = h->kp;
     scan_tc_kernel<<<h->scan_ctas, kThreads, kTileRegion + 1024, s>>>(maps.x, maps.q32, maps.q64, maps.q128,
                                                                      maps.q256, a);

@@ -75,12 +75,20 @@ __device__ __forceinline__ void warp_sort_desc(u64 (&v)[ITEMS]) {
     }
 }
 
-// One (block, query) candidate buffer: sort its *cnt entries (at most CAP), keep the best kp,
-// raise the block's threshold to the kp-th score and publish it (atomic max on the ordered
-// form) for the other blocks.  Called by a whole warp; the entries were written by threads
-// of the same block before a barrier.
+// One (block, query) candidate buffer: sort its *cnt entries (at most CAP), keep the best kp and
+// raise the block's threshold to the kp-th score.  Called by a whole warp; the entries were
+// written by threads of the same block before a barrier.
+//
+// Thresholds are shared between blocks through two arrays.  thr_g_q holds the best known lower
+// bound of the query's global kp-th best score (ordered-uint form, atomic max).  top_q[b] holds
+// the j-th best score block b has found (j = 1 for kp <= 128, else 2): since blocks scan disjoint
+// rows, the r-th largest entry of top_q, r = ceil(kp / j), is exceeded or matched by at least kp
+// distinct rows, so it is such a lower bound, and a much tighter one than any single block's
+// kp-th best.  With prune set, entries below the shared bound are dropped as well (they cannot
+// be among the global best kp).
 template <int CAP>
-__device__ __forceinline__ void warp_compact(u64 *qbuf, int *cnt, float *thr, uint32_t *thr_g_q, int kp) {
+__device__ __forceinline__ void warp_compact(u64 *qbuf, int *cnt, float *thr, uint32_t *thr_g_q, int kp,
+                                             uint32_t *top_q, int block, int n_blocks, bool prune) {
     const int lane = threadIdx.x & 31;
     const int n = *cnt < CAP ? *cnt : CAP;
     u64 v[CAP / 32];
@@ -90,22 +98,61 @@ __device__ __forceinline__ void warp_compact(u64 *qbuf, int *cnt, float *thr, ui
         v[it] = (e < n) ? qbuf[e] : 0ull;
     }
     warp_sort_desc<CAP / 32>(v);
-    const int keep = n < kp ? n : kp;
+    int keep = n < kp ? n : kp;
     u64 kth = 0ull;
 #pragma unroll
     for (int it = 0; it < CAP / 32; ++it) {
         const int e = it * 32 + lane;
-        if (e < keep) qbuf[e] = v[it];
         kth |= (e == kp - 1) ? v[it] : 0ull;             // only the owning lane picks it up
     }
     kth = __shfl_sync(0xffffffffu, kth, (kp - 1) & 31);
+    uint32_t bound = (n >= kp) ? (uint32_t)(kth >> 32) : 0u;
+
+    // publish this block's j-th best and derive the bound from all blocks' values
+    const int j = (kp + 127) >> 7;
+    const int r = (kp + j - 1) / j;
+    if (top_q != nullptr && r <= n_blocks && n_blocks <= 256) {
+        const uint32_t mine = (uint32_t)(__shfl_sync(0xffffffffu, v[0], j - 1) >> 32);
+        if (lane == 0 && n >= j) top_q[block] = mine;
+        u64 t[8];
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int e = it * 32 + lane;
+            uint32_t o = (e < n_blocks) ? __ldcg(&top_q[e]) : 0u;
+            if (e == block && n >= j) o = mine;
+            t[it] = (u64)o;
+        }
+        warp_sort_desc<8>(t);
+        u64 rth = 0ull;
+#pragma unroll
+        for (int it = 0; it < 8; ++it) rth |= (it * 32 + lane == r - 1) ? t[it] : 0ull;
+        rth = __shfl_sync(0xffffffffu, rth, (r - 1) & 31);
+        if ((uint32_t)rth > bound) bound = (uint32_t)rth;
+    }
+    uint32_t g = bound;
+    if (lane == 0 && bound != 0u) {
+        const uint32_t old = atomicMax(thr_g_q, bound);
+        g = old > bound ? old : bound;
+    }
+    g = __shfl_sync(0xffffffffu, g, 0);
+    if (prune && g != 0u) {
+        int ge = 0;
+#pragma unroll
+        for (int it = 0; it < CAP / 32; ++it)
+            ge += __popc(__ballot_sync(0xffffffffu, (uint32_t)(v[it] >> 32) >= g && v[it] != 0ull));
+        if (ge < keep) keep = ge;
+    }
+#pragma unroll
+    for (int it = 0; it < CAP / 32; ++it) {
+        const int e = it * 32 + lane;
+        if (e < keep) qbuf[e] = v[it];
+    }
     __syncwarp();
     if (lane == 0) {
         *cnt = keep;
-        if (n >= kp) {
-            const float s = entry_score(kth);
+        if (g != 0u) {
+            const float s = o2f(g);
             if (s > *thr) *thr = s;
-            atomicMax(thr_g_q, (uint32_t)(kth >> 32));
         }
     }
 }
