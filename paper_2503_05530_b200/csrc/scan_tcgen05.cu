@@ -2,7 +2,7 @@
 // every corpus row and up to 256 miss queries per pass, with the per-query best-k' selection
 // fused into the accumulator read-out (Algorithm 1, line 6: the database call of the misses).
 //
-// One persistent block per SM, 10 warps:
+// One persistent block per SM, 11 warps:
 //   warp 0   one lane issues TMA loads (cp.async.bulk.tensor, no multicast) of 128-row x 64-col
 //            bf16 corpus tiles, and of the matching query tile unless the whole query block
 //            fits in shared memory and is loaded once, into a ring of mbarrier-guarded stages;
@@ -13,6 +13,7 @@
 //            tensor-memory lane quarter splitting the columns), subtract the row's half norm,
 //            compare with the query's threshold and append survivors to the block's candidate
 //            buffers; they sort and cut a buffer when it could overflow.
+//   warp 10  keeps the score bounds that the blocks share fresh (see the bound warp below).
 // Every wait on an mbarrier is bounded in time; on expiry the block latches PROX_ERR_TIMEOUT,
 // stops issuing work, lets copies in flight land, frees its tensor memory and returns.
 #include <cuda.h>
@@ -26,7 +27,7 @@ namespace prox {
 
 namespace {
 
-constexpr int kThreads = 320;                        // 2 control warps + 8 read-out warps
+constexpr int kThreads = 352;                        // 2 control warps + 8 read-out warps + 1 bound warp
 constexpr int kMaxStages = 8;
 constexpr int kChunkK = 64;                          // bf16 elements per 128-byte swizzle row
 constexpr int kATileBytes = kTileRows * 128;         // 16 KB
@@ -131,7 +132,7 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
 
 // Thresholds and survivors of 32 accumulator columns (queries c0 .. c0+31) of one corpus row.
 __device__ __forceinline__ void readout32(const uint32_t (&v)[32], int c0, float hn, int32_t row,
-                                          const float *thr, int *cnt, int *need, u64 *mybuf) {
+                                          const float *thr, int *cnt, uint32_t *best, int *need, u64 *mybuf) {
     uint32_t pass = 0;
 #pragma unroll
     for (int j4 = 0; j4 < 8; ++j4) {
@@ -147,7 +148,9 @@ __device__ __forceinline__ void readout32(const uint32_t (&v)[32], int c0, float
             if (pass & (1u << j)) {
                 const int q = c0 + j;
                 const int pos = atomicAdd(&cnt[q], 1);
-                if (pos < kBufCap) mybuf[(size_t)q * kBufCap + pos] = pack_entry(__uint_as_float(v[j]) - hn, row);
+                const u64 ent = pack_entry(__uint_as_float(v[j]) - hn, row);
+                if (pos < kBufCap) mybuf[(size_t)q * kBufCap + pos] = ent;
+                atomicMax(&best[q], (uint32_t)(ent >> 32));
                 if (pos >= kBufCap - kTileRows) *need = 1;        // this buffer must be cut before the next tile
             }
         }
@@ -173,6 +176,8 @@ struct Control {
     int abort_flag;        // set by any role whose wait ran out
     int abort_epi;         // written by read-out threads only, read after their barrier
     int need[3];           // per tile (mod 3): some candidate buffer must be cut before the next tile
+    int done;              // read-out finished: the bound warp may stop
+    uint32_t best[kScanQ]; // best score this block has appended per query (ordered-uint form)
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -219,10 +224,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         ctl.abort_flag = 0;
         ctl.abort_epi = 0;
         ctl.need[0] = ctl.need[1] = ctl.need[2] = 0;
+        ctl.done = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    for (int q = tid; q < kScanQ; q += kThreads) { ctl.thr[q] = q < nq ? -INFINITY : INFINITY; ctl.cnt[q] = 0; }
+    for (int q = tid; q < kScanQ; q += kThreads) { ctl.thr[q] = q < nq ? -INFINITY : INFINITY; ctl.cnt[q] = 0; ctl.best[q] = 0u; }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&ctl.tmem_base)), "r"(kTmemCols) : "memory");
@@ -285,7 +291,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 if (ok) tc_commit(smem_u32(&ctl.tmem_full[b]));   // accumulator complete
             }
         }
-    } else {
+    } else if (warp < 10) {
         // ------------------------------------------------------------ accumulator read-out
         // Eight warps: warp w may read tensor-memory lanes 32 (w mod 4) .. +31; the two warps that
         // share a lane quarter split the columns.  Thread et owns query et for threshold upkeep.
@@ -296,7 +302,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         const int cw = n_pad >= 64 ? n_pad / 2 : 32;              // columns per warp
         const int col_begin = half * cw;
         const bool active = col_begin < n_pad;
-        uint32_t it = 0;
+        uint32_t it = 0, published = 0u;
         long long row = (long long)blockIdx.x * kTileRows + quarter * 32 + lane;
         float hn = (blockIdx.x < ntiles && row < a.N) ? a.xh[row] : INFINITY;
         for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
@@ -321,8 +327,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                         tc_ld32(taddr + c0, v0);
                         if (two) tc_ld32(taddr + c0 + 32, v1);
                         tc_wait_ld();
-                        readout32(v0, c0, hn, (int32_t)row, ctl.thr, ctl.cnt, &ctl.need[flag_now], mybuf);
-                        if (two) readout32(v1, c0 + 32, hn, (int32_t)row, ctl.thr, ctl.cnt, &ctl.need[flag_now], mybuf);
+                        readout32(v0, c0, hn, (int32_t)row, ctl.thr, ctl.cnt, ctl.best, &ctl.need[flag_now], mybuf);
+                        if (two) readout32(v1, c0 + 32, hn, (int32_t)row, ctl.thr, ctl.cnt, ctl.best, &ctl.need[flag_now], mybuf);
                     }
                 }
                 tc_fence_before();
@@ -338,6 +344,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             if (et < nq) {
                 const float g = o2f(g_thr);
                 if (g > ctl.thr[et]) ctl.thr[et] = g;
+                const uint32_t bq = ctl.best[et];
+                if (bq > published) {                             // let the other blocks see this block's best
+                    top1[(size_t)et * gridDim.x + blockIdx.x] = bq;
+                    published = bq;
+                }
             }
             if (ctl.need[flag_now]) {
                 const bool mine = et < nq && ctl.cnt[et] > kBufCap - kTileRows;
@@ -347,13 +358,14 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     m &= m - 1;
                     const int qq = e * 32 + l;
                     warp_compact<kBufCap>(mybuf + (size_t)qq * kBufCap, &ctl.cnt[qq], &ctl.thr[qq], &thr_g[qq], a.kp,
-                                          top1 + (size_t)qq * gridDim.x, blockIdx.x, gridDim.x, false);
+                                          nullptr, blockIdx.x, gridDim.x, false);
                 }
                 asm volatile("bar.sync 1, 256;" ::: "memory");
             }
             row = row_next;
             hn = hn_next;
         }
+        if (et == 0) ctl.done = 1;
         if (!ctl.abort_epi) {
             asm volatile("bar.sync 1, 256;" ::: "memory");
             for (int q = e; q < nq; q += 8)
@@ -363,6 +375,36 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             for (int q = et; q < nq; q += 256) a.buf_cnt[(size_t)blockIdx.x * kScanQ + q] = ctl.cnt[q];
         } else {
             for (int q = et; q < nq; q += 256) a.buf_cnt[(size_t)blockIdx.x * kScanQ + q] = 0;
+        }
+    } else {
+        // ------------------------------------------------------------ bound warp
+        // Blocks scan disjoint rows, so the r-th largest of the blocks' best scores for a query,
+        // r = k', is matched or exceeded by at least k' distinct rows: a lower bound of the
+        // query's global k'-th best that tightens as every block publishes better rows.  Each
+        // block keeps the bounds of the queries q = block (mod blocks) fresh.
+        const int P = gridDim.x;
+        if (a.kp <= P && P <= 256) {
+            volatile int *done = &ctl.done;
+            int jq = blockIdx.x;
+            while (!*done && !*abort_flag) {
+                if (jq >= nq) jq = blockIdx.x;
+                if (jq < nq) {
+                    u64 t[8];
+#pragma unroll
+                    for (int i8 = 0; i8 < 8; ++i8) {
+                        const int eidx = i8 * 32 + lane;
+                        t[i8] = (eidx < P) ? (u64)__ldcg(&top1[(size_t)jq * P + eidx]) : 0ull;
+                    }
+                    warp_sort_desc<8>(t);
+                    u64 rth = 0ull;
+#pragma unroll
+                    for (int i8 = 0; i8 < 8; ++i8) rth |= (i8 * 32 + lane == a.kp - 1) ? t[i8] : 0ull;
+                    rth = __shfl_sync(0xffffffffu, rth, (a.kp - 1) & 31);
+                    if (lane == 0 && (uint32_t)rth != 0u) atomicMax(&thr_g[jq], (uint32_t)rth);
+                }
+                jq += P;
+                __nanosleep(1000);
+            }
         }
     }
 
