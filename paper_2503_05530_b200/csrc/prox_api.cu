@@ -141,7 +141,9 @@ extern "C" prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, i
     ok = ok && dev_alloc(h->miss_list, MB) && dev_alloc(h->miss_rank, MB);
     ok = ok && dev_alloc(h->qb, MB * d) && dev_alloc(h->qbn, MB) && dev_alloc(h->qerr, MB) && dev_alloc(h->thr_g, MB);
     ok = ok && dev_alloc(h->top1, MB * P);
-    ok = ok && dev_alloc(h->buf, P * kScanQ * kBufCap) && dev_alloc(h->buf_cnt, P * kScanQ);
+    h->tc_cap = h->kp <= 128 ? 256 : 512;               // four warp-private lists per block in the tensor-core scan
+    const size_t buf_entries = P * kScanQ * (size_t)(4 * h->tc_cap > kBufCap ? 4 * h->tc_cap : kBufCap);
+    ok = ok && dev_alloc(h->buf, buf_entries) && dev_alloc(h->buf_cnt, 4 * P * kScanQ);
     ok = ok && dev_alloc(h->cand_id, MB * kMaxKp) && dev_alloc(h->cand_score, MB * kMaxKp);
     ok = ok && dev_alloc(h->cand_n, MB) && dev_alloc(h->cand_sk, MB);
     ok = ok && dev_alloc(h->res_ids, MB * k) && dev_alloc(h->res_dists, MB * k);
@@ -157,7 +159,7 @@ extern "C" prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, i
     }
     cudaMemset(h->st, 0, sizeof(DevState));
     cudaMemset(h->qb, 0, MB * d * sizeof(__nv_bfloat16));
-    cudaMemset(h->buf_cnt, 0, P * kScanQ * sizeof(int32_t));
+    cudaMemset(h->buf_cnt, 0, 4 * P * kScanQ * sizeof(int32_t));
     launch_convert_corpus(h, 0);
     launch_reset(h, 0);
     const cudaError_t e = cudaDeviceSynchronize();

@@ -87,9 +87,12 @@ struct prox_handle {
     float *qerr;                      // kMaxBatch: upper bound of |q - bf16(q)|
     uint32_t *thr_g;                  // kMaxBatch: shared score thresholds (ordered-uint form)
     uint32_t *top1;                   // kMaxBatch x P: each block's best score per miss query (ordered-uint form)
-    unsigned long long *buf;          // P x kScanQ x kBufCap candidate entries
-    int32_t *buf_cnt;                 // P x kScanQ
+    unsigned long long *buf;          // candidate lists of the scan blocks (layout set by the scan that ran)
+    int32_t *buf_cnt;                 // entries per list
     int32_t scan_ctas;                // P
+    int32_t scan_lists;               // lists per query written by the last scan pass
+    int32_t scan_list_stride;         // entries between consecutive (list, query) buffers
+    int32_t tc_cap;                   // entries per (warp, query) buffer of the tensor-core scan
     int32_t *cand_id;                 // kMaxBatch x kMaxKp
     float *cand_score;                // kMaxBatch x kMaxKp
     int32_t *cand_n;                  // kMaxBatch

@@ -214,28 +214,60 @@ scan_cc_kernel(const DevState *__restrict__ st, const __nv_bfloat16 *__restrict_
 }
 
 // ------------------------------------------------------------------------------------------
-// Merge: per query, the k' best entries over all blocks' buffers (each already cut to k').
-// Radix select on the 32-bit ordered score, then a collection pass.
+// Merge: per query, the k' best entries over all candidate lists of the pass (every list was
+// already cut to at most k' entries).  The entries are staged in shared memory when they fit;
+// radix select on the 32-bit ordered score, then a collection pass.
 // ------------------------------------------------------------------------------------------
+constexpr int kMergeStage = 8192;                  // entries staged in shared memory
+
+struct MergeSrc {
+    const u64 *buf;                                // lists of this query: list p at buf + p * list_stride
+    const int32_t *cnt;                            // cnt[p * cnt_stride]
+    size_t list_stride;
+    int cnt_stride, n_lists, kp, total;
+    const u64 *stage;                              // non-null: all entries are in stage[0 .. total)
+    __device__ __forceinline__ int span() const { return stage ? total : n_lists * kp; }
+    __device__ __forceinline__ bool get(int idx, u64 &ent) const {
+        if (stage) { ent = stage[idx]; return true; }
+        const int p = idx / kp, e = idx - p * kp;
+        if (e >= cnt[(size_t)p * cnt_stride]) return false;
+        ent = buf[(size_t)p * list_stride + e];
+        return true;
+    }
+};
+
 __global__ void __launch_bounds__(1024)
-merge_select_kernel(const DevState *__restrict__ st, int pass, int P, int kp, const u64 *__restrict__ buf,
-                    const int32_t *__restrict__ buf_cnt, int32_t *cand_id, float *cand_score,
-                    int32_t *cand_n, float *cand_sk) {
+merge_select_kernel(const DevState *__restrict__ st, int pass, int n_lists, int stride, int kp,
+                    const u64 *__restrict__ buf, const int32_t *__restrict__ buf_cnt, int32_t *cand_id,
+                    float *cand_score, int32_t *cand_n, float *cand_sk) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    u64 *stage = reinterpret_cast<u64 *>(smem_raw);
     __shared__ unsigned hist[256];
     __shared__ uint32_t s_prefix, s_mask;
     __shared__ int s_remaining, s_total, s_gt, s_eq;
-    const int q = blockIdx.x, tid = threadIdx.x;
+    const int q = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m = pass * kScanQ + q;
     if (m >= st->n_miss) return;
 
     if (tid == 0) { s_total = 0; s_gt = 0; s_eq = 0; }
     __syncthreads();
-    int local = 0;
-    for (int p = tid; p < P; p += blockDim.x) local += buf_cnt[(size_t)p * kScanQ + q];
-    if (local) atomicAdd(&s_total, local);
+    for (int p = warp; p < n_lists; p += 32) {
+        const int c = buf_cnt[(size_t)p * kScanQ + q];
+        int base = 0;
+        if (lane == 0 && c > 0) base = atomicAdd(&s_total, c);
+        base = __shfl_sync(0xffffffffu, base, 0);
+        if (base + c <= kMergeStage)
+            for (int e = lane; e < c; e += 32) stage[base + e] = buf[((size_t)p * kScanQ + q) * stride + e];
+    }
     __syncthreads();
-    const int total = s_total;
-    const int span = P * kp;                       // entry (p, e) <-> idx = p * kp + e, e < cnt[p]
+    MergeSrc src;
+    src.buf = buf + (size_t)q * stride;
+    src.cnt = buf_cnt + q;
+    src.list_stride = (size_t)kScanQ * stride;
+    src.cnt_stride = kScanQ;
+    src.n_lists = n_lists; src.kp = kp; src.total = s_total;
+    src.stage = (s_total <= kMergeStage) ? stage : nullptr;
+    const int total = src.total, span = src.span();
 
     uint32_t T = 0;                                // ordered score of the k'-th best (0: keep all)
     if (total >= kp) {
@@ -245,9 +277,9 @@ merge_select_kernel(const DevState *__restrict__ st, int pass, int P, int kp, co
             __syncthreads();
             const uint32_t prefix = s_prefix, mask = s_mask;
             for (int idx = tid; idx < span; idx += blockDim.x) {
-                const int p = idx / kp, e = idx - p * kp;
-                if (e < buf_cnt[(size_t)p * kScanQ + q]) {
-                    const uint32_t o = (uint32_t)(buf[((size_t)p * kScanQ + q) * kBufCap + e] >> 32);
+                u64 ent;
+                if (src.get(idx, ent)) {
+                    const uint32_t o = (uint32_t)(ent >> 32);
                     if ((o & mask) == prefix) atomicAdd(&hist[(o >> (8 * dg)) & 255u], 1u);
                 }
             }
@@ -266,9 +298,8 @@ merge_select_kernel(const DevState *__restrict__ st, int pass, int P, int kp, co
     // entries above T all go in; entries equal to T fill what is left
     const int keep = total < kp ? total : kp;
     for (int idx = tid; idx < span; idx += blockDim.x) {
-        const int p = idx / kp, e = idx - p * kp;
-        if (e < buf_cnt[(size_t)p * kScanQ + q]) {
-            const u64 ent = buf[((size_t)p * kScanQ + q) * kBufCap + e];
+        u64 ent;
+        if (src.get(idx, ent)) {
             const uint32_t o = (uint32_t)(ent >> 32);
             if (o > T || total < kp) {
                 const int pos = atomicAdd(&s_gt, 1);
@@ -281,15 +312,12 @@ merge_select_kernel(const DevState *__restrict__ st, int pass, int P, int kp, co
     const int n_gt = s_gt;
     if (total >= kp) {
         for (int idx = tid; idx < span; idx += blockDim.x) {
-            const int p = idx / kp, e = idx - p * kp;
-            if (e < buf_cnt[(size_t)p * kScanQ + q]) {
-                const u64 ent = buf[((size_t)p * kScanQ + q) * kBufCap + e];
-                if ((uint32_t)(ent >> 32) == T) {
-                    const int pos = n_gt + atomicAdd(&s_eq, 1);
-                    if (pos < kp) {
-                        cand_id[(size_t)m * kMaxKp + pos] = entry_row(ent);
-                        cand_score[(size_t)m * kMaxKp + pos] = o2f(T);
-                    }
+            u64 ent;
+            if (src.get(idx, ent) && (uint32_t)(ent >> 32) == T) {
+                const int pos = n_gt + atomicAdd(&s_eq, 1);
+                if (pos < kp) {
+                    cand_id[(size_t)m * kMaxKp + pos] = entry_row(ent);
+                    cand_score[(size_t)m * kMaxKp + pos] = o2f(T);
                 }
             }
         }
@@ -476,6 +504,8 @@ void launch_prep_miss(prox_handle *h, const float *q, int B, cudaStream_t s) {
 }
 
 void launch_scan_pass(prox_handle *h, int pass, cudaStream_t s) {
+    h->scan_lists = h->scan_ctas;                         // one candidate list per block and query
+    h->scan_list_stride = kBufCap;
     scan_cc_kernel<<<h->scan_ctas, 256, 0, s>>>(h->st, h->xb, h->xh, h->qb, (long long)h->N, h->d, pass,
                                                 h->kp, h->thr_g, h->top1, h->buf, h->buf_cnt);
     h->launches++;
@@ -485,8 +515,14 @@ void launch_merge_select(prox_handle *h, int pass, int B, cudaStream_t s) {
     int nq = B - pass * kScanQ;
     if (nq > kScanQ) nq = kScanQ;
     if (nq <= 0) return;
-    merge_select_kernel<<<nq, 1024, 0, s>>>(h->st, pass, h->scan_ctas, h->kp, h->buf, h->buf_cnt, h->cand_id,
-                                            h->cand_score, h->cand_n, h->cand_sk);
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(merge_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeStage * 8);
+        attr_set = true;
+    }
+    merge_select_kernel<<<nq, 1024, kMergeStage * 8, s>>>(h->st, pass, h->scan_lists, h->scan_list_stride, h->kp,
+                                                          h->buf, h->buf_cnt, h->cand_id, h->cand_score, h->cand_n,
+                                                          h->cand_sk);
     h->launches++;
 }
 

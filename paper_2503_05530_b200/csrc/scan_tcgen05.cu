@@ -2,18 +2,18 @@
 // every corpus row and up to 256 miss queries per pass, with the per-query best-k' selection
 // fused into the accumulator read-out (Algorithm 1, line 6: the database call of the misses).
 //
-// One persistent block per SM, 11 warps:
+// One persistent block per SM, 12 warps:
 //   warp 0   one lane issues TMA loads (cp.async.bulk.tensor, no multicast) of 128-row x 64-col
 //            bf16 corpus tiles, and of the matching query tile unless the whole query block
 //            fits in shared memory and is loaded once, into a ring of mbarrier-guarded stages;
 //   warp 1   allocates tensor memory; one lane issues tcgen05.mma (M = 128 corpus rows,
 //            N = padded query count, K = 16 per instruction, fp32 accumulators in tensor memory,
 //            two accumulator buffers so that the read-out of tile t overlaps the products of t+1);
-//   warps 2-9  read the accumulators (tcgen05.ld, one corpus row per thread, two warps per
+//   warp 2   keeps the score bounds that the blocks share fresh (see the bound warp below);
+//   warps 4-11 read the accumulators (tcgen05.ld, one corpus row per thread, two warps per
 //            tensor-memory lane quarter splitting the columns), subtract the row's half norm,
-//            compare with the query's threshold and append survivors to the block's candidate
-//            buffers; they sort and cut a buffer when it could overflow.
-//   warp 10  keeps the score bounds that the blocks share fresh (see the bound warp below).
+//            compare with the query's threshold and append survivors to warp-private candidate
+//            lists; a warp sorts and cuts a list of its own when it could overflow.
 // Every wait on an mbarrier is bounded in time; on expiry the block latches PROX_ERR_TIMEOUT,
 // stops issuing work, lets copies in flight land, frees its tensor memory and returns.
 #include <cuda.h>
@@ -27,11 +27,12 @@ namespace prox {
 
 namespace {
 
-constexpr int kThreads = 352;                        // 2 control warps + 8 read-out warps + 1 bound warp
+constexpr int kThreads = 384;                        // producer, MMA, bound, (idle), 8 read-out warps
+constexpr int kReadWarps = 8;
 constexpr int kMaxStages = 8;
 constexpr int kChunkK = 64;                          // bf16 elements per 128-byte swizzle row
 constexpr int kATileBytes = kTileRows * 128;         // 16 KB
-constexpr int kTileRegion = 220 * 1024;              // shared memory for operand tiles
+constexpr int kTileRegion = 216 * 1024;              // shared memory for operand tiles
 constexpr int kQResidentMax = 128 * 1024;            // query block kept resident up to this size
 constexpr int kTmemCols = 512;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -130,33 +131,6 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
 }
 
-// Thresholds and survivors of 32 accumulator columns (queries c0 .. c0+31) of one corpus row.
-__device__ __forceinline__ void readout32(const uint32_t (&v)[32], int c0, float hn, int32_t row,
-                                          const float *thr, int *cnt, uint32_t *best, int *need, u64 *mybuf) {
-    uint32_t pass = 0;
-#pragma unroll
-    for (int j4 = 0; j4 < 8; ++j4) {
-        const float4 t4 = *reinterpret_cast<const float4 *>(&thr[c0 + 4 * j4]);
-        pass |= (__uint_as_float(v[4 * j4]) - hn > t4.x) ? (1u << (4 * j4)) : 0u;
-        pass |= (__uint_as_float(v[4 * j4 + 1]) - hn > t4.y) ? (2u << (4 * j4)) : 0u;
-        pass |= (__uint_as_float(v[4 * j4 + 2]) - hn > t4.z) ? (4u << (4 * j4)) : 0u;
-        pass |= (__uint_as_float(v[4 * j4 + 3]) - hn > t4.w) ? (8u << (4 * j4)) : 0u;
-    }
-    if (pass) {                                                   // rare once the thresholds have settled
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            if (pass & (1u << j)) {
-                const int q = c0 + j;
-                const int pos = atomicAdd(&cnt[q], 1);
-                const u64 ent = pack_entry(__uint_as_float(v[j]) - hn, row);
-                if (pos < kBufCap) mybuf[(size_t)q * kBufCap + pos] = ent;
-                atomicMax(&best[q], (uint32_t)(ent >> 32));
-                if (pos >= kBufCap - kTileRows) *need = 1;        // this buffer must be cut before the next tile
-            }
-        }
-    }
-}
-
 struct ScanArgs {
     DevState *st;
     const float *xh;
@@ -170,16 +144,54 @@ struct ScanArgs {
 
 struct Control {
     unsigned long long full[kMaxStages], empty[kMaxStages], tmem_full[2], tmem_empty[2], q_full;
-    alignas(16) float thr[kScanQ];
-    int cnt[kScanQ];
+    alignas(16) float thr[kScanQ];   // per query: scores at or below it cannot be among the best k'
+    uint32_t best[kScanQ];           // best score this block has appended per query (ordered-uint form)
+    int wcnt[kReadWarps][kScanQ / 2];  // entries in each read-out warp's private candidate lists
     uint32_t tmem_base;
-    int abort_flag;        // set by any role whose wait ran out
-    int abort_epi;         // written by read-out threads only, read after their barrier
-    int need[3];           // per tile (mod 3): some candidate buffer must be cut before the next tile
-    int done;              // read-out finished: the bound warp may stop
-    uint32_t best[kScanQ]; // best score this block has appended per query (ordered-uint form)
+    int abort_flag;                  // set by any thread whose wait ran out
+    int done;                        // read-out warps that have finished (the bound warp stops at kReadWarps)
 };
 
+// One read-out warp owns, for every query column it reads, a private candidate list in global
+// memory (CAP entries): it appends the scores that beat the query's threshold and, when a list
+// could overflow during the next tile, sorts it and keeps the best k'.  No other warp touches the
+// list, so the read-out needs no block-wide barrier.
+template <int CAP>
+__device__ __forceinline__ void append32(const uint32_t (&v)[32], int c0, int lc0, float hn, int32_t row,
+                                         const float *thr, int *wcnt, uint32_t *best, u64 *lists, bool &need) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        if (__uint_as_float(v[j]) - thr[c0 + j] > hn) {           // the same arithmetic as the shortcut
+            const float s = __uint_as_float(v[j]) - hn;
+            const int pos = atomicAdd(&wcnt[lc0 + j], 1);
+            const u64 ent = pack_entry(s, row);
+            if (pos < CAP) lists[(size_t)(c0 + j) * CAP + pos] = ent;
+            atomicMax(&best[c0 + j], (uint32_t)(ent >> 32));
+            if (pos >= CAP - 33) need = true;                     // this list must be cut before the next tile
+        }
+    }
+}
+
+// 32 accumulator columns (queries c0 .. c0+31) of one corpus row.  A column passes when
+// acc - thr > half norm, i.e. score = acc - half norm beats the threshold up to one rounding
+// (the certificate's slack covers it); the common case, no column passes, is decided by one
+// maximum over the 32 differences.
+template <int CAP>
+__device__ __forceinline__ void readout32(const uint32_t (&v)[32], int c0, int lc0, float hn,
+                                          int32_t row, const float *thr, int *wcnt, uint32_t *best, u64 *lists,
+                                          bool &need) {
+    float m = -INFINITY;
+#pragma unroll
+    for (int j4 = 0; j4 < 8; ++j4) {
+        const float4 t4 = *reinterpret_cast<const float4 *>(&thr[c0 + 4 * j4]);
+        const float a0 = __uint_as_float(v[4 * j4]) - t4.x, a1 = __uint_as_float(v[4 * j4 + 1]) - t4.y;
+        const float a2 = __uint_as_float(v[4 * j4 + 2]) - t4.z, a3 = __uint_as_float(v[4 * j4 + 3]) - t4.w;
+        m = fmaxf(m, fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)));
+    }
+    if (m > hn) append32<CAP>(v, c0, lc0, hn, row, thr, wcnt, best, lists, need);
+}
+
+template <int CAP>
 __global__ void __launch_bounds__(kThreads, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_q32,
                const __grid_constant__ CUtensorMap tm_q64, const __grid_constant__ CUtensorMap tm_q128,
@@ -208,7 +220,6 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     volatile int *abort_flag = &ctl.abort_flag;
     uint32_t *thr_g = a.thr_g + q0;
     uint32_t *top1 = a.top1 + (size_t)q0 * gridDim.x;
-    u64 *mybuf = a.buf + (size_t)blockIdx.x * kScanQ * kBufCap;
     const long long ntiles = (a.N + kTileRows - 1) / kTileRows;
 
     if (tid == 0) {
@@ -218,17 +229,16 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl.tmem_full[b]), 1);
-            mbar_init(smem_u32(&ctl.tmem_empty[b]), 8);
+            mbar_init(smem_u32(&ctl.tmem_empty[b]), kReadWarps);
         }
         mbar_init(smem_u32(&ctl.q_full), 1);
         ctl.abort_flag = 0;
-        ctl.abort_epi = 0;
-        ctl.need[0] = ctl.need[1] = ctl.need[2] = 0;
         ctl.done = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    for (int q = tid; q < kScanQ; q += kThreads) { ctl.thr[q] = q < nq ? -INFINITY : INFINITY; ctl.cnt[q] = 0; ctl.best[q] = 0u; }
+    for (int q = tid; q < kScanQ; q += kThreads) { ctl.thr[q] = q < nq ? -INFINITY : INFINITY; ctl.best[q] = 0u; }
+    for (int i = tid; i < kReadWarps * (kScanQ / 2); i += kThreads) (&ctl.wcnt[0][0])[i] = 0;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&ctl.tmem_base)), "r"(kTmemCols) : "memory");
@@ -291,102 +301,17 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 if (ok) tc_commit(smem_u32(&ctl.tmem_full[b]));   // accumulator complete
             }
         }
-    } else if (warp < 10) {
-        // ------------------------------------------------------------ accumulator read-out
-        // Eight warps: warp w may read tensor-memory lanes 32 (w mod 4) .. +31; the two warps that
-        // share a lane quarter split the columns.  Thread et owns query et for threshold upkeep.
-        const int e = warp - 2;                                   // 0..7
-        const int quarter = warp & 3;
-        const int half = e >> 2;
-        const int et = e * 32 + lane;                             // 0..255
-        const int cw = n_pad >= 64 ? n_pad / 2 : 32;              // columns per warp
-        const int col_begin = half * cw;
-        const bool active = col_begin < n_pad;
-        uint32_t it = 0, published = 0u;
-        long long row = (long long)blockIdx.x * kTileRows + quarter * 32 + lane;
-        float hn = (blockIdx.x < ntiles && row < a.N) ? a.xh[row] : INFINITY;
-        for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
-            const uint32_t b = it & 1u, bph = (it >> 1) & 1u;
-            const int flag_now = it % 3, flag_next = (it + 1) % 3;
-            // loads whose latency should hide behind the wait and the read-out
-            const long long row_next = row + (long long)gridDim.x * kTileRows;
-            const float hn_next = (tile + gridDim.x < ntiles && row_next < a.N) ? a.xh[row_next] : INFINITY;
-            const uint32_t g_thr = et < nq ? __ldcg(&thr_g[et]) : 0u;
-            if (et == 0) ctl.need[flag_next] = 0;                 // last read two tiles ago
-            bool ok = mbar_wait(smem_u32(&ctl.tmem_full[b]), bph, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (ok) {
-                tc_fence_after();
-                // rows past the end carry an infinite half norm, columns past nq an infinite
-                // threshold: neither can pass, so the compare loop needs no bounds tests
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)kScanQ;
-                if (active) {
-                    for (int c0 = col_begin; c0 < col_begin + cw; c0 += 64) {
-                        const bool two = c0 + 32 < col_begin + cw;
-                        uint32_t v0[32], v1[32];
-                        tc_ld32(taddr + c0, v0);
-                        if (two) tc_ld32(taddr + c0 + 32, v1);
-                        tc_wait_ld();
-                        readout32(v0, c0, hn, (int32_t)row, ctl.thr, ctl.cnt, ctl.best, &ctl.need[flag_now], mybuf);
-                        if (two) readout32(v1, c0 + 32, hn, (int32_t)row, ctl.thr, ctl.cnt, ctl.best, &ctl.need[flag_now], mybuf);
-                    }
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[b]));
-            } else if (lane == 0) {
-                ctl.abort_epi = 1;
-            }
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (ctl.abort_epi) break;
-            // threshold upkeep: a stale (lower) threshold only lets more rows through, so no
-            // barrier is needed unless some buffer has to be cut before the next tile
-            if (et < nq) {
-                const float g = o2f(g_thr);
-                if (g > ctl.thr[et]) ctl.thr[et] = g;
-                const uint32_t bq = ctl.best[et];
-                if (bq > published) {                             // let the other blocks see this block's best
-                    top1[(size_t)et * gridDim.x + blockIdx.x] = bq;
-                    published = bq;
-                }
-            }
-            if (ctl.need[flag_now]) {
-                const bool mine = et < nq && ctl.cnt[et] > kBufCap - kTileRows;
-                unsigned m = __ballot_sync(0xffffffffu, mine);
-                while (m) {
-                    const int l = __ffs(m) - 1;
-                    m &= m - 1;
-                    const int qq = e * 32 + l;
-                    warp_compact<kBufCap>(mybuf + (size_t)qq * kBufCap, &ctl.cnt[qq], &ctl.thr[qq], &thr_g[qq], a.kp,
-                                          nullptr, blockIdx.x, gridDim.x, false);
-                }
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-            }
-            row = row_next;
-            hn = hn_next;
-        }
-        if (et == 0) ctl.done = 1;
-        if (!ctl.abort_epi) {
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            for (int q = e; q < nq; q += 8)
-                warp_compact<kBufCap>(mybuf + (size_t)q * kBufCap, &ctl.cnt[q], &ctl.thr[q], &thr_g[q], a.kp,
-                                      top1 + (size_t)q * gridDim.x, blockIdx.x, gridDim.x, true);
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            for (int q = et; q < nq; q += 256) a.buf_cnt[(size_t)blockIdx.x * kScanQ + q] = ctl.cnt[q];
-        } else {
-            for (int q = et; q < nq; q += 256) a.buf_cnt[(size_t)blockIdx.x * kScanQ + q] = 0;
-        }
-    } else {
+    } else if (warp == 2) {
         // ------------------------------------------------------------ bound warp
-        // Blocks scan disjoint rows, so the r-th largest of the blocks' best scores for a query,
-        // r = k', is matched or exceeded by at least k' distinct rows: a lower bound of the
-        // query's global k'-th best that tightens as every block publishes better rows.  Each
-        // block keeps the bounds of the queries q = block (mod blocks) fresh.
+        // Blocks scan disjoint rows, so the k'-th largest of the blocks' best scores for a query
+        // is matched or exceeded by at least k' distinct rows: a lower bound of the query's global
+        // k'-th best that tightens as every block publishes better rows.  Each block keeps the
+        // bounds of the queries q = block (mod blocks) fresh while its read-out runs.
         const int P = gridDim.x;
         if (a.kp <= P && P <= 256) {
             volatile int *done = &ctl.done;
             int jq = blockIdx.x;
-            while (!*done && !*abort_flag) {
+            while (*done < kReadWarps && !*abort_flag) {
                 if (jq >= nq) jq = blockIdx.x;
                 if (jq < nq) {
                     u64 t[8];
@@ -403,9 +328,110 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     if (lane == 0 && (uint32_t)rth != 0u) atomicMax(&thr_g[jq], (uint32_t)rth);
                 }
                 jq += P;
-                __nanosleep(1000);
+                __nanosleep(2000);
             }
         }
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------ accumulator read-out
+        // Eight warps: warp w may read tensor-memory lanes 32 (w mod 4) .. +31 (one corpus row per
+        // thread); the two warps that share a lane quarter split the query columns.
+        const int e = warp - 4;                                   // 0..7
+        const int quarter = warp & 3;
+        const int half = e >> 2;
+        const int cw = n_pad >= 64 ? n_pad / 2 : 32;              // columns per warp
+        const int col_begin = half * cw;
+        const bool active = col_begin < n_pad;
+        const int ncol = active ? (nq - col_begin < cw ? (nq - col_begin > 0 ? nq - col_begin : 0) : cw) : 0;
+        int *wcnt = ctl.wcnt[e];
+        // lists of this warp: [(block * 4 + quarter) * kScanQ + query] * CAP
+        u64 *lists = a.buf + ((size_t)(blockIdx.x * 4 + quarter) * kScanQ) * CAP;
+        int32_t *lists_cnt = a.buf_cnt + (size_t)(blockIdx.x * 4 + quarter) * kScanQ;
+        uint32_t it = 0;
+        uint32_t published[4] = {0u, 0u, 0u, 0u};
+        long long row = (long long)blockIdx.x * kTileRows + quarter * 32 + lane;
+        float hn = (blockIdx.x < ntiles && row < a.N) ? a.xh[row] : INFINITY;
+        bool alive = true;
+        for (long long tile = blockIdx.x; alive && tile < ntiles; tile += gridDim.x, ++it) {
+            const uint32_t b = it & 1u, bph = (it >> 1) & 1u;
+            // loads whose latency hides behind the wait and the read-out
+            const long long row_next = row + (long long)gridDim.x * kTileRows;
+            const float hn_next = (tile + gridDim.x < ntiles && row_next < a.N) ? a.xh[row_next] : INFINITY;
+            uint32_t g_thr[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int c = col_begin + lane + 32 * i;
+                g_thr[i] = (lane + 32 * i < ncol) ? __ldcg(&thr_g[c]) : 0u;
+            }
+            bool ok = mbar_wait(smem_u32(&ctl.tmem_full[b]), bph, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) { alive = false; break; }
+            tc_fence_after();
+            // rows past the end carry an infinite half norm, columns past nq an infinite threshold:
+            // neither can pass, so the compare loop needs no bounds tests
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)kScanQ;
+            bool need = false;
+            if (active) {
+                for (int c0 = col_begin; c0 < col_begin + cw; c0 += 64) {
+                    const bool two = c0 + 32 < col_begin + cw;
+                    uint32_t v0[32], v1[32];
+                    tc_ld32(taddr + c0, v0);
+                    if (two) tc_ld32(taddr + c0 + 32, v1);
+                    tc_wait_ld();
+                    readout32<CAP>(v0, c0, c0 - col_begin, hn, (int32_t)row, ctl.thr, wcnt, ctl.best, lists, need);
+                    if (two)
+                        readout32<CAP>(v1, c0 + 32, c0 + 32 - col_begin, hn, (int32_t)row, ctl.thr, wcnt,
+                                       ctl.best, lists, need);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[b]));
+            // threshold upkeep for this warp's columns: a stale (lower) threshold only lets more
+            // rows through, so plain stores shared with the other warps are enough
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int lc = lane + 32 * i;
+                if (lc < ncol) {
+                    const int c = col_begin + lc;
+                    const float g = o2f(g_thr[i]);
+                    if (g > ctl.thr[c]) ctl.thr[c] = g;
+                    if (quarter == 0) {                           // one warp per column publishes the block's best
+                        const uint32_t bq = ctl.best[c];
+                        if (bq > published[i]) {
+                            top1[(size_t)c * gridDim.x + blockIdx.x] = bq;
+                            published[i] = bq;
+                        }
+                    }
+                }
+            }
+            if (__any_sync(0xffffffffu, need)) {
+                __syncwarp();
+                for (int i = 0; i < 4; ++i) {
+                    const int lc = lane + 32 * i;
+                    unsigned mm = __ballot_sync(0xffffffffu, lc < ncol && wcnt[lc] > CAP - 33);
+                    while (mm) {
+                        const int l = __ffs(mm) - 1;
+                        mm &= mm - 1;
+                        const int lcc = l + 32 * i, c = col_begin + lcc;
+                        warp_compact<CAP>(lists + (size_t)c * CAP, &wcnt[lcc], &ctl.thr[c], &thr_g[c], a.kp, nullptr,
+                                          blockIdx.x, gridDim.x, false);
+                    }
+                }
+                __syncwarp();
+            }
+            row = row_next;
+            hn = hn_next;
+        }
+        // final cut of every list, dropping what the shared bound has already ruled out
+        __syncwarp();
+        for (int lc = 0; lc < ncol; ++lc) {
+            const int c = col_begin + lc;
+            if (alive)
+                warp_compact<CAP>(lists + (size_t)c * CAP, &wcnt[lc], &ctl.thr[c], &thr_g[c], a.kp, nullptr, blockIdx.x,
+                                  gridDim.x, true);
+            if (lane == 0) lists_cnt[c] = alive ? wcnt[lc] : 0;
+        }
+        if (lane == 0) atomicAdd(&ctl.done, 1);
     }
 
     // ---------------------------------------------------------------- teardown
@@ -479,15 +505,22 @@ int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s) {
                 make_map(&m->q64, h->qb, kMaxBatch, (uint64_t)h->d, 64) &&
                 make_map(&m->q128, h->qb, kMaxBatch, (uint64_t)h->d, 128) &&
                 make_map(&m->q256, h->qb, kMaxBatch, (uint64_t)h->d, 256);
-        cudaFuncSetAttribute(scan_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
+        cudaFuncSetAttribute(scan_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
+        cudaFuncSetAttribute(scan_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
     }
     Maps &maps = *static_cast<Maps *>(h->tc_state);
     if (!maps.ok) return 1;
     ScanArgs a;
     a.st = h->st; a.xh = h->xh; a.thr_g = h->thr_g; a.top1 = h->top1; a.buf = h->buf; a.buf_cnt = h->buf_cnt;
     a.N = (long long)h->N; a.d = h->d; a.pass = pass; a.kp = h->kp;
-    scan_tc_kernel<<<h->scan_ctas, kThreads, kTileRegion + 1024, s>>>(maps.x, maps.q32, maps.q64, maps.q128,
-                                                                     maps.q256, a);
+    h->scan_lists = 4 * h->scan_ctas;                     // one candidate list per read-out lane quarter
+    h->scan_list_stride = h->tc_cap;
+    if (h->tc_cap == 256)
+        scan_tc_kernel<256><<<h->scan_ctas, kThreads, kTileRegion + 1024, s>>>(maps.x, maps.q32, maps.q64, maps.q128,
+                                                                              maps.q256, a);
+    else
+        scan_tc_kernel<512><<<h->scan_ctas, kThreads, kTileRegion + 1024, s>>>(maps.x, maps.q32, maps.q64, maps.q128,
+                                                                              maps.q256, a);
     h->launches++;
     return 0;
 }
