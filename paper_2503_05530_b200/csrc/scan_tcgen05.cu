@@ -156,20 +156,33 @@ struct Control {
 // memory (CAP entries): it appends the scores that beat the query's threshold and, when a list
 // could overflow during the next tile, sorts it and keeps the best k'.  No other warp touches the
 // list, so the read-out needs no block-wide barrier.
+// Slow path of the read-out, entered by the whole warp when some lane has a passing column:
+// per column, the passing lanes take consecutive slots of the warp's list (the counter is
+// private to the warp, so a ballot replaces atomics) and the warp's best score is folded in.
 template <int CAP>
 __device__ __forceinline__ void append32(const uint32_t (&v)[32], int c0, int lc0, float hn, int32_t row,
                                          const float *thr, int *wcnt, uint32_t *best, u64 *lists, bool &need) {
+    const int lane = threadIdx.x & 31;
+    const unsigned lt = (1u << lane) - 1u;
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
-        if (__uint_as_float(v[j]) - thr[c0 + j] > hn) {           // the same arithmetic as the shortcut
-            const float s = __uint_as_float(v[j]) - hn;
-            const int pos = atomicAdd(&wcnt[lc0 + j], 1);
-            const u64 ent = pack_entry(s, row);
-            if (pos < CAP) lists[(size_t)(c0 + j) * CAP + pos] = ent;
-            atomicMax(&best[c0 + j], (uint32_t)(ent >> 32));
-            if (pos >= CAP - 33) need = true;                     // this list must be cut before the next tile
+        const bool p = __uint_as_float(v[j]) - thr[c0 + j] > hn;    // the same arithmetic as the shortcut
+        const unsigned mask = __ballot_sync(0xffffffffu, p);
+        if (mask) {
+            const int base = wcnt[lc0 + j];
+            const u64 ent = pack_entry(__uint_as_float(v[j]) - hn, row);
+            const int pos = base + __popc(mask & lt);
+            if (p && pos < CAP) lists[(size_t)(c0 + j) * CAP + pos] = ent;
+            const uint32_t mx = __reduce_max_sync(0xffffffffu, p ? (uint32_t)(ent >> 32) : 0u);
+            const int n_new = base + __popc(mask);
+            if (lane == 0) {
+                wcnt[lc0 + j] = n_new;
+                atomicMax(&best[c0 + j], mx);
+            }
+            if (n_new > CAP - 33) need = true;                    // this list must be cut before the next tile
         }
     }
+    __syncwarp();
 }
 
 // 32 accumulator columns (queries c0 .. c0+31) of one corpus row.  A column passes when
@@ -188,7 +201,7 @@ __device__ __forceinline__ void readout32(const uint32_t (&v)[32], int c0, int l
         const float a2 = __uint_as_float(v[4 * j4 + 2]) - t4.z, a3 = __uint_as_float(v[4 * j4 + 3]) - t4.w;
         m = fmaxf(m, fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)));
     }
-    if (m > hn) append32<CAP>(v, c0, lc0, hn, row, thr, wcnt, best, lists, need);
+    if (__any_sync(0xffffffffu, m > hn)) append32<CAP>(v, c0, lc0, hn, row, thr, wcnt, best, lists, need);
 }
 
 template <int CAP>
@@ -404,7 +417,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     }
                 }
             }
-            if (__any_sync(0xffffffffu, need)) {
+            if (need) {                                           // warp-uniform
                 __syncwarp();
                 for (int i = 0; i < 4; ++i) {
                     const int lc = lane + 32 * i;

@@ -97,6 +97,31 @@ __device__ __forceinline__ void warp_compact(u64 *qbuf, int *cnt, float *thr, ui
         const int e = it * 32 + lane;
         v[it] = (e < n) ? qbuf[e] : 0ull;
     }
+    {
+        // cheap first: drop what the shared bound already rules out; if at most kp entries are
+        // left, the list need not be sorted (its order does not matter to anyone)
+        const uint32_t g0 = __ldcg(thr_g_q);
+        int cnt_ge[CAP / 32], ge = 0;
+#pragma unroll
+        for (int it = 0; it < CAP / 32; ++it) {
+            const unsigned mk = __ballot_sync(0xffffffffu, v[it] != 0ull && (uint32_t)(v[it] >> 32) >= g0);
+            cnt_ge[it] = ge + __popc(mk & ((1u << lane) - 1u));
+            ge += __popc(mk);
+        }
+        if (ge <= kp && g0 != 0u) {
+            __syncwarp();
+#pragma unroll
+            for (int it = 0; it < CAP / 32; ++it)
+                if (v[it] != 0ull && (uint32_t)(v[it] >> 32) >= g0) qbuf[cnt_ge[it]] = v[it];
+            __syncwarp();
+            if (lane == 0) {
+                *cnt = ge;
+                const float s = o2f(g0);
+                if (s > *thr) *thr = s;
+            }
+            return;
+        }
+    }
     warp_sort_desc<CAP / 32>(v);
     int keep = n < kp ? n : kp;
     u64 kth = 0ull;
