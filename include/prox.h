@@ -171,6 +171,37 @@ int32_t prox_profile(prox_handle *h, uint32_t stage_mask);
  */
 int32_t prox_profile_read(prox_handle *h, double *ms_by_stage, int64_t *launches_by_stage, void *stream);
 
+/* ---- a lookup for callers that must not allocate ------------------------------------------ */
+
+enum {
+    PROX_STATIC_MAX_BATCH = 256,        /* largest B of prox_nearest_key_static */
+    PROX_STATIC_MAX_KEYS = 1 << 22      /* largest n_keys of prox_nearest_key_static */
+};
+
+/*
+ * prox_nearest_key_static -- for every query the nearest of n_keys keys and its squared distance
+ * (the argmin of Algorithm 1's lines 2-3; the paper has no counterpart of this entry point, it is
+ * an addition of this library).  It is meant for callers that cannot allocate device memory at
+ * the time of the call: code embedded in an application that owns all GPU memory and forbids
+ * further allocations, code running with a fixed memory budget, a thread that must not touch the
+ * allocator.  The call needs no handle, calls no cudaMalloc / cudaFree and no allocating library
+ * routine; the partial results its blocks exchange live in an array of about 192 KB that is part
+ * of the library image on every GPU that loads it, until the process exits.
+ *   keys      DEVICE, n_keys x d fp32 row-major, 1 <= n_keys <= PROX_STATIC_MAX_KEYS, 1 <= d <= 4096.
+ *   queries   DEVICE, B x d fp32 row-major, 1 <= B <= PROX_STATIC_MAX_BATCH.
+ *   out_slot  DEVICE, B int32: row of the nearest key (lowest row on a tie).
+ *   out_dist  DEVICE, B fp32: its squared distance (fp64 sum over the fp32 values, rounded once).
+ * Sizes beyond these limits are rejected with PROX_ERR_INVALID_ARG and a text in prox_last_error();
+ * nothing is launched then.  Asynchronous on stream.
+ * The first call on a GPU looks up the device address of the built-in array (once per GPU, with
+ * that GPU current); make that first call outside any stream capture.
+ * All calls on one GPU share the array, which keeps the last call's contents (the call clears the
+ * counters it needs at zero itself): calls that could run at the same time on one GPU race with
+ * each other, so order them on one stream.
+ */
+int32_t prox_nearest_key_static(const float *keys, int64_t n_keys, int32_t d, const float *queries, int32_t B,
+                                int32_t *out_slot, float *out_dist, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -61,6 +61,16 @@ static void set_err(const char *fmt, ...) {
 
 extern "C" const char *prox_last_error(void) { return g_err; }
 
+namespace prox {
+// For entry points that live in other files: same thread-local text as set_err.
+void set_last_error(const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+}  // namespace prox
+
 template <typename T>
 static bool dev_alloc(T *&p, size_t n) {
     void *q = nullptr;

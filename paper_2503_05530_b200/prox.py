@@ -76,6 +76,8 @@ def load_library():
     L.prox_profile.argtypes = [vp, C.c_uint32]
     L.prox_profile_read.restype = i32
     L.prox_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64), vp]
+    L.prox_nearest_key_static.restype = i32
+    L.prox_nearest_key_static.argtypes = [vp, i64, i32, vp, i32, vp, vp, vp]
     _lib = L
     return L
 
@@ -99,6 +101,16 @@ def _dev_f32(t: torch.Tensor, what: str) -> torch.Tensor:
     if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and t.dim() == 2):
         raise ProxError(f"{what} must be a contiguous 2-d float32 CUDA tensor")
     return t
+
+
+def nearest_key_static(keys: torch.Tensor, queries: torch.Tensor, out_slot: torch.Tensor, out_dist: torch.Tensor,
+                       stream=None):
+    """prox_nearest_key_static: nearest key per query, for callers that may not allocate device memory.
+    Every tensor is the caller's (CUDA, contiguous; keys/queries float32, out_slot int32, out_dist float32);
+    the binding allocates nothing either."""
+    _check(load_library().prox_nearest_key_static(keys.data_ptr(), keys.shape[0], keys.shape[1], queries.data_ptr(),
+                                                  queries.shape[0], out_slot.data_ptr(), out_dist.data_ptr(),
+                                                  _stream_ptr(stream)))
 
 
 class Prox:
