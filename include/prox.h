@@ -46,8 +46,9 @@ enum {
 enum {
     PROX_MAX_K = 64,            /* largest k */
     PROX_MAX_BATCH = 1024,      /* largest B of one call */
-    PROX_SCAN_AUTO = 0,         /* prox_set_scan_mode: tensor-core scan (default) */
-    PROX_SCAN_CUDA_CORE = 1     /* prox_set_scan_mode: plain CUDA-core scan of the same bf16 scores */
+    PROX_SCAN_AUTO = 0,         /* prox_set_scan_mode: tensor-core scan, two blocks per MMA (default) */
+    PROX_SCAN_CUDA_CORE = 1,    /* prox_set_scan_mode: plain CUDA-core scan of the same bf16 scores */
+    PROX_SCAN_TC_SINGLE = 2     /* prox_set_scan_mode: tensor-core scan, one block per MMA */
 };
 
 /*
@@ -143,7 +144,7 @@ int32_t prox_get_stats(prox_handle *h, prox_stats *out, void *stream);
 /* prox_status -- synchronises the stream and returns the latched device error (PROX_OK if none). */
 int32_t prox_status(prox_handle *h, void *stream);
 
-/* prox_set_scan_mode -- PROX_SCAN_AUTO or PROX_SCAN_CUDA_CORE (for cross-checks and timing). */
+/* prox_set_scan_mode -- one of the PROX_SCAN_* values (for cross-checks and timing). */
 int32_t prox_set_scan_mode(prox_handle *h, int32_t mode);
 
 /* prox_kernel_launches -- kernels launched by this handle so far (host-side count). */

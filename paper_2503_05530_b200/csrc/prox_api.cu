@@ -311,7 +311,7 @@ extern "C" int32_t prox_status(prox_handle *h, void *stream) {
 
 extern "C" int32_t prox_set_scan_mode(prox_handle *h, int32_t mode) {
     g_err[0] = 0;
-    if (!h || (mode != PROX_SCAN_AUTO && mode != PROX_SCAN_CUDA_CORE)) {
+    if (!h || (mode != PROX_SCAN_AUTO && mode != PROX_SCAN_CUDA_CORE && mode != PROX_SCAN_TC_SINGLE)) {
         set_err("bad handle or mode");
         return PROX_ERR_INVALID_ARG;
     }

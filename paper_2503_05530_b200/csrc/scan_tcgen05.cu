@@ -21,9 +21,13 @@
 #include <new>
 
 #include "prox_internal.h"
+#include "scan_readout.cuh"
+#include "sm100_ptx.cuh"
 #include "topk_device.cuh"
 
 namespace prox {
+
+using namespace sm100;
 
 namespace {
 
@@ -35,101 +39,6 @@ constexpr int kATileBytes = kTileRows * 128;         // 16 KB
 constexpr int kTileRegion = 216 * 1024;              // shared memory for operand tiles
 constexpr int kQResidentMax = 128 * 1024;            // query block kept resident up to this size
 constexpr int kTmemCols = 512;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
-
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait: false if the limit ran out or another thread of the block gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-#pragma unroll 1
-    for (int i = 0; i < 128; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-#pragma unroll 1
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (global_ns() - t0 > kWaitLimitNs) {
-            *abort_flag = 1;
-            return false;
-        }
-        __nanosleep(32);
-    }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
-        : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                            uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor of a K-major operand tile whose rows are 128 bytes
-// (64 bf16) written by TMA with the 128-byte swizzle: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-    uint64_t desc = 0;
-    desc |= (uint64_t)((addr & 0x3ffffu) >> 4);          // start address, 16-byte units
-    desc |= (uint64_t)(1024u >> 4) << 32;                // stride between 8-row groups
-    desc |= 1ull << 46;                                  // descriptor version of sm_100
-    desc |= 2ull << 61;                                  // 128-byte swizzle
-    return desc;
-}
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
-}
 
 struct ScanArgs {
     DevState *st;
@@ -156,71 +65,34 @@ struct Control {
 // memory (CAP entries): it appends the scores that beat the query's threshold and, when a list
 // could overflow during the next tile, sorts it and keeps the best k'.  No other warp touches the
 // list, so the read-out needs no block-wide barrier.
-// Slow path of the read-out, entered by the whole warp when some lane has a passing column:
-// per column, the passing lanes take consecutive slots of the warp's list (the counter is
-// private to the warp, so a ballot replaces atomics) and the warp's best score is folded in.
-template <int CAP>
-__device__ __forceinline__ void append32(const uint32_t (&v)[32], int c0, int lc0, float hn, int32_t row,
-                                         const float *thr, int *wcnt, uint32_t *best, u64 *lists, bool &need) {
-    const int lane = threadIdx.x & 31;
-    const unsigned lt = (1u << lane) - 1u;
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        const bool p = __uint_as_float(v[j]) - thr[c0 + j] > hn;    // the same arithmetic as the shortcut
-        const unsigned mask = __ballot_sync(0xffffffffu, p);
-        if (mask) {
-            const int base = wcnt[lc0 + j];
-            const u64 ent = pack_entry(__uint_as_float(v[j]) - hn, row);
-            const int pos = base + __popc(mask & lt);
-            if (p && pos < CAP) lists[(size_t)(c0 + j) * CAP + pos] = ent;
-            const uint32_t mx = __reduce_max_sync(0xffffffffu, p ? (uint32_t)(ent >> 32) : 0u);
-            const int n_new = base + __popc(mask);
-            if (lane == 0) {
-                wcnt[lc0 + j] = n_new;
-                atomicMax(&best[c0 + j], mx);
-            }
-            if (n_new > CAP - 33) need = true;                    // this list must be cut before the next tile
-        }
-    }
-    __syncwarp();
-}
-
-// 32 accumulator columns (queries c0 .. c0+31) of one corpus row.  A column passes when
-// acc - thr > half norm, i.e. score = acc - half norm beats the threshold up to one rounding
-// (the certificate's slack covers it); the common case, no column passes, is decided by one
-// maximum over the 32 differences.
-template <int CAP>
-__device__ __forceinline__ void readout32(const uint32_t (&v)[32], int c0, int lc0, float hn,
-                                          int32_t row, const float *thr, int *wcnt, uint32_t *best, u64 *lists,
-                                          bool &need) {
-    float m = -INFINITY;
-#pragma unroll
-    for (int j4 = 0; j4 < 8; ++j4) {
-        const float4 t4 = *reinterpret_cast<const float4 *>(&thr[c0 + 4 * j4]);
-        const float a0 = __uint_as_float(v[4 * j4]) - t4.x, a1 = __uint_as_float(v[4 * j4 + 1]) - t4.y;
-        const float a2 = __uint_as_float(v[4 * j4 + 2]) - t4.z, a3 = __uint_as_float(v[4 * j4 + 3]) - t4.w;
-        m = fmaxf(m, fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)));
-    }
-    if (__any_sync(0xffffffffu, m > hn)) append32<CAP>(v, c0, lc0, hn, row, thr, wcnt, best, lists, need);
-}
-
-template <int CAP>
+//
+// PAIR = true runs two blocks per MMA (a cluster of two, tcgen05 cta_group::2): a pair takes 256
+// corpus rows per tile, each block loading its own 128 rows and half of the query rows, so a
+// block ingests a third less per corpus row than alone.  Block 0 of the pair issues the MMAs.
+template <int CAP, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
-scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_q32,
-               const __grid_constant__ CUtensorMap tm_q64, const __grid_constant__ CUtensorMap tm_q128,
-               const __grid_constant__ CUtensorMap tm_q256, const ScanArgs a) {
+scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_q16,
+               const __grid_constant__ CUtensorMap tm_q32, const __grid_constant__ CUtensorMap tm_q64,
+               const __grid_constant__ CUtensorMap tm_q128, const __grid_constant__ CUtensorMap tm_q256,
+               const ScanArgs a) {
     extern __shared__ unsigned char smem_dyn[];
     __shared__ Control ctl;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = PAIR ? cluster_rank() : 0u;        // 0: the block of the pair that issues MMAs
+    const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;      // pair (or block) index
+    const int n_units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    constexpr int kUnitRows = PAIR ? 2 * kTileRows : kTileRows;            // corpus rows per tile of a unit
 
     const int q0 = a.pass * kScanQ;
     int nq = a.st->n_miss - q0;
     if (nq > kScanQ) nq = kScanQ;
     if (nq <= 0) return;                                  // nothing missed in this pass
     const int n_pad = nq <= 32 ? 32 : (nq <= 64 ? 64 : (nq <= 128 ? 128 : 256));
-    const CUtensorMap *tm_q = n_pad == 32 ? &tm_q32 : (n_pad == 64 ? &tm_q64 : (n_pad == 128 ? &tm_q128 : &tm_q256));
+    const int q_rows = PAIR ? n_pad / 2 : n_pad;             // query rows this block stages (half of B in a pair)
+    const CUtensorMap *tm_q = q_rows == 16 ? &tm_q16 : (q_rows == 32 ? &tm_q32 : (q_rows == 64 ? &tm_q64 : (q_rows == 128 ? &tm_q128 : &tm_q256)));
+    const int q_row0 = q0 + (int)rank * q_rows;
     const int nk = a.d / kChunkK;
-    const int b_tile_bytes = n_pad * 128;
+    const int b_tile_bytes = q_rows * 128;
     const int q_block_bytes = b_tile_bytes * nk;
     const bool resident = q_block_bytes <= kQResidentMax;
     const int stage_bytes = resident ? kATileBytes : kATileBytes + b_tile_bytes;
@@ -233,7 +105,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     volatile int *abort_flag = &ctl.abort_flag;
     uint32_t *thr_g = a.thr_g + q0;
     uint32_t *top1 = a.top1 + (size_t)q0 * gridDim.x;
-    const long long ntiles = (a.N + kTileRows - 1) / kTileRows;
+    const long long ntiles = (a.N + kUnitRows - 1) / kUnitRows;
+    // barriers the MMA-issuing block waits on: in a pair, both blocks signal block 0's copy
+    const uint32_t tx_mult = PAIR ? 2u : 1u;
 
     if (tid == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
@@ -242,7 +116,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl.tmem_full[b]), 1);
-            mbar_init(smem_u32(&ctl.tmem_empty[b]), kReadWarps);
+            mbar_init(smem_u32(&ctl.tmem_empty[b]), PAIR ? 2 * kReadWarps : kReadWarps);
         }
         mbar_init(smem_u32(&ctl.q_full), 1);
         ctl.abort_flag = 0;
@@ -252,48 +126,55 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     }
     for (int q = tid; q < kScanQ; q += kThreads) { ctl.thr[q] = q < nq ? -INFINITY : INFINITY; ctl.best[q] = 0u; }
     for (int i = tid; i < kReadWarps * (kScanQ / 2); i += kThreads) (&ctl.wcnt[0][0])[i] = 0;
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&ctl.tmem_base)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+    if (warp == 1) tmem_alloc<PAIR>(smem_u32(&ctl.tmem_base), kTmemCols);
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();               // both blocks' barriers exist before any remote signal
     tc_fence_after();
     const uint32_t tmem_base = ctl.tmem_base;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
+            const uint32_t q_full_bar = PAIR ? map_to_rank(smem_u32(&ctl.q_full), 0) : smem_u32(&ctl.q_full);
             if (resident) {
-                mbar_expect_tx(smem_u32(&ctl.q_full), (uint32_t)q_block_bytes);
-                for (int kc = 0; kc < nk; ++kc)
-                    tma_load_2d(q_res0 + kc * b_tile_bytes, tm_q, kc * kChunkK, q0, smem_u32(&ctl.q_full));
+                if (rank == 0) mbar_expect_tx(smem_u32(&ctl.q_full), tx_mult * (uint32_t)q_block_bytes);
+                for (int kc = 0; kc < nk; ++kc) {
+                    if constexpr (PAIR) tma_load_2d_pair(q_res0 + kc * b_tile_bytes, tm_q, kc * kChunkK, q_row0, q_full_bar);
+                    else tma_load_2d(q_res0 + kc * b_tile_bytes, tm_q, kc * kChunkK, q_row0, q_full_bar);
+                }
             }
             uint32_t g = 0;
             bool ok = true;
-            for (long long tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
-                const int row0 = (int)(tile * kTileRows);
+            for (long long tile = unit; ok && tile < ntiles; tile += n_units) {
+                const int row0 = (int)(tile * kUnitRows) + (int)rank * kTileRows;
                 for (int kc = 0; kc < nk; ++kc, ++g) {
                     const int s = g % stages;
                     const uint32_t ph = (g / stages) & 1u;
                     if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t fb = smem_u32(&ctl.full[s]);
                     const uint32_t dst = stage0 + s * stage_bytes;
-                    mbar_expect_tx(fb, (uint32_t)stage_bytes);
-                    tma_load_2d(dst, &tm_x, kc * kChunkK, row0, fb);
-                    if (!resident) tma_load_2d(dst + kATileBytes, tm_q, kc * kChunkK, q0, fb);
+                    if constexpr (PAIR) {
+                        const uint32_t fb = map_to_rank(smem_u32(&ctl.full[s]), 0);
+                        if (rank == 0) mbar_expect_tx(smem_u32(&ctl.full[s]), 2u * (uint32_t)stage_bytes);
+                        tma_load_2d_pair(dst, &tm_x, kc * kChunkK, row0, fb);
+                        if (!resident) tma_load_2d_pair(dst + kATileBytes, tm_q, kc * kChunkK, q_row0, fb);
+                    } else {
+                        const uint32_t fb = smem_u32(&ctl.full[s]);
+                        mbar_expect_tx(fb, (uint32_t)stage_bytes);
+                        tma_load_2d(dst, &tm_x, kc * kChunkK, row0, fb);
+                        if (!resident) tma_load_2d(dst + kATileBytes, tm_q, kc * kChunkK, q_row0, fb);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = instr_desc_bf16(n_pad);
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = instr_desc_bf16(kUnitRows, n_pad);
             bool ok = true;
             if (resident) ok = mbar_wait(smem_u32(&ctl.q_full), 0, abort_flag);
             uint32_t g = 0, it = 0;
-            for (long long tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x, ++it) {
+            for (long long tile = unit; ok && tile < ntiles; tile += n_units, ++it) {
                 const uint32_t b = it & 1u, bph = (it >> 1) & 1u;
                 if (!mbar_wait(smem_u32(&ctl.tmem_empty[b]), bph ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -307,11 +188,18 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     const uint32_t b_addr = resident ? q_res0 + kc * b_tile_bytes : a_addr + kATileBytes;
                     const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(b_addr);
 #pragma unroll
-                    for (int k4 = 0; k4 < kChunkK / 16; ++k4)     // 16 bf16 = 32 bytes = 2 descriptor units
-                        tc_mma_bf16(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (kc | k4) ? 1u : 0u);
-                    tc_commit(smem_u32(&ctl.empty[s]));           // the stage is free once these are done
+                    for (int k4 = 0; k4 < kChunkK / 16; ++k4) {   // 16 bf16 = 32 bytes = 2 descriptor units
+                        if constexpr (PAIR) tc_mma_bf16_pair(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (kc | k4) ? 1u : 0u);
+                        else tc_mma_bf16(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (kc | k4) ? 1u : 0u);
+                    }
+                    // the stage is free (in both blocks of a pair) once these are done
+                    if constexpr (PAIR) tc_commit_pair(smem_u32(&ctl.empty[s]));
+                    else tc_commit(smem_u32(&ctl.empty[s]));
                 }
-                if (ok) tc_commit(smem_u32(&ctl.tmem_full[b]));   // accumulator complete
+                if (ok) {                                         // accumulator complete
+                    if constexpr (PAIR) tc_commit_pair(smem_u32(&ctl.tmem_full[b]));
+                    else tc_commit(smem_u32(&ctl.tmem_full[b]));
+                }
             }
         }
     } else if (warp == 2) {
@@ -361,14 +249,16 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         int32_t *lists_cnt = a.buf_cnt + (size_t)(blockIdx.x * 4 + quarter) * kScanQ;
         uint32_t it = 0;
         uint32_t published[4] = {0u, 0u, 0u, 0u};
-        long long row = (long long)blockIdx.x * kTileRows + quarter * 32 + lane;
-        float hn = (blockIdx.x < ntiles && row < a.N) ? a.xh[row] : INFINITY;
+        long long row = (long long)unit * kUnitRows + (long long)rank * kTileRows + quarter * 32 + lane;
+        float hn = (unit < ntiles && row < a.N) ? a.xh[row] : INFINITY;
         bool alive = true;
-        for (long long tile = blockIdx.x; alive && tile < ntiles; tile += gridDim.x, ++it) {
+        const uint32_t empty_bar0 = PAIR ? map_to_rank(smem_u32(&ctl.tmem_empty[0]), 0) : smem_u32(&ctl.tmem_empty[0]);
+        const uint32_t empty_bar1 = PAIR ? map_to_rank(smem_u32(&ctl.tmem_empty[1]), 0) : smem_u32(&ctl.tmem_empty[1]);
+        for (long long tile = unit; alive && tile < ntiles; tile += n_units, ++it) {
             const uint32_t b = it & 1u, bph = (it >> 1) & 1u;
             // loads whose latency hides behind the wait and the read-out
-            const long long row_next = row + (long long)gridDim.x * kTileRows;
-            const float hn_next = (tile + gridDim.x < ntiles && row_next < a.N) ? a.xh[row_next] : INFINITY;
+            const long long row_next = row + (long long)n_units * kUnitRows;
+            const float hn_next = (tile + n_units < ntiles && row_next < a.N) ? a.xh[row_next] : INFINITY;
             uint32_t g_thr[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -398,7 +288,10 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[b]));
+            if (lane == 0) {
+                if constexpr (PAIR) mbar_arrive_cluster(b ? empty_bar1 : empty_bar0);
+                else mbar_arrive(b ? empty_bar1 : empty_bar0);
+            }
             // threshold upkeep for this warp's columns: a stale (lower) threshold only lets more
             // rows through, so plain stores shared with the other warps are enough
 #pragma unroll
@@ -450,6 +343,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();               // no signal to the other block is still under way
     if (ctl.abort_flag) {
         if (tid == 0) atomicCAS(&a.st->error, 0, PROX_ERR_TIMEOUT);
         // let copies and products that were already issued finish before memory is handed back
@@ -459,7 +353,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     }
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        tmem_dealloc<PAIR>(tmem_base, kTmemCols);
     }
 }
 
@@ -498,7 +392,7 @@ bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, 
 }
 
 struct Maps {
-    CUtensorMap x, q32, q64, q128, q256;
+    CUtensorMap x, q16, q32, q64, q128, q256;
     bool ok = false;
 };
 
@@ -514,26 +408,45 @@ int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s) {
         if (!m) return 1;
         h->tc_state = m;
         m->ok = make_map(&m->x, h->xb, (uint64_t)h->N, (uint64_t)h->d, kTileRows) &&
+                make_map(&m->q16, h->qb, kMaxBatch, (uint64_t)h->d, 16) &&
                 make_map(&m->q32, h->qb, kMaxBatch, (uint64_t)h->d, 32) &&
                 make_map(&m->q64, h->qb, kMaxBatch, (uint64_t)h->d, 64) &&
                 make_map(&m->q128, h->qb, kMaxBatch, (uint64_t)h->d, 128) &&
                 make_map(&m->q256, h->qb, kMaxBatch, (uint64_t)h->d, 256);
-        cudaFuncSetAttribute(scan_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
-        cudaFuncSetAttribute(scan_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
+        cudaFuncSetAttribute(scan_tc_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
+        cudaFuncSetAttribute(scan_tc_kernel<512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
+        cudaFuncSetAttribute(scan_tc_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
+        cudaFuncSetAttribute(scan_tc_kernel<512, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
     }
     Maps &maps = *static_cast<Maps *>(h->tc_state);
     if (!maps.ok) return 1;
     ScanArgs a;
     a.st = h->st; a.xh = h->xh; a.thr_g = h->thr_g; a.top1 = h->top1; a.buf = h->buf; a.buf_cnt = h->buf_cnt;
     a.N = (long long)h->N; a.d = h->d; a.pass = pass; a.kp = h->kp;
-    h->scan_lists = 4 * h->scan_ctas;                     // one candidate list per read-out lane quarter
+    const bool pair = h->scan_mode != PROX_SCAN_TC_SINGLE && h->scan_ctas >= 2 && h->N >= 2 * kTileRows;
+    const int grid = pair ? (h->scan_ctas & ~1) : h->scan_ctas;
+    h->scan_lists = 4 * grid;                             // one candidate list per read-out lane quarter
     h->scan_list_stride = h->tc_cap;
-    if (h->tc_cap == 256)
-        scan_tc_kernel<256><<<h->scan_ctas, kThreads, kTileRegion + 1024, s>>>(maps.x, maps.q32, maps.q64, maps.q128,
-                                                                              maps.q256, a);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kTileRegion + 1024;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = pair ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
+    if (pair)
+        e = h->tc_cap == 256 ? cudaLaunchKernelEx(&cfg, scan_tc_kernel<256, true>, maps.x, maps.q16, maps.q32, maps.q64, maps.q128, maps.q256, a)
+                             : cudaLaunchKernelEx(&cfg, scan_tc_kernel<512, true>, maps.x, maps.q16, maps.q32, maps.q64, maps.q128, maps.q256, a);
     else
-        scan_tc_kernel<512><<<h->scan_ctas, kThreads, kTileRegion + 1024, s>>>(maps.x, maps.q32, maps.q64, maps.q128,
-                                                                              maps.q256, a);
+        e = h->tc_cap == 256 ? cudaLaunchKernelEx(&cfg, scan_tc_kernel<256, false>, maps.x, maps.q16, maps.q32, maps.q64, maps.q128, maps.q256, a)
+                             : cudaLaunchKernelEx(&cfg, scan_tc_kernel<512, false>, maps.x, maps.q16, maps.q32, maps.q64, maps.q128, maps.q256, a);
+    if (e != cudaSuccess) return 1;                       // the caller falls back to the CUDA-core scan
     h->launches++;
     return 0;
 }

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libprox.so")
 LRU, FIFO = 0, 1
 OK, ERR_INVALID_ARG, ERR_OOM, ERR_CUDA, ERR_UNSUPPORTED, ERR_TIMEOUT, ERR_INTERNAL = range(7)
 MAX_K, MAX_BATCH = 64, 1024
-SCAN_AUTO, SCAN_CUDA_CORE = 0, 1
+SCAN_AUTO, SCAN_CUDA_CORE, SCAN_TC_SINGLE = 0, 1, 2
 STAGES = ("risk_select", "probe", "candidates", "resolve", "gather", "prep_miss", "scan", "merge",
           "rerank", "exact_pass", "scatter")
 _POLICY = {"lru": LRU, "fifo": FIFO, LRU: LRU, FIFO: FIFO}

@@ -172,12 +172,18 @@ def test_host_buffer_entry_point_equals_device_entry_point():
         assert np.array_equal(x, y)
 
 
-def test_cuda_core_scan_equals_default_scan():
-    X, Q = stream(9001, 768, 8, 200, 40, 1.1, 0.02, seed=10)
-    a = run_gpu(X.to(DEV), Q.to(DEV), 10, 30, 0.25, "lru", 64)
-    b = run_gpu(X.to(DEV), Q.to(DEV), 10, 30, 0.25, "lru", 64, scan_mode=prox.SCAN_CUDA_CORE)
-    for x, y in zip(a[:3], b[:3]):
-        assert np.array_equal(x, y)
+@pytest.mark.parametrize("d,batch", [(768, 64), (128, 256), (256, 24)])
+def test_the_three_scan_kernels_agree(d, batch):
+    """Two-block tensor-core scan (default), one-block tensor-core scan and CUDA-core scan."""
+    X, Q = stream(9001, d, 8, 520, 40, 1.1, 0.02, seed=10)
+    a = run_gpu(X.to(DEV), Q.to(DEV), 10, 30, 0.25, "lru", batch)
+    b = run_gpu(X.to(DEV), Q.to(DEV), 10, 30, 0.25, "lru", batch, scan_mode=prox.SCAN_CUDA_CORE)
+    c = run_gpu(X.to(DEV), Q.to(DEV), 10, 30, 0.25, "lru", batch, scan_mode=prox.SCAN_TC_SINGLE)
+    for x, y, z in zip(a[:3], b[:3], c[:3]):
+        assert np.array_equal(x, y) and np.array_equal(x, z)
+    ids, dists = oracle.exact_topk(X.numpy(), Q.numpy()[:40], 10)
+    miss = a[2][:40] == 0
+    assert np.array_equal(a[0][:40][miss], ids[miss])
 
 
 def test_reset_cache_and_argument_checks():
