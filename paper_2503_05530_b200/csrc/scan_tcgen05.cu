@@ -183,7 +183,6 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     const int s = g % stages;
                     const uint32_t ph = (g / stages) & 1u;
                     if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
                     const uint32_t a_addr = stage0 + s * stage_bytes;
                     const uint32_t b_addr = resident ? q_res0 + kc * b_tile_bytes : a_addr + kATileBytes;
                     const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(b_addr);
