@@ -49,6 +49,7 @@ struct ScanArgs {
     int32_t *buf_cnt;
     long long N;
     int d, pass, kp;
+    int ks;                 // 64-column groups per pipeline stage (1 or 2; the tensor maps' boxes match)
 };
 
 struct Control {
@@ -91,11 +92,13 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     const int q_rows = PAIR ? n_pad / 2 : n_pad;             // query rows this block stages (half of B in a pair)
     const CUtensorMap *tm_q = q_rows == 16 ? &tm_q16 : (q_rows == 32 ? &tm_q32 : (q_rows == 64 ? &tm_q64 : (q_rows == 128 ? &tm_q128 : &tm_q256)));
     const int q_row0 = q0 + (int)rank * q_rows;
-    const int nk = a.d / kChunkK;
+    const int nk = a.d / kChunkK;                            // 64-column groups of a row
+    const int ks = a.ks;                                     // column groups per stage (one barrier round trip)
+    const int nst = nk / ks;                                 // stages per tile
     const int b_tile_bytes = q_rows * 128;
     const int q_block_bytes = b_tile_bytes * nk;
     const bool resident = q_block_bytes <= kQResidentMax;
-    const int stage_bytes = resident ? kATileBytes : kATileBytes + b_tile_bytes;
+    const int stage_bytes = ks * (resident ? kATileBytes : kATileBytes + b_tile_bytes);
     int stages = (kTileRegion - (resident ? q_block_bytes : 0)) / stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
 
@@ -139,30 +142,30 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             const uint32_t q_full_bar = PAIR ? map_to_rank(smem_u32(&ctl.q_full), 0) : smem_u32(&ctl.q_full);
             if (resident) {
                 if (rank == 0) mbar_expect_tx(smem_u32(&ctl.q_full), tx_mult * (uint32_t)q_block_bytes);
-                for (int kc = 0; kc < nk; ++kc) {
-                    if constexpr (PAIR) tma_load_2d_pair(q_res0 + kc * b_tile_bytes, tm_q, kc * kChunkK, q_row0, q_full_bar);
-                    else tma_load_2d(q_res0 + kc * b_tile_bytes, tm_q, kc * kChunkK, q_row0, q_full_bar);
+                for (int st = 0; st < nst; ++st) {
+                    if constexpr (PAIR) tma_load_3d_pair(q_res0 + st * ks * b_tile_bytes, tm_q, 0, q_row0, st * ks, q_full_bar);
+                    else tma_load_3d(q_res0 + st * ks * b_tile_bytes, tm_q, 0, q_row0, st * ks, q_full_bar);
                 }
             }
             uint32_t g = 0;
             bool ok = true;
             for (long long tile = unit; ok && tile < ntiles; tile += n_units) {
                 const int row0 = (int)(tile * kUnitRows) + (int)rank * kTileRows;
-                for (int kc = 0; kc < nk; ++kc, ++g) {
+                for (int st = 0; st < nst; ++st, ++g) {
                     const int s = g % stages;
                     const uint32_t ph = (g / stages) & 1u;
                     if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t dst = stage0 + s * stage_bytes;
+                    const uint32_t dst = stage0 + s * stage_bytes;        // [ks corpus groups][ks query groups]
                     if constexpr (PAIR) {
                         const uint32_t fb = map_to_rank(smem_u32(&ctl.full[s]), 0);
                         if (rank == 0) mbar_expect_tx(smem_u32(&ctl.full[s]), 2u * (uint32_t)stage_bytes);
-                        tma_load_2d_pair(dst, &tm_x, kc * kChunkK, row0, fb);
-                        if (!resident) tma_load_2d_pair(dst + kATileBytes, tm_q, kc * kChunkK, q_row0, fb);
+                        tma_load_3d_pair(dst, &tm_x, 0, row0, st * ks, fb);
+                        if (!resident) tma_load_3d_pair(dst + ks * kATileBytes, tm_q, 0, q_row0, st * ks, fb);
                     } else {
                         const uint32_t fb = smem_u32(&ctl.full[s]);
                         mbar_expect_tx(fb, (uint32_t)stage_bytes);
-                        tma_load_2d(dst, &tm_x, kc * kChunkK, row0, fb);
-                        if (!resident) tma_load_2d(dst + kATileBytes, tm_q, kc * kChunkK, q_row0, fb);
+                        tma_load_3d(dst, &tm_x, 0, row0, st * ks, fb);
+                        if (!resident) tma_load_3d(dst + ks * kATileBytes, tm_q, 0, q_row0, st * ks, fb);
                     }
                 }
             }
@@ -179,17 +182,21 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 if (!mbar_wait(smem_u32(&ctl.tmem_empty[b]), bph ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + b * (uint32_t)kScanQ;
-                for (int kc = 0; kc < nk; ++kc, ++g) {
+                for (int st = 0; st < nst; ++st, ++g) {
                     const int s = g % stages;
                     const uint32_t ph = (g / stages) & 1u;
                     if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag)) { ok = false; break; }
                     const uint32_t a_addr = stage0 + s * stage_bytes;
-                    const uint32_t b_addr = resident ? q_res0 + kc * b_tile_bytes : a_addr + kATileBytes;
-                    const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(b_addr);
+                    const uint32_t b_addr = resident ? q_res0 + st * ks * b_tile_bytes : a_addr + ks * kATileBytes;
+                    for (int ka = 0; ka < ks; ++ka) {
+                        const uint64_t a_desc = smem_desc_sw128(a_addr + ka * kATileBytes);
+                        const uint64_t b_desc = smem_desc_sw128(b_addr + ka * b_tile_bytes);
 #pragma unroll
-                    for (int k4 = 0; k4 < kChunkK / 16; ++k4) {   // 16 bf16 = 32 bytes = 2 descriptor units
-                        if constexpr (PAIR) tc_mma_bf16_pair(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (kc | k4) ? 1u : 0u);
-                        else tc_mma_bf16(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (kc | k4) ? 1u : 0u);
+                        for (int k4 = 0; k4 < kChunkK / 16; ++k4) {   // 16 bf16 = 32 bytes = 2 descriptor units
+                            const uint32_t acc = (st | ka | k4) ? 1u : 0u;
+                            if constexpr (PAIR) tc_mma_bf16_pair(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, acc);
+                            else tc_mma_bf16(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, acc);
+                        }
                     }
                     // the stage is free (in both blocks of a pair) once these are done
                     if constexpr (PAIR) tc_commit_pair(smem_u32(&ctl.empty[s]));
@@ -378,20 +385,23 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+// A row-major bf16 matrix seen as (64-column group, row, column within the group): one box is
+// box_rows rows of ks neighbouring groups, landing in shared memory group after group.
+bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t ks) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * 2};
-    const cuuint32_t box[2] = {kChunkK, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+    const cuuint64_t dims[3] = {kChunkK, rows, cols / kChunkK};
+    const cuuint64_t strides[2] = {cols * 2, kChunkK * 2};
+    const cuuint32_t box[3] = {kChunkK, box_rows, ks};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 struct Maps {
     CUtensorMap x, q16, q32, q64, q128, q256;
+    int ks = 1;
     bool ok = false;
 };
 
@@ -406,12 +416,14 @@ int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s) {
         Maps *m = new (std::nothrow) Maps();
         if (!m) return 1;
         h->tc_state = m;
-        m->ok = make_map(&m->x, h->xb, (uint64_t)h->N, (uint64_t)h->d, kTileRows) &&
-                make_map(&m->q16, h->qb, kMaxBatch, (uint64_t)h->d, 16) &&
-                make_map(&m->q32, h->qb, kMaxBatch, (uint64_t)h->d, 32) &&
-                make_map(&m->q64, h->qb, kMaxBatch, (uint64_t)h->d, 64) &&
-                make_map(&m->q128, h->qb, kMaxBatch, (uint64_t)h->d, 128) &&
-                make_map(&m->q256, h->qb, kMaxBatch, (uint64_t)h->d, 256);
+        const uint32_t ks = ((h->d / kChunkK) % 2 == 0) ? 2 : 1;
+        m->ks = (int)ks;
+        m->ok = make_map(&m->x, h->xb, (uint64_t)h->N, (uint64_t)h->d, kTileRows, ks) &&
+                make_map(&m->q16, h->qb, kMaxBatch, (uint64_t)h->d, 16, ks) &&
+                make_map(&m->q32, h->qb, kMaxBatch, (uint64_t)h->d, 32, ks) &&
+                make_map(&m->q64, h->qb, kMaxBatch, (uint64_t)h->d, 64, ks) &&
+                make_map(&m->q128, h->qb, kMaxBatch, (uint64_t)h->d, 128, ks) &&
+                make_map(&m->q256, h->qb, kMaxBatch, (uint64_t)h->d, 256, ks);
         cudaFuncSetAttribute(scan_tc_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
         cudaFuncSetAttribute(scan_tc_kernel<512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
         cudaFuncSetAttribute(scan_tc_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
@@ -421,7 +433,7 @@ int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s) {
     if (!maps.ok) return 1;
     ScanArgs a;
     a.st = h->st; a.xh = h->xh; a.thr_g = h->thr_g; a.top1 = h->top1; a.buf = h->buf; a.buf_cnt = h->buf_cnt;
-    a.N = (long long)h->N; a.d = h->d; a.pass = pass; a.kp = h->kp;
+    a.N = (long long)h->N; a.d = h->d; a.pass = pass; a.kp = h->kp; a.ks = maps.ks;
     const bool pair = h->scan_mode != PROX_SCAN_TC_SINGLE && h->scan_ctas >= 2 && h->N >= 2 * kTileRows;
     const int grid = pair ? (h->scan_ctas & ~1) : h->scan_ctas;
     h->scan_lists = 4 * grid;                             // one candidate list per read-out lane quarter
