@@ -151,6 +151,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             bool ok = true;
             for (long long tile = unit; ok && tile < ntiles; tile += n_units) {
                 const int row0 = (int)(tile * kUnitRows) + (int)rank * kTileRows;
+                // the ring holds less than a tile, little to cover DRAM latency with: have the next
+                // tile's corpus rows brought into L2 while this one is consumed
+                if (tile + n_units < ntiles) {
+                    const int row_n = row0 + n_units * kUnitRows;
+                    for (int st = 0; st < nst; ++st) tma_prefetch_l2_3d(&tm_x, 0, row_n, st * ks);
+                }
                 for (int st = 0; st < nst; ++st, ++g) {
                     const int s = g % stages;
                     const uint32_t ph = (g / stages) & 1u;
