@@ -223,7 +223,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         const int P = gridDim.x;
         if (a.kp <= P && P <= 256) {
             volatile int *done = &ctl.done;
-            int jq = blockIdx.x;
+            int jq = blockIdx.x, jobs = 0;
             while (*done < kReadWarps && !*abort_flag) {
                 if (jq >= nq) jq = blockIdx.x;
                 if (jq < nq) {
@@ -241,7 +241,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     if (lane == 0 && (uint32_t)rth != 0u) atomicMax(&thr_g[jq], (uint32_t)rth);
                 }
                 jq += P;
-                __nanosleep(2000);
+                // bounds move fast while the first tiles come in and slowly afterwards; this warp
+                // shares an issue port with read-out warps, so it backs off once they have settled
+                __nanosleep(++jobs < 48 ? 2000 : 20000);
             }
         }
     } else if (warp >= 4) {
