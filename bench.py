@@ -392,7 +392,7 @@ def main():
     ap.add_argument("--rows", type=int, default=0, help="override the corpus size (profiling runs)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling runs)")
     ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--default-steps", type=int, default=200)
+    ap.add_argument("--default-steps", type=int, default=800, help="cap of the timed batches when --steps is 0 (a whole query stream if it is shorter)")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--stages", action="store_true", help="also print the time of every stage (one extra run)")

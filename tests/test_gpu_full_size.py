@@ -1,0 +1,91 @@
+"""Parity at the full sizes of the benchmark workloads, in the launch configuration bench.py times.
+
+The oracle cannot answer every miss at 24 million or 100 million rows, so the check is split the
+way the method allows: hit / miss decisions, matched keys and evictions depend on the query stream
+alone, so the oracle replays the whole prefix of the stream without a corpus and every flag is
+compared; a hit must return exactly the list of the miss that created its key (checked on the GPU
+output itself); and for a seeded sample of misses the oracle computes the exact k nearest rows from
+the corpus bytes copied off the device in chunks."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2503_05530_b200 import prox, workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+POL = {"lru": oracle.LRU, "fifo": oracle.FIFO}
+
+
+def run_full_size(cfg, tau, n_batches, n_samples, seed=0, chunk_rows=1 << 20):
+    need = cfg.N * cfg.d * 6 + (8 << 30)
+    free, _ = torch.cuda.mem_get_info()
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GB of device memory")
+    corpus = W.make_corpus(cfg.N, cfg.d, cfg.n_components, seed, DEV)
+    n = n_batches * cfg.batch
+    queries, _, _ = W.make_query_stream(corpus, n, cfg.n_topics, cfg.zipf_s, cfg.sigma, seed)
+    p = prox.Prox(corpus, cfg.k, cfg.capacity, tau, cfg.policy)
+    ids = torch.empty(n, cfg.k, dtype=torch.int64, device=DEV)
+    dists = torch.empty(n, cfg.k, dtype=torch.float32, device=DEV)
+    hit = torch.empty(n, dtype=torch.uint8, device=DEV)
+    for a in range(0, n, cfg.batch):
+        p.query_batch(queries[a:a + cfg.batch], ids[a:a + cfg.batch], dists[a:a + cfg.batch], hit[a:a + cfg.batch])
+    torch.cuda.synchronize()
+    assert p.status() == prox.OK, prox.last_error()
+    stats = p.stats()
+    p.close()
+    ids, dists, hit = ids.cpu().numpy(), dists.cpu().numpy(), hit.cpu().numpy()
+    Q = queries.cpu().numpy()
+
+    # 1. the cache trace of the whole prefix (needs no corpus)
+    o = oracle.Oracle(None, cfg.d, cfg.k, cfg.capacity, float(np.float32(tau)), POL[cfg.policy])
+    r = o.query(Q)
+    o.close()
+    assert np.array_equal(hit, r["hit"]), f"first differing flag at query {np.nonzero(hit != r['hit'])[0][0]}"
+    assert stats["hits"] == int(r["hit"].sum()) and stats["evictions"] == int((r["evicted"] >= 0).sum())
+    assert stats["unresolved"] == 0
+
+    # 2. a hit returns the list of the miss that made its key
+    hits = np.nonzero(r["hit"] == 1)[0]
+    for i in hits:
+        src = int(r["origin"][i])
+        assert np.array_equal(ids[i], ids[src]) and np.array_equal(dists[i], dists[src])
+
+    # 3. sampled misses against the oracle's exact top-k over the corpus bytes
+    misses = np.nonzero(r["hit"] == 0)[0]
+    rng = np.random.default_rng(seed)
+    sample = np.sort(rng.choice(misses, size=min(n_samples, len(misses)), replace=False))
+    tops = [oracle.ChunkedTopK(Q[i], cfg.k) for i in sample]
+    for r0 in range(0, cfg.N, chunk_rows):
+        chunk = corpus[r0:r0 + chunk_rows].cpu().numpy()
+        for t in tops:
+            t.feed(chunk)
+    for i, t in zip(sample, tops):
+        assert np.array_equal(ids[i], t.ids), f"ids differ at sampled miss {i}"
+        assert np.allclose(dists[i], t.dists, rtol=1e-4, atol=1e-12)
+        assert np.all(np.diff(dists[i]) >= 0)
+    # every miss list is sorted and made of valid, distinct rows
+    m_ids = ids[misses]
+    assert m_ids.min() >= 0 and m_ids.max() < cfg.N
+    assert all(len(set(row)) == cfg.k for row in m_ids[:: max(1, len(m_ids) // 500)])
+    return dict(hit_rate=float(r["hit"].mean()), stats=stats)
+
+
+def test_one_million_rows_batch64_lru_full_size():
+    cfg = W.CONFIGS["1m"]
+    res = run_full_size(cfg, 0.5, n_batches=100, n_samples=24)
+    assert 0.3 < res["hit_rate"] < 0.95 and res["stats"]["evictions"] > 0
+
+
+def test_24m_rows_batch256_lru_full_size():
+    cfg = W.CONFIGS["large"]
+    res = run_full_size(cfg, 1.0, n_batches=24, n_samples=6)
+    assert 0.2 < res["hit_rate"] < 0.95
+
+
+def test_100m_rows_d128_batch1024_fifo_full_size():
+    cfg = W.CONFIGS["lowhit"]
+    res = run_full_size(cfg, 0.3, n_batches=4, n_samples=6)
+    assert res["hit_rate"] < 0.5
