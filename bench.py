@@ -270,14 +270,18 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    misses = head["stats"]["misses"]
-    scan_batches = max(1, head["stats"]["scan_batches"])
-    scan_ms_per = head["scan_ms"] / max(1, head["scan_n"])
-    roof = roofline_of_scan(cfg, misses / scan_batches, scan_ms_per, peaks)
+    def scan_roofline(r):
+        """Roofline of the scan over the launches that had misses to scan (a launch takes up to 256 of them;
+        launches of batches without misses return at once and only add their few microseconds)."""
+        sb = max(1, r["stats"]["scan_batches"])
+        per_batch = r["stats"]["misses"] / sb
+        working = sb * max(1, -(-int(round(per_batch)) // 256))
+        return roofline_of_scan(cfg, r["stats"]["misses"] / working, r["scan_ms"] / working, peaks)
+
+    roof = scan_roofline(head)
     sweep = []
     for tau, r in results.items():
-        sb = max(1, r["stats"]["scan_batches"])
-        rf = roofline_of_scan(cfg, r["stats"]["misses"] / sb, r["scan_ms"] / max(1, r["scan_n"]), peaks)
+        rf = scan_roofline(r)
         sweep.append(dict(tau=tau, value=round(K * cfg.batch / (r["ms"] * 1e-3), 1), hit_rate=round(r["hit_rate"], 4),
                           ms_per_step=round(r["ms"] / K, 4), scan_frac_of_roofline=rf["frac"], scan_bound=rf["bound"],
                           scan_ms_per_launch=rf["ms_per_launch"], uncertified=r["stats"]["uncertified"],
@@ -381,13 +385,71 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_probe(args):
+    """Probe-only workload: a cache pre-filled with C keys, batches of 1024 queries (half near
+    random keys, half fresh mixture draws), tau = 0.5; times probe + resolve + key insertion
+    (prox_probe_batch) and reports GB/s of keys scanned per cache size and policy."""
+    from paper_2503_05530_b200 import prox
+    import __graft_entry__ as g
+    g.build()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    B, d, tau = 1024, 768, 0.5
+    K = args.steps if args.steps > 0 else 50
+    sizes = [c for c in W.PROBE_SIZES if c <= (args.rows or W.PROBE_SIZES[-1])]
+    fp64_peak = 148 * 64 * 1.965e9                      # DADD/DFMA issue slots per second (64 per SM and clock)
+    out = []
+    for C in sizes:
+        keys, centres = W.make_probe_keys(C, d, 4096, args.seed, dev)
+        batches = [W.make_probe_batch(keys, centres, B, 0.02, args.seed, b) for b in range(K + args.warmup)]
+        for policy in ("lru", "fifo"):
+            p = prox.Prox(keys[:64].contiguous(), 1, C, tau, policy)
+            p.cache_load(keys)
+            for q in batches[K:]:
+                p.probe_batch(q)
+            torch.cuda.synchronize()
+            p.cache_load(keys)
+            p.profile(None)
+            p.profile_read()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            hits = []
+            e0.record()
+            for q in batches[:K]:
+                hits.append(p.probe_batch(q)[0])
+            e1.record()
+            torch.cuda.synchronize()
+            prof = p.profile_read()
+            assert p.status() == prox.OK, prox.last_error()
+            ms = e0.elapsed_time(e1) / K
+            hit_rate = float(torch.stack(hits).float().mean().item())
+            key_bytes = C * d * 4
+            instr = 2.0 * B * C * d                     # one subtraction and one fused multiply-add per element
+            out.append(dict(C=C, policy=policy, us_per_batch=round(ms * 1e3, 1), keys_GBps=round(key_bytes / ms / 1e6, 1),
+                            hit_rate=round(hit_rate, 4), queries_per_s=round(B / ms * 1e3, 1),
+                            probe_us=round(prof["probe"][0] / K * 1e3, 1), resolve_us=round(prof["resolve"][0] / K * 1e3, 1),
+                            risk_select_us=round(prof["risk_select"][0] / K * 1e3, 1),
+                            frac_of_fp64_alu=round(instr / (prof["probe"][0] / K * 1e-3) / fp64_peak, 4)))
+            p.close()
+        del keys, batches
+    big = out[-1]
+    print(json.dumps(dict(metric="probe_keys_scanned", value=big["keys_GBps"], unit="GB/s", n_gpus=1, steps=K,
+                          warmup=args.warmup, ms_per_step=round(big["us_per_batch"] / 1e3, 4), higher_is_better=True,
+                          scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                          config=dict(workload=f"probe-only: B={B} d={d} tau={tau} keys from a 4096-component mixture, "
+                                               f"C={big['C']} policy={big['policy']}", l2="keys_exceed_l2" if big["C"] * d * 4 > 126e6 else "keys_fit_l2"),
+                          roofline=dict(bound="alu", achieved=round(big["frac_of_fp64_alu"] * fp64_peak / 1e12, 2),
+                                        peak=round(fp64_peak / 1e12, 2), unit="T fp64 instr/s", frac=big["frac_of_fp64_alu"],
+                                        traffic=None, kernel="probe_kernel"),
+                          points=out)), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=0, help="timed batches (0: a default that ends within minutes)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="auto", choices=["auto"] + list(W.CONFIGS))
+    ap.add_argument("--workload", default="auto", choices=["auto", "probe"] + list(W.CONFIGS))
     ap.add_argument("--tau", type=float, default=None, help="one tolerance instead of the workload's sweep")
     ap.add_argument("--rows", type=int, default=0, help="override the corpus size (profiling runs)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling runs)")
@@ -401,6 +463,8 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "probe":
+        run_probe(args)
     else:
         run_ours(args)
 
