@@ -136,6 +136,7 @@ typedef struct prox_stats {
     int64_t fallback_rows;              /* rows collected by the exact fp32 pass for those misses */
     int64_t unresolved;                 /* misses whose exact pass overflowed (result best effort) */
     int64_t count;                      /* |C| now */
+    int64_t probe_uncertified;          /* queries whose coarse (tensor-core) probe fell back to the exact fp64 probe */
 } prox_stats;
 
 /* prox_get_stats -- synchronises the stream, then copies the device counters to *out (HOST). */

@@ -100,8 +100,11 @@ risk_select_kernel(DevState *st, const u64 *__restrict__ stamp, int32_t *risk_po
 // ------------------------------------------------------------------------------------------
 // Probe: squared distances, in fp64 over the fp32 values and in difference form (so that a
 // bitwise duplicate is at distance exactly 0), from each query to every valid key and to
-// every earlier query of the batch.  Columns are [0, count) = slots, then [count, count+B) =
-// the batch itself.  Tile: 32 queries x 64 columns per block, d in chunks of 32.
+// every earlier query of the batch.  Tile: 32 queries x 64 columns per block, d in chunks of 32.
+//   mode 0  columns = slots [0, count) then the batch [count, count + B): everything in fp64.
+//   mode 1  columns = the R at-risk slots then the batch: what the resolve needs as full rows
+//           when the safe slots are handled by the coarse tensor-core probe.
+//   mode 2  queries = those the coarse probe could not certify (pfail_list), columns = slots.
 // ------------------------------------------------------------------------------------------
 constexpr int PQ = 32, PC = 64, PD = 32;
 
@@ -109,19 +112,28 @@ __global__ void __launch_bounds__(256)
 probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
              const float *__restrict__ queries, const int32_t *__restrict__ risk_pos, int B, int d,
              double *__restrict__ part_min, int32_t *__restrict__ part_arg,
-             double *__restrict__ d_risk, double *__restrict__ d_intra) {
+             double *__restrict__ d_risk, double *__restrict__ d_intra, int mode,
+             const int32_t *__restrict__ risk_slot, const int32_t *__restrict__ pfail_list) {
     __shared__ double qs[PQ][PD + 1];
     __shared__ double ks[PC][PD + 1];
+    __shared__ int q_index[PQ];
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
     const long long count = st->count;
-    const long long ncols = count + B;
+    const int R = st->n_risk;
+    const int nq = mode == 2 ? st->n_pfail : B;            // queries this launch serves
+    if ((int)blockIdx.x * PQ >= nq) return;
+    const long long nslot_cols = mode == 1 ? R : count;      // columns that are cached keys
+    const long long ncols = mode == 2 ? count : nslot_cols + B;
+    if (tid < PQ) {
+        const int r = blockIdx.x * PQ + tid;
+        q_index[tid] = r < nq ? (mode == 2 ? pfail_list[r] : r) : -1;
+    }
+    __syncthreads();
     const long long ntiles = (ncols + PC - 1) / PC;
     const int S = gridDim.y, sp = blockIdx.y;
     const long long per = (ntiles + S - 1) / S;
     const long long t_begin = sp * per;
     const long long t_end = (t_begin + per < ntiles) ? t_begin + per : ntiles;
-    const int q0 = blockIdx.x * PQ;
-
     double best_d[2] = {INFINITY, INFINITY};
     int best_s[2] = {0x7fffffff, 0x7fffffff};
 
@@ -138,8 +150,8 @@ probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
 #pragma unroll
             for (int it = 0; it < (PQ * PD) / 256; ++it) {
                 const int idx = it * 256 + tid, r = idx / PD, c = idx % PD;
-                const int qi = q0 + r;
-                qs[r][c] = (qi < B && kc + c < d) ? (double)queries[(size_t)qi * d + kc + c] : 0.0;
+                const int qi = q_index[r];
+                qs[r][c] = (qi >= 0 && kc + c < d) ? (double)queries[(size_t)qi * d + kc + c] : 0.0;
             }
 #pragma unroll
             for (int it = 0; it < (PC * PD) / 256; ++it) {
@@ -147,8 +159,8 @@ probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
                 const long long col = c0 + r;
                 double v = 0.0;
                 if (col < ncols && kc + c < d) {
-                    const float *src = (col < count) ? keys + (size_t)col * d
-                                                     : queries + (size_t)(col - count) * d;
+                    const float *src = (col >= nslot_cols) ? queries + (size_t)(col - nslot_cols) * d
+                                       : keys + (size_t)(mode == 1 ? risk_slot[col] : col) * d;
                     v = (double)src[kc + c];
                 }
                 ks[r][c] = v;
@@ -168,23 +180,23 @@ probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
         }
 #pragma unroll
         for (int a = 0; a < 2; ++a) {
-            const int i = q0 + ty * 2 + a;
-            if (i >= B) continue;
+            const int i = q_index[ty * 2 + a];
+            if (i < 0) continue;
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
                 const long long col = c0 + tx + 16 * b;
                 if (col >= ncols) continue;
                 const double v = acc[a][b];
-                if (col < count) {
-                    const int rp = risk_pos[col];
+                if (col < nslot_cols) {
+                    const int rp = mode == 1 ? (int)col : risk_pos[col];
                     if (rp >= 0) {
-                        d_risk[(size_t)i * kMaxBatch + rp] = v;
+                        if (mode != 2) d_risk[(size_t)i * kMaxBatch + rp] = v;
                     } else if (v < best_d[a] || (v == best_d[a] && (int)col < best_s[a])) {
                         best_d[a] = v;
                         best_s[a] = (int)col;
                     }
                 } else {
-                    const int j = (int)(col - count);
+                    const int j = (int)(col - nslot_cols);
                     if (j < i) d_intra[(size_t)i * kMaxBatch + j] = v;
                 }
             }
@@ -199,8 +211,8 @@ probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
             const int os = __shfl_xor_sync(0xffffffffu, best_s[a], m);
             if (od < best_d[a] || (od == best_d[a] && os < best_s[a])) { best_d[a] = od; best_s[a] = os; }
         }
-        const int i = q0 + ty * 2 + a;
-        if (tx == 0 && i < B) {
+        const int i = q_index[ty * 2 + a];
+        if (tx == 0 && i >= 0 && mode != 1) {
             part_min[(size_t)i * kProbeSplitMax + sp] = best_d[a];
             part_arg[(size_t)i * kProbeSplitMax + sp] = best_s[a];
         }
@@ -216,13 +228,13 @@ build_candidates_kernel(const DevState *__restrict__ st, int B, int S, double ta
                         const double *__restrict__ part_min, const int32_t *__restrict__ part_arg,
                         const double *__restrict__ d_risk, const double *__restrict__ d_intra,
                         double *safe_min, int32_t *safe_arg, double *cand_d, int32_t *cand_code,
-                        int32_t *n_cand) {
+                        int32_t *n_cand, const int32_t *__restrict__ use_partial) {
     __shared__ int s_n;
     const int i = blockIdx.x, tid = threadIdx.x;
     if (i >= B) return;
     if (tid == 0) s_n = 0;
     __syncthreads();
-    if (tid < 32) {
+    if (tid < 32 && (use_partial == nullptr || use_partial[i])) {   // else the coarse probe has set them
         double bd = INFINITY;
         int bs = 0x7fffffff;
         for (int s = tid; s < S; s += 32) {
@@ -510,7 +522,9 @@ __global__ void scatter_kernel(int B, int d, int k, int with_values, const float
                                const int32_t *__restrict__ miss_rank,
                                const int32_t *__restrict__ res_ids,
                                const double *__restrict__ res_dists, float *keys, int32_t *val_ids,
-                               float *val_dists, int64_t *out_ids, float *out_dists) {
+                               float *val_dists, int64_t *out_ids, float *out_dists, __nv_bfloat16 *keys_b,
+                               float *kh, DevState *st) {
+    __shared__ float red[2][4];
     const int i = blockIdx.x;
     if (i >= B) return;
     const int kind = src_kind[i];
@@ -524,11 +538,37 @@ __global__ void scatter_kernel(int B, int d, int k, int with_values, const float
     }
     const int slot = ins_slot[i];
     if (slot >= 0) {
-        for (int j = threadIdx.x; j < d; j += blockDim.x)
-            keys[(size_t)slot * d + j] = queries[(size_t)i * d + j];
+        float nn = 0.f, ee = 0.f;
+        for (int j = threadIdx.x; j < d; j += blockDim.x) {
+            const float v = queries[(size_t)i * d + j];
+            keys[(size_t)slot * d + j] = v;
+            if (keys_b) {                                 // bf16 copy for the coarse probe
+                const __nv_bfloat16 b = __float2bfloat16_rn(v);
+                const float f = __bfloat162float(b);
+                keys_b[(size_t)slot * d + j] = b;
+                nn += f * f;
+                ee += (v - f) * (v - f);
+            }
+        }
         for (int r = threadIdx.x; r < k; r += blockDim.x) {
             val_ids[(size_t)slot * k + r] = with_values ? res_ids[(size_t)m * k + r] : -1;
             val_dists[(size_t)slot * k + r] = with_values ? (float)res_dists[(size_t)m * k + r] : 0.f;
+        }
+        if (keys_b) {
+#pragma unroll
+            for (int sft = 16; sft > 0; sft >>= 1) {
+                nn += __shfl_xor_sync(0xffffffffu, nn, sft);
+                ee += __shfl_xor_sync(0xffffffffu, ee, sft);
+            }
+            if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = nn; red[1][threadIdx.x >> 5] = ee; }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                const float n2 = red[0][0] + red[0][1] + red[0][2] + red[0][3];
+                const float e2 = red[1][0] + red[1][1] + red[1][2] + red[1][3];
+                kh[slot] = 0.5f * n2;
+                atomicMax(reinterpret_cast<int *>(&st->ke_max), __float_as_int(sqrtf(e2) * 1.0001f));
+                atomicMax(reinterpret_cast<int *>(&st->kn_max), __float_as_int(sqrtf(n2) * 1.0001f));
+            }
         }
     }
 }
@@ -542,14 +582,18 @@ __global__ void copy_probe_outputs_kernel(int B, const int32_t *__restrict__ evt
     if (out_min_dist) out_min_dist[i] = evt_dist[i];
 }
 
-__global__ void reset_kernel(DevState *st, int32_t *risk_pos, long long C, long long n_loaded) {
+__global__ void reset_kernel(DevState *st, int32_t *risk_pos, long long C, long long n_loaded, float *kh) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < C) risk_pos[i] = -1;
+    if (i < C) {
+        risk_pos[i] = -1;
+        if (kh) kh[i] = INFINITY;                         // an empty slot can never pass the coarse probe
+    }
     if (i == 0) {
-        const float e_max = st->e_max;
+        const float e_max = st->e_max, xn_max = st->xn_max;
         const int err = st->error;
         *st = DevState{};
         st->e_max = e_max;
+        st->xn_max = xn_max;
         st->error = err;
         st->count = n_loaded;
         st->clock = n_loaded;
@@ -557,10 +601,39 @@ __global__ void reset_kernel(DevState *st, int32_t *risk_pos, long long C, long 
 }
 
 __global__ void cache_load_kernel(long long n, int d, int k, const float *__restrict__ src, float *keys,
-                                  int32_t *val_ids, float *val_dists, u64 *stamp) {
+                                  int32_t *val_ids, float *val_dists, u64 *stamp, __nv_bfloat16 *keys_b, float *kh,
+                                  DevState *st) {
+    __shared__ float red[2][4];
     const long long s = blockIdx.x;
     if (s >= n) return;
-    for (int j = threadIdx.x; j < d; j += blockDim.x) keys[(size_t)s * d + j] = src[(size_t)s * d + j];
+    float nn = 0.f, ee = 0.f;
+    for (int j = threadIdx.x; j < d; j += blockDim.x) {
+        const float v = src[(size_t)s * d + j];
+        keys[(size_t)s * d + j] = v;
+        if (keys_b) {
+            const __nv_bfloat16 b = __float2bfloat16_rn(v);
+            const float f = __bfloat162float(b);
+            keys_b[(size_t)s * d + j] = b;
+            nn += f * f;
+            ee += (v - f) * (v - f);
+        }
+    }
+    if (keys_b) {
+#pragma unroll
+        for (int sft = 16; sft > 0; sft >>= 1) {
+            nn += __shfl_xor_sync(0xffffffffu, nn, sft);
+            ee += __shfl_xor_sync(0xffffffffu, ee, sft);
+        }
+        if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = nn; red[1][threadIdx.x >> 5] = ee; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const float n2 = red[0][0] + red[0][1] + red[0][2] + red[0][3];
+            const float e2 = red[1][0] + red[1][1] + red[1][2] + red[1][3];
+            kh[s] = 0.5f * n2;
+            atomicMax(reinterpret_cast<int *>(&st->ke_max), __float_as_int(sqrtf(e2) * 1.0001f));
+            atomicMax(reinterpret_cast<int *>(&st->kn_max), __float_as_int(sqrtf(n2) * 1.0001f));
+        }
+    }
     for (int r = threadIdx.x; r < k; r += blockDim.x) {
         val_ids[(size_t)s * k + r] = -1;
         val_dists[(size_t)s * k + r] = 0.f;
@@ -587,17 +660,23 @@ void launch_risk_select(prox_handle *h, int B, cudaStream_t s) {
     h->launches++;
 }
 
-void launch_probe(prox_handle *h, const float *q, int B, cudaStream_t s) {
-    dim3 grid((B + PQ - 1) / PQ, probe_splits(h, B));
+void launch_probe(prox_handle *h, const float *q, int B, int mode, cudaStream_t s) {
+    int splits = probe_splits(h, B);
+    if (mode == 1) {                                      // at most 2 * kMaxBatch columns
+        const int tiles = (2 * B + PC - 1) / PC;
+        if (splits > tiles) splits = tiles;
+    }
+    dim3 grid((B + PQ - 1) / PQ, splits);
     probe_kernel<<<grid, 256, 0, s>>>(h->st, h->keys, q, h->risk_pos, B, h->d, h->part_min, h->part_arg,
-                                      h->d_risk, h->d_intra);
+                                      h->d_risk, h->d_intra, mode, h->risk_slot, h->pfail_list);
     h->launches++;
 }
 
 void launch_build_candidates(prox_handle *h, int B, cudaStream_t s) {
     build_candidates_kernel<<<B, 128, 0, s>>>(h->st, B, probe_splits(h, B), (double)h->tau, h->part_min,
                                               h->part_arg, h->d_risk, h->d_intra, h->safe_min,
-                                              h->safe_arg, h->cand_d, h->cand_code, h->n_cand);
+                                              h->safe_arg, h->cand_d, h->cand_code, h->n_cand,
+                                              h->probe_tc ? h->use_partial : nullptr);
     h->launches++;
 }
 
@@ -625,7 +704,8 @@ void launch_scatter(prox_handle *h, const float *q, int B, int64_t *out_ids, flo
                     int with_values, cudaStream_t s) {
     scatter_kernel<<<B, 128, 0, s>>>(B, h->d, h->k, with_values, q, h->src, h->src_kind, h->ins_slot,
                                      h->miss_rank, h->res_ids, h->res_dists, h->keys, h->val_ids,
-                                     h->val_dists, out_ids, out_dists);
+                                     h->val_dists, out_ids, out_dists, h->probe_tc ? h->keys_b : nullptr, h->kh,
+                                     h->st);
     h->launches++;
 }
 
@@ -637,17 +717,18 @@ void launch_probe_outputs(prox_handle *h, int B, int32_t *out_slot, float *out_m
 
 void launch_reset(prox_handle *h, cudaStream_t s) {
     const long long C = h->C;
-    reset_kernel<<<(unsigned)((C + 255) / 256), 256, 0, s>>>(h->st, h->risk_pos, C, 0);
+    reset_kernel<<<(unsigned)((C + 255) / 256), 256, 0, s>>>(h->st, h->risk_pos, C, 0, h->probe_tc ? h->kh : nullptr);
     h->launches++;
 }
 
 void launch_cache_load(prox_handle *h, const float *keys, int64_t n, cudaStream_t s) {
     const long long C = h->C;
-    reset_kernel<<<(unsigned)((C + 255) / 256), 256, 0, s>>>(h->st, h->risk_pos, C, (long long)n);
+    reset_kernel<<<(unsigned)((C + 255) / 256), 256, 0, s>>>(h->st, h->risk_pos, C, (long long)n, h->probe_tc ? h->kh : nullptr);
     h->launches++;
     if (n > 0) {
         cache_load_kernel<<<(unsigned)n, 128, 0, s>>>((long long)n, h->d, h->k, keys, h->keys, h->val_ids,
-                                                      h->val_dists, h->stamp);
+                                                      h->val_dists, h->stamp, h->probe_tc ? h->keys_b : nullptr,
+                                                      h->kh, h->st);
         h->launches++;
     }
 }

@@ -90,7 +90,8 @@ static void free_all(prox_handle *h) {
                     h->ins_slot, h->evt_slot, h->evt_dist, h->miss_list, h->miss_rank, h->qb, h->qbn,
                     h->qerr, h->thr_g, h->top1, h->buf, h->buf_cnt, h->cand_id, h->cand_score, h->cand_n,
                     h->cand_sk, h->res_ids, h->res_dists, h->fail_list, h->fail_radius, h->coll_id,
-                    h->coll_n, h->stage_q, h->stage_ids, h->stage_dists, h->stage_hit};
+                    h->coll_n, h->stage_q, h->stage_ids, h->stage_dists, h->stage_hit, h->keys_b, h->kh, h->pqb,
+                    h->pqbn, h->pqerr, h->use_partial, h->pfail_list};
     for (void *p : ptrs)
         if (p) cudaFree(p);
 }
@@ -159,6 +160,13 @@ extern "C" prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, i
     ok = ok && dev_alloc(h->res_ids, MB * k) && dev_alloc(h->res_dists, MB * k);
     ok = ok && dev_alloc(h->fail_list, MB) && dev_alloc(h->fail_radius, MB);
     ok = ok && dev_alloc(h->coll_id, MB * kCollectCap) && dev_alloc(h->coll_n, MB);
+    // caches of a few thousand keys and more are probed on the tensor cores first (bf16 copies of the keys)
+    h->probe_tc = (d % 64 == 0 && capacity >= 4096) ? 1 : 0;
+    ok = ok && dev_alloc(h->use_partial, MB) && dev_alloc(h->pfail_list, MB);
+    if (h->probe_tc) {
+        ok = ok && dev_alloc(h->keys_b, C * d) && dev_alloc(h->kh, C);
+        ok = ok && dev_alloc(h->pqb, MB * d) && dev_alloc(h->pqbn, MB) && dev_alloc(h->pqerr, MB);
+    }
     ok = ok && dev_alloc(h->stage_q, MB * d) && dev_alloc(h->stage_ids, MB * k);
     ok = ok && dev_alloc(h->stage_dists, MB * k) && dev_alloc(h->stage_hit, MB);
     if (!ok) {
@@ -169,6 +177,10 @@ extern "C" prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, i
     }
     cudaMemset(h->st, 0, sizeof(DevState));
     cudaMemset(h->qb, 0, MB * d * sizeof(__nv_bfloat16));
+    if (h->probe_tc) {
+        cudaMemset(h->pqb, 0, MB * d * sizeof(__nv_bfloat16));
+        cudaMemset(h->keys_b, 0, C * d * sizeof(__nv_bfloat16));
+    }
     cudaMemset(h->buf_cnt, 0, 4 * P * kScanQ * sizeof(int32_t));
     launch_convert_corpus(h, 0);
     launch_reset(h, 0);
@@ -202,7 +214,28 @@ static int check_batch_args(prox_handle *h, const void *queries, int32_t B) {
 static void enqueue_probe_and_resolve(prox_handle *h, const float *queries, int32_t B, uint8_t *out_hit,
                                       cudaStream_t s) {
     { StageScope t(h, PROX_STAGE_RISK_SELECT, s); launch_risk_select(h, B, s); }
-    { StageScope t(h, PROX_STAGE_PROBE, s); launch_probe(h, queries, B, s); }
+    {
+        StageScope t(h, PROX_STAGE_PROBE, s);
+        bool coarse = h->probe_tc && h->scan_mode != PROX_SCAN_CUDA_CORE;
+        if (coarse) {
+            // safe slots: coarse scores on the tensor cores, exact recheck of the best few;
+            // at-risk slots and the batch itself: full fp64 rows; uncertified queries: fp64 over all slots
+            launch_prep_probe(h, queries, B, s);
+            const int passes = (B + kScanQ - 1) / kScanQ;
+            for (int p = 0; p < passes && coarse; ++p) {
+                if (launch_probe_scan_tc(h, p, s) != 0) { coarse = false; break; }
+                launch_merge_select(h, p, B, 1, s);
+            }
+        }
+        if (coarse) {
+            launch_probe_exact(h, queries, B, s);
+            launch_probe(h, queries, B, 1, s);
+            launch_probe(h, queries, B, 2, s);
+        } else {
+            if (h->probe_tc) cudaMemsetAsync(h->use_partial, 0xff, sizeof(int32_t) * kMaxBatch, s);   // all from partials
+            launch_probe(h, queries, B, 0, s);
+        }
+    }
     { StageScope t(h, PROX_STAGE_CANDIDATES, s); launch_build_candidates(h, B, s); }
     { StageScope t(h, PROX_STAGE_RESOLVE, s); launch_resolve(h, B, out_hit, s); }
 }
@@ -223,7 +256,7 @@ extern "C" int32_t prox_query_batch(prox_handle *h, const float *queries, int32_
             StageScope t(h, PROX_STAGE_SCAN, s);
             if (h->scan_mode == PROX_SCAN_CUDA_CORE || launch_scan_pass_tc(h, p, s) != 0) launch_scan_pass(h, p, s);
         }
-        { StageScope t(h, PROX_STAGE_MERGE, s); launch_merge_select(h, p, B, s); }
+        { StageScope t(h, PROX_STAGE_MERGE, s); launch_merge_select(h, p, B, 0, s); }
     }
     { StageScope t(h, PROX_STAGE_RERANK, s); launch_rerank(h, queries, B, s); }
     { StageScope t(h, PROX_STAGE_EXACT_PASS, s); launch_fallback(h, queries, B, s); }
@@ -294,6 +327,7 @@ extern "C" int32_t prox_get_stats(prox_handle *h, prox_stats *out, void *stream)
     out->intra_batch_hits = st.intra_hits; out->evictions = st.evictions;
     out->scan_batches = st.scan_batches; out->uncertified = st.uncertified;
     out->fallback_rows = st.fallback_rows; out->unresolved = st.unresolved; out->count = st.count;
+    out->probe_uncertified = st.probe_uncertified;
     return PROX_OK;
 }
 

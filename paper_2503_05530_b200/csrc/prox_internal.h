@@ -16,6 +16,7 @@ constexpr int kTileRows = 128;               // corpus rows per scan tile (MMA M
 constexpr int kBufCap = 512;                 // entries of one (CTA, query) candidate buffer
 constexpr int kCollectCap = 2048;            // rows the exact pass may collect per query
 constexpr int kProbeSplitMax = 64;           // column splits of the probe grid
+constexpr int kProbeKp = 64;                 // slots per query the coarse probe keeps for the exact recheck
 
 // Device-resident scalars of a handle.
 struct DevState {
@@ -27,9 +28,13 @@ struct DevState {
     int error;                // latched PROX_ERR_* found on the device
     float e_max;              // upper bound of |x - bf16(x)| over corpus rows
     float xn_max;             // upper bound of |bf16(x)| over corpus rows
+    float ke_max;             // upper bound of |key - bf16(key)| over the keys inserted since the last reset
+    float kn_max;             // upper bound of |bf16(key)| over those keys
+    int n_probe;              // queries of the current batch (read by the coarse probe's kernels)
+    int n_pfail;              // queries whose coarse probe was not certified
     // statistics
     long long queries, hits, misses, intra_hits, evictions, scan_batches, uncertified,
-        fallback_rows, unresolved;
+        fallback_rows, unresolved, probe_uncertified;
 };
 
 struct Profiler;
@@ -60,6 +65,8 @@ struct prox_handle {
     float *val_dists;         // C x k
     unsigned long long *stamp;  // C
     int32_t *risk_pos;        // C: position in the at-risk list or -1
+    __nv_bfloat16 *keys_b;    // C x d: bf16 copies of the keys for the tensor-core probe
+    float *kh;                // C: 0.5 * |bf16(key)|^2, +inf for an empty slot
     prox::DevState *st;
 
     // per-batch scratch
@@ -79,6 +86,13 @@ struct prox_handle {
     int32_t *ins_slot;                // kMaxBatch: slot written at batch end or -1
     int32_t *evt_slot;                // kMaxBatch: matched / written slot at the time of the lookup
     float *evt_dist;                  // kMaxBatch: distance to the matched key (+inf on a miss)
+    __nv_bfloat16 *pqb;               // kMaxBatch x d: bf16 copies of all batch queries (coarse probe)
+    float *pqbn;                      // kMaxBatch: |bf16(q)|^2
+    float *pqerr;                     // kMaxBatch: upper bound of |q - bf16(q)|
+    int32_t *use_partial;             // kMaxBatch: 1 = the safe minimum comes from the fp64 probe's partial minima
+    int32_t *pfail_list;              // kMaxBatch: queries that take the exact fp64 probe
+    int32_t probe_tc;                 // 1 = coarse tensor-core probe in use for this handle
+    void *tc_state_keys;              // tensor maps of the coarse probe
     int32_t *miss_list;               // kMaxBatch
     int32_t *miss_rank;               // kMaxBatch
 
@@ -116,7 +130,7 @@ namespace prox {
 void launch_convert_corpus(prox_handle *h, cudaStream_t s);
 // cache kernels
 void launch_risk_select(prox_handle *h, int B, cudaStream_t s);
-void launch_probe(prox_handle *h, const float *q, int B, cudaStream_t s);
+void launch_probe(prox_handle *h, const float *q, int B, int mode, cudaStream_t s);   // 0 all slots, 1 at-risk + batch, 2 failed queries
 void launch_build_candidates(prox_handle *h, int B, cudaStream_t s);
 void launch_resolve(prox_handle *h, int B, uint8_t *out_hit, cudaStream_t s);
 void launch_gather_hits(prox_handle *h, int B, int64_t *out_ids, float *out_dists, cudaStream_t s);
@@ -127,10 +141,13 @@ void launch_cache_load(prox_handle *h, const float *keys, int64_t n, cudaStream_
 void launch_reset(prox_handle *h, cudaStream_t s);
 // scan kernels
 void launch_prep_miss(prox_handle *h, const float *q, int B, cudaStream_t s);
+void launch_prep_probe(prox_handle *h, const float *q, int B, cudaStream_t s);
+int launch_probe_scan_tc(prox_handle *h, int pass, cudaStream_t s);    // coarse probe over the bf16 keys; nonzero = not available
+void launch_probe_exact(prox_handle *h, const float *q, int B, cudaStream_t s);
 void launch_scan_pass(prox_handle *h, int pass, cudaStream_t s);       // CUDA-core scan
 int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s);     // tcgen05 scan; nonzero = not available
 void free_scan_tc(prox_handle *h);
-void launch_merge_select(prox_handle *h, int pass, int B, cudaStream_t s);
+void launch_merge_select(prox_handle *h, int pass, int B, int for_probe, cudaStream_t s);
 void launch_rerank(prox_handle *h, const float *q, int B, cudaStream_t s);
 void launch_fallback(prox_handle *h, const float *q, int B, cudaStream_t s);
 }  // namespace prox

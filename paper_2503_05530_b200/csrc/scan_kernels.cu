@@ -133,7 +133,7 @@ scan_cc_kernel(const DevState *__restrict__ st, const __nv_bfloat16 *__restrict_
     __shared__ float qs[64][33];
     __shared__ float thr[kScanQ];
     __shared__ int cnt[kScanQ];
-    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4, warp = tid >> 5;
     const int q0 = pass * kScanQ;
     int nq = st->n_miss - q0;
     if (nq > kScanQ) nq = kScanQ;
@@ -237,7 +237,7 @@ struct MergeSrc {
 };
 
 __global__ void __launch_bounds__(1024)
-merge_select_kernel(const DevState *__restrict__ st, int pass, int n_lists, int stride, int kp,
+merge_select_kernel(const int *__restrict__ n_active, int pass, int n_lists, int stride, int kp,
                     const u64 *__restrict__ buf, const int32_t *__restrict__ buf_cnt, int32_t *cand_id,
                     float *cand_score, int32_t *cand_n, float *cand_sk) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -247,7 +247,7 @@ merge_select_kernel(const DevState *__restrict__ st, int pass, int n_lists, int 
     __shared__ int s_remaining, s_total, s_gt, s_eq;
     const int q = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m = pass * kScanQ + q;
-    if (m >= st->n_miss) return;
+    if (m >= *n_active) return;
 
     if (tid == 0) { s_total = 0; s_gt = 0; s_eq = 0; }
     __syncthreads();
@@ -487,6 +487,104 @@ fallback_collect_kernel(DevState *st, const float *__restrict__ corpus, const fl
 }
 
 // ------------------------------------------------------------------------------------------
+// Coarse tensor-core probe (Algorithm 1, lines 2-3, for large caches): the scan kernel run over
+// the bf16 copies of the keys gives, per query, the kProbeKp slots with the best coarse scores;
+// here their exact fp64 distances give the nearest safe slot, with the same kind of
+// certificate as the corpus scan.  At-risk slots are left out (the fp64 probe measures them as
+// full rows).  Only a safe minimum within tau matters to the resolve, so a query is settled if
+//   - every valid slot was a candidate, or
+//   - the best safe candidate is nearer than any slot outside the candidates can be, or
+//   - no slot outside the candidates can be within tau.
+// Otherwise the query is handed to the exact fp64 probe over all slots.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+prep_probe_kernel(DevState *st, const float *__restrict__ queries, int B, int d, __nv_bfloat16 *pqb, float *pqbn,
+                  float *pqerr, uint32_t *thr_g, uint32_t *top1, int n_blocks, int32_t *use_partial) {
+    __shared__ float red[2][4];
+    const int m = blockIdx.x, tid = threadIdx.x;
+    if (m == 0) {
+        for (int i = tid; i < kMaxBatch; i += blockDim.x) thr_g[i] = f2o(-INFINITY);
+        if (tid == 0) { st->n_probe = B; st->n_pfail = 0; }
+    }
+    for (int i = tid; i < n_blocks; i += blockDim.x) top1[(size_t)m * n_blocks + i] = 0u;
+    if (m >= B) {
+        for (int j = tid; j < d; j += blockDim.x) pqb[(size_t)m * d + j] = __float2bfloat16_rn(0.f);
+        return;
+    }
+    if (tid == 0) use_partial[m] = 0;
+    const float *src = queries + (size_t)m * d;
+    float nn = 0.f, ee = 0.f;
+    for (int j = tid; j < d; j += blockDim.x) {
+        const float v = src[j];
+        const __nv_bfloat16 b = __float2bfloat16_rn(v);
+        const float f = __bfloat162float(b);
+        pqb[(size_t)m * d + j] = b;
+        nn += f * f;
+        ee += (v - f) * (v - f);
+    }
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) {
+        nn += __shfl_xor_sync(0xffffffffu, nn, s);
+        ee += __shfl_xor_sync(0xffffffffu, ee, s);
+    }
+    if ((tid & 31) == 0) { red[0][tid >> 5] = nn; red[1][tid >> 5] = ee; }
+    __syncthreads();
+    if (tid == 0) {
+        pqbn[m] = red[0][0] + red[0][1] + red[0][2] + red[0][3];
+        pqerr[m] = sqrtf(red[1][0] + red[1][1] + red[1][2] + red[1][3]) * 1.0001f;
+    }
+}
+
+__global__ void __launch_bounds__(128)
+probe_exact_kernel(DevState *st, const float *__restrict__ keys, const float *__restrict__ queries, int B, int d,
+                   double tau, const int32_t *__restrict__ risk_pos, const int32_t *__restrict__ cand_id,
+                   const int32_t *__restrict__ cand_n, const float *__restrict__ cand_sk,
+                   const float *__restrict__ pqbn, const float *__restrict__ pqerr, double *safe_min,
+                   int32_t *safe_arg, int32_t *use_partial, int32_t *pfail_list) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *q_sm = reinterpret_cast<float *>(smem_raw);
+    __shared__ double w_d[4];
+    __shared__ int w_s[4];
+    const int i = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (i >= B) return;
+    for (int j = tid; j < d; j += blockDim.x) q_sm[j] = queries[(size_t)i * d + j];
+    __syncthreads();
+    const int n = cand_n[i];
+    double bd = INFINITY;
+    int bs = 0x7fffffff;
+    for (int c = warp; c < n; c += 4) {
+        const int slot = cand_id[(size_t)i * kMaxKp + c];
+        if (risk_pos[slot] >= 0) continue;                        // measured as a full row by the fp64 probe
+        const double v = exact_sqdist_warp(q_sm, keys + (size_t)slot * d, d);
+        if (v < bd || (v == bd && slot < bs)) { bd = v; bs = slot; }
+    }
+    if (lane == 0) { w_d[warp] = bd; w_s[warp] = bs; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < 4; ++w)
+            if (w_d[w] < bd || (w_d[w] == bd && w_s[w] < bs)) { bd = w_d[w]; bs = w_s[w]; }
+        const float sk = cand_sk[i];
+        bool settled = true;
+        if (sk != -INFINITY) {                                    // slots outside the candidate set exist
+            const double qn = sqrt((double)pqbn[i]), kn = (double)st->kn_max;
+            const double slack = 4.0 * (double)(d + 16) * 5.9604644775390625e-08 * (2.0 * qn * kn + kn * kn + qn * qn);
+            const double cprime = (double)pqbn[i] - 2.0 * (double)sk - slack;
+            const double g = (double)pqerr[i] + (double)st->ke_max;
+            const double root = cprime > 0.0 ? sqrt(cprime) : 0.0;
+            const double lower = root > g ? (root - g) * (root - g) : 0.0;    // no outside slot is nearer than this
+            settled = (bd < lower) || (lower > tau);
+        }
+        safe_min[i] = bd;
+        safe_arg[i] = (bs == 0x7fffffff) ? -1 : bs;
+        if (!settled) {
+            use_partial[i] = 1;
+            pfail_list[atomicAdd(&st->n_pfail, 1)] = i;
+            atomicAdd((u64 *)&st->probe_uncertified, 1ull);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // Launchers
 // ------------------------------------------------------------------------------------------
 void launch_convert_corpus(prox_handle *h, cudaStream_t s) {
@@ -511,7 +609,7 @@ void launch_scan_pass(prox_handle *h, int pass, cudaStream_t s) {
     h->launches++;
 }
 
-void launch_merge_select(prox_handle *h, int pass, int B, cudaStream_t s) {
+void launch_merge_select(prox_handle *h, int pass, int B, int for_probe, cudaStream_t s) {
     int nq = B - pass * kScanQ;
     if (nq > kScanQ) nq = kScanQ;
     if (nq <= 0) return;
@@ -520,7 +618,8 @@ void launch_merge_select(prox_handle *h, int pass, int B, cudaStream_t s) {
         cudaFuncSetAttribute(merge_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeStage * 8);
         attr_set = true;
     }
-    merge_select_kernel<<<nq, 1024, kMergeStage * 8, s>>>(h->st, pass, h->scan_lists, h->scan_list_stride, h->kp,
+    merge_select_kernel<<<nq, 1024, kMergeStage * 8, s>>>(for_probe ? &h->st->n_probe : &h->st->n_miss, pass,
+                                                          h->scan_lists, h->scan_list_stride, for_probe ? kProbeKp : h->kp,
                                                           h->buf, h->buf_cnt, h->cand_id, h->cand_score, h->cand_n,
                                                           h->cand_sk);
     h->launches++;
@@ -556,4 +655,21 @@ void launch_fallback(prox_handle *h, const float *q, int B, cudaStream_t s) {
     h->launches++;
 }
 
+}  // namespace prox
+
+namespace prox {
+void launch_prep_probe(prox_handle *h, const float *q, int B, cudaStream_t s) {
+    int rows = ((B + kScanQ - 1) / kScanQ) * kScanQ;
+    if (rows > kMaxBatch) rows = kMaxBatch;
+    prep_probe_kernel<<<rows, 128, 0, s>>>(h->st, q, B, h->d, h->pqb, h->pqbn, h->pqerr, h->thr_g, h->top1,
+                                           h->scan_ctas, h->use_partial);
+    h->launches++;
+}
+
+void launch_probe_exact(prox_handle *h, const float *q, int B, cudaStream_t s) {
+    probe_exact_kernel<<<B, 128, (size_t)h->d * 4, s>>>(h->st, h->keys, q, B, h->d, (double)h->tau, h->risk_pos,
+                                                         h->cand_id, h->cand_n, h->cand_sk, h->pqbn, h->pqerr,
+                                                         h->safe_min, h->safe_arg, h->use_partial, h->pfail_list);
+    h->launches++;
+}
 }  // namespace prox

@@ -42,6 +42,7 @@ constexpr int kTmemCols = 512;
 
 struct ScanArgs {
     DevState *st;
+    const int *n_active;    // device: how many queries the whole call serves (misses, or the batch for the probe)
     const float *xh;
     uint32_t *thr_g;
     uint32_t *top1;
@@ -85,7 +86,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     constexpr int kUnitRows = PAIR ? 2 * kTileRows : kTileRows;            // corpus rows per tile of a unit
 
     const int q0 = a.pass * kScanQ;
-    int nq = a.st->n_miss - q0;
+    int nq = *a.n_active - q0;
     if (nq > kScanQ) nq = kScanQ;
     if (nq <= 0) return;                                  // nothing missed in this pass
     const int n_pad = nq <= 32 ? 32 : (nq <= 64 ? 64 : (nq <= 128 ? 128 : 256));
@@ -415,34 +416,34 @@ struct Maps {
 
 }  // namespace
 
-// Returns nonzero when the tensor-core path cannot take this handle (d not a multiple of 64,
-// fewer corpus rows than one tile, or no tensor-map encoder in the driver); the caller then
-// runs the CUDA-core scan.
-int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s) {
-    if (h->d % kChunkK || h->N < kTileRows) return 1;
-    if (!h->tc_state) {
+// One pass of the tensor-core scan of `rows` bf16 rows (xb, half norms xh) against the bf16 query
+// block qb.  Returns nonzero when the tensor-core path cannot run (no tensor-map encoder in the
+// driver, out of memory for the maps); the caller then falls back.
+static int launch_scan_generic(prox_handle *h, void **state, const __nv_bfloat16 *xb, const float *xh, long long rows,
+                               const __nv_bfloat16 *qb, const int *n_active, int kp, int pass, cudaStream_t s) {
+    if (!*state) {
         Maps *m = new (std::nothrow) Maps();
         if (!m) return 1;
-        h->tc_state = m;
+        *state = m;
         const uint32_t ks = ((h->d / kChunkK) % 2 == 0) ? 2 : 1;
         m->ks = (int)ks;
-        m->ok = make_map(&m->x, h->xb, (uint64_t)h->N, (uint64_t)h->d, kTileRows, ks) &&
-                make_map(&m->q16, h->qb, kMaxBatch, (uint64_t)h->d, 16, ks) &&
-                make_map(&m->q32, h->qb, kMaxBatch, (uint64_t)h->d, 32, ks) &&
-                make_map(&m->q64, h->qb, kMaxBatch, (uint64_t)h->d, 64, ks) &&
-                make_map(&m->q128, h->qb, kMaxBatch, (uint64_t)h->d, 128, ks) &&
-                make_map(&m->q256, h->qb, kMaxBatch, (uint64_t)h->d, 256, ks);
+        m->ok = make_map(&m->x, xb, (uint64_t)rows, (uint64_t)h->d, kTileRows, ks) &&
+                make_map(&m->q16, qb, kMaxBatch, (uint64_t)h->d, 16, ks) &&
+                make_map(&m->q32, qb, kMaxBatch, (uint64_t)h->d, 32, ks) &&
+                make_map(&m->q64, qb, kMaxBatch, (uint64_t)h->d, 64, ks) &&
+                make_map(&m->q128, qb, kMaxBatch, (uint64_t)h->d, 128, ks) &&
+                make_map(&m->q256, qb, kMaxBatch, (uint64_t)h->d, 256, ks);
         cudaFuncSetAttribute(scan_tc_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
         cudaFuncSetAttribute(scan_tc_kernel<512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
         cudaFuncSetAttribute(scan_tc_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
         cudaFuncSetAttribute(scan_tc_kernel<512, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
     }
-    Maps &maps = *static_cast<Maps *>(h->tc_state);
+    Maps &maps = *static_cast<Maps *>(*state);
     if (!maps.ok) return 1;
     ScanArgs a;
-    a.st = h->st; a.xh = h->xh; a.thr_g = h->thr_g; a.top1 = h->top1; a.buf = h->buf; a.buf_cnt = h->buf_cnt;
-    a.N = (long long)h->N; a.d = h->d; a.pass = pass; a.kp = h->kp; a.ks = maps.ks;
-    const bool pair = h->scan_mode != PROX_SCAN_TC_SINGLE && h->scan_ctas >= 2 && h->N >= 2 * kTileRows;
+    a.st = h->st; a.n_active = n_active; a.xh = xh; a.thr_g = h->thr_g; a.top1 = h->top1; a.buf = h->buf;
+    a.buf_cnt = h->buf_cnt; a.N = rows; a.d = h->d; a.pass = pass; a.kp = kp; a.ks = maps.ks;
+    const bool pair = h->scan_mode != PROX_SCAN_TC_SINGLE && h->scan_ctas >= 2 && rows >= 2 * kTileRows;
     const int grid = pair ? (h->scan_ctas & ~1) : h->scan_ctas;
     h->scan_lists = 4 * grid;                             // one candidate list per read-out lane quarter
     h->scan_list_stride = h->tc_cap;
@@ -465,14 +466,30 @@ int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s) {
     else
         e = h->tc_cap == 256 ? cudaLaunchKernelEx(&cfg, scan_tc_kernel<256, false>, maps.x, maps.q16, maps.q32, maps.q64, maps.q128, maps.q256, a)
                              : cudaLaunchKernelEx(&cfg, scan_tc_kernel<512, false>, maps.x, maps.q16, maps.q32, maps.q64, maps.q128, maps.q256, a);
-    if (e != cudaSuccess) return 1;                       // the caller falls back to the CUDA-core scan
+    if (e != cudaSuccess) return 1;
     h->launches++;
     return 0;
+}
+
+// The corpus scan of the misses.  Nonzero: the handle cannot take the tensor-core path (d not a
+// multiple of 64, fewer corpus rows than one tile); the caller then runs the CUDA-core scan.
+int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s) {
+    if (h->d % kChunkK || h->N < kTileRows) return 1;
+    return launch_scan_generic(h, &h->tc_state, h->xb, h->xh, (long long)h->N, h->qb, &h->st->n_miss, h->kp, pass, s);
+}
+
+// The coarse probe: the same scan over the bf16 copies of the cached keys, all batch queries,
+// keeping the kProbeKp best slots per query.
+int launch_probe_scan_tc(prox_handle *h, int pass, cudaStream_t s) {
+    return launch_scan_generic(h, &h->tc_state_keys, h->keys_b, h->kh, (long long)h->C, h->pqb, &h->st->n_probe,
+                               kProbeKp, pass, s);
 }
 
 void free_scan_tc(prox_handle *h) {
     delete static_cast<Maps *>(h->tc_state);
     h->tc_state = nullptr;
+    delete static_cast<Maps *>(h->tc_state_keys);
+    h->tc_state_keys = nullptr;
 }
 
 }  // namespace prox

@@ -143,11 +143,12 @@ def test_uncertified_queries_take_the_exact_pass():
 
 # ------------------------------------------------------------------ probe only, pre-filled cache
 @pytest.mark.parametrize("policy", ["lru", "fifo"])
-def test_probe_only_prefilled_cache(policy):
-    keys, centres = W.make_probe_keys(3000, 768, 4096, seed=8)
-    p = prox.Prox(keys[:64].contiguous().to(DEV), 1, 3000, 0.5, policy)
+@pytest.mark.parametrize("n_keys", [3000, 6000])        # fp64 probe / coarse tensor-core probe with exact recheck
+def test_probe_only_prefilled_cache(policy, n_keys):
+    keys, centres = W.make_probe_keys(n_keys, 768, 4096, seed=8)
+    p = prox.Prox(keys[:64].contiguous().to(DEV), 1, n_keys, 0.5, policy)
     p.cache_load(keys.to(DEV))
-    o = oracle.Oracle(None, 768, 1, 3000, float(np.float32(0.5)), oracle.LRU if policy == "lru" else oracle.FIFO)
+    o = oracle.Oracle(None, 768, 1, n_keys, float(np.float32(0.5)), oracle.LRU if policy == "lru" else oracle.FIFO)
     o.cache_load(keys.numpy())
     for b in range(3):
         Q = W.make_probe_batch(keys, centres, 1024, 0.02, 8, b)
@@ -161,6 +162,55 @@ def test_probe_only_prefilled_cache(policy):
         assert 0.3 < r["hit"].mean() < 0.9
     assert p.status() == prox.OK
     p.close()
+
+
+def test_large_cache_stream_with_coarse_probe():
+    """Capacity above the switch-over to the tensor-core probe, pre-filled and full, so that the
+    stream evicts from its first miss on; lists of pre-filled keys are the empty ones on both sides."""
+    X, Q = stream(20011, 256, 64, 1600, 500, 1.0, 0.03, seed=13)
+    keys = torch.cat([Q[800:], W.make_corpus(4400, 256, 64, seed=14)]).contiguous()     # some keys near later queries
+    Qs = Q[:800].contiguous()
+    k, cap, tau = 10, keys.shape[0], 0.5
+    p = prox.Prox(X.to(DEV), k, cap, tau, "lru")
+    p.cache_load(keys.to(DEV))
+    outs = [p.query_batch(Qs[a:a + 256].to(DEV)) for a in range(0, 800, 256)]
+    torch.cuda.synchronize()
+    assert p.status() == prox.OK
+    st = p.stats()
+    p.close()
+    ids = torch.cat([o_[0] for o_ in outs]).cpu().numpy()
+    dists = torch.cat([o_[1] for o_ in outs]).cpu().numpy()
+    hit = torch.cat([o_[2] for o_ in outs]).cpu().numpy()
+    o = oracle.Oracle(X.numpy(), 256, k, cap, float(np.float32(tau)), oracle.LRU)
+    o.cache_load(keys.numpy())
+    r = o.query(Qs.numpy())
+    assert np.array_equal(hit, r["hit"]) and 0.1 < r["hit"].mean() < 0.95
+    assert np.array_equal(ids, r["ids"])
+    assert np.allclose(dists, r["dists"], rtol=1e-4, atol=1e-12)
+    assert st["evictions"] == int((r["evicted"] >= 0).sum()) > 0
+
+
+def test_coarse_probe_hands_tight_clusters_to_the_exact_probe():
+    g = torch.Generator().manual_seed(17)
+    c = torch.randn(128, generator=g)
+    keys = c + 3e-4 * torch.randn(5000, 128, generator=g)
+    keys = (keys / keys.norm(dim=1, keepdim=True)).contiguous()
+    Q = keys[:300] + 1e-4 * torch.randn(300, 128, generator=g)
+    Q = (Q / Q.norm(dim=1, keepdim=True)).contiguous()
+    tau = 2e-5
+    p = prox.Prox(keys[:64].contiguous().to(DEV), 1, 5000, tau, "fifo")
+    p.cache_load(keys.to(DEV))
+    hit, slot, dist = p.probe_batch(Q.to(DEV))
+    torch.cuda.synchronize()
+    st = p.stats()
+    assert p.status() == prox.OK
+    p.close()
+    o = oracle.Oracle(None, 128, 1, 5000, float(np.float32(tau)), oracle.FIFO)
+    o.cache_load(keys.numpy())
+    r = o.query(Q.numpy())
+    assert st["probe_uncertified"] > 0
+    assert np.array_equal(hit.cpu().numpy(), r["hit"]) and np.array_equal(slot.cpu().numpy(), r["slot"])
+    assert 0.05 < r["hit"].mean() < 0.999
 
 
 # ------------------------------------------------------------------ API behaviour
