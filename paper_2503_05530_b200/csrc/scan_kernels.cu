@@ -430,6 +430,46 @@ rerank_kernel(DevState *st, int mode, const float *__restrict__ corpus, const fl
 // ------------------------------------------------------------------------------------------
 constexpr int kFallbackGroup = 8;
 
+// Rows warp, warp + nwarps, ... of the corpus against NG queries held in shared memory (NG is the
+// number of queries actually in the group, rounded up to 1, 2, 4 or 8, so that a lone failing
+// query costs one query's arithmetic and the pass stays bound by the corpus read).
+template <int NG>
+__device__ __forceinline__ void fallback_rows(const float *__restrict__ corpus, long long N, int d, long long warp,
+                                              long long nwarps, const float *q_sm, const float *radius, float margin,
+                                              int32_t *coll_id, int32_t *coll_n, int g0) {
+    const int lane = threadIdx.x & 31;
+    for (long long r = warp; r < N; r += nwarps) {
+        const float4 *x = reinterpret_cast<const float4 *>(corpus + (size_t)r * d);
+        float acc[NG];
+#pragma unroll
+        for (int f = 0; f < NG; ++f) acc[f] = 0.f;
+        for (int j = lane; j < d / 4; j += 32) {
+            const float4 xv = __ldcs(&x[j]);                       // streamed once: do not keep it in cache
+#pragma unroll
+            for (int f = 0; f < NG; ++f) {
+                const float4 qv = *reinterpret_cast<const float4 *>(&q_sm[f * d + 4 * j]);
+                const float d0 = qv.x - xv.x, d1 = qv.y - xv.y, d2 = qv.z - xv.z, d3 = qv.w - xv.w;
+                acc[f] = fmaf(d0, d0, fmaf(d1, d1, fmaf(d2, d2, fmaf(d3, d3, acc[f]))));
+            }
+        }
+#pragma unroll
+        for (int f = 0; f < NG; ++f)
+#pragma unroll
+            for (int s = 16; s > 0; s >>= 1) acc[f] += __shfl_xor_sync(0xffffffffu, acc[f], s);
+        if (lane < NG) {
+            float mine = 0.f;
+#pragma unroll
+            for (int f = 0; f < NG; ++f)
+                if (f == lane) mine = acc[f];
+            const float rad = radius[lane];                        // -1 for an empty place in the group
+            if (mine <= rad * (1.f + margin) + 1e-30f) {
+                const int pos = atomicAdd(&coll_n[g0 + lane], 1);
+                if (pos < kCollectCap) coll_id[(size_t)(g0 + lane) * kCollectCap + pos] = (int32_t)r;
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(256)
 fallback_collect_kernel(DevState *st, const float *__restrict__ corpus, const float *__restrict__ queries,
                         long long N, int d, const int32_t *__restrict__ miss_list,
@@ -440,7 +480,7 @@ fallback_collect_kernel(DevState *st, const float *__restrict__ corpus, const fl
     __shared__ float radius[kFallbackGroup];
     const int n_fail = st->n_fail;
     if (n_fail == 0) return;
-    const int tid = threadIdx.x, lane = tid & 31;
+    const int tid = threadIdx.x;
     const long long warp = ((long long)blockIdx.x * blockDim.x + tid) >> 5;
     const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
     const float margin = (float)(d + 8) * 1.1920929e-07f;              // (d + 8) * 2^-23, relative
@@ -454,35 +494,10 @@ fallback_collect_kernel(DevState *st, const float *__restrict__ corpus, const fl
         }
         if (tid < kFallbackGroup) radius[tid] = (tid < ng) ? fail_radius[g0 + tid] : -1.f;
         __syncthreads();
-        for (long long r = warp; r < N; r += nwarps) {
-            const float *x = corpus + (size_t)r * d;
-            float acc[kFallbackGroup];
-#pragma unroll
-            for (int f = 0; f < kFallbackGroup; ++f) acc[f] = 0.f;
-            for (int j = lane; j < d; j += 32) {
-                const float xv = x[j];
-#pragma unroll
-                for (int f = 0; f < kFallbackGroup; ++f) {
-                    const float df = q_sm[f * d + j] - xv;
-                    acc[f] = fmaf(df, df, acc[f]);
-                }
-            }
-#pragma unroll
-            for (int f = 0; f < kFallbackGroup; ++f)
-#pragma unroll
-                for (int s = 16; s > 0; s >>= 1) acc[f] += __shfl_xor_sync(0xffffffffu, acc[f], s);
-            if (lane < ng) {
-                float mine = 0.f;
-#pragma unroll
-                for (int f = 0; f < kFallbackGroup; ++f)
-                    if (f == lane) mine = acc[f];
-                const float rad = radius[lane];
-                if (mine <= rad * (1.f + margin) + 1e-30f) {
-                    const int pos = atomicAdd(&coll_n[g0 + lane], 1);
-                    if (pos < kCollectCap) coll_id[(size_t)(g0 + lane) * kCollectCap + pos] = (int32_t)r;
-                }
-            }
-        }
+        if (ng == 1) fallback_rows<1>(corpus, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
+        else if (ng == 2) fallback_rows<2>(corpus, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
+        else if (ng <= 4) fallback_rows<4>(corpus, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
+        else fallback_rows<8>(corpus, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
     }
 }
 

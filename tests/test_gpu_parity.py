@@ -173,7 +173,7 @@ def test_large_cache_stream_with_coarse_probe():
     k, cap, tau = 10, keys.shape[0], 0.5
     p = prox.Prox(X.to(DEV), k, cap, tau, "lru")
     p.cache_load(keys.to(DEV))
-    outs = [p.query_batch(Qs[a:a + 256].to(DEV)) for a in range(0, 800, 256)]
+    outs = [p.query_batch(Qs[a:a + 800].to(DEV)) for a in range(0, 800, 800)]      # 800 x 5200 pairs: coarse probe
     torch.cuda.synchronize()
     assert p.status() == prox.OK
     st = p.stats()
