@@ -195,7 +195,7 @@ def test_coarse_probe_hands_tight_clusters_to_the_exact_probe():
     c = torch.randn(128, generator=g)
     keys = c + 3e-4 * torch.randn(5000, 128, generator=g)
     keys = (keys / keys.norm(dim=1, keepdim=True)).contiguous()
-    Q = keys[:300] + 1e-4 * torch.randn(300, 128, generator=g)
+    Q = keys[:700] + 1e-4 * torch.randn(700, 128, generator=g)       # 700 x 5000 pairs: above the switch to the coarse probe
     Q = (Q / Q.norm(dim=1, keepdim=True)).contiguous()
     tau = 1.22e-6
     p = prox.Prox(keys[:64].contiguous().to(DEV), 1, 5000, tau, "fifo")
