@@ -1,60 +1,84 @@
-// Accumulator read-out shared by the tensor-core scan kernels: threshold test of 32 accumulator
-// columns of one corpus row and ballot-aggregated appends to warp-private candidate lists.
+// Accumulator read-out of the tensor-core scan kernel: threshold test of the accumulator columns
+// of one corpus row per lane and ballot-aggregated appends to warp-private candidate lists.
 #pragma once
 #include "topk_device.cuh"
 
 namespace prox {
 
-// 32 accumulator columns (queries c0 .. c0+31) of one corpus row, one row per lane.
-//
-// A column passes when acc - thr > half norm, i.e. score = acc - half norm beats the threshold up
-// to one rounding (the certificate's slack covers it).  Three levels, cheapest first:
-//   1. one maximum over the 32 differences decides the common case that nothing passes;
-//   2. else every lane forms its 32 pass bits and one OR across the warp names the columns in
-//      which some lane passes;
-//   3. only those columns are visited: the passing lanes take consecutive slots of the warp's
-//      private list (a ballot replaces atomics) and the warp's best score is folded in.
+// v[j] for a run-time j without indexing the register array: a tree of 31 selects.
+__device__ __forceinline__ uint32_t select32(const uint32_t (&v)[32], int j) {
+    uint32_t a[16], b[8], c[4], d[2];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) a[i] = (j & 1) ? v[2 * i + 1] : v[2 * i];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) b[i] = (j & 2) ? a[2 * i + 1] : a[2 * i];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) c[i] = (j & 4) ? b[2 * i + 1] : b[2 * i];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) d[i] = (j & 8) ? c[2 * i + 1] : c[2 * i];
+    return (j & 16) ? d[1] : d[0];
+}
+
+// Appends of one group of 32 accumulator columns (queries c0 .. c0+31) of one corpus row per
+// lane.  Every lane forms its 32 pass bits and walks its own set bits: it takes the next slot of
+// the warp's private list of that query with a shared-memory atomic and folds its score into
+// the block's best.  Lanes and columns do not wait for one another, so a row that passes for
+// many queries at once (queries on one topic) costs a few atomic latencies, and the code stays
+// small: this path runs for about one tile in ten and must not crowd the common path out of
+// the instruction cache.
 template <int CAP>
-__device__ __forceinline__ void readout32(const uint32_t (&v)[32], int c0, int lc0, float hn, int32_t row,
-                                          const float *__restrict__ thr, int *wcnt, uint32_t *best, u64 *lists,
-                                          bool &need) {
-    float dlt[32];
+__device__ __forceinline__ void append32(const uint32_t (&v)[32], int c0, int lc0, float hn, int32_t row,
+                                         const float *thr, int *wcnt, uint32_t *best, u64 *lists, bool &need) {
+    uint32_t pass = 0;
+#pragma unroll
+    for (int j4 = 0; j4 < 8; ++j4) {
+        const float4 t4 = *reinterpret_cast<const float4 *>(&thr[c0 + 4 * j4]);
+        pass |= (__uint_as_float(v[4 * j4]) - t4.x > hn) ? (1u << (4 * j4)) : 0u;
+        pass |= (__uint_as_float(v[4 * j4 + 1]) - t4.y > hn) ? (2u << (4 * j4)) : 0u;
+        pass |= (__uint_as_float(v[4 * j4 + 2]) - t4.z > hn) ? (4u << (4 * j4)) : 0u;
+        pass |= (__uint_as_float(v[4 * j4 + 3]) - t4.w > hn) ? (8u << (4 * j4)) : 0u;
+    }
+    bool full = false;
+#pragma unroll 1
+    while (pass) {
+        const int j = __ffs(pass) - 1;
+        pass &= pass - 1;
+        const u64 ent = pack_entry(__uint_as_float(select32(v, j)) - hn, row);
+        const int pos = atomicAdd(&wcnt[lc0 + j], 1);
+        if (pos < CAP) lists[(size_t)(c0 + j) * CAP + pos] = ent;
+        atomicMax(&best[c0 + j], (uint32_t)(ent >> 32));
+        full |= pos + 1 > CAP - 33;                              // this list must be cut before the next tile
+    }
+    if (__any_sync(0xffffffffu, full)) need = true;
+}
+
+// Largest of acc - thr over 32 accumulator columns of this lane's row.
+__device__ __forceinline__ float max_margin32(const uint32_t (&v)[32], const float *__restrict__ thr, int c0) {
     float m = -INFINITY;
 #pragma unroll
     for (int j4 = 0; j4 < 8; ++j4) {
         const float4 t4 = *reinterpret_cast<const float4 *>(&thr[c0 + 4 * j4]);
-        dlt[4 * j4] = __uint_as_float(v[4 * j4]) - t4.x;
-        dlt[4 * j4 + 1] = __uint_as_float(v[4 * j4 + 1]) - t4.y;
-        dlt[4 * j4 + 2] = __uint_as_float(v[4 * j4 + 2]) - t4.z;
-        dlt[4 * j4 + 3] = __uint_as_float(v[4 * j4 + 3]) - t4.w;
-        m = fmaxf(m, fmaxf(fmaxf(dlt[4 * j4], dlt[4 * j4 + 1]), fmaxf(dlt[4 * j4 + 2], dlt[4 * j4 + 3])));
+        m = fmaxf(m, fmaxf(fmaxf(__uint_as_float(v[4 * j4]) - t4.x, __uint_as_float(v[4 * j4 + 1]) - t4.y),
+                           fmaxf(__uint_as_float(v[4 * j4 + 2]) - t4.z, __uint_as_float(v[4 * j4 + 3]) - t4.w)));
     }
-    if (!__any_sync(0xffffffffu, m > hn)) return;
-    uint32_t pass = 0;
-#pragma unroll
-    for (int j = 0; j < 32; ++j) pass |= (dlt[j] > hn) ? (1u << j) : 0u;
-    const uint32_t cols = __reduce_or_sync(0xffffffffu, pass);
-    const int lane = threadIdx.x & 31;
-    const unsigned lt = (1u << lane) - 1u;
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        if (cols & (1u << j)) {                                   // warp-uniform
-            const bool p = (pass >> j) & 1u;
-            const unsigned mask = __ballot_sync(0xffffffffu, p);
-            const int base = wcnt[lc0 + j];
-            const u64 ent = pack_entry(__uint_as_float(v[j]) - hn, row);
-            const int pos = base + __popc(mask & lt);
-            if (p && pos < CAP) lists[(size_t)(c0 + j) * CAP + pos] = ent;
-            const uint32_t mx = __reduce_max_sync(0xffffffffu, p ? (uint32_t)(ent >> 32) : 0u);
-            const int n_new = base + __popc(mask);
-            if (lane == 0) {
-                wcnt[lc0 + j] = n_new;
-                atomicMax(&best[c0 + j], mx);
-            }
-            if (n_new > CAP - 33) need = true;                    // this list must be cut before the next tile
-        }
-    }
-    __syncwarp();
+    return m;
+}
+
+// Up to 64 accumulator columns (queries c0 .. c0+63; the second 32 only when `two`) of one corpus
+// row per lane, already in registers.  A column passes when acc - thr > half norm, i.e. score =
+// acc - half norm beats the threshold up to one rounding (the certificate's slack covers it).
+// One maximum per group and a single vote decide the common case that nothing passes.
+template <int CAP>
+__device__ __forceinline__ void readout64(const uint32_t (&v0)[32], const uint32_t (&v1)[32], bool two, int c0,
+                                          int lc0, float hn, int32_t row, const float *thr, int *wcnt,
+                                          uint32_t *best, u64 *lists, bool &need) {
+    const float m0 = max_margin32(v0, thr, c0);
+    const float m1 = two ? max_margin32(v1, thr, c0 + 32) : -INFINITY;
+    const unsigned any = __ballot_sync(0xffffffffu, fmaxf(m0, m1) > hn);
+    if (any == 0u) return;
+    if (__any_sync(0xffffffffu, m0 > hn)) append32<CAP>(v0, c0, lc0, hn, row, thr, wcnt, best, lists, need);
+    if (two && __any_sync(0xffffffffu, m1 > hn))
+        append32<CAP>(v1, c0 + 32, lc0 + 32, hn, row, thr, wcnt, best, lists, need);
 }
 
 }  // namespace prox

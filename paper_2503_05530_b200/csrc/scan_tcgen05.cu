@@ -2,7 +2,7 @@
 // every corpus row and up to 256 miss queries per pass, with the per-query best-k' selection
 // fused into the accumulator read-out (Algorithm 1, line 6: the database call of the misses).
 //
-// One persistent block per SM, 12 warps:
+// One persistent block per SM, 4 + 8 warps:
 //   warp 0   one lane issues TMA loads (cp.async.bulk.tensor, no multicast) of 128-row x 64-col
 //            bf16 corpus tiles, and of the matching query tile unless the whole query block
 //            fits in shared memory and is loaded once, into a ring of mbarrier-guarded stages;
@@ -10,10 +10,11 @@
 //            N = padded query count, K = 16 per instruction, fp32 accumulators in tensor memory,
 //            two accumulator buffers so that the read-out of tile t overlaps the products of t+1);
 //   warp 2   keeps the score bounds that the blocks share fresh (see the bound warp below);
-//   warps 4-11 read the accumulators (tcgen05.ld, one corpus row per thread, two warps per
-//            tensor-memory lane quarter splitting the columns), subtract the row's half norm,
-//            compare with the query's threshold and append survivors to warp-private candidate
-//            lists; a warp sorts and cuts a list of its own when it could overflow.
+//   warps 4-   read the accumulators (tcgen05.ld, one corpus row per thread, the warps of a
+//            tensor-memory lane quarter splitting the columns) into registers, hand the
+//            accumulator buffer back at once, then compare every score with the query's
+//            threshold and append survivors to warp-private candidate lists; a warp sorts and
+//            cuts a list of its own when it could overflow.
 // Every wait on an mbarrier is bounded in time; on expiry the block latches PROX_ERR_TIMEOUT,
 // stops issuing work, lets copies in flight land, frees its tensor memory and returns.
 #include <cuda.h>
@@ -31,8 +32,14 @@ using namespace sm100;
 
 namespace {
 
-constexpr int kThreads = 384;                        // producer, MMA, bound, (idle), 8 read-out warps
-constexpr int kReadWarps = 8;
+#ifndef PROX_READ_WARPS
+#define PROX_READ_WARPS 8
+#endif
+constexpr int kReadWarps = PROX_READ_WARPS;          // 8 or 16
+constexpr int kReadPerQuarter = kReadWarps / 4;      // warps that share a tensor-memory lane quarter
+constexpr int kReadCols = kScanQ / kReadPerQuarter;  // most query columns one read-out warp takes
+constexpr int kReadGroups = kReadCols / 32;
+constexpr int kThreads = 128 + 32 * kReadWarps;      // producer, MMA, bound, (idle), read-out warps
 constexpr int kMaxStages = 8;
 constexpr int kChunkK = 64;                          // bf16 elements per 128-byte swizzle row
 constexpr int kATileBytes = kTileRows * 128;         // 16 KB
@@ -57,7 +64,7 @@ struct Control {
     unsigned long long full[kMaxStages], empty[kMaxStages], tmem_full[2], tmem_empty[2], q_full;
     alignas(16) float thr[kScanQ];   // per query: scores at or below it cannot be among the best k'
     uint32_t best[kScanQ];           // best score this block has appended per query (ordered-uint form)
-    int wcnt[kReadWarps][kScanQ / 2];  // entries in each read-out warp's private candidate lists
+    int wcnt[kReadWarps][kReadCols];   // entries in each read-out warp's private candidate lists
     uint32_t tmem_base;
     int abort_flag;                  // set by any thread whose wait ran out
     int done;                        // read-out warps that have finished (the bound warp stops at kReadWarps)
@@ -129,7 +136,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     for (int q = tid; q < kScanQ; q += kThreads) { ctl.thr[q] = q < nq ? -INFINITY : INFINITY; ctl.best[q] = 0u; }
-    for (int i = tid; i < kReadWarps * (kScanQ / 2); i += kThreads) (&ctl.wcnt[0][0])[i] = 0;
+    for (int i = tid; i < kReadWarps * kReadCols; i += kThreads) (&ctl.wcnt[0][0])[i] = 0;
     if (warp == 1) tmem_alloc<PAIR>(smem_u32(&ctl.tmem_base), kTmemCols);
     tc_fence_before();
     __syncthreads();
@@ -249,21 +256,26 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         }
     } else if (warp >= 4) {
         // ------------------------------------------------------------ accumulator read-out
-        // Eight warps: warp w may read tensor-memory lanes 32 (w mod 4) .. +31 (one corpus row per
-        // thread); the two warps that share a lane quarter split the query columns.
-        const int e = warp - 4;                                   // 0..7
+        // Warp w may read tensor-memory lanes 32 (w mod 4) .. +31 (one corpus row per thread); the
+        // warps that share a lane quarter split the query columns.  A warp copies
+        // its columns into registers and frees the accumulator buffer before it looks at them, so
+        // a slow tile (appends, a list to cut) does not hold back the products two tiles on.
+        const int e = warp - 4;                                   // 0..15
         const int quarter = warp & 3;
-        const int half = e >> 2;
-        const int cw = n_pad >= 64 ? n_pad / 2 : 32;              // columns per warp
-        const int col_begin = half * cw;
+        const int part = e >> 2;
+        const int cw = n_pad >= 32 * kReadPerQuarter ? n_pad / kReadPerQuarter : 32;   // columns per warp
+        const int col_begin = part * cw;
         const bool active = col_begin < n_pad;
+        const int ngr = cw / 32;                                  // groups of 32 columns: 1, 2 or 4
         const int ncol = active ? (nq - col_begin < cw ? (nq - col_begin > 0 ? nq - col_begin : 0) : cw) : 0;
         int *wcnt = ctl.wcnt[e];
         // lists of this warp: [(block * 4 + quarter) * kScanQ + query] * CAP
         u64 *lists = a.buf + ((size_t)(blockIdx.x * 4 + quarter) * kScanQ) * CAP;
         int32_t *lists_cnt = a.buf_cnt + (size_t)(blockIdx.x * 4 + quarter) * kScanQ;
         uint32_t it = 0;
-        uint32_t published[4] = {0u, 0u, 0u, 0u};
+        uint32_t published[kReadGroups];
+#pragma unroll
+        for (int i = 0; i < kReadGroups; ++i) published[i] = 0u;
         long long row = (long long)unit * kUnitRows + (long long)rank * kTileRows + quarter * 32 + lane;
         float hn = (unit < ntiles && row < a.N) ? a.xh[row] : INFINITY;
         bool alive = true;
@@ -274,9 +286,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             // loads whose latency hides behind the wait and the read-out
             const long long row_next = row + (long long)n_units * kUnitRows;
             const float hn_next = (tile + n_units < ntiles && row_next < a.N) ? a.xh[row_next] : INFINITY;
-            uint32_t g_thr[4];
+            uint32_t g_thr[kReadGroups];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < kReadGroups; ++i) {
                 const int c = col_begin + lane + 32 * i;
                 g_thr[i] = (lane + 32 * i < ncol) ? __ldcg(&thr_g[c]) : 0u;
             }
@@ -284,33 +296,38 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { alive = false; break; }
             tc_fence_after();
-            // rows past the end carry an infinite half norm, columns past nq an infinite threshold:
-            // neither can pass, so the compare loop needs no bounds tests
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)kScanQ;
+            // 64 columns at a time; the accumulator buffer goes back to the MMA issuer as soon as
+            // the last of them are in registers, before they are looked at.  Rows past the end carry
+            // an infinite half norm, columns past nq an infinite threshold: neither can pass, so
+            // the compare loop needs no bounds tests.
             bool need = false;
-            if (active) {
-                for (int c0 = col_begin; c0 < col_begin + cw; c0 += 64) {
-                    const bool two = c0 + 32 < col_begin + cw;
-                    uint32_t v0[32], v1[32];
-                    tc_ld32(taddr + c0, v0);
-                    if (two) tc_ld32(taddr + c0 + 32, v1);
+#pragma unroll 1
+            for (int c0 = 0; c0 < kReadCols; c0 += 64) {
+                const bool last = c0 + 64 >= cw;
+                uint32_t v0[32], v1[32];
+                if (active && c0 < cw) {
+                    tc_ld32(taddr + col_begin + c0, v0);
+                    if (c0 + 32 < cw) tc_ld32(taddr + col_begin + c0 + 32, v1);
                     tc_wait_ld();
-                    readout32<CAP>(v0, c0, c0 - col_begin, hn, (int32_t)row, ctl.thr, wcnt, ctl.best, lists, need);
-                    if (two)
-                        readout32<CAP>(v1, c0 + 32, c0 + 32 - col_begin, hn, (int32_t)row, ctl.thr, wcnt,
-                                       ctl.best, lists, need);
                 }
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                if constexpr (PAIR) mbar_arrive_cluster(b ? empty_bar1 : empty_bar0);
-                else mbar_arrive(b ? empty_bar1 : empty_bar0);
+                if (last) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if constexpr (PAIR) mbar_arrive_cluster(b ? empty_bar1 : empty_bar0);
+                        else mbar_arrive(b ? empty_bar1 : empty_bar0);
+                    }
+                }
+                if (active && c0 < cw)
+                    readout64<CAP>(v0, v1, c0 + 32 < cw, col_begin + c0, c0, hn, (int32_t)row, ctl.thr, wcnt, ctl.best,
+                                   lists, need);
+                if (last) break;
             }
             // threshold upkeep for this warp's columns: a stale (lower) threshold only lets more
             // rows through, so plain stores shared with the other warps are enough
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < kReadGroups; ++i) {
                 const int lc = lane + 32 * i;
                 if (lc < ncol) {
                     const int c = col_begin + lc;
@@ -327,7 +344,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             }
             if (need) {                                           // warp-uniform
                 __syncwarp();
-                for (int i = 0; i < 4; ++i) {
+                for (int i = 0; i < kReadGroups; ++i) {
                     const int lc = lane + 32 * i;
                     unsigned mm = __ballot_sync(0xffffffffu, lc < ncol && wcnt[lc] > CAP - 33);
                     while (mm) {

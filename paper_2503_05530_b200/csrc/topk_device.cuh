@@ -30,40 +30,55 @@ __device__ __forceinline__ u64 shfl_xor_u64(u64 v, int m) {
     return ((u64)hi << 32) | lo;
 }
 
+// One compare-exchange pass of the bitonic network between the register slots it and it ^ DJ of
+// every lane (keys 32 * DJ apart); k is the size of the bitonic blocks being merged.
+template <int ITEMS, int DJ>
+__device__ __forceinline__ void sort_pass_regs(u64 (&v)[ITEMS], int k, int lane) {
+#pragma unroll
+    for (int it = 0; it < ITEMS; ++it) {
+        const int partner = it ^ DJ;
+        if (partner > it) {
+            const int e = it * 32 + lane;
+            const bool desc = ((e & k) == 0);
+            const u64 a = v[it], b = v[partner];
+            const bool swap = desc ? (a < b) : (a > b);
+            v[it] = swap ? b : a;
+            v[partner] = swap ? a : b;
+        }
+    }
+}
+
 // Sorts ITEMS*32 keys held by one warp, DESCENDING.  Element e lives in
 // v[e / 32] of lane e % 32, so after the sort v[0] of lane 0 is the largest key,
 // v[0] of lane 1 the next, ... v[1] of lane 0 the 33rd, and so on.
+// The passes of the network run in rolled loops (only the register slots are unrolled): the
+// sort is rare next to the code that calls it, and a fully unrolled network is tens of
+// kilobytes of instructions that would push that code out of the instruction cache.
 template <int ITEMS>
 __device__ __forceinline__ void warp_sort_desc(u64 (&v)[ITEMS]) {
     constexpr int LOG = (ITEMS == 1 ? 5 : ITEMS == 2 ? 6 : ITEMS == 4 ? 7 : ITEMS == 8 ? 8 : ITEMS == 16 ? 9 : 10);
     static_assert((32 << (LOG - 5)) == ITEMS * 32, "ITEMS must be a power of two up to 32");
     const int lane = threadIdx.x & 31;
-#pragma unroll
+#pragma unroll 1
     for (int lk = 1; lk <= LOG; ++lk) {
         const int k = 1 << lk;
-#pragma unroll
+#pragma unroll 1
         for (int lj = lk - 1; lj >= 0; --lj) {
             const int j = 1 << lj;
             if (j >= 32) {
-                const int dj = j >> 5;
-#pragma unroll
-                for (int it = 0; it < ITEMS; ++it) {
-                    const int partner = it ^ dj;
-                    if (partner > it) {
-                        const int e = it * 32 + lane;
-                        const bool desc = ((e & k) == 0);
-                        const u64 a = v[it], b = v[partner];
-                        const bool swap = desc ? (a < b) : (a > b);
-                        v[it] = swap ? b : a;
-                        v[partner] = swap ? a : b;
-                    }
+                switch (j >> 5) {
+                    case 1: if constexpr (ITEMS >= 2) sort_pass_regs<ITEMS, 1>(v, k, lane); break;
+                    case 2: if constexpr (ITEMS >= 4) sort_pass_regs<ITEMS, 2>(v, k, lane); break;
+                    case 4: if constexpr (ITEMS >= 8) sort_pass_regs<ITEMS, 4>(v, k, lane); break;
+                    case 8: if constexpr (ITEMS >= 16) sort_pass_regs<ITEMS, 8>(v, k, lane); break;
+                    default: if constexpr (ITEMS >= 32) sort_pass_regs<ITEMS, 16>(v, k, lane); break;
                 }
             } else {
+                const bool lower = ((lane & j) == 0);           // this lane holds the lower index of the pair
 #pragma unroll
                 for (int it = 0; it < ITEMS; ++it) {
                     const int e = it * 32 + lane;
                     const bool desc = ((e & k) == 0);
-                    const bool lower = ((lane & j) == 0);       // this lane holds the lower index of the pair
                     const u64 mine = v[it];
                     const u64 other = shfl_xor_u64(mine, j);
                     // descending block: lower index keeps the max; ascending block: lower keeps the min
@@ -87,8 +102,8 @@ __device__ __forceinline__ void warp_sort_desc(u64 (&v)[ITEMS]) {
 // kp-th best.  With prune set, entries below the shared bound are dropped as well (they cannot
 // be among the global best kp).
 template <int CAP>
-__device__ __forceinline__ void warp_compact(u64 *qbuf, int *cnt, float *thr, uint32_t *thr_g_q, int kp,
-                                             uint32_t *top_q, int block, int n_blocks, bool prune) {
+__device__ __noinline__ void warp_compact(u64 *qbuf, int *cnt, float *thr, uint32_t *thr_g_q, int kp,
+                                          uint32_t *top_q, int block, int n_blocks, bool prune) {
     const int lane = threadIdx.x & 31;
     const int n = *cnt < CAP ? *cnt : CAP;
     u64 v[CAP / 32];
