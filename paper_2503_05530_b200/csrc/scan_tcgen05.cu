@@ -297,6 +297,18 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             if (!ok) { alive = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)kScanQ;
+            // the shared bounds read above go into the block's thresholds before this tile is tested
+            // (a stale, lower threshold only lets more rows through, so plain stores that the
+            // warps of a column share are enough)
+#pragma unroll
+            for (int i = 0; i < kReadGroups; ++i) {
+                const int lc = lane + 32 * i;
+                if (lc < ncol) {
+                    const float g = o2f(g_thr[i]);
+                    if (g > ctl.thr[col_begin + lc]) ctl.thr[col_begin + lc] = g;
+                }
+            }
+            __syncwarp();
             // 64 columns at a time; the accumulator buffer goes back to the MMA issuer as soon as
             // the last of them are in registers, before they are looked at.  Rows past the end carry
             // an infinite half norm, columns past nq an infinite threshold: neither can pass, so
@@ -324,16 +336,13 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                                    lists, need);
                 if (last) break;
             }
-            // threshold upkeep for this warp's columns: a stale (lower) threshold only lets more
-            // rows through, so plain stores shared with the other warps are enough
+            // one warp per column publishes the block's best score
+            if (quarter == 0) {
 #pragma unroll
-            for (int i = 0; i < kReadGroups; ++i) {
-                const int lc = lane + 32 * i;
-                if (lc < ncol) {
-                    const int c = col_begin + lc;
-                    const float g = o2f(g_thr[i]);
-                    if (g > ctl.thr[c]) ctl.thr[c] = g;
-                    if (quarter == 0) {                           // one warp per column publishes the block's best
+                for (int i = 0; i < kReadGroups; ++i) {
+                    const int lc = lane + 32 * i;
+                    if (lc < ncol) {
+                        const int c = col_begin + lc;
                         const uint32_t bq = ctl.best[c];
                         if (bq > published[i]) {
                             top1[(size_t)c * gridDim.x + blockIdx.x] = bq;
