@@ -214,9 +214,10 @@ scan_cc_kernel(const DevState *__restrict__ st, const __nv_bfloat16 *__restrict_
 }
 
 // ------------------------------------------------------------------------------------------
-// Merge: per query, the k' best entries over all candidate lists of the pass (every list was
-// already cut to at most k' entries).  The entries are staged in shared memory when they fit;
-// radix select on the 32-bit ordered score, then a collection pass.
+// Merge: per query, the k' best entries over all candidate lists of the pass.  A list holds up to
+// `stride` entries as the scan left them; entries below the query's shared score bound (a lower
+// bound of its global k'-th best) are dropped on the way in.  What is left is staged in shared
+// memory when it fits; radix select on the 32-bit ordered score, then a collection pass.
 // ------------------------------------------------------------------------------------------
 constexpr int kMergeStage = 8192;                  // entries staged in shared memory
 
@@ -224,22 +225,24 @@ struct MergeSrc {
     const u64 *buf;                                // lists of this query: list p at buf + p * list_stride
     const int32_t *cnt;                            // cnt[p * cnt_stride]
     size_t list_stride;
-    int cnt_stride, n_lists, kp, total;
+    int cnt_stride, n_lists, cap, total;
+    uint32_t g0;                                   // entries whose ordered score is below it do not count
     const u64 *stage;                              // non-null: all entries are in stage[0 .. total)
-    __device__ __forceinline__ int span() const { return stage ? total : n_lists * kp; }
+    __device__ __forceinline__ int span() const { return stage ? total : n_lists * cap; }
     __device__ __forceinline__ bool get(int idx, u64 &ent) const {
         if (stage) { ent = stage[idx]; return true; }
-        const int p = idx / kp, e = idx - p * kp;
+        const int p = idx / cap, e = idx - p * cap;
         if (e >= cnt[(size_t)p * cnt_stride]) return false;
         ent = buf[(size_t)p * list_stride + e];
-        return true;
+        return (uint32_t)(ent >> 32) >= g0;
     }
 };
 
 __global__ void __launch_bounds__(1024)
 merge_select_kernel(const int *__restrict__ n_active, int pass, int n_lists, int stride, int kp,
-                    const u64 *__restrict__ buf, const int32_t *__restrict__ buf_cnt, int32_t *cand_id,
-                    float *cand_score, int32_t *cand_n, float *cand_sk) {
+                    const u64 *__restrict__ buf, const int32_t *__restrict__ buf_cnt,
+                    const uint32_t *__restrict__ thr_g, int32_t *cand_id, float *cand_score, int32_t *cand_n,
+                    float *cand_sk) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     u64 *stage = reinterpret_cast<u64 *>(smem_raw);
     __shared__ unsigned hist[256];
@@ -251,13 +254,29 @@ merge_select_kernel(const int *__restrict__ n_active, int pass, int n_lists, int
 
     if (tid == 0) { s_total = 0; s_gt = 0; s_eq = 0; }
     __syncthreads();
-    for (int p = warp; p < n_lists; p += 32) {
-        const int c = buf_cnt[(size_t)p * kScanQ + q];
-        int base = 0;
-        if (lane == 0 && c > 0) base = atomicAdd(&s_total, c);
-        base = __shfl_sync(0xffffffffu, base, 0);
-        if (base + c <= kMergeStage)
-            for (int e = lane; e < c; e += 32) stage[base + e] = buf[((size_t)p * kScanQ + q) * stride + e];
+    const uint32_t g0 = thr_g[m];
+    // warp w takes the lists w, w + 32, ...: their counts come in with one load per 32 lists
+    for (int p0 = warp; p0 < n_lists; p0 += 32 * 32) {
+        int my_c = 0;
+        if (p0 + 32 * lane < n_lists) {
+            my_c = buf_cnt[(size_t)(p0 + 32 * lane) * kScanQ + q];
+            if (my_c > stride) my_c = stride;
+        }
+        for (int i = 0; i < 32 && p0 + 32 * i < n_lists; ++i) {
+            const int p = p0 + 32 * i;
+            const int c = __shfl_sync(0xffffffffu, my_c, i);
+            const u64 *list = buf + ((size_t)p * kScanQ + q) * stride;
+            for (int e0 = 0; e0 < c; e0 += 32) {
+                const u64 ent = (e0 + lane < c) ? list[e0 + lane] : 0ull;
+                const bool keep = ent != 0ull && (uint32_t)(ent >> 32) >= g0;
+                const unsigned mask = __ballot_sync(0xffffffffu, keep);
+                if (mask == 0u) continue;
+                int base = 0;
+                if (lane == 0) base = atomicAdd(&s_total, __popc(mask));
+                base = __shfl_sync(0xffffffffu, base, 0) + __popc(mask & ((1u << lane) - 1u));
+                if (keep && base < kMergeStage) stage[base] = ent;
+            }
+        }
     }
     __syncthreads();
     MergeSrc src;
@@ -265,7 +284,7 @@ merge_select_kernel(const int *__restrict__ n_active, int pass, int n_lists, int
     src.cnt = buf_cnt + q;
     src.list_stride = (size_t)kScanQ * stride;
     src.cnt_stride = kScanQ;
-    src.n_lists = n_lists; src.kp = kp; src.total = s_total;
+    src.n_lists = n_lists; src.cap = stride; src.g0 = g0; src.total = s_total;
     src.stage = (s_total <= kMergeStage) ? stage : nullptr;
     const int total = src.total, span = src.span();
 
@@ -635,8 +654,8 @@ void launch_merge_select(prox_handle *h, int pass, int B, int for_probe, cudaStr
     }
     merge_select_kernel<<<nq, 1024, kMergeStage * 8, s>>>(for_probe ? &h->st->n_probe : &h->st->n_miss, pass,
                                                           h->scan_lists, h->scan_list_stride, for_probe ? kProbeKp : h->kp,
-                                                          h->buf, h->buf_cnt, h->cand_id, h->cand_score, h->cand_n,
-                                                          h->cand_sk);
+                                                          h->buf, h->buf_cnt, h->thr_g, h->cand_id, h->cand_score,
+                                                          h->cand_n, h->cand_sk);
     h->launches++;
 }
 

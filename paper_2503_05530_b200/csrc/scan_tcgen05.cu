@@ -369,14 +369,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             row = row_next;
             hn = hn_next;
         }
-        // final cut of every list, dropping what the shared bound has already ruled out
+        // the lists go to the merge as they are: it drops what the shared bound has ruled out
         __syncwarp();
-        for (int lc = 0; lc < ncol; ++lc) {
-            const int c = col_begin + lc;
-            if (alive)
-                warp_compact<CAP>(lists + (size_t)c * CAP, &wcnt[lc], &ctl.thr[c], &thr_g[c], a.kp, nullptr, blockIdx.x,
-                                  gridDim.x, true);
-            if (lane == 0) lists_cnt[c] = alive ? wcnt[lc] : 0;
+        for (int lc = lane; lc < ncol; lc += 32) {
+            const int n = wcnt[lc] < CAP ? wcnt[lc] : CAP;
+            lists_cnt[col_begin + lc] = alive ? n : 0;
         }
         if (lane == 0) atomicAdd(&ctl.done, 1);
     }
