@@ -87,6 +87,23 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm))
 
 
+def stream_seed(seed: int, rank: int) -> int:
+    """Every rank serves its own query stream over its own copy of the corpus."""
+    return seed + rank
+
+
+def aggregate_over_ranks(ms_local: float, queries_local: int, dist=None, device="cpu"):
+    """Whole-job figures of a run of independent replicas: the slowest rank's time and the
+    queries of all ranks.  `dist` is torch.distributed with an initialised group, or None."""
+    if dist is None:
+        return float(ms_local), int(queries_local)
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    n = torch.tensor([queries_local], dtype=torch.int64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(n.item())
+
+
 def pick_workload(name: str, free_bytes: int) -> W.Config:
     if name != "auto":
         return W.CONFIGS[name]
@@ -176,7 +193,7 @@ def run_ours(args):
                          name=cfg.name + "-cut", n_components=max(1, cfg.n_components * (args.rows or cfg.N) // cfg.N),
                          n_topics=min(cfg.n_topics, (args.rows or cfg.N) // 4))
     peaks = load_peaks()
-    seed = args.seed + rank                                    # each rank serves its own stream
+    seed = stream_seed(args.seed, rank)
     K, Wm = args.steps, args.warmup
     n_batches_total = (cfg.n_queries + cfg.batch - 1) // cfg.batch
     if K <= 0:
@@ -248,17 +265,9 @@ def run_ours(args):
         del p
 
     # max over ranks of the times, sum over ranks of the queries
-    def allmax(x):
-        if not dist:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
     head = results[head_tau]
-    ms = allmax(head["ms"])
-    ms_e2e = allmax(head["ms_e2e"])
-    total_q = K * cfg.batch * world
+    ms, total_q = aggregate_over_ranks(head["ms"], K * cfg.batch, dist, dev)
+    ms_e2e, _ = aggregate_over_ranks(head["ms_e2e"], K * cfg.batch, dist, dev)
     value = total_q / (ms * 1e-3)
     e2e = total_q / (ms_e2e * 1e-3)
 
