@@ -21,6 +21,72 @@ namespace prox {
 // At-risk list: the R entries with the smallest stamps, in stamp order (Section 3.3.2: the
 // victim is always the entry with the oldest insertion (FIFO) or oldest use (LRU)).
 // ------------------------------------------------------------------------------------------
+// The R smallest of n unique keys (vals[i], or i when vals is null, rides along), left in
+// s_key / s_val (1024 entries each, unused ones at the maximum) for a block of 1024 threads;
+// clock bounds the keys from above.  Returns how many were found (R unless the keys repeat).
+__device__ int select_smallest(const u64 *__restrict__ keys, const int32_t *__restrict__ vals, long long n, int R,
+                               long long clock, unsigned *hist, u64 *s_key, int *s_val, u64 *s_prefix, u64 *s_mask,
+                               int *s_remaining, int *s_n) {
+    const int tid = threadIdx.x;
+    u64 T = ~0ull;                       // R-th smallest key
+    if ((long long)R < n) {
+        int nd = 1;
+        while (nd < 8 && (clock >> (8 * nd)) != 0) ++nd;
+        if (tid == 0) { *s_prefix = 0; *s_mask = 0; *s_remaining = R; }
+        for (int p = nd - 1; p >= 0; --p) {
+            if (tid < 256) hist[tid] = 0;
+            __syncthreads();
+            const u64 prefix = *s_prefix, mask = *s_mask;
+            for (long long s = tid; s < n; s += blockDim.x) {
+                const u64 v = keys[s];
+                if ((v & mask) == prefix) atomicAdd(&hist[(unsigned)(v >> (8 * p)) & 255u], 1u);
+            }
+            __syncthreads();
+            if (tid == 0) {
+                int rem = *s_remaining, b = 0;
+                while (b < 255 && (int)hist[b] < rem) { rem -= (int)hist[b]; ++b; }
+                *s_remaining = rem;
+                *s_prefix = prefix | ((u64)b << (8 * p));
+                *s_mask = mask | (0xffull << (8 * p));
+            }
+            __syncthreads();
+        }
+        T = *s_prefix;
+    }
+    if (tid == 0) *s_n = 0;
+    s_key[tid] = ~0ull;
+    s_val[tid] = 0x7fffffff;
+    __syncthreads();
+    for (long long s = tid; s < n; s += blockDim.x) {
+        const u64 v = keys[s];
+        if (v <= T) {
+            const int pos = atomicAdd(s_n, 1);
+            if (pos < 1024) { s_key[pos] = v; s_val[pos] = vals ? vals[s] : (int)s; }
+        }
+    }
+    __syncthreads();
+    return *s_n;
+}
+
+// Sorts the R selected (stamp, slot) pairs and publishes the at-risk list.
+__device__ void publish_risk_list(DevState *st, int R, u64 *s_key, int *s_val, int32_t *risk_pos,
+                                  int32_t *risk_slot, u64 *risk_stamp) {
+    const int tid = threadIdx.x;
+    int n2 = 1;
+    while (n2 < R) n2 <<= 1;
+    block_sort_asc(s_key, s_val, n2);
+    if (tid < R) {
+        risk_slot[tid] = s_val[tid];
+        risk_stamp[tid] = s_key[tid];
+        risk_pos[s_val[tid]] = tid;
+    }
+    if (tid == 0) st->n_risk = R;
+}
+
+__device__ __forceinline__ int risk_count(long long count, int B, long long C) {
+    return (count + B > C) ? (int)(count < (long long)B ? count : (long long)B) : 0;
+}
+
 __global__ void __launch_bounds__(1024)
 risk_select_kernel(DevState *st, const u64 *__restrict__ stamp, int32_t *risk_pos,
                    int32_t *risk_slot, u64 *risk_stamp, int B, long long C) {
@@ -37,64 +103,139 @@ risk_select_kernel(DevState *st, const u64 *__restrict__ stamp, int32_t *risk_po
     const long long clock = st->clock;
     __syncthreads();
 
-    int R = 0;
-    if (count + B > C) R = (int)(count < (long long)B ? count : (long long)B);
+    const int R = risk_count(count, B, C);
     if (R == 0) {
         if (tid == 0) st->n_risk = 0;
         return;
     }
-
-    u64 T = ~0ull;                       // R-th smallest stamp
-    if ((long long)R < count) {
-        int nd = 1;
-        while (nd < 8 && (clock >> (8 * nd)) != 0) ++nd;
-        if (tid == 0) { s_prefix = 0; s_mask = 0; s_remaining = R; }
-        for (int p = nd - 1; p >= 0; --p) {
-            if (tid < 256) hist[tid] = 0;
-            __syncthreads();
-            const u64 prefix = s_prefix, mask = s_mask;
-            for (long long s = tid; s < count; s += blockDim.x) {
-                const u64 v = stamp[s];
-                if ((v & mask) == prefix) atomicAdd(&hist[(unsigned)(v >> (8 * p)) & 255u], 1u);
-            }
-            __syncthreads();
-            if (tid == 0) {
-                int rem = s_remaining, b = 0;
-                while (b < 255 && (int)hist[b] < rem) { rem -= (int)hist[b]; ++b; }
-                s_remaining = rem;
-                s_prefix = prefix | ((u64)b << (8 * p));
-                s_mask = mask | (0xffull << (8 * p));
-            }
-            __syncthreads();
-        }
-        T = s_prefix;
-    }
-
-    if (tid == 0) s_n = 0;
-    s_key[tid] = ~0ull;
-    s_val[tid] = 0x7fffffff;
-    __syncthreads();
-    for (long long s = tid; s < count; s += blockDim.x) {
-        const u64 v = stamp[s];
-        if (v <= T) {
-            const int pos = atomicAdd(&s_n, 1);
-            if (pos < 1024) { s_key[pos] = v; s_val[pos] = (int)s; }
-        }
-    }
-    __syncthreads();
-    if (s_n != R) {                      // stamps must be unique; anything else is a broken state
+    const int found = select_smallest(stamp, nullptr, count, R, clock, hist, s_key, s_val, &s_prefix, &s_mask,
+                                      &s_remaining, &s_n);
+    if (found != R) {                    // stamps must be unique; anything else is a broken state
         if (tid == 0) { atomicCAS(&st->error, 0, PROX_ERR_INTERNAL); st->n_risk = 0; }
         return;
     }
-    int n2 = 1;
-    while (n2 < R) n2 <<= 1;
-    block_sort_asc(s_key, s_val, n2);
-    if (tid < R) {
-        risk_slot[tid] = s_val[tid];
-        risk_stamp[tid] = s_key[tid];
-        risk_pos[s_val[tid]] = tid;
+    publish_risk_list(st, R, s_key, s_val, risk_pos, risk_slot, risk_stamp);
+}
+
+// Large caches: the same selection spread over the whole GPU.  A 65536-bin histogram of the
+// stamps' leading bits names the bin that holds the R-th smallest; stamps in lower bins are at
+// risk for certain, the stamps of that one bin (few, stamps being unique) are settled by one
+// block.  Work area: histogram, the two lists and their counters.
+constexpr int kRiskBins = 1 << 16;
+constexpr int kRiskEdgeCap = 1 << 20;
+struct RiskWork {
+    unsigned hist[kRiskBins];
+    int n_sure, n_edge, bin, shift;
+    u64 sure_key[kMaxBatch];
+    int32_t sure_val[kMaxBatch];
+    u64 edge_key[kRiskEdgeCap];
+    int32_t edge_val[kRiskEdgeCap];
+};
+
+__device__ __forceinline__ int risk_shift(long long clock) {
+    int bits = 0;
+    while (bits < 63 && (clock >> bits) != 0) ++bits;
+    return bits > 16 ? bits - 16 : 0;
+}
+
+__global__ void __launch_bounds__(256)
+risk_hist_kernel(const DevState *st, const u64 *__restrict__ stamp, int32_t *risk_pos,
+                 const int32_t *__restrict__ risk_slot, RiskWork *w, int B, long long C) {
+    const long long gtid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long nth = (long long)gridDim.x * blockDim.x;
+    const int prev = st->n_risk;
+    for (long long r = gtid; r < prev; r += nth) risk_pos[risk_slot[r]] = -1;
+    const long long count = st->count;
+    const int R = risk_count(count, B, C);
+    if (R == 0 || (long long)R >= count) return;
+    const int shift = risk_shift(st->clock);
+    for (long long s = gtid; s < count; s += nth) atomicAdd(&w->hist[(unsigned)(stamp[s] >> shift)], 1u);
+}
+
+__global__ void __launch_bounds__(1024)
+risk_pick_kernel(const DevState *st, RiskWork *w, int B, long long C) {
+    __shared__ unsigned part[1024];
+    const int tid = threadIdx.x;
+    const long long count = st->count;
+    const int R = risk_count(count, B, C);
+    if (tid == 0) { w->n_sure = 0; w->n_edge = 0; w->shift = risk_shift(st->clock); }
+    if (R == 0 || (long long)R >= count) {
+        if (tid == 0) w->bin = kRiskBins;                // every entry (or none) is at risk
+        return;
     }
-    if (tid == 0) st->n_risk = R;
+    constexpr int per = kRiskBins / 1024;
+    unsigned sum = 0;
+    for (int i = 0; i < per; ++i) sum += w->hist[tid * per + i];
+    part[tid] = sum;
+    __syncthreads();
+    if (tid == 0) {
+        unsigned acc = 0;
+        int t = 0;
+        while (t < 1023 && acc + part[t] < (unsigned)R) { acc += part[t]; ++t; }
+        int b = t * per;
+        while (b < kRiskBins - 1 && acc + w->hist[b] < (unsigned)R) { acc += w->hist[b]; ++b; }
+        w->bin = b;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+risk_collect_kernel(const DevState *st, const u64 *__restrict__ stamp, RiskWork *w, int B, long long C) {
+    const long long count = st->count;
+    if (risk_count(count, B, C) == 0) return;
+    const long long gtid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long nth = (long long)gridDim.x * blockDim.x;
+    const unsigned bin = (unsigned)w->bin;
+    const int shift = w->shift;
+    for (long long s = gtid; s < count; s += nth) {
+        const u64 v = stamp[s];
+        const unsigned bn = bin == (unsigned)kRiskBins ? 0u : (unsigned)(v >> shift);
+        if (bn < bin) {
+            const int pos = atomicAdd(&w->n_sure, 1);
+            if (pos < kMaxBatch) { w->sure_key[pos] = v; w->sure_val[pos] = (int32_t)s; }
+        } else if (bn == bin) {
+            const int pos = atomicAdd(&w->n_edge, 1);
+            if (pos < kRiskEdgeCap) { w->edge_key[pos] = v; w->edge_val[pos] = (int32_t)s; }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(1024)
+risk_finish_kernel(DevState *st, RiskWork *w, int32_t *risk_pos, int32_t *risk_slot, u64 *risk_stamp, int B,
+                   long long C) {
+    __shared__ unsigned hist[256];
+    __shared__ u64 s_key[1024];
+    __shared__ int s_val[1024];
+    __shared__ u64 s_prefix, s_mask;
+    __shared__ int s_remaining, s_n;
+    const int tid = threadIdx.x;
+    const long long count = st->count;
+    const int R = risk_count(count, B, C);
+    if (R == 0) {
+        if (tid == 0) st->n_risk = 0;
+        return;
+    }
+    const int n_sure = w->n_sure, n_edge = w->n_edge;
+    const int need = R - n_sure;
+    bool ok = n_sure <= R && need <= n_edge && n_edge <= kRiskEdgeCap;
+    int found = 0;
+    if (ok) {
+        found = need > 0 ? select_smallest(w->edge_key, w->edge_val, n_edge, need, st->clock, hist, s_key, s_val,
+                                           &s_prefix, &s_mask, &s_remaining, &s_n)
+                         : 0;
+        if (need <= 0) {
+            s_key[tid] = ~0ull;
+            s_val[tid] = 0x7fffffff;
+            __syncthreads();
+        }
+        ok = found == (need > 0 ? need : 0);
+    }
+    if (!ok) {                           // stamps must be unique; anything else is a broken state
+        if (tid == 0) { atomicCAS(&st->error, 0, PROX_ERR_INTERNAL); st->n_risk = 0; }
+        return;
+    }
+    if (tid < n_sure) { s_key[found + tid] = w->sure_key[tid]; s_val[found + tid] = w->sure_val[tid]; }
+    __syncthreads();
+    publish_risk_list(st, R, s_key, s_val, risk_pos, risk_slot, risk_stamp);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -655,9 +796,23 @@ static int probe_splits(const prox_handle *h, int B) {
 }
 
 void launch_risk_select(prox_handle *h, int B, cudaStream_t s) {
-    risk_select_kernel<<<1, 1024, 0, s>>>(h->st, h->stamp, h->risk_pos, h->risk_slot, h->risk_stamp, B,
-                                          (long long)h->C);
-    h->launches++;
+    // one block reads a small cache faster than four launches do
+    if (h->C <= (1 << 16)) {
+        risk_select_kernel<<<1, 1024, 0, s>>>(h->st, h->stamp, h->risk_pos, h->risk_slot, h->risk_stamp, B,
+                                              (long long)h->C);
+        h->launches++;
+        return;
+    }
+    // the work area borrows the candidate table of the resolve, which is filled later in the batch
+    static_assert(sizeof(RiskWork) <= sizeof(double) * (size_t)kMaxBatch * 2 * kMaxBatch, "work area too large");
+    RiskWork *w = reinterpret_cast<RiskWork *>(h->cand_d);
+    cudaMemsetAsync(w->hist, 0, sizeof(w->hist), s);
+    const int grid = h->num_sms * 8;
+    risk_hist_kernel<<<grid, 256, 0, s>>>(h->st, h->stamp, h->risk_pos, h->risk_slot, w, B, (long long)h->C);
+    risk_pick_kernel<<<1, 1024, 0, s>>>(h->st, w, B, (long long)h->C);
+    risk_collect_kernel<<<grid, 256, 0, s>>>(h->st, h->stamp, w, B, (long long)h->C);
+    risk_finish_kernel<<<1, 1024, 0, s>>>(h->st, w, h->risk_pos, h->risk_slot, h->risk_stamp, B, (long long)h->C);
+    h->launches += 4;
 }
 
 void launch_probe(prox_handle *h, const float *q, int B, int mode, cudaStream_t s) {

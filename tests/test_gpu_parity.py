@@ -164,6 +164,31 @@ def test_probe_only_prefilled_cache(policy, n_keys):
     p.close()
 
 
+@pytest.mark.parametrize("policy", ["lru", "fifo"])
+def test_probe_only_cache_above_the_multi_block_risk_selection(policy):
+    """More than 65536 keys: the at-risk entries are picked by the histogram kernels spread over
+    the GPU; the slots that misses overwrite show the eviction order."""
+    n_keys, d = 70000, 64
+    keys, centres = W.make_probe_keys(n_keys, d, 512, seed=21)
+    tau = 0.02                                              # queries around keys hit, fresh draws mostly miss
+    p = prox.Prox(keys[:64].contiguous().to(DEV), 1, n_keys, tau, policy)
+    p.cache_load(keys.to(DEV))
+    o = oracle.Oracle(None, d, 1, n_keys, float(np.float32(tau)), oracle.LRU if policy == "lru" else oracle.FIFO)
+    o.cache_load(keys.numpy())
+    misses = 0
+    for b in range(4):
+        Q = W.make_probe_batch(keys, centres, 1000, 0.01, 21, b)
+        hit, slot, dist = p.probe_batch(Q.to(DEV))
+        torch.cuda.synchronize()
+        r = o.query(Q.numpy())
+        assert np.array_equal(hit.cpu().numpy(), r["hit"])
+        assert np.array_equal(slot.cpu().numpy(), r["slot"])
+        misses += int((r["hit"] == 0).sum())
+    assert 100 < misses < 3900
+    assert p.status() == prox.OK
+    p.close()
+
+
 def test_large_cache_stream_with_coarse_probe():
     """Capacity above the switch-over to the tensor-core probe, pre-filled and full, so that the
     stream evicts from its first miss on; lists of pre-filled keys are the empty ones on both sides."""
