@@ -220,6 +220,7 @@ scan_cc_kernel(const DevState *__restrict__ st, const __nv_bfloat16 *__restrict_
 // memory when it fits; radix select on the 32-bit ordered score, then a collection pass.
 // ------------------------------------------------------------------------------------------
 constexpr int kMergeStage = 8192;                  // entries staged in shared memory
+constexpr int kMergeStageMax = 24576;              // ... when few rows were scanned, so that every row may be an entry
 
 struct MergeSrc {
     const u64 *buf;                                // lists of this query: list p at buf + p * list_stride
@@ -239,7 +240,7 @@ struct MergeSrc {
 };
 
 __global__ void __launch_bounds__(1024)
-merge_select_kernel(const int *__restrict__ n_active, int pass, int n_lists, int stride, int kp,
+merge_select_kernel(const int *__restrict__ n_active, int pass, int n_lists, int stride, int kp, int stage_cap,
                     const u64 *__restrict__ buf, const int32_t *__restrict__ buf_cnt,
                     const uint32_t *__restrict__ thr_g, int32_t *cand_id, float *cand_score, int32_t *cand_n,
                     float *cand_sk) {
@@ -274,7 +275,7 @@ merge_select_kernel(const int *__restrict__ n_active, int pass, int n_lists, int
                 int base = 0;
                 if (lane == 0) base = atomicAdd(&s_total, __popc(mask));
                 base = __shfl_sync(0xffffffffu, base, 0) + __popc(mask & ((1u << lane) - 1u));
-                if (keep && base < kMergeStage) stage[base] = ent;
+                if (keep && base < stage_cap) stage[base] = ent;
             }
         }
     }
@@ -285,7 +286,7 @@ merge_select_kernel(const int *__restrict__ n_active, int pass, int n_lists, int
     src.list_stride = (size_t)kScanQ * stride;
     src.cnt_stride = kScanQ;
     src.n_lists = n_lists; src.cap = stride; src.g0 = g0; src.total = s_total;
-    src.stage = (s_total <= kMergeStage) ? stage : nullptr;
+    src.stage = (s_total <= stage_cap) ? stage : nullptr;
     const int total = src.total, span = src.span();
 
     uint32_t T = 0;                                // ordered score of the k'-th best (0: keep all)
@@ -649,11 +650,14 @@ void launch_merge_select(prox_handle *h, int pass, int B, int for_probe, cudaStr
     if (nq <= 0) return;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaFuncSetAttribute(merge_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeStage * 8);
+        cudaFuncSetAttribute(merge_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeStageMax * 8);
         attr_set = true;
     }
-    merge_select_kernel<<<nq, 1024, kMergeStage * 8, s>>>(for_probe ? &h->st->n_probe : &h->st->n_miss, pass,
-                                                          h->scan_lists, h->scan_list_stride, for_probe ? kProbeKp : h->kp,
+    // a scan of few rows never tightens its bounds, so every row may still be in the lists: stage them all
+    const long long rows = for_probe ? (long long)h->C : (long long)h->N;
+    const int stage_cap = rows <= kMergeStageMax ? (int)((rows + 1023) / 1024 * 1024) : kMergeStage;
+    merge_select_kernel<<<nq, 1024, (size_t)stage_cap * 8, s>>>(for_probe ? &h->st->n_probe : &h->st->n_miss, pass,
+                                                          h->scan_lists, h->scan_list_stride, for_probe ? kProbeKp : h->kp, stage_cap,
                                                           h->buf, h->buf_cnt, h->thr_g, h->cand_id, h->cand_score,
                                                           h->cand_n, h->cand_sk);
     h->launches++;
