@@ -45,6 +45,8 @@ def lib():
         L.oracle_sqdist.argtypes = [fp, fp, C.c_int32]
         L.oracle_create.restype = C.c_void_p
         L.oracle_create.argtypes = [fp, C.c_int64, C.c_int32, C.c_int32, C.c_int64, C.c_double, C.c_int32]
+        L.oracle_create_rho.restype = C.c_void_p
+        L.oracle_create_rho.argtypes = [fp, C.c_int64, C.c_int32, C.c_int32, C.c_int64, C.c_double, C.c_int32, C.c_int32]
         L.oracle_destroy.argtypes = [C.c_void_p]
         L.oracle_reset.argtypes = [C.c_void_p]
         L.oracle_counters.argtypes = [C.c_void_p, ip]
@@ -116,16 +118,19 @@ class ChunkedTopK:
 
 class Oracle:
     """Algorithm 1 as a sequential state machine.  ``corpus=None`` gives the cache trace only
-    (hits, slots, evictions depend on the query stream alone; lists are then filled with -1)."""
+    (hits, slots, evictions depend on the query stream alone; lists are then filled with -1).
+    ``rho`` is the re-ranking factor: rho * k neighbours are fetched and stored per miss, and a
+    hit returns the k of them nearest to the current query (rho = 1: the stored list as it is)."""
 
-    def __init__(self, corpus, d: int, k: int, capacity: int, tau: float, policy: int):
+    def __init__(self, corpus, d: int, k: int, capacity: int, tau: float, policy: int, rho: int = 1):
         self._X = None if corpus is None else _f32(corpus)
         N = 0 if self._X is None else self._X.shape[0]
         if self._X is not None:
             assert self._X.shape[1] == d
         self.d, self.k, self.capacity, self.tau, self.policy = d, k, capacity, float(tau), policy
-        self._h = lib().oracle_create(None if self._X is None else _ptr(self._X, C.c_float),
-                                      N, d, k, capacity, float(tau), policy)
+        self.rho = int(rho)
+        self._h = lib().oracle_create_rho(None if self._X is None else _ptr(self._X, C.c_float),
+                                          N, d, k, capacity, float(tau), policy, self.rho)
         if not self._h:
             raise ValueError("oracle_create rejected the arguments")
 

@@ -28,7 +28,12 @@
  *   - every query owns one logical time stamp; an insert counts as a use;
  *   - a hit returns the stored list (and the stored distances of the key's own
  *     query) unchanged and alters nothing but the LRU stamp;
- *   - an empty cache is a miss; capacity 0 is rejected.
+ *   - an empty cache is a miss; capacity 0 is rejected;
+ *   - re-ranking factor rho (Section 3.3, "The re-ranking factor"): a miss asks the database for
+ *     m = rho * k neighbours, stores all m under the key and returns the k nearest of them; a hit
+ *     measures the m stored rows against the CURRENT query and returns the k nearest (distance
+ *     ascending, ties to the lower row id) with those distances.  rho = 1 is "no re-ranking"
+ *     (Section 4): the stored list comes back as it is, as above.
  *
  * All sums are taken in double precision over the float inputs, one term
  * after the other in index order.  OpenMP only splits independent rows over
@@ -50,13 +55,14 @@ typedef struct {
     const float *corpus;   /* N x d, borrowed; NULL = trace-only (no database) */
     int64_t N;
     int32_t d, k;
+    int32_t rho, m;        /* re-ranking factor and m = rho * k entries per value list */
     int64_t capacity;
     double tau;
     int32_t policy;
     /* the dict C: slot s holds a key (copy of the query), its value list */
     float *keys;           /* capacity x d */
-    int64_t *val_ids;      /* capacity x k */
-    double *val_dists;     /* capacity x k */
+    int64_t *val_ids;      /* capacity x m */
+    double *val_dists;     /* capacity x m */
     int64_t *stamp;        /* capacity: LRU = last use, FIFO = insertion time */
     int64_t *origin;       /* capacity: stream index of the query that made the key */
     uint8_t *valid;        /* capacity */
@@ -131,23 +137,29 @@ void oracle_exact_topk(const float *corpus, int64_t N, int32_t d, const float *q
     for (int32_t r = have; r < k; ++r) { out_ids[r] = -1; out_dists[r] = INFINITY; }
 }
 
-oracle_t *oracle_create(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
-                        double tau, int32_t policy) {
-    if (d < 1 || k < 1 || capacity < 1 || !(tau >= 0.0)) return NULL;
+oracle_t *oracle_create_rho(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
+                            double tau, int32_t policy, int32_t rho) {
+    if (d < 1 || k < 1 || capacity < 1 || rho < 1 || !(tau >= 0.0)) return NULL;
     if (policy != ORACLE_LRU && policy != ORACLE_FIFO) return NULL;
-    if (corpus && (N < 1 || k > N)) return NULL;
+    const int32_t m = rho * k;
+    if (corpus && (N < 1 || m > N)) return NULL;
     oracle_t *o = (oracle_t *)calloc(1, sizeof(oracle_t));
     if (!o) return NULL;
-    o->corpus = corpus; o->N = N; o->d = d; o->k = k;
+    o->corpus = corpus; o->N = N; o->d = d; o->k = k; o->rho = rho; o->m = m;
     o->capacity = capacity; o->tau = tau; o->policy = policy;
     o->keys = (float *)calloc((size_t)capacity * d, sizeof(float));
-    o->val_ids = (int64_t *)calloc((size_t)capacity * k, sizeof(int64_t));
-    o->val_dists = (double *)calloc((size_t)capacity * k, sizeof(double));
+    o->val_ids = (int64_t *)calloc((size_t)capacity * m, sizeof(int64_t));
+    o->val_dists = (double *)calloc((size_t)capacity * m, sizeof(double));
     o->stamp = (int64_t *)calloc((size_t)capacity, sizeof(int64_t));
     o->origin = (int64_t *)calloc((size_t)capacity, sizeof(int64_t));
     o->valid = (uint8_t *)calloc((size_t)capacity, 1);
     o->scratch = corpus ? (double *)malloc(sizeof(double) * (size_t)N) : NULL;
     return o;
+}
+
+oracle_t *oracle_create(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
+                        double tau, int32_t policy) {
+    return oracle_create_rho(corpus, N, d, k, capacity, tau, policy, 1);
 }
 
 void oracle_destroy(oracle_t *o) {
@@ -174,7 +186,7 @@ int oracle_cache_load(oracle_t *o, const float *keys, int64_t n) {
     memcpy(o->keys, keys, sizeof(float) * (size_t)n * o->d);
     for (int64_t s = 0; s < n; ++s) {
         o->valid[s] = 1; o->stamp[s] = s; o->origin[s] = -1 - s;
-        for (int32_t r = 0; r < o->k; ++r) { o->val_ids[s * o->k + r] = -1; o->val_dists[s * o->k + r] = 0.0; }
+        for (int32_t r = 0; r < o->m; ++r) { o->val_ids[s * o->m + r] = -1; o->val_dists[s * o->m + r] = 0.0; }
     }
     o->count = n; o->clock = n;
     return 0;
@@ -196,7 +208,7 @@ int oracle_cache_load(oracle_t *o, const float *keys, int64_t n) {
  */
 void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids, double *out_dists,
                    int64_t *trace, double *dtrace) {
-    const int32_t d = o->d, k = o->k;
+    const int32_t d = o->d, k = o->k, m = o->m;
     const int64_t t = o->clock++;                 /* this query's time stamp */
 
     /* lines 2-3 of Algorithm 1: all key distances, then the minimum (first minimum in slot order) */
@@ -217,18 +229,41 @@ void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids,
 
     if (hit) {                                     /* line 5: return C[key] */
         if (o->policy == ORACLE_LRU) o->stamp[best_slot] = t;   /* a hit is a use (LRU only) */
-        if (out_ids) memcpy(out_ids, o->val_ids + best_slot * k, sizeof(int64_t) * k);
-        if (out_dists) memcpy(out_dists, o->val_dists + best_slot * k, sizeof(double) * k);
+        const int64_t *sid = o->val_ids + best_slot * m;
+        if (o->rho == 1 || !o->corpus) {           /* no re-ranking: the stored list, as it is */
+            if (out_ids) memcpy(out_ids, sid, sizeof(int64_t) * k);
+            if (out_dists) memcpy(out_dists, o->val_dists + best_slot * m, sizeof(double) * k);
+        } else {
+            /* re-ranking: the m stored rows measured against this query, the k nearest returned;
+               insertion in (distance, row id) order, one stored row after the other */
+            int64_t *rid = (int64_t *)malloc(sizeof(int64_t) * m);
+            double *rd = (double *)malloc(sizeof(double) * m);
+            int32_t have = 0;
+            for (int32_t r = 0; r < m; ++r) {
+                if (sid[r] < 0) continue;          /* the corpus had fewer than m rows */
+                const double v = oracle_sqdist(q, o->corpus + sid[r] * (int64_t)d, d);
+                int32_t pos = have;
+                while (pos > 0 && (rd[pos - 1] > v || (rd[pos - 1] == v && rid[pos - 1] > sid[r]))) {
+                    rd[pos] = rd[pos - 1]; rid[pos] = rid[pos - 1]; --pos;
+                }
+                rd[pos] = v; rid[pos] = sid[r]; ++have;
+            }
+            for (int32_t r = 0; r < k; ++r) {
+                if (out_ids) out_ids[r] = r < have ? rid[r] : -1;
+                if (out_dists) out_dists[r] = r < have ? rd[r] : INFINITY;
+            }
+            free(rid); free(rd);
+        }
         if (trace) { trace[0] = 1; trace[1] = best_slot; trace[2] = o->origin[best_slot]; trace[3] = -1; }
         o->n_hits++;
         return;
     }
 
     /* line 6: I <- D.retrieveDocumentIndices(q) */
-    int64_t *ids = (int64_t *)malloc(sizeof(int64_t) * k);
-    double *dists = (double *)malloc(sizeof(double) * k);
-    if (o->corpus) oracle_exact_topk(o->corpus, o->N, d, q, k, o->scratch, ids, dists);
-    else for (int32_t r = 0; r < k; ++r) { ids[r] = -1; dists[r] = 0.0; }
+    int64_t *ids = (int64_t *)malloc(sizeof(int64_t) * m);
+    double *dists = (double *)malloc(sizeof(double) * m);
+    if (o->corpus) oracle_exact_topk(o->corpus, o->N, d, q, m, o->scratch, ids, dists);   /* m = rho * k neighbours */
+    else for (int32_t r = 0; r < m; ++r) { ids[r] = -1; dists[r] = 0.0; }
 
     /* lines 7-8: if |C| >= c evict one entry (the smallest stamp; stamps are unique) */
     int64_t slot, evicted = -1;
@@ -244,12 +279,12 @@ void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids,
 
     /* line 9: C[q] <- I */
     memcpy(o->keys + slot * d, q, sizeof(float) * d);
-    memcpy(o->val_ids + slot * k, ids, sizeof(int64_t) * k);
-    memcpy(o->val_dists + slot * k, dists, sizeof(double) * k);
+    memcpy(o->val_ids + slot * m, ids, sizeof(int64_t) * m);
+    memcpy(o->val_dists + slot * m, dists, sizeof(double) * m);
     o->valid[slot] = 1; o->stamp[slot] = t; o->origin[slot] = t; o->count++;
     o->n_misses++;
 
-    /* line 10: return I */
+    /* line 10: return I (its k nearest when more were fetched) */
     if (out_ids) memcpy(out_ids, ids, sizeof(int64_t) * k);
     if (out_dists) memcpy(out_dists, dists, sizeof(double) * k);
     if (trace) { trace[0] = 0; trace[1] = slot; trace[2] = t; trace[3] = evicted; }

@@ -225,3 +225,76 @@ def test_forced_decisions_follow_the_branch():
     r = o.query(Q, force)
     assert r["hit"][5] == 1 and np.array_equal(r["ids"][5], r["ids"][r["origin"][5]])
     assert r["hit"].sum() == 1
+
+
+# ---------------------------------------------------------------- re-ranking factor rho (Section 3.3)
+def np_sq(q, rows):
+    return ((q.astype(np.float64)[None, :] - rows.astype(np.float64)) ** 2).sum(1)
+
+
+def test_rho_one_is_the_plain_cache():
+    X, Q, _ = small_workload(seed=3)
+    a = oracle.Oracle(X, X.shape[1], 5, 10, 0.5, oracle.LRU).query(Q)
+    b = oracle.Oracle(X, X.shape[1], 5, 10, 0.5, oracle.LRU, rho=1).query(Q)
+    for key in ("ids", "dists", "hit", "slot", "evicted"):
+        assert np.array_equal(a[key], b[key])
+
+
+def test_rho_hand_worked_line():
+    """Points on a line, k = 1, rho = 2.  Query 0.0 misses and stores its two nearest points
+    (0.1 -> row 0, -0.3 -> row 1) and returns row 0.  Query -0.25 lies within tau of that key:
+    among the stored rows the one nearest to -0.25 is row 1 at 0.05^2; without re-ranking the
+    stored head, row 0, would come back with the key's own distance 0.1^2."""
+    X = np.array([[0.1], [-0.3], [0.9], [-2.0]], np.float32)
+    Q = np.array([[0.0], [-0.25]], np.float32)
+    r = oracle.Oracle(X, 1, 1, 4, 0.1, oracle.FIFO, rho=2).query(Q)
+    assert r["hit"].tolist() == [0, 1]
+    assert r["ids"][:, 0].tolist() == [0, 1]
+    assert r["dists"][0, 0] == pytest.approx(np.float64(np.float32(0.1)) ** 2, rel=1e-15)
+    assert r["dists"][1, 0] == pytest.approx((np.float64(np.float32(-0.25)) - np.float64(np.float32(-0.3))) ** 2, rel=1e-15)
+    r1 = oracle.Oracle(X, 1, 1, 4, 0.1, oracle.FIFO, rho=1).query(Q)
+    assert r1["ids"][:, 0].tolist() == [0, 0] and r1["dists"][1, 0] == r1["dists"][0, 0]
+
+
+@pytest.mark.parametrize("rho", [2, 4])
+def test_rho_miss_returns_knn_and_hit_reranks_the_stored_rows(rho):
+    X, Q, _ = small_workload(seed=5, N=600, nq=200)
+    k = 5
+    o = oracle.Oracle(X, X.shape[1], k, 4, 0.5, oracle.LRU, rho=rho)      # four entries: topics keep falling out
+    r = o.query(Q)
+    assert 0.2 < r["hit"].mean() < 0.95
+    wide_ids, _ = oracle.exact_topk(X, Q, rho * k)
+    for i in range(len(Q)):
+        if r["hit"][i] == 0:                                   # the k nearest of the rho k fetched
+            full = np_sq(Q[i], X)
+            order = np.lexsort((np.arange(len(X)), full))[:k]
+            assert np.array_equal(r["ids"][i], order)
+            assert np.allclose(r["dists"][i], full[order], rtol=1e-12)
+        else:                                                  # the k of the key's rho k rows nearest to THIS query
+            stored = wide_ids[r["origin"][i]]
+            dd = np_sq(Q[i], X[stored])
+            order = np.lexsort((stored, dd))[:k]
+            assert np.array_equal(r["ids"][i], stored[order])
+            assert np.allclose(r["dists"][i], dd[order], rtol=1e-12)
+            # a re-ranked list can never beat the true neighbours of the query
+            true = np.sort(np_sq(Q[i], X))[:k]
+            assert np.all(r["dists"][i] >= true * (1 - 1e-12))
+
+
+def test_rho_storing_the_whole_corpus_makes_every_hit_exact():
+    """rho * k = N: every key stores all rows, so a re-ranked hit is the exact answer for the
+    current query, whatever key matched."""
+    X, Q, _ = small_workload(seed=6, N=40, nq=60, topics=5)
+    k, rho = 5, 8
+    r = oracle.Oracle(X, X.shape[1], k, 6, 1.0, oracle.FIFO, rho=rho).query(Q)
+    assert r["hit"].sum() > 10
+    ids, dists = oracle.exact_topk(X, Q, k)
+    assert np.array_equal(r["ids"], ids) and np.allclose(r["dists"], dists, rtol=1e-12)
+
+
+def test_rho_duplicate_query_gets_the_head_of_the_stored_list():
+    X, Q, _ = small_workload(seed=7)
+    Q2 = np.concatenate([Q[:1], Q[:1]])
+    r = oracle.Oracle(X, X.shape[1], 4, 5, 0.0, oracle.LRU, rho=3).query(Q2)
+    assert r["hit"].tolist() == [0, 1]
+    assert np.array_equal(r["ids"][0], r["ids"][1]) and np.array_equal(r["dists"][0], r["dists"][1])
