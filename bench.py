@@ -212,7 +212,7 @@ def run_ours(args):
     results = {}
     handle_args = None
     for tau in taus:
-        p = prox.Prox(corpus, k, cfg.capacity, tau, cfg.policy)
+        p = prox.Prox(corpus, k, cfg.capacity, tau, cfg.policy, rho=args.rho)
         B = cfg.batch
         n_use = K * B
         ids = torch.empty(n_use, k, dtype=torch.int64, device=dev)
@@ -302,7 +302,7 @@ def run_ours(args):
         config=dict(workload=f"{cfg.name}: N={cfg.N} d={cfg.d} k={cfg.k} capacity={cfg.capacity} policy={cfg.policy} "
                              f"batch={cfg.batch} tau={head_tau} topics={cfg.n_topics} zipf={cfg.zipf_s} sigma={cfg.sigma}",
                     tau=head_tau, hit_rate=round(head["hit_rate"], 4), l2="inputs_exceed_l2" if cfg.N * cfg.d * 2 > 126e6 else "corpus_fits_l2",
-                    parallelism=f"replica x{world}", seed=args.seed, gen_seconds=round(t_gen, 1)),
+                    parallelism=f"replica x{world}", rho=args.rho, seed=args.seed, gen_seconds=round(t_gen, 1)),
         clocks=head["clocks"],
         e2e=dict(value=round(e2e, 1), unit=UNIT, h2d_bytes_per_step=head["h2d"], d2h_bytes_per_step=head["d2h"]),
         gpu_launches=int(head["launches"]),
@@ -469,6 +469,7 @@ def main():
     ap.add_argument("--tau", type=float, default=None, help="one tolerance instead of the workload's sweep")
     ap.add_argument("--rows", type=int, default=0, help="override the corpus size (profiling runs)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling runs)")
+    ap.add_argument("--rho", type=int, default=1, help="re-ranking factor: rho * k rows fetched and stored per miss (1 = none)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--default-steps", type=int, default=800, help="cap of the timed batches when --steps is 0 (a whole query stream if it is shorter)")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)

@@ -45,6 +45,7 @@ enum {
 
 enum {
     PROX_MAX_K = 64,            /* largest k */
+    PROX_MAX_FETCH = 128,       /* largest rho * k (neighbours fetched and stored per miss) */
     PROX_MAX_BATCH = 1024,      /* largest B of one call */
     PROX_SCAN_AUTO = 0,         /* prox_set_scan_mode: tensor-core scan, two blocks per MMA (default) */
     PROX_SCAN_CUDA_CORE = 1,    /* prox_set_scan_mode: plain CUDA-core scan of the same bf16 scores */
@@ -70,6 +71,17 @@ prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, int32_t k, i
                          float tau, int32_t policy);
 
 /*
+ * prox_create_rho -- prox_create with the re-ranking factor rho >= 1 of Section 3.3
+ * ("The re-ranking factor"): a miss fetches the rho * k nearest corpus rows, stores all of
+ * them under the key and returns the k nearest; a hit measures the rho * k stored rows
+ * against the CURRENT query (exact squared distances) and returns the k nearest of them,
+ * nearest first, ties by lower id, with those distances.  rho = 1 is prox_create: no
+ * re-ranking, the stored list comes back as it is.  rho * k <= min(N, PROX_MAX_FETCH).
+ */
+prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
+                             float tau, int32_t policy, int32_t rho);
+
+/*
  * prox_query_batch -- LOOKUP(q) of Algorithm 1 for queries 0..B-1, with the
  * outcome of processing them strictly in index order: query i sees the inserts,
  * evictions and LRU touches of queries 0..i-1 of the same batch.
@@ -79,6 +91,8 @@ prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, int32_t k, i
  *             ties by lower id).  On a hit: the list stored with the matched key.
  *   out_dists DEVICE, B x k fp32: squared distances belonging to out_ids.  On a hit these
  *             are the distances stored with the key, i.e. those of the key's own query.
+ *             (With rho > 1, see prox_create_rho: a hit returns the k stored rows nearest
+ *             to this query with their distances to this query.)
  *   out_hit   DEVICE, B bytes: 1 = cache hit (Algorithm 1, line 5), 0 = miss (lines 6-10).
  *   stream    a cudaStream_t (NULL = the default stream).
  * Misses are answered by an exact k-nearest-neighbour search over the whole corpus

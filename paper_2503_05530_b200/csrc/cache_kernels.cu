@@ -657,7 +657,7 @@ __global__ void gather_hits_kernel(int B, int k, const int32_t *__restrict__ src
 
 // Misses return their fresh list (line 10); hits on a key inserted earlier in the batch return
 // that query's list; entries that own a slot at batch end are written (line 9).
-__global__ void scatter_kernel(int B, int d, int k, int with_values, const float *__restrict__ queries,
+__global__ void scatter_kernel(int B, int d, int k, int k_out, int with_values, const float *__restrict__ queries,
                                const int32_t *__restrict__ src, const int32_t *__restrict__ src_kind,
                                const int32_t *__restrict__ ins_slot,
                                const int32_t *__restrict__ miss_rank,
@@ -671,10 +671,12 @@ __global__ void scatter_kernel(int B, int d, int k, int with_values, const float
     const int kind = src_kind[i];
     const int owner = (kind == 0) ? i : (kind == 2 ? src[i] : -1);
     const int m = (owner >= 0) ? miss_rank[owner] : -1;
-    if (with_values && m >= 0) {
-        for (int r = threadIdx.x; r < k; r += blockDim.x) {
-            out_ids[(size_t)i * k + r] = (int64_t)res_ids[(size_t)m * k + r];
-            out_dists[(size_t)i * k + r] = (float)res_dists[(size_t)m * k + r];
+    // a miss returns the k_out nearest of the k rows it fetched; with re-ranking (k > k_out) a hit
+    // on a key of this batch was answered by the re-ranking kernel
+    if (with_values && m >= 0 && (kind == 0 || k == k_out)) {
+        for (int r = threadIdx.x; r < k_out; r += blockDim.x) {
+            out_ids[(size_t)i * k_out + r] = (int64_t)res_ids[(size_t)m * k + r];
+            out_dists[(size_t)i * k_out + r] = (float)res_dists[(size_t)m * k + r];
         }
     }
     const int slot = ins_slot[i];
@@ -857,7 +859,7 @@ void launch_gather_hits(prox_handle *h, int B, int64_t *out_ids, float *out_dist
 
 void launch_scatter(prox_handle *h, const float *q, int B, int64_t *out_ids, float *out_dists,
                     int with_values, cudaStream_t s) {
-    scatter_kernel<<<B, 128, 0, s>>>(B, h->d, h->k, with_values, q, h->src, h->src_kind, h->ins_slot,
+    scatter_kernel<<<B, 128, 0, s>>>(B, h->d, h->k, h->k_out, with_values, q, h->src, h->src_kind, h->ins_slot,
                                      h->miss_rank, h->res_ids, h->res_dists, h->keys, h->val_ids,
                                      h->val_dists, out_ids, out_dists, h->probe_tc ? h->keys_b : nullptr, h->kh,
                                      h->st);

@@ -107,11 +107,22 @@ static int check_launch(const char *what) {
 
 extern "C" prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, int32_t k,
                                     int64_t capacity, float tau, int32_t policy) {
+    return prox_create_rho(corpus, N, d, k, capacity, tau, policy, 1);
+}
+
+extern "C" prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t d, int32_t k_out,
+                                        int64_t capacity, float tau, int32_t policy, int32_t rho) {
     g_err[0] = 0;
+    if (rho < 1) { set_err("rho must be >= 1"); return nullptr; }
+    if (k_out < 1 || k_out > kMaxK || k_out > N) { set_err("k must be in [1, min(N, %d)]", kMaxK); return nullptr; }
+    if ((long long)rho * k_out > kMaxFetch || (long long)rho * k_out > N) {
+        set_err("rho * k must be at most min(N, %d)", kMaxFetch);
+        return nullptr;
+    }
+    const int32_t k = rho * k_out;                        // entries fetched and stored per miss
     if (!corpus) { set_err("corpus is NULL"); return nullptr; }
     if (N < 1 || N >= (1LL << 31)) { set_err("N must be in [1, 2^31)"); return nullptr; }
     if (d < 16 || d > 4096 || d % 16) { set_err("d must be a multiple of 16 in [16, 4096]"); return nullptr; }
-    if (k < 1 || k > kMaxK || k > N) { set_err("k must be in [1, min(N, %d)]", kMaxK); return nullptr; }
     if (capacity < 1 || capacity >= (1LL << 31)) { set_err("capacity must be in [1, 2^31)"); return nullptr; }
     if (!(tau >= 0.f) || std::isinf(tau)) { set_err("tau must be finite and >= 0"); return nullptr; }
     if (policy != PROX_LRU && policy != PROX_FIFO) { set_err("policy must be PROX_LRU or PROX_FIFO"); return nullptr; }
@@ -119,7 +130,7 @@ extern "C" prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, i
     prox_handle *h = new (std::nothrow) prox_handle();
     if (!h) { set_err("out of host memory"); return nullptr; }
     std::memset(h, 0, sizeof(*h));
-    h->corpus = corpus; h->N = N; h->d = d; h->k = k; h->C = capacity; h->tau = tau; h->policy = policy;
+    h->corpus = corpus; h->N = N; h->d = d; h->k = k; h->k_out = k_out; h->rho = rho; h->C = capacity; h->tau = tau; h->policy = policy;
     h->kp = 4 * k < 64 ? 64 : (4 * k > kMaxKp ? kMaxKp : 4 * k);
     h->scan_mode = PROX_SCAN_AUTO;
     cudaDeviceProp prop;
@@ -250,7 +261,11 @@ extern "C" int32_t prox_query_batch(prox_handle *h, const float *queries, int32_
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
     enqueue_probe_and_resolve(h, queries, B, out_hit, s);
-    { StageScope t(h, PROX_STAGE_GATHER, s); launch_gather_hits(h, B, out_ids, out_dists, s); }
+    {
+        StageScope t(h, PROX_STAGE_GATHER, s);
+        if (h->rho == 1) launch_gather_hits(h, B, out_ids, out_dists, s);
+        else launch_hit_rerank(h, queries, B, 1, out_ids, out_dists, s);     // before the scatter rewrites slots
+    }
     { StageScope t(h, PROX_STAGE_PREP_MISS, s); launch_prep_miss(h, queries, B, s); }
     const int passes = (B + kScanQ - 1) / kScanQ;
     for (int p = 0; p < passes; ++p) {
@@ -262,7 +277,11 @@ extern "C" int32_t prox_query_batch(prox_handle *h, const float *queries, int32_
     }
     { StageScope t(h, PROX_STAGE_RERANK, s); launch_rerank(h, queries, B, s); }
     { StageScope t(h, PROX_STAGE_EXACT_PASS, s); launch_fallback(h, queries, B, s); }
-    { StageScope t(h, PROX_STAGE_SCATTER, s); launch_scatter(h, queries, B, out_ids, out_dists, 1, s); }
+    {
+        StageScope t(h, PROX_STAGE_SCATTER, s);
+        if (h->rho > 1) launch_hit_rerank(h, queries, B, 2, out_ids, out_dists, s);   // hits on keys of this batch
+        launch_scatter(h, queries, B, out_ids, out_dists, 1, s);
+    }
     return check_launch("prox_query_batch");
 }
 
@@ -272,7 +291,7 @@ extern "C" int32_t prox_query_batch_host(prox_handle *h, const float *queries, i
     if (rc) return rc;
     if (!out_ids || !out_dists || !out_hit) { set_err("an output pointer is NULL"); return PROX_ERR_INVALID_ARG; }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const size_t k = h->k;
+    const size_t k = h->k_out;
     if (cudaMemcpyAsync(h->stage_q, queries, (size_t)B * h->d * sizeof(float), cudaMemcpyHostToDevice, s) !=
         cudaSuccess)
         return check_launch("copy of the queries");

@@ -9,6 +9,7 @@
 namespace prox {
 
 constexpr int kMaxK = PROX_MAX_K;            // largest k
+constexpr int kMaxFetch = PROX_MAX_FETCH;    // largest rho * k
 constexpr int kMaxKp = 256;                  // largest k' (candidates kept by the coarse scan)
 constexpr int kMaxBatch = PROX_MAX_BATCH;    // largest B
 constexpr int kScanQ = 256;                  // queries per scan pass (MMA N dimension)
@@ -45,7 +46,8 @@ struct prox_handle {
     // stored state of Algorithm 1
     const float *corpus;      // N x d fp32, borrowed
     int64_t N;
-    int32_t d, k, kp;
+    int32_t d, k, kp;         // k: entries of a value list (rho * k_out)
+    int32_t k_out, rho;       // neighbours returned per query; re-ranking factor
     int64_t C;
     float tau;
     int32_t policy;
@@ -134,6 +136,8 @@ void launch_probe(prox_handle *h, const float *q, int B, int mode, cudaStream_t 
 void launch_build_candidates(prox_handle *h, int B, cudaStream_t s);
 void launch_resolve(prox_handle *h, int B, uint8_t *out_hit, cudaStream_t s);
 void launch_gather_hits(prox_handle *h, int B, int64_t *out_ids, float *out_dists, cudaStream_t s);
+void launch_hit_rerank(prox_handle *h, const float *q, int B, int kind, int64_t *out_ids, float *out_dists,
+                       cudaStream_t s);   // rho > 1: hits of that kind (1 stored key, 2 key of this batch)
 void launch_scatter(prox_handle *h, const float *q, int B, int64_t *out_ids, float *out_dists,
                     int with_values, cudaStream_t s);
 void launch_probe_outputs(prox_handle *h, int B, int32_t *out_slot, float *out_min_dist, cudaStream_t s);

@@ -444,6 +444,45 @@ rerank_kernel(DevState *st, int mode, const float *__restrict__ corpus, const fl
 }
 
 // ------------------------------------------------------------------------------------------
+// Re-ranking of a hit (Section 3.3, re-ranking factor rho > 1): the k stored rows of the matched
+// key measured against the current query in fp64, sorted by (distance, row id), the k_out
+// nearest returned.  kind 1: key stored before the batch (list in the value slots); kind 2: key
+// inserted earlier in this batch (list in the batch's results).  Stored id -1 (a pre-loaded key
+// without a list) sorts last and comes back as -1 with an infinite distance.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+hit_rerank_kernel(int B, int d, int k, int k_out, int kind, const float *__restrict__ corpus,
+                  const float *__restrict__ queries, const int32_t *__restrict__ src,
+                  const int32_t *__restrict__ src_kind, const int32_t *__restrict__ miss_rank,
+                  const int32_t *__restrict__ val_ids, const int32_t *__restrict__ res_ids, int64_t *out_ids,
+                  float *out_dists) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *sd = reinterpret_cast<double *>(smem_raw);                 // kMaxFetch
+    int *sid = reinterpret_cast<int *>(sd + kMaxFetch);                // kMaxFetch
+    float *q_sm = reinterpret_cast<float *>(sid + kMaxFetch);          // d
+    const int i = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (i >= B || src_kind[i] != kind) return;
+    const int32_t *ids = kind == 1 ? val_ids + (size_t)src[i] * k : res_ids + (size_t)miss_rank[src[i]] * k;
+    for (int j = tid; j < d; j += blockDim.x) q_sm[j] = queries[(size_t)i * d + j];
+    int n2 = 1;
+    while (n2 < k) n2 <<= 1;
+    for (int e = tid; e < n2; e += blockDim.x) { sd[e] = INFINITY; sid[e] = 0x7fffffff; }
+    __syncthreads();
+    for (int c = warp; c < k; c += 8) {
+        const int row = ids[c];
+        if (row < 0) continue;
+        const double v = exact_sqdist_warp(q_sm, corpus + (size_t)row * d, d);
+        if (lane == 0) { sd[c] = v; sid[c] = row; }
+    }
+    block_sort_asc(sd, sid, n2);
+    for (int r = tid; r < k_out; r += blockDim.x) {
+        const bool have = sid[r] != 0x7fffffff;
+        out_ids[(size_t)i * k_out + r] = have ? (int64_t)sid[r] : -1;
+        out_dists[(size_t)i * k_out + r] = have ? (float)sd[r] : INFINITY;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // Exact pass for uncertified queries: every corpus row within the radius (the exact k-th
 // candidate distance) in fp32 difference form, with the fp32 rounding margin on top.
 // Eight queries per sweep of the corpus; one warp per row.
@@ -678,6 +717,14 @@ void launch_rerank(prox_handle *h, const float *q, int B, cudaStream_t s) {
                                                     h->miss_list, h->cand_id, h->cand_n, h->cand_sk, h->qbn,
                                                     h->qerr, h->res_ids, h->res_dists, h->fail_list,
                                                     h->fail_radius, h->coll_id, h->coll_n);
+    h->launches++;
+}
+
+void launch_hit_rerank(prox_handle *h, const float *q, int B, int kind, int64_t *out_ids, float *out_dists,
+                       cudaStream_t s) {
+    const size_t smem = (size_t)kMaxFetch * 12 + (size_t)h->d * 4;
+    hit_rerank_kernel<<<B, 256, smem, s>>>(B, h->d, h->k, h->k_out, kind, h->corpus, q, h->src, h->src_kind,
+                                           h->miss_rank, h->val_ids, h->res_ids, out_ids, out_dists);
     h->launches++;
 }
 

@@ -51,6 +51,8 @@ def load_library():
     vp, i32, i64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
     L.prox_create.restype = vp
     L.prox_create.argtypes = [vp, i64, i32, i32, i64, f32, i32]
+    L.prox_create_rho.restype = vp
+    L.prox_create_rho.argtypes = [vp, i64, i32, i32, i64, f32, i32, i32]
     L.prox_query_batch.restype = i32
     L.prox_query_batch.argtypes = [vp, vp, i32, vp, vp, vp, vp]
     L.prox_query_batch_host.restype = i32
@@ -116,15 +118,16 @@ def nearest_key_static(keys: torch.Tensor, queries: torch.Tensor, out_slot: torc
 class Prox:
     """prox_create / prox_query_batch / prox_reset_cache / prox_destroy with tensors."""
 
-    def __init__(self, corpus: torch.Tensor, k: int, capacity: int, tau: float, policy="lru"):
+    def __init__(self, corpus: torch.Tensor, k: int, capacity: int, tau: float, policy="lru", rho: int = 1):
         self._lib = load_library()
         self._corpus = _dev_f32(corpus, "corpus")      # borrowed by the library: keep it alive
         self.N, self.d = corpus.shape
         self.k, self.capacity, self.tau = int(k), int(capacity), float(tau)
         self.policy = _POLICY[policy]
+        self.rho = int(rho)                            # re-ranking factor (prox_create_rho); 1 = prox_create
         with torch.cuda.device(corpus.device):
-            self._h = self._lib.prox_create(corpus.data_ptr(), self.N, self.d, self.k, self.capacity,
-                                            self.tau, self.policy)
+            self._h = self._lib.prox_create_rho(corpus.data_ptr(), self.N, self.d, self.k, self.capacity,
+                                                self.tau, self.policy, self.rho)
         if not self._h:
             raise ProxError(f"prox_create failed: {last_error()}")
         self.device = corpus.device

@@ -16,9 +16,9 @@ REL_TIE = 1e-5
 REL_DIST = 1e-4
 
 
-def run_gpu(corpus_t, queries_t, k, capacity, tau, policy, batch, scan_mode=None, host_api=False):
+def run_gpu(corpus_t, queries_t, k, capacity, tau, policy, batch, scan_mode=None, host_api=False, rho=1):
     """corpus_t, queries_t: CUDA float32 tensors.  Returns numpy (ids, dists, hit) and the stats."""
-    p = prox.Prox(corpus_t, k, capacity, tau, policy)
+    p = prox.Prox(corpus_t, k, capacity, tau, policy, rho=rho)
     try:
         if scan_mode is not None:
             p.set_scan_mode(scan_mode)
@@ -45,7 +45,7 @@ def run_gpu(corpus_t, queries_t, k, capacity, tau, policy, batch, scan_mode=None
     return ids.cpu().numpy(), dists.cpu().numpy(), hit.cpu().numpy(), stats
 
 
-def run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=None, max_forced=16):
+def run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=None, max_forced=16, rho=1):
     """Oracle on the same bytes.  tau is rounded to float32 first, as the C ABI takes a float.
     If gpu_hit is given, queries whose decision ties with tau (rule (i)) adopt the GPU's
     decision so that both state machines stay in step; returns the list of such queries."""
@@ -54,7 +54,7 @@ def run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=None, max_forc
     force = np.full(len(queries), -1, np.int32)
     forced = []
     while True:
-        o = oracle.Oracle(corpus, d, k, capacity, tau32, POL[policy])
+        o = oracle.Oracle(corpus, d, k, capacity, tau32, POL[policy], rho=rho)
         r = o.query(queries, force)
         o.close()
         if gpu_hit is None:
@@ -80,9 +80,9 @@ def knn_tie_excused(corpus, q, k):
     return bool(np.any(gaps < REL_TIE * np.maximum(d[1:], 1e-300)))
 
 
-def compare(corpus, queries, k, capacity, tau, policy, gpu, max_excused_frac=1e-3):
+def compare(corpus, queries, k, capacity, tau, policy, gpu, max_excused_frac=1e-3, rho=1):
     ids, dists, hit, stats = gpu
-    ref, forced = run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=hit)
+    ref, forced = run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=hit, rho=rho)
     n = len(queries)
     bad_hit = np.nonzero(ref["hit"] != hit)[0]
     assert len(bad_hit) == 0, f"hit/miss differs first at query {bad_hit[0]} (best={ref['best'][bad_hit[0]]}, tau={tau})"
@@ -91,8 +91,12 @@ def compare(corpus, queries, k, capacity, tau, policy, gpu, max_excused_frac=1e-
     for i in rows_bad:
         origin = int(ref["origin"][i])                       # the miss whose list is returned
         src = origin if origin >= 0 else i
-        assert knn_tie_excused(corpus, queries[src], k), \
-            f"ids differ at query {i} (list of query {src}): oracle {ref['ids'][i]} gpu {ids[i]}"
+        tie = knn_tie_excused(corpus, queries[src], k * rho)
+        if not tie and rho > 1 and src != i:                 # re-ranked hit: a tie among the stored rows for this query
+            stored, _ = oracle.exact_topk(corpus, queries[src], k * rho)
+            dd = np.sort(((queries[i].astype(np.float64)[None, :] - corpus[stored[0]].astype(np.float64)) ** 2).sum(1))
+            tie = bool(np.any(np.diff(dd) < REL_TIE * np.maximum(dd[1:], 1e-300)))
+        assert tie, f"ids differ at query {i} (list of query {src}): oracle {ref['ids'][i]} gpu {ids[i]}"
         excused.add(int(i))
     ok_rows = np.setdiff1d(np.arange(n), rows_bad)
     rd, gd = ref["dists"][ok_rows], dists[ok_rows].astype(np.float64)

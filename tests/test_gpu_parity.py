@@ -21,7 +21,7 @@ def stream(N, d, comps, nq, topics, s, sigma, seed=0):
 
 def check(X, Q, k, cap, tau, policy, batch, **kw):
     gpu = run_gpu(X.to(DEV), Q.to(DEV), k, cap, tau, policy, batch, **kw)
-    return compare(X.numpy(), Q.numpy(), k, cap, tau, policy, gpu), gpu
+    return compare(X.numpy(), Q.numpy(), k, cap, tau, policy, gpu, rho=kw.get("rho", 1)), gpu
 
 
 # ------------------------------------------------------------------ hand-traced sequences
@@ -139,6 +139,34 @@ def test_uncertified_queries_take_the_exact_pass():
     ids, dists = oracle.exact_topk(X.numpy(), Q.numpy(), 10)
     assert np.array_equal(gpu[0], ids)
     assert np.allclose(gpu[1], dists, rtol=1e-4, atol=1e-12)
+
+
+# ------------------------------------------------------------------ re-ranking factor (Section 3.3)
+@pytest.mark.parametrize("policy,batch,rho,k", [("lru", 64, 4, 10), ("fifo", 1, 2, 5), ("lru", 200, 2, 32),
+                                                ("fifo", 1024, 4, 32)])
+def test_reranking_factor_matches_the_oracle(policy, batch, rho, k):
+    """rho * k rows fetched and stored per miss, hits re-ranked against the current query: hits on
+    stored keys, hits on keys of the same batch and capacity below the batch size all occur."""
+    X, Q = stream(30011, 128, 48, 2300, 120, 1.0, 0.03, seed=31)
+    res, gpu = check(X, Q, k, 40, 0.25, policy, batch, rho=rho)
+    assert 0.3 < res["hit_rate"] < 0.97
+    if batch > 1:
+        assert gpu[3]["intra_batch_hits"] > 0
+    # a re-ranked list differs from the stored head for a good share of the hits
+    plain = run_gpu(X.to(DEV), Q.to(DEV), k, 40, 0.25, policy, batch, rho=1)
+    h = res["ref"]["hit"] == 1
+    assert (plain[0][h] != gpu[0][h]).any(axis=1).mean() > 0.05
+
+
+def test_reranking_factor_argument_checks():
+    Xd = torch.randn(500, 64, device=DEV).contiguous()
+    lib = prox.load_library()
+    for k, rho in [(10, 0), (33, 4), (64, 3), (10, 60)]:
+        assert not lib.prox_create_rho(Xd.data_ptr(), 500, 64, k, 8, 0.5, 0, rho), (k, rho)
+        assert "rho" in prox.last_error()
+    h = lib.prox_create_rho(Xd.data_ptr(), 500, 64, 32, 8, 0.5, 0, 4)
+    assert h
+    lib.prox_destroy(h)
 
 
 # ------------------------------------------------------------------ probe only, pre-filled cache
