@@ -47,6 +47,11 @@ def lib():
         L.oracle_create.argtypes = [fp, C.c_int64, C.c_int32, C.c_int32, C.c_int64, C.c_double, C.c_int32]
         L.oracle_create_rho.restype = C.c_void_p
         L.oracle_create_rho.argtypes = [fp, C.c_int64, C.c_int32, C.c_int32, C.c_int64, C.c_double, C.c_int32, C.c_int32]
+        L.oracle_create_lsh.restype = C.c_void_p
+        L.oracle_create_lsh.argtypes = [fp, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32, fp, C.c_double,
+                                        C.c_int32, C.c_int32]
+        L.oracle_lsh_hash.restype = C.c_int64
+        L.oracle_lsh_hash.argtypes = [fp, C.c_int32, C.c_int32, fp]
         L.oracle_destroy.argtypes = [C.c_void_p]
         L.oracle_reset.argtypes = [C.c_void_p]
         L.oracle_counters.argtypes = [C.c_void_p, ip]
@@ -96,6 +101,13 @@ def exact_topk(corpus, queries, k: int):
     return ids, dists
 
 
+def lsh_hash(planes, q) -> int:
+    """h(q) of PROXIMITY-LSH: bit l is (q . r_l >= 0) for the l-th row of ``planes``."""
+    P, v = _f32(planes), _f32(q).ravel()
+    assert P.ndim == 2 and P.shape[1] == v.size
+    return int(lib().oracle_lsh_hash(_ptr(P, C.c_float), P.shape[0], P.shape[1], _ptr(v, C.c_float)))
+
+
 class ChunkedTopK:
     """The database call for ONE query with the corpus fed in ascending row chunks."""
 
@@ -120,17 +132,27 @@ class Oracle:
     """Algorithm 1 as a sequential state machine.  ``corpus=None`` gives the cache trace only
     (hits, slots, evictions depend on the query stream alone; lists are then filled with -1).
     ``rho`` is the re-ranking factor: rho * k neighbours are fetched and stored per miss, and a
-    hit returns the k of them nearest to the current query (rho = 1: the stored list as it is)."""
+    hit returns the k of them nearest to the current query (rho = 1: the stored list as it is).
+    ``lsh_planes`` (L x d) with ``lsh_bucket`` = b switches to PROXIMITY-LSH: 2^L buckets of b entries."""
 
-    def __init__(self, corpus, d: int, k: int, capacity: int, tau: float, policy: int, rho: int = 1):
+    def __init__(self, corpus, d: int, k: int, capacity: int, tau: float, policy: int, rho: int = 1,
+                 lsh_planes=None, lsh_bucket: int = 0):
         self._X = None if corpus is None else _f32(corpus)
         N = 0 if self._X is None else self._X.shape[0]
         if self._X is not None:
             assert self._X.shape[1] == d
         self.d, self.k, self.capacity, self.tau, self.policy = d, k, capacity, float(tau), policy
         self.rho = int(rho)
-        self._h = lib().oracle_create_rho(None if self._X is None else _ptr(self._X, C.c_float),
-                                          N, d, k, capacity, float(tau), policy, self.rho)
+        xp = None if self._X is None else _ptr(self._X, C.c_float)
+        if lsh_planes is None:
+            self._h = lib().oracle_create_rho(xp, N, d, k, capacity, float(tau), policy, self.rho)
+        else:
+            # PROXIMITY-LSH: one bucket of lsh_bucket entries per hash code; capacity = 2^L * lsh_bucket
+            self._P = _f32(lsh_planes).reshape(-1, d)
+            L_ = self._P.shape[0]
+            assert capacity == (1 << L_) * lsh_bucket, "capacity must be 2^L * bucket size"
+            self._h = lib().oracle_create_lsh(xp, N, d, k, L_, lsh_bucket, _ptr(self._P, C.c_float) if L_ else None,
+                                              float(tau), policy, self.rho)
         if not self._h:
             raise ValueError("oracle_create rejected the arguments")
 

@@ -33,7 +33,15 @@
  *     m = rho * k neighbours, stores all m under the key and returns the k nearest of them; a hit
  *     measures the m stored rows against the CURRENT query and returns the k nearest (distance
  *     ascending, ties to the lower row id) with those distances.  rho = 1 is "no re-ranking"
- *     (Section 4): the stored list comes back as it is, as above.
+ *     (Section 4): the stored list comes back as it is, as above;
+ *   - PROXIMITY-LSH (Section 3.2): L random hyperplanes through the origin, given by the caller
+ *     as L normal vectors; bit l of the hash is (q . r_l >= 0), the dot product taken in fp64
+ *     in index order; the 2^L buckets are PROXIMITY-FLAT caches of b entries each, every one
+ *     with its own FIFO / LRU eviction (Section 3.3.2, last sentence); bucket h owns the slots
+ *     h*b .. h*b+b-1, filled in that order; time stamps stay global (one per query), which
+ *     orders the entries of a bucket exactly as bucket-local stamps would.  Memory for all
+ *     buckets is taken at once (the paper allocates a bucket at its first insert; the contents
+ *     are the same).
  *
  * All sums are taken in double precision over the float inputs, one term
  * after the other in index order.  OpenMP only splits independent rows over
@@ -56,6 +64,9 @@ typedef struct {
     int64_t N;
     int32_t d, k;
     int32_t rho, m;        /* re-ranking factor and m = rho * k entries per value list */
+    int32_t lsh_L, lsh_b;  /* PROXIMITY-LSH: hyperplanes and bucket size; lsh_L < 0 = PROXIMITY-FLAT */
+    float *planes;         /* lsh_L x d normal vectors (copy) */
+    int64_t *bucket_count; /* 2^lsh_L */
     int64_t capacity;
     double tau;
     int32_t policy;
@@ -145,7 +156,7 @@ oracle_t *oracle_create_rho(const float *corpus, int64_t N, int32_t d, int32_t k
     if (corpus && (N < 1 || m > N)) return NULL;
     oracle_t *o = (oracle_t *)calloc(1, sizeof(oracle_t));
     if (!o) return NULL;
-    o->corpus = corpus; o->N = N; o->d = d; o->k = k; o->rho = rho; o->m = m;
+    o->corpus = corpus; o->N = N; o->d = d; o->k = k; o->rho = rho; o->m = m; o->lsh_L = -1;
     o->capacity = capacity; o->tau = tau; o->policy = policy;
     o->keys = (float *)calloc((size_t)capacity * d, sizeof(float));
     o->val_ids = (int64_t *)calloc((size_t)capacity * m, sizeof(int64_t));
@@ -162,8 +173,33 @@ oracle_t *oracle_create(const float *corpus, int64_t N, int32_t d, int32_t k, in
     return oracle_create_rho(corpus, N, d, k, capacity, tau, policy, 1);
 }
 
+/* h(q) of Section 3.2: bit l = (q . r_l >= 0). */
+int64_t oracle_lsh_hash(const float *planes, int32_t L, int32_t d, const float *q) {
+    int64_t h = 0;
+    for (int32_t l = 0; l < L; ++l) {
+        double dot = 0.0;
+        for (int32_t j = 0; j < d; ++j) dot += (double)q[j] * (double)planes[(int64_t)l * d + j];
+        if (dot >= 0.0) h |= (int64_t)1 << l;
+    }
+    return h;
+}
+
+/* PROXIMITY-LSH: 2^L buckets of b entries; total capacity 2^L * b (Section 3.3.1). */
+oracle_t *oracle_create_lsh(const float *corpus, int64_t N, int32_t d, int32_t k, int32_t L, int32_t b,
+                            const float *planes, double tau, int32_t policy, int32_t rho) {
+    if (L < 0 || L > 24 || b < 1 || (L > 0 && !planes)) return NULL;
+    oracle_t *o = oracle_create_rho(corpus, N, d, k, ((int64_t)1 << L) * b, tau, policy, rho);
+    if (!o) return NULL;
+    o->lsh_L = L; o->lsh_b = b;
+    o->planes = (float *)malloc(sizeof(float) * (size_t)(L > 0 ? L : 1) * d);
+    if (L > 0) memcpy(o->planes, planes, sizeof(float) * (size_t)L * d);
+    o->bucket_count = (int64_t *)calloc((size_t)1 << L, sizeof(int64_t));
+    return o;
+}
+
 void oracle_destroy(oracle_t *o) {
     if (!o) return;
+    free(o->planes); free(o->bucket_count);
     free(o->keys); free(o->val_ids); free(o->val_dists); free(o->stamp);
     free(o->origin); free(o->valid); free(o->scratch); free(o);
 }
@@ -171,6 +207,7 @@ void oracle_destroy(oracle_t *o) {
 void oracle_reset(oracle_t *o) {
     memset(o->valid, 0, (size_t)o->capacity);
     o->count = 0; o->clock = 0;
+    if (o->bucket_count) memset(o->bucket_count, 0, sizeof(int64_t) << o->lsh_L);
     o->probe_madds = 0; o->n_hits = o->n_misses = o->n_evictions = 0;
 }
 
@@ -212,9 +249,16 @@ void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids,
     const int64_t t = o->clock++;                 /* this query's time stamp */
 
     /* lines 2-3 of Algorithm 1: all key distances, then the minimum (first minimum in slot order) */
+    /* PROXIMITY-LSH: only the bucket that the hash names is looked at and updated */
+    int64_t s_begin = 0, s_end = o->capacity, bucket = -1;
+    if (o->lsh_L >= 0) {
+        bucket = oracle_lsh_hash(o->planes, o->lsh_L, d, q);
+        o->probe_madds += (int64_t)o->lsh_L * d;
+        s_begin = bucket * o->lsh_b; s_end = s_begin + o->lsh_b;
+    }
     double best = INFINITY, second = INFINITY;
     int64_t best_slot = -1;
-    for (int64_t s = 0; s < o->capacity; ++s) {
+    for (int64_t s = s_begin; s < s_end; ++s) {
         if (!o->valid[s]) continue;
         double dist = oracle_sqdist(q, o->keys + s * d, d);
         o->probe_madds += d;
@@ -267,14 +311,16 @@ void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids,
 
     /* lines 7-8: if |C| >= c evict one entry (the smallest stamp; stamps are unique) */
     int64_t slot, evicted = -1;
-    if (o->count >= o->capacity) {
+    const int64_t held = bucket >= 0 ? o->bucket_count[bucket] : o->count;      /* |C| of this (bucket's) cache */
+    if (held >= s_end - s_begin) {
         slot = -1;
-        for (int64_t s = 0; s < o->capacity; ++s)
+        for (int64_t s = s_begin; s < s_end; ++s)
             if (o->valid[s] && (slot < 0 || o->stamp[s] < o->stamp[slot])) slot = s;
         o->valid[slot] = 0; o->count--; o->n_evictions++;
+        if (bucket >= 0) o->bucket_count[bucket]--;
         evicted = slot;
     } else {
-        slot = o->count;                           /* slots fill in index order */
+        slot = s_begin + held;                     /* slots fill in index order */
     }
 
     /* line 9: C[q] <- I */
@@ -282,6 +328,7 @@ void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids,
     memcpy(o->val_ids + slot * m, ids, sizeof(int64_t) * m);
     memcpy(o->val_dists + slot * m, dists, sizeof(double) * m);
     o->valid[slot] = 1; o->stamp[slot] = t; o->origin[slot] = t; o->count++;
+    if (bucket >= 0) o->bucket_count[bucket]++;
     o->n_misses++;
 
     /* line 10: return I (its k nearest when more were fetched) */

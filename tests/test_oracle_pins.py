@@ -298,3 +298,74 @@ def test_rho_duplicate_query_gets_the_head_of_the_stored_list():
     r = oracle.Oracle(X, X.shape[1], 4, 5, 0.0, oracle.LRU, rho=3).query(Q2)
     assert r["hit"].tolist() == [0, 1]
     assert np.array_equal(r["ids"][0], r["ids"][1]) and np.array_equal(r["dists"][0], r["dists"][1])
+
+
+# ---------------------------------------------------------------- PROXIMITY-LSH (Section 3.2)
+def planes_for(L, d, seed):
+    return np.random.default_rng(seed).standard_normal((L, d)).astype(np.float32)
+
+
+def test_lsh_hash_is_the_sign_pattern():
+    P = planes_for(10, 48, 1)
+    for q in unit_rows(50, 48, 2):
+        bits = (P.astype(np.float64) @ q.astype(np.float64)) >= 0
+        assert oracle.lsh_hash(P, q) == int(sum(1 << l for l in range(10) if bits[l]))
+    assert oracle.lsh_hash(P, np.zeros(48, np.float32)) == (1 << 10) - 1          # 0 >= 0 on every plane
+    assert oracle.lsh_hash(P[:3], -P[1]) & 2 == 0 and oracle.lsh_hash(P[:3], P[1]) & 2 == 2
+
+
+@pytest.mark.parametrize("policy", ["lru", "fifo"])
+def test_lsh_with_no_hyperplane_is_the_flat_cache(policy):
+    X, Q, _ = small_workload(seed=9)
+    d = X.shape[1]
+    flat = oracle.Oracle(X, d, 5, 12, 0.5, POL[policy]).query(Q)
+    lsh = oracle.Oracle(X, d, 5, 12, 0.5, POL[policy], lsh_planes=np.zeros((0, d), np.float32), lsh_bucket=12).query(Q)
+    for key in ("ids", "dists", "hit", "slot", "evicted", "best"):
+        assert np.array_equal(flat[key], lsh[key])
+
+
+def test_lsh_buckets_are_independent_flat_caches():
+    """Queries are dealt to their buckets; every bucket must behave like a flat cache of b
+    entries fed with its own queries alone (own eviction, Section 3.3.2), with slots h*b.."""
+    X, Q, _ = small_workload(seed=10, nq=300, topics=40)
+    d, L, b = X.shape[1], 3, 2
+    P = planes_for(L, d, 4)
+    r = oracle.Oracle(X, d, 4, (1 << L) * b, 0.6, oracle.LRU, lsh_planes=P, lsh_bucket=b).query(Q)
+    code = np.array([oracle.lsh_hash(P, q) for q in Q])
+    assert len(np.unique(code)) >= 4 and r["evicted"].max() >= 0
+    for h in np.unique(code):
+        sel = np.nonzero(code == h)[0]
+        f = oracle.Oracle(X, d, 4, b, 0.6, oracle.LRU).query(Q[sel])
+        assert np.array_equal(f["hit"], r["hit"][sel]) and np.array_equal(f["ids"], r["ids"][sel])
+        assert np.array_equal(f["slot"] + h * b, r["slot"][sel])
+        ev = f["evicted"].copy(); ev[ev >= 0] += h * b
+        assert np.array_equal(ev, r["evicted"][sel])
+
+
+def test_lsh_never_matches_across_buckets_even_with_a_huge_tau():
+    X, Q, _ = small_workload(seed=11)
+    d = X.shape[1]
+    P = planes_for(4, d, 5)
+    r = oracle.Oracle(X, d, 3, 16 * 5, 100.0, oracle.FIFO, lsh_planes=P, lsh_bucket=5).query(Q)
+    code = np.array([oracle.lsh_hash(P, q) for q in Q])
+    first = {}
+    for i, h in enumerate(code):
+        assert r["hit"][i] == (1 if h in first else 0)                # only the first query of a bucket misses
+        first.setdefault(h, i)
+        assert r["slot"][i] == h * 5
+
+
+def test_lsh_operation_count_of_the_papers_example():
+    """Section 3.2: c = 10 000, d = 768, b = 20, L = 10: (L + b) d = 23 040 operations per lookup
+    once the bucket is full, against 7.68 million for the flat cache."""
+    d, L, b = 768, 10, 20
+    rng = np.random.default_rng(0)
+    base = rng.standard_normal(d).astype(np.float32)
+    Q = (base[None, :] + 1e-3 * rng.standard_normal((b + 1, d))).astype(np.float32)   # one bucket, distinct keys
+    P = planes_for(L, d, 6)
+    assert len({oracle.lsh_hash(P, q) for q in Q}) == 1
+    o = oracle.Oracle(None, d, 1, (1 << L) * b, 0.0, oracle.FIFO, lsh_planes=P, lsh_bucket=b)
+    o.query(Q[:b])
+    before = o.counters()["probe_madds"]
+    o.query(Q[b:])
+    assert o.counters()["probe_madds"] - before == (L + b) * d == 23040
