@@ -212,7 +212,12 @@ def run_ours(args):
     results = {}
     handle_args = None
     for tau in taus:
-        p = prox.Prox(corpus, k, cfg.capacity, tau, cfg.policy, rho=args.rho)
+        if args.lsh_bits >= 0:                                 # PROXIMITY-LSH: 2^L buckets of b entries
+            planes = torch.randn(args.lsh_bits, cfg.d, device=dev, generator=torch.Generator(device=dev).manual_seed(args.seed + 77))
+            p = prox.Prox(corpus, k, (1 << args.lsh_bits) * args.lsh_bucket, tau, cfg.policy, rho=args.rho,
+                          lsh_planes=planes, lsh_bucket=args.lsh_bucket)
+        else:
+            p = prox.Prox(corpus, k, cfg.capacity, tau, cfg.policy, rho=args.rho)
         B = cfg.batch
         n_use = K * B
         ids = torch.empty(n_use, k, dtype=torch.int64, device=dev)
@@ -302,7 +307,8 @@ def run_ours(args):
         config=dict(workload=f"{cfg.name}: N={cfg.N} d={cfg.d} k={cfg.k} capacity={cfg.capacity} policy={cfg.policy} "
                              f"batch={cfg.batch} tau={head_tau} topics={cfg.n_topics} zipf={cfg.zipf_s} sigma={cfg.sigma}",
                     tau=head_tau, hit_rate=round(head["hit_rate"], 4), l2="inputs_exceed_l2" if cfg.N * cfg.d * 2 > 126e6 else "corpus_fits_l2",
-                    parallelism=f"replica x{world}", rho=args.rho, seed=args.seed, gen_seconds=round(t_gen, 1)),
+                    parallelism=f"replica x{world}", rho=args.rho,
+                    cache="flat" if args.lsh_bits < 0 else f"lsh L={args.lsh_bits} b={args.lsh_bucket}", seed=args.seed, gen_seconds=round(t_gen, 1)),
         clocks=head["clocks"],
         e2e=dict(value=round(e2e, 1), unit=UNIT, h2d_bytes_per_step=head["h2d"], d2h_bytes_per_step=head["d2h"]),
         gpu_launches=int(head["launches"]),
@@ -449,6 +455,36 @@ def run_probe(args):
                                           kernel="scan_tc_kernel over the keys" if coarse else "probe_kernel")))
             p.close()
         del keys, batches
+    # PROXIMITY-LSH at the paper's setting (L = 10, b = 20, capacity 20 480): filled by a pass of keys, then timed
+    lsh = None
+    if not args.rows or args.rows >= 20480:
+        Lb, bb = 10, 20
+        keys, centres = W.make_probe_keys(1 << 15, d, 4096, args.seed, dev)
+        planes = torch.randn(Lb, d, device=dev, generator=torch.Generator(device=dev).manual_seed(args.seed + 77))
+        p = prox.Prox(keys[:64].contiguous(), 1, (1 << Lb) * bb, tau, "lru", lsh_planes=planes, lsh_bucket=bb)
+        for a in range(0, keys.shape[0], B):
+            p.probe_batch(keys[a:a + B])
+        batches = [W.make_probe_batch(keys, centres, B, 0.02, args.seed, b_) for b_ in range(K + args.warmup)]
+        for q in batches[K:]:
+            p.probe_batch(q)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        hits = []
+        e0.record()
+        for q in batches[:K]:
+            hits.append(p.probe_batch(q)[0])
+        e1.record()
+        torch.cuda.synchronize()
+        assert p.status() == prox.OK, prox.last_error()
+        ms = e0.elapsed_time(e1) / K
+        st = p.stats()
+        alg_bytes = B * (Lb + bb) * d * 4                  # every query reads the hyperplanes and its bucket's keys
+        lsh = dict(L=Lb, b=bb, capacity=(1 << Lb) * bb, held=st["count"], us_per_batch=round(ms * 1e3, 1),
+                   queries_per_s=round(B / ms * 1e3, 1), hit_rate=round(float(torch.stack(hits).float().mean().item()), 4),
+                   roofline=dict(bound="hbm", achieved=round(alg_bytes / ms / 1e6, 1), peak=peaks["hbm_gbs"], unit="GB/s",
+                                 frac=round(alg_bytes / ms / 1e6 / peaks["hbm_gbs"], 4), traffic=None,
+                                 kernel="lsh_resolve_kernel (gather of one bucket per query, replay in order)"))
+        p.close()
     big = out[-1]
     print(json.dumps(dict(metric="probe_keys_scanned", value=big["keys_GBps"], unit="GB/s", n_gpus=1, steps=K,
                           warmup=args.warmup, ms_per_step=round(big["us_per_batch"] / 1e3, 4), higher_is_better=True,
@@ -456,7 +492,7 @@ def run_probe(args):
                           config=dict(workload=f"probe-only: B={B} d={d} tau={tau} keys from a 4096-component mixture, "
                                                f"C={big['C']} policy={big['policy']}", l2="keys_exceed_l2" if big["C"] * d * 4 > 126e6 else "keys_fit_l2"),
                           roofline=big["roofline"],
-                          points=out)), flush=True)
+                          points=out, lsh=lsh)), flush=True)
 
 
 def main():
@@ -470,6 +506,8 @@ def main():
     ap.add_argument("--rows", type=int, default=0, help="override the corpus size (profiling runs)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling runs)")
     ap.add_argument("--rho", type=int, default=1, help="re-ranking factor: rho * k rows fetched and stored per miss (1 = none)")
+    ap.add_argument("--lsh-bits", type=int, default=-1, help="PROXIMITY-LSH with this many hyperplanes (-1: flat cache)")
+    ap.add_argument("--lsh-bucket", type=int, default=20, help="entries per LSH bucket")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--default-steps", type=int, default=800, help="cap of the timed batches when --steps is 0 (a whole query stream if it is shorter)")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)

@@ -82,6 +82,24 @@ prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t d, int32_t 
                              float tau, int32_t policy, int32_t rho);
 
 /*
+ * prox_create_lsh -- PROXIMITY-LSH of Section 3.2: the cache is split into 2^L buckets of b
+ * entries; a query is looked up in, and on a miss inserted into, the one bucket that its hash
+ * h(q) = (q . r_1 >= 0, ..., q . r_L >= 0) names (bit l-1 of the bucket number belongs to r_l;
+ * dot products in fp64).  Every bucket is a PROXIMITY-FLAT cache with its own FIFO / LRU
+ * eviction (Section 3.3.2); bucket h owns the slots h*b .. h*b+b-1.  Total capacity 2^L * b.
+ *   planes   DEVICE, L x d fp32 row-major: the hyperplanes' normal vectors r_1..r_L, drawn by
+ *            the caller (the library draws no random numbers); copied.  May be NULL when L = 0.
+ *   L        0 <= L <= 20 (L = 0: one bucket, i.e. a flat cache of b entries).
+ *   b        bucket size, 1 <= b <= 64 (the paper uses 20), 2^L * b < 2^31.
+ *   rho      re-ranking factor as in prox_create_rho (1 = none).
+ * All buckets are allocated at once (the paper allocates a bucket at its first insert; with
+ * the memory of this GPU the difference is moot).  prox_cache_load is not available for such
+ * a handle.  Everything else (prox_query_batch, prox_probe_batch, ...) works as for a flat cache.
+ */
+prox_handle *prox_create_lsh(const float *corpus, int64_t N, int32_t d, int32_t k, int32_t L, int32_t b,
+                             const float *planes, float tau, int32_t policy, int32_t rho);
+
+/*
  * prox_query_batch -- LOOKUP(q) of Algorithm 1 for queries 0..B-1, with the
  * outcome of processing them strictly in index order: query i sees the inserts,
  * evictions and LRU touches of queries 0..i-1 of the same batch.

@@ -84,7 +84,7 @@ static bool dev_alloc(T *&p, size_t n) {
 }
 
 static void free_all(prox_handle *h) {
-    void *ptrs[] = {h->xb, h->xh, h->keys, h->val_ids, h->val_dists, h->stamp, h->risk_pos, h->st,
+    void *ptrs[] = {h->planes, h->bucket_count, h->lsh_code, h->lsh_order, h->lsh_seg, h->lsh_work, h->xb, h->xh, h->keys, h->val_ids, h->val_dists, h->stamp, h->risk_pos, h->st,
                     h->risk_slot, h->risk_stamp, h->part_min, h->part_arg, h->d_risk, h->d_intra,
                     h->safe_min, h->safe_arg, h->cand_d, h->cand_code, h->n_cand, h->src, h->src_kind,
                     h->ins_slot, h->evt_slot, h->evt_dist, h->miss_list, h->miss_rank, h->qb, h->qbn,
@@ -130,7 +130,7 @@ extern "C" prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t 
     prox_handle *h = new (std::nothrow) prox_handle();
     if (!h) { set_err("out of host memory"); return nullptr; }
     std::memset(h, 0, sizeof(*h));
-    h->corpus = corpus; h->N = N; h->d = d; h->k = k; h->k_out = k_out; h->rho = rho; h->C = capacity; h->tau = tau; h->policy = policy;
+    h->corpus = corpus; h->N = N; h->d = d; h->k = k; h->k_out = k_out; h->rho = rho; h->lsh_L = -1; h->C = capacity; h->tau = tau; h->policy = policy;
     h->kp = 4 * k < 64 ? 64 : (4 * k > kMaxKp ? kMaxKp : 4 * k);
     h->scan_mode = PROX_SCAN_AUTO;
     cudaDeviceProp prop;
@@ -205,6 +205,35 @@ extern "C" prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t 
     return h;
 }
 
+extern "C" prox_handle *prox_create_lsh(const float *corpus, int64_t N, int32_t d, int32_t k, int32_t L, int32_t b,
+                                        const float *planes, float tau, int32_t policy, int32_t rho) {
+    g_err[0] = 0;
+    if (L < 0 || L > 20) { set_err("L must be in [0, 20]"); return nullptr; }
+    if (b < 1 || b > 64) { set_err("the bucket size b must be in [1, 64]"); return nullptr; }
+    if (L > 0 && !planes) { set_err("planes is NULL"); return nullptr; }
+    if (((int64_t)b << L) >= (1LL << 31)) { set_err("2^L * b must be below 2^31"); return nullptr; }
+    prox_handle *h = prox_create_rho(corpus, N, d, k, (int64_t)b << L, tau, policy, rho);
+    if (!h) return nullptr;
+    h->lsh_L = L; h->lsh_b = b;
+    h->probe_tc = 0;                                      // buckets are probed directly; no bf16 key copies
+    const size_t MB = kMaxBatch;
+    bool ok = dev_alloc(h->planes, (size_t)(L > 0 ? L : 1) * d) && dev_alloc(h->bucket_count, (size_t)1 << L) &&
+              dev_alloc(h->lsh_code, MB) && dev_alloc(h->lsh_order, MB) && dev_alloc(h->lsh_seg, MB + 1) &&
+              dev_alloc(h->lsh_work, 4);
+    if (ok) {
+        if (L > 0) cudaMemcpy(h->planes, planes, (size_t)L * d * sizeof(float), cudaMemcpyDeviceToDevice);
+        cudaMemset(h->bucket_count, 0, sizeof(int32_t) << L);
+        ok = cudaDeviceSynchronize() == cudaSuccess;
+    }
+    if (!ok) {
+        set_err("out of device memory for the buckets: %s", cudaGetErrorString(cudaGetLastError()));
+        free_all(h);
+        delete h;
+        return nullptr;
+    }
+    return h;
+}
+
 extern "C" void prox_destroy(prox_handle *h) {
     if (!h) return;
     cudaDeviceSynchronize();
@@ -224,6 +253,11 @@ static int check_batch_args(prox_handle *h, const void *queries, int32_t B) {
 
 static void enqueue_probe_and_resolve(prox_handle *h, const float *queries, int32_t B, uint8_t *out_hit,
                                       cudaStream_t s) {
+    if (h->lsh_L >= 0) {                                  // PROXIMITY-LSH: the query's bucket only
+        StageScope t(h, PROX_STAGE_PROBE, s);
+        launch_lsh_probe(h, queries, B, out_hit, s);
+        return;
+    }
     { StageScope t(h, PROX_STAGE_RISK_SELECT, s); launch_risk_select(h, B, s); }
     {
         StageScope t(h, PROX_STAGE_PROBE, s);
@@ -324,6 +358,7 @@ extern "C" int32_t prox_reset_cache(prox_handle *h, void *stream) {
     g_err[0] = 0;
     if (!h) { set_err("handle is NULL"); return PROX_ERR_INVALID_ARG; }
     launch_reset(h, static_cast<cudaStream_t>(stream));
+    if (h->lsh_L >= 0) cudaMemsetAsync(h->bucket_count, 0, sizeof(int32_t) << h->lsh_L, static_cast<cudaStream_t>(stream));
     return check_launch("prox_reset_cache");
 }
 
@@ -332,6 +367,7 @@ extern "C" int32_t prox_cache_load(prox_handle *h, const float *keys, int64_t n,
     if (!h) { set_err("handle is NULL"); return PROX_ERR_INVALID_ARG; }
     if (n < 0 || n > h->C) { set_err("n must be in [0, capacity]"); return PROX_ERR_INVALID_ARG; }
     if (n > 0 && !keys) { set_err("keys is NULL"); return PROX_ERR_INVALID_ARG; }
+    if (h->lsh_L >= 0) { set_err("prox_cache_load is not available for a PROXIMITY-LSH handle"); return PROX_ERR_UNSUPPORTED; }
     launch_cache_load(h, keys, n, static_cast<cudaStream_t>(stream));
     return check_launch("prox_cache_load");
 }

@@ -48,6 +48,14 @@ struct prox_handle {
     int64_t N;
     int32_t d, k, kp;         // k: entries of a value list (rho * k_out)
     int32_t k_out, rho;       // neighbours returned per query; re-ranking factor
+    // PROXIMITY-LSH (lsh_L < 0: flat cache)
+    int32_t lsh_L, lsh_b;
+    float *planes;            // lsh_L x d normal vectors
+    int32_t *bucket_count;    // 2^lsh_L: entries held by each bucket
+    int32_t *lsh_code;        // kMaxBatch: bucket of each batch query
+    int32_t *lsh_order;       // kMaxBatch: batch queries sorted by (bucket, index)
+    int32_t *lsh_seg;         // kMaxBatch + 1: where each bucket's run starts in lsh_order
+    int32_t *lsh_work;        // [0] number of runs, [1] evictions, [2] hits on keys of this batch
     int64_t C;
     float tau;
     int32_t policy;
@@ -140,6 +148,7 @@ void launch_hit_rerank(prox_handle *h, const float *q, int B, int kind, int64_t 
                        cudaStream_t s);   // rho > 1: hits of that kind (1 stored key, 2 key of this batch)
 void launch_scatter(prox_handle *h, const float *q, int B, int64_t *out_ids, float *out_dists,
                     int with_values, cudaStream_t s);
+void launch_lsh_probe(prox_handle *h, const float *q, int B, uint8_t *out_hit, cudaStream_t s);   // hash, group, replay per bucket
 void launch_probe_outputs(prox_handle *h, int B, int32_t *out_slot, float *out_min_dist, cudaStream_t s);
 void launch_cache_load(prox_handle *h, const float *keys, int64_t n, cudaStream_t s);
 void launch_reset(prox_handle *h, cudaStream_t s);

@@ -53,6 +53,8 @@ def load_library():
     L.prox_create.argtypes = [vp, i64, i32, i32, i64, f32, i32]
     L.prox_create_rho.restype = vp
     L.prox_create_rho.argtypes = [vp, i64, i32, i32, i64, f32, i32, i32]
+    L.prox_create_lsh.restype = vp
+    L.prox_create_lsh.argtypes = [vp, i64, i32, i32, i32, i32, vp, f32, i32, i32]
     L.prox_query_batch.restype = i32
     L.prox_query_batch.argtypes = [vp, vp, i32, vp, vp, vp, vp]
     L.prox_query_batch_host.restype = i32
@@ -118,7 +120,8 @@ def nearest_key_static(keys: torch.Tensor, queries: torch.Tensor, out_slot: torc
 class Prox:
     """prox_create / prox_query_batch / prox_reset_cache / prox_destroy with tensors."""
 
-    def __init__(self, corpus: torch.Tensor, k: int, capacity: int, tau: float, policy="lru", rho: int = 1):
+    def __init__(self, corpus: torch.Tensor, k: int, capacity: int, tau: float, policy="lru", rho: int = 1,
+                 lsh_planes: torch.Tensor | None = None, lsh_bucket: int = 0):
         self._lib = load_library()
         self._corpus = _dev_f32(corpus, "corpus")      # borrowed by the library: keep it alive
         self.N, self.d = corpus.shape
@@ -126,8 +129,17 @@ class Prox:
         self.policy = _POLICY[policy]
         self.rho = int(rho)                            # re-ranking factor (prox_create_rho); 1 = prox_create
         with torch.cuda.device(corpus.device):
-            self._h = self._lib.prox_create_rho(corpus.data_ptr(), self.N, self.d, self.k, self.capacity,
-                                                self.tau, self.policy, self.rho)
+            if lsh_planes is None:
+                self._h = self._lib.prox_create_rho(corpus.data_ptr(), self.N, self.d, self.k, self.capacity,
+                                                    self.tau, self.policy, self.rho)
+            else:
+                # PROXIMITY-LSH (prox_create_lsh): 2^L buckets of lsh_bucket entries; capacity = 2^L * lsh_bucket
+                P = _dev_f32(lsh_planes.reshape(-1, self.d), "lsh_planes")
+                L_ = P.shape[0]
+                if self.capacity != (1 << L_) * lsh_bucket:
+                    raise ProxError("capacity must equal 2^L * lsh_bucket")
+                self._h = self._lib.prox_create_lsh(corpus.data_ptr(), self.N, self.d, self.k, L_, int(lsh_bucket),
+                                                    P.data_ptr() if L_ else None, self.tau, self.policy, self.rho)
         if not self._h:
             raise ProxError(f"prox_create failed: {last_error()}")
         self.device = corpus.device

@@ -16,9 +16,11 @@ REL_TIE = 1e-5
 REL_DIST = 1e-4
 
 
-def run_gpu(corpus_t, queries_t, k, capacity, tau, policy, batch, scan_mode=None, host_api=False, rho=1):
+def run_gpu(corpus_t, queries_t, k, capacity, tau, policy, batch, scan_mode=None, host_api=False, rho=1,
+            lsh_planes=None, lsh_bucket=0):
     """corpus_t, queries_t: CUDA float32 tensors.  Returns numpy (ids, dists, hit) and the stats."""
-    p = prox.Prox(corpus_t, k, capacity, tau, policy, rho=rho)
+    planes_t = None if lsh_planes is None else torch.as_tensor(lsh_planes).to(corpus_t.device)
+    p = prox.Prox(corpus_t, k, capacity, tau, policy, rho=rho, lsh_planes=planes_t, lsh_bucket=lsh_bucket)
     try:
         if scan_mode is not None:
             p.set_scan_mode(scan_mode)
@@ -45,7 +47,8 @@ def run_gpu(corpus_t, queries_t, k, capacity, tau, policy, batch, scan_mode=None
     return ids.cpu().numpy(), dists.cpu().numpy(), hit.cpu().numpy(), stats
 
 
-def run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=None, max_forced=16, rho=1):
+def run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=None, max_forced=16, rho=1, lsh_planes=None,
+               lsh_bucket=0):
     """Oracle on the same bytes.  tau is rounded to float32 first, as the C ABI takes a float.
     If gpu_hit is given, queries whose decision ties with tau (rule (i)) adopt the GPU's
     decision so that both state machines stay in step; returns the list of such queries."""
@@ -54,7 +57,7 @@ def run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=None, max_forc
     force = np.full(len(queries), -1, np.int32)
     forced = []
     while True:
-        o = oracle.Oracle(corpus, d, k, capacity, tau32, POL[policy], rho=rho)
+        o = oracle.Oracle(corpus, d, k, capacity, tau32, POL[policy], rho=rho, lsh_planes=lsh_planes, lsh_bucket=lsh_bucket)
         r = o.query(queries, force)
         o.close()
         if gpu_hit is None:
@@ -80,9 +83,10 @@ def knn_tie_excused(corpus, q, k):
     return bool(np.any(gaps < REL_TIE * np.maximum(d[1:], 1e-300)))
 
 
-def compare(corpus, queries, k, capacity, tau, policy, gpu, max_excused_frac=1e-3, rho=1):
+def compare(corpus, queries, k, capacity, tau, policy, gpu, max_excused_frac=1e-3, rho=1, lsh_planes=None, lsh_bucket=0):
     ids, dists, hit, stats = gpu
-    ref, forced = run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=hit, rho=rho)
+    ref, forced = run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=hit, rho=rho, lsh_planes=lsh_planes,
+                             lsh_bucket=lsh_bucket)
     n = len(queries)
     bad_hit = np.nonzero(ref["hit"] != hit)[0]
     assert len(bad_hit) == 0, f"hit/miss differs first at query {bad_hit[0]} (best={ref['best'][bad_hit[0]]}, tau={tau})"

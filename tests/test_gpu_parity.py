@@ -21,7 +21,8 @@ def stream(N, d, comps, nq, topics, s, sigma, seed=0):
 
 def check(X, Q, k, cap, tau, policy, batch, **kw):
     gpu = run_gpu(X.to(DEV), Q.to(DEV), k, cap, tau, policy, batch, **kw)
-    return compare(X.numpy(), Q.numpy(), k, cap, tau, policy, gpu, rho=kw.get("rho", 1)), gpu
+    return compare(X.numpy(), Q.numpy(), k, cap, tau, policy, gpu, rho=kw.get("rho", 1),
+                   lsh_planes=kw.get("lsh_planes"), lsh_bucket=kw.get("lsh_bucket", 0)), gpu
 
 
 # ------------------------------------------------------------------ hand-traced sequences
@@ -167,6 +168,41 @@ def test_reranking_factor_argument_checks():
     h = lib.prox_create_rho(Xd.data_ptr(), 500, 64, 32, 8, 0.5, 0, 4)
     assert h
     lib.prox_destroy(h)
+
+
+# ------------------------------------------------------------------ PROXIMITY-LSH (Section 3.2)
+@pytest.mark.parametrize("policy,batch,L,b,rho", [("lru", 1, 4, 3, 1), ("fifo", 64, 4, 3, 1), ("lru", 1000, 6, 2, 1),
+                                                  ("fifo", 256, 0, 7, 1), ("lru", 300, 5, 4, 2)])
+def test_lsh_cache_matches_the_oracle(policy, batch, L, b, rho):
+    """Buckets of a few entries and batches far larger than a bucket: hits on stored keys, on keys
+    of the same batch, and evictions of entries that the same batch inserted all occur."""
+    X, Q = stream(20011, 128, 32, 2400, 150, 0.9, 0.03, seed=41)
+    planes = torch.randn(L, 128, generator=torch.Generator().manual_seed(5)).numpy()
+    res, gpu = check(X, Q, 8, (1 << L) * b, 0.3, policy, batch, rho=rho, lsh_planes=planes, lsh_bucket=b)
+    assert 0.1 < res["hit_rate"] < 0.97
+    assert gpu[3]["evictions"] == int((res["ref"]["evicted"] >= 0).sum()) > 0
+    if batch > 1:
+        assert gpu[3]["intra_batch_hits"] > 0
+
+
+def test_lsh_probe_only_slots_and_argument_checks():
+    X, Q = stream(5000, 64, 16, 700, 60, 0.9, 0.03, seed=42)
+    planes = torch.randn(5, 64, generator=torch.Generator().manual_seed(6))
+    p = prox.Prox(X.to(DEV), 4, 32 * 3, 0.3, "lru", lsh_planes=planes.to(DEV), lsh_bucket=3)
+    o = oracle.Oracle(None, 64, 4, 32 * 3, float(np.float32(0.3)), oracle.LRU, lsh_planes=planes.numpy(), lsh_bucket=3)
+    for a in range(0, 700, 350):
+        hit, slot, dist = p.probe_batch(Q[a:a + 350].to(DEV))
+        torch.cuda.synchronize()
+        r = o.query(Q[a:a + 350].numpy())
+        assert np.array_equal(hit.cpu().numpy(), r["hit"]) and np.array_equal(slot.cpu().numpy(), r["slot"])
+    assert p.status() == prox.OK
+    with pytest.raises(prox.ProxError):
+        p.cache_load(Q[:8].to(DEV))
+    p.close()
+    lib = prox.load_library()
+    Xd = X.to(DEV)
+    for L, b in [(-1, 4), (21, 4), (3, 0), (3, 65)]:
+        assert not lib.prox_create_lsh(Xd.data_ptr(), 5000, 64, 4, L, b, planes.to(DEV).data_ptr(), 0.3, 0, 1)
 
 
 # ------------------------------------------------------------------ probe only, pre-filled cache
