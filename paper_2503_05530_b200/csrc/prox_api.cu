@@ -162,7 +162,7 @@ extern "C" prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t 
     ok = ok && dev_alloc(h->evt_slot, MB) && dev_alloc(h->evt_dist, MB);
     ok = ok && dev_alloc(h->miss_list, MB) && dev_alloc(h->miss_rank, MB);
     ok = ok && dev_alloc(h->qb, MB * d) && dev_alloc(h->qbn, MB) && dev_alloc(h->qerr, MB) && dev_alloc(h->thr_g, MB);
-    ok = ok && dev_alloc(h->top1, MB * P);
+    ok = ok && dev_alloc(h->top1, MB * 4 * P);          // per query: best score of every block's lane quarter
     h->tc_cap = h->kp <= 128 ? 256 : 512;               // four warp-private lists per block in the tensor-core scan
     const size_t buf_entries = P * kScanQ * (size_t)(4 * h->tc_cap > kBufCap ? 4 * h->tc_cap : kBufCap);
     ok = ok && dev_alloc(h->buf, buf_entries) && dev_alloc(h->buf_cnt, 4 * P * kScanQ);

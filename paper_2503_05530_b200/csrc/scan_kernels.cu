@@ -671,7 +671,7 @@ void launch_prep_miss(prox_handle *h, const float *q, int B, cudaStream_t s) {
     int rows = ((B + kScanQ - 1) / kScanQ) * kScanQ;      // zero the padding rows of the last pass too
     if (rows > kMaxBatch) rows = kMaxBatch;
     prep_miss_kernel<<<rows, 128, 0, s>>>(h->st, q, B, h->d, h->miss_list, h->qb, h->qbn, h->qerr, h->thr_g,
-                                          h->coll_n, h->top1, h->scan_ctas);
+                                          h->coll_n, h->top1, 4 * h->scan_ctas);
     h->launches++;
 }
 
@@ -747,7 +747,7 @@ void launch_prep_probe(prox_handle *h, const float *q, int B, cudaStream_t s) {
     int rows = ((B + kScanQ - 1) / kScanQ) * kScanQ;
     if (rows > kMaxBatch) rows = kMaxBatch;
     prep_probe_kernel<<<rows, 128, 0, s>>>(h->st, q, B, h->d, h->pqb, h->pqbn, h->pqerr, h->thr_g, h->top1,
-                                           h->scan_ctas, h->use_partial);
+                                           4 * h->scan_ctas, h->use_partial);
     h->launches++;
 }
 

@@ -63,7 +63,7 @@ struct ScanArgs {
 struct Control {
     unsigned long long full[kMaxStages], empty[kMaxStages], tmem_full[2], tmem_empty[2], q_full;
     alignas(16) float thr[kScanQ];   // per query: scores at or below it cannot be among the best k'
-    uint32_t best[kScanQ];           // best score this block has appended per query (ordered-uint form)
+    uint32_t best[4][kScanQ];        // best score appended per query by each lane quarter (ordered-uint form)
     int wcnt[kReadWarps][kReadCols];   // entries in each read-out warp's private candidate lists
     uint32_t tmem_base;
     int abort_flag;                  // set by any thread whose wait ran out
@@ -115,7 +115,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     const uint32_t stage0 = tiles0 + (resident ? (uint32_t)q_block_bytes : 0u);
     volatile int *abort_flag = &ctl.abort_flag;
     uint32_t *thr_g = a.thr_g + q0;
-    uint32_t *top1 = a.top1 + (size_t)q0 * gridDim.x;
+    uint32_t *top1 = a.top1 + (size_t)q0 * 4 * gridDim.x;      // [query][block][lane quarter]
     const long long ntiles = (a.N + kUnitRows - 1) / kUnitRows;
     // barriers the MMA-issuing block waits on: in a pair, both blocks signal block 0's copy
     const uint32_t tx_mult = PAIR ? 2u : 1u;
@@ -135,7 +135,10 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    for (int q = tid; q < kScanQ; q += kThreads) { ctl.thr[q] = q < nq ? -INFINITY : INFINITY; ctl.best[q] = 0u; }
+    for (int q = tid; q < kScanQ; q += kThreads) {
+        ctl.thr[q] = q < nq ? -INFINITY : INFINITY;
+        ctl.best[0][q] = 0u; ctl.best[1][q] = 0u; ctl.best[2][q] = 0u; ctl.best[3][q] = 0u;
+    }
     for (int i = tid; i < kReadWarps * kReadCols; i += kThreads) (&ctl.wcnt[0][0])[i] = 0;
     if (warp == 1) tmem_alloc<PAIR>(smem_u32(&ctl.tmem_base), kTmemCols);
     tc_fence_before();
@@ -228,27 +231,35 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         // is matched or exceeded by at least k' distinct rows: a lower bound of the query's global
         // k'-th best that tightens as every block publishes better rows.  Each block keeps the
         // bounds of the queries q = block (mod blocks) fresh while its read-out runs.
-        const int P = gridDim.x;
-        if (a.kp <= P && P <= 256) {
+        // The rows of a block split further into its four lane quarters, so there are four times
+        // as many disjoint row sets as blocks: a tighter bound, and one that exists for k' up to that.
+        const int P = 4 * gridDim.x;
+        if (a.kp <= P && P <= 1024) {
             volatile int *done = &ctl.done;
             int jq = blockIdx.x, jobs = 0;
             while (*done < kReadWarps && !*abort_flag) {
                 if (jq >= nq) jq = blockIdx.x;
                 if (jq < nq) {
-                    u64 t[8];
+                    uint32_t t[32];
 #pragma unroll
-                    for (int i8 = 0; i8 < 8; ++i8) {
+                    for (int i8 = 0; i8 < 32; ++i8) {
                         const int eidx = i8 * 32 + lane;
-                        t[i8] = (eidx < P) ? (u64)__ldcg(&top1[(size_t)jq * P + eidx]) : 0ull;
+                        t[i8] = (eidx < P) ? __ldcg(&top1[(size_t)jq * P + eidx]) : 0u;
                     }
-                    warp_sort_desc<8>(t);
-                    u64 rth = 0ull;
+                    // the k'-th largest of them, bit by bit: the largest value that at least k' reach
+                    uint32_t rth = 0u;
+#pragma unroll 1
+                    for (int bit = 31; bit >= 0; --bit) {
+                        const uint32_t cand = rth | (1u << bit);
+                        int n_ge = 0;
 #pragma unroll
-                    for (int i8 = 0; i8 < 8; ++i8) rth |= (i8 * 32 + lane == a.kp - 1) ? t[i8] : 0ull;
-                    rth = __shfl_sync(0xffffffffu, rth, (a.kp - 1) & 31);
-                    if (lane == 0 && (uint32_t)rth != 0u) atomicMax(&thr_g[jq], (uint32_t)rth);
+                        for (int i8 = 0; i8 < 32; ++i8) n_ge += t[i8] >= cand ? 1 : 0;
+                        n_ge = __reduce_add_sync(0xffffffffu, n_ge);
+                        if (n_ge >= a.kp) rth = cand;
+                    }
+                    if (lane == 0 && rth != 0u) atomicMax(&thr_g[jq], rth);
                 }
-                jq += P;
+                jq += gridDim.x;
                 // bounds move fast while the first tiles come in and slowly afterwards; this warp
                 // shares an issue port with read-out warps, so it backs off once they have settled
                 __nanosleep(++jobs < 48 ? 2000 : 20000);
@@ -332,22 +343,20 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     }
                 }
                 if (active && c0 < cw)
-                    readout64<CAP>(v0, v1, c0 + 32 < cw, col_begin + c0, c0, hn, (int32_t)row, ctl.thr, wcnt, ctl.best,
+                    readout64<CAP>(v0, v1, c0 + 32 < cw, col_begin + c0, c0, hn, (int32_t)row, ctl.thr, wcnt, ctl.best[quarter],
                                    lists, need);
                 if (last) break;
             }
-            // one warp per column publishes the block's best score
-            if (quarter == 0) {
+            // the warp publishes the best score of its lane quarter for each of its columns
 #pragma unroll
-                for (int i = 0; i < kReadGroups; ++i) {
-                    const int lc = lane + 32 * i;
-                    if (lc < ncol) {
-                        const int c = col_begin + lc;
-                        const uint32_t bq = ctl.best[c];
-                        if (bq > published[i]) {
-                            top1[(size_t)c * gridDim.x + blockIdx.x] = bq;
-                            published[i] = bq;
-                        }
+            for (int i = 0; i < kReadGroups; ++i) {
+                const int lc = lane + 32 * i;
+                if (lc < ncol) {
+                    const int c = col_begin + lc;
+                    const uint32_t bq = ctl.best[quarter][c];
+                    if (bq > published[i]) {
+                        top1[((size_t)c * gridDim.x + blockIdx.x) * 4 + quarter] = bq;
+                        published[i] = bq;
                     }
                 }
             }
