@@ -52,16 +52,36 @@ __device__ __forceinline__ void append32(const uint32_t (&v)[32], int c0, int lc
     if (__any_sync(0xffffffffu, full)) need = true;
 }
 
+// Two fp32 differences with one instruction (sub.f32x2 on register pairs), and the maximum of
+// three values with one (max.f32 with three inputs): both are sm_100 forms.  The threshold test
+// is the only arithmetic that touches every accumulator, so halving its instruction count
+// halves the issue slots the read-out takes.
+__device__ __forceinline__ void sub2(uint32_t a0, uint32_t a1, float b0, float b1, float &d0, float &d1) {
+    unsigned long long pa, pb, pd;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(pa) : "r"(a0), "r"(a1));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(pb) : "f"(b0), "f"(b1));
+    asm("sub.f32x2 %0, %1, %2;" : "=l"(pd) : "l"(pa), "l"(pb));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d0), "=f"(d1) : "l"(pd));
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float m;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(m) : "f"(a), "f"(b), "f"(c));
+    return m;
+}
+
 // Largest of acc - thr over 32 accumulator columns of this lane's row.
 __device__ __forceinline__ float max_margin32(const uint32_t (&v)[32], const float *__restrict__ thr, int c0) {
-    float m = -INFINITY;
+    float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
     for (int j4 = 0; j4 < 8; ++j4) {
         const float4 t4 = *reinterpret_cast<const float4 *>(&thr[c0 + 4 * j4]);
-        m = fmaxf(m, fmaxf(fmaxf(__uint_as_float(v[4 * j4]) - t4.x, __uint_as_float(v[4 * j4 + 1]) - t4.y),
-                           fmaxf(__uint_as_float(v[4 * j4 + 2]) - t4.z, __uint_as_float(v[4 * j4 + 3]) - t4.w)));
+        float d0, d1, d2, d3;
+        sub2(v[4 * j4], v[4 * j4 + 1], t4.x, t4.y, d0, d1);
+        sub2(v[4 * j4 + 2], v[4 * j4 + 3], t4.z, t4.w, d2, d3);
+        m0 = max3(m0, d0, d1);
+        m1 = max3(m1, d2, d3);
     }
-    return m;
+    return fmaxf(m0, m1);
 }
 
 // Up to 64 accumulator columns (queries c0 .. c0+63; the second 32 only when `two`) of one corpus

@@ -35,10 +35,10 @@ namespace {
 #ifndef PROX_READ_WARPS
 #define PROX_READ_WARPS 8
 #endif
-constexpr int kReadWarps = PROX_READ_WARPS;          // 8 or 16
+constexpr int kReadWarps = PROX_READ_WARPS;          // 8, 12 or 16
 constexpr int kReadPerQuarter = kReadWarps / 4;      // warps that share a tensor-memory lane quarter
-constexpr int kReadCols = kScanQ / kReadPerQuarter;  // most query columns one read-out warp takes
-constexpr int kReadGroups = kReadCols / 32;
+constexpr int kReadGroups = (kScanQ / 32 + kReadPerQuarter - 1) / kReadPerQuarter;   // most 32-column groups of one warp
+constexpr int kReadCols = 32 * kReadGroups;          // most query columns one read-out warp takes
 constexpr int kThreads = 128 + 32 * kReadWarps;      // producer, MMA, bound, (idle), read-out warps
 constexpr int kMaxStages = 8;
 constexpr int kChunkK = 64;                          // bf16 elements per 128-byte swizzle row
@@ -274,10 +274,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         const int e = warp - 4;                                   // 0..15
         const int quarter = warp & 3;
         const int part = e >> 2;
-        const int cw = n_pad >= 32 * kReadPerQuarter ? n_pad / kReadPerQuarter : 32;   // columns per warp
-        const int col_begin = part * cw;
-        const bool active = col_begin < n_pad;
-        const int ngr = cw / 32;                                  // groups of 32 columns: 1, 2 or 4
+        // the 32-column groups of the query block are dealt to the warps of the quarter as evenly as they go
+        const int n_grp = n_pad / 32, g_base = n_grp / kReadPerQuarter, g_rem = n_grp % kReadPerQuarter;
+        const int cw = 32 * (g_base + (part < g_rem ? 1 : 0));    // columns of this warp
+        const int col_begin = 32 * (part * g_base + (part < g_rem ? part : g_rem));
+        const bool active = cw > 0;
         const int ncol = active ? (nq - col_begin < cw ? (nq - col_begin > 0 ? nq - col_begin : 0) : cw) : 0;
         int *wcnt = ctl.wcnt[e];
         // lists of this warp: [(block * 4 + quarter) * kScanQ + query] * CAP
@@ -308,18 +309,23 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             if (!ok) { alive = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)kScanQ;
-            // the shared bounds read above go into the block's thresholds before this tile is tested
-            // (a stale, lower threshold only lets more rows through, so plain stores that the
-            // warps of a column share are enough)
+            // The shared bounds read above go into the block's thresholds (a stale, lower threshold
+            // only lets more rows through, so plain stores that the warps of a column share are
+            // enough).  While the first tiles come in every tile that is still tested against an
+            // open threshold floods the lists, so the bounds are applied before the test; later
+            // they are applied after it, where the latency of their load is hidden.
+            const bool early = it < 8;
+            if (early) {
 #pragma unroll
-            for (int i = 0; i < kReadGroups; ++i) {
-                const int lc = lane + 32 * i;
-                if (lc < ncol) {
-                    const float g = o2f(g_thr[i]);
-                    if (g > ctl.thr[col_begin + lc]) ctl.thr[col_begin + lc] = g;
+                for (int i = 0; i < kReadGroups; ++i) {
+                    const int lc = lane + 32 * i;
+                    if (lc < ncol) {
+                        const float g = o2f(g_thr[i]);
+                        if (g > ctl.thr[col_begin + lc]) ctl.thr[col_begin + lc] = g;
+                    }
                 }
+                __syncwarp();
             }
-            __syncwarp();
             // 64 columns at a time; the accumulator buffer goes back to the MMA issuer as soon as
             // the last of them are in registers, before they are looked at.  Rows past the end carry
             // an infinite half norm, columns past nq an infinite threshold: neither can pass, so
@@ -347,16 +353,29 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                                    lists, need);
                 if (last) break;
             }
-            // the warp publishes the best score of its lane quarter for each of its columns
+            if (!early) {
 #pragma unroll
-            for (int i = 0; i < kReadGroups; ++i) {
-                const int lc = lane + 32 * i;
-                if (lc < ncol) {
-                    const int c = col_begin + lc;
-                    const uint32_t bq = ctl.best[quarter][c];
-                    if (bq > published[i]) {
-                        top1[((size_t)c * gridDim.x + blockIdx.x) * 4 + quarter] = bq;
-                        published[i] = bq;
+                for (int i = 0; i < kReadGroups; ++i) {
+                    const int lc = lane + 32 * i;
+                    if (lc < ncol) {
+                        const float g = o2f(g_thr[i]);
+                        if (g > ctl.thr[col_begin + lc]) ctl.thr[col_begin + lc] = g;
+                    }
+                }
+            }
+            // the warp publishes the best score of its lane quarter for each of its columns (every
+            // tile at first, every fourth once the bounds move slowly)
+            if (it < 16 || (it & 3u) == 0u) {
+#pragma unroll
+                for (int i = 0; i < kReadGroups; ++i) {
+                    const int lc = lane + 32 * i;
+                    if (lc < ncol) {
+                        const int c = col_begin + lc;
+                        const uint32_t bq = ctl.best[quarter][c];
+                        if (bq > published[i]) {
+                            top1[((size_t)c * gridDim.x + blockIdx.x) * 4 + quarter] = bq;
+                            published[i] = bq;
+                        }
                     }
                 }
             }
