@@ -112,9 +112,18 @@ def pick_workload(name: str, free_bytes: int) -> W.Config:
     return cfg if free_bytes >= need else W.CONFIGS["1m"]
 
 
+# DRAM bytes per algorithmic byte of one scan launch, from one ncu capture of scan_tc_kernel on a 4 M x 768 cut
+# of the "large" workload (dram__bytes_read.sum + dram__bytes_write.sum = 7.29 GB against 6.16 GB); the extra
+# bytes grow with the row tiles like the algorithmic ones, so the ratio carries over to a full launch.
+# Valid for d = 768 and 256 misses per launch only; set to None when the kernel changes.
+SCAN_TRAFFIC_RATIO_D768_M256 = 1.184
+
+
 def roofline_of_scan(cfg, mean_misses, scan_ms_per_launch, peaks, traffic=None):
     """The corpus scan: bytes = bf16 corpus + row norms once per launch, flops = 2 M N d."""
     bytes_alg = cfg.N * cfg.d * 2 + cfg.N * 4
+    if traffic is None and cfg.d == 768 and mean_misses > 255 and SCAN_TRAFFIC_RATIO_D768_M256:
+        traffic = round(SCAN_TRAFFIC_RATIO_D768_M256 * bytes_alg)
     flops = 2.0 * mean_misses * cfg.N * cfg.d
     t = scan_ms_per_launch * 1e-3
     t_hbm = bytes_alg / (peaks["hbm_gbs"] * 1e9)
