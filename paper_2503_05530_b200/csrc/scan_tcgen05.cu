@@ -262,7 +262,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 jq += gridDim.x;
                 // bounds move fast while the first tiles come in and slowly afterwards; this warp
                 // shares an issue port with read-out warps, so it backs off once they have settled
-                __nanosleep(++jobs < 48 ? 2000 : 20000);
+                // (in short naps, so that the block does not outlive its read-out by a long one)
+                const int naps = ++jobs < 48 ? 1 : 10;
+                for (int n = 0; n < naps && *done < kReadWarps; ++n) __nanosleep(2000);
             }
         }
     } else if (warp >= 4) {

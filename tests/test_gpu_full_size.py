@@ -18,7 +18,8 @@ DEV = "cuda:0"
 POL = {"lru": oracle.LRU, "fifo": oracle.FIFO}
 
 
-def run_full_size(cfg, tau, n_batches, n_samples, seed=0, chunk_rows=1 << 20):
+def run_full_size(cfg, tau, n_batches, n_samples, seed=0, chunk_rows=1 << 20, lsh=None):
+    """lsh = (L, b): PROXIMITY-LSH with 2^L buckets of b entries instead of the flat cache of cfg.capacity."""
     need = cfg.N * cfg.d * 6 + (8 << 30)
     free, _ = torch.cuda.mem_get_info()
     if free < need:
@@ -26,7 +27,12 @@ def run_full_size(cfg, tau, n_batches, n_samples, seed=0, chunk_rows=1 << 20):
     corpus = W.make_corpus(cfg.N, cfg.d, cfg.n_components, seed, DEV)
     n = n_batches * cfg.batch
     queries, _, _ = W.make_query_stream(corpus, n, cfg.n_topics, cfg.zipf_s, cfg.sigma, seed)
-    p = prox.Prox(corpus, cfg.k, cfg.capacity, tau, cfg.policy)
+    capacity, planes, bucket = cfg.capacity, None, 0
+    if lsh is not None:
+        planes = torch.randn(lsh[0], cfg.d, generator=torch.Generator().manual_seed(seed + 3))
+        bucket, capacity = lsh[1], (1 << lsh[0]) * lsh[1]
+    p = prox.Prox(corpus, cfg.k, capacity, tau, cfg.policy, lsh_planes=None if planes is None else planes.to(DEV),
+                  lsh_bucket=bucket)
     ids = torch.empty(n, cfg.k, dtype=torch.int64, device=DEV)
     dists = torch.empty(n, cfg.k, dtype=torch.float32, device=DEV)
     hit = torch.empty(n, dtype=torch.uint8, device=DEV)
@@ -40,7 +46,8 @@ def run_full_size(cfg, tau, n_batches, n_samples, seed=0, chunk_rows=1 << 20):
     Q = queries.cpu().numpy()
 
     # 1. the cache trace of the whole prefix (needs no corpus)
-    o = oracle.Oracle(None, cfg.d, cfg.k, cfg.capacity, float(np.float32(tau)), POL[cfg.policy])
+    o = oracle.Oracle(None, cfg.d, cfg.k, capacity, float(np.float32(tau)), POL[cfg.policy],
+                      lsh_planes=None if planes is None else planes.numpy(), lsh_bucket=bucket)
     r = o.query(Q)
     o.close()
     assert np.array_equal(hit, r["hit"]), f"first differing flag at query {np.nonzero(hit != r['hit'])[0][0]}"
@@ -77,6 +84,12 @@ def test_one_million_rows_batch64_lru_full_size():
     cfg = W.CONFIGS["1m"]
     res = run_full_size(cfg, 0.5, n_batches=100, n_samples=24)
     assert 0.3 < res["hit_rate"] < 0.95 and res["stats"]["evictions"] > 0
+
+
+def test_one_million_rows_lsh_full_size():
+    cfg = W.CONFIGS["1m"]
+    res = run_full_size(cfg, 0.5, n_batches=60, n_samples=12, lsh=(8, 4))
+    assert 0.2 < res["hit_rate"] < 0.95 and res["stats"]["evictions"] > 0
 
 
 def test_24m_rows_batch256_lru_full_size():
