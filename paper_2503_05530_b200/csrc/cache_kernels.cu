@@ -286,27 +286,55 @@ probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
 #pragma unroll
             for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
 
+        // operands of the next 32 dimensions are fetched into registers while the current ones are
+        // multiplied: small problems (few blocks per SM) are bound by this latency, not by the fp64 rate
+        const float *q_src[(PQ * PD) / 256];
+        const float *k_src[(PC * PD) / 256];
+#pragma unroll
+        for (int it = 0; it < (PQ * PD) / 256; ++it) {
+            const int idx = it * 256 + tid, r = idx / PD, c = idx % PD;
+            const int qi = q_index[r];
+            q_src[it] = qi >= 0 ? queries + (size_t)qi * d + c : nullptr;
+        }
+#pragma unroll
+        for (int it = 0; it < (PC * PD) / 256; ++it) {
+            const int idx = it * 256 + tid, r = idx / PD, c = idx % PD;
+            const long long col = c0 + r;
+            k_src[it] = nullptr;
+            if (col < ncols)
+                k_src[it] = ((col >= nslot_cols) ? queries + (size_t)(col - nslot_cols) * d
+                                                 : keys + (size_t)(mode == 1 ? risk_slot[col] : col) * d) + c;
+        }
+        float q_next[(PQ * PD) / 256], k_next[(PC * PD) / 256];
+#pragma unroll
+        for (int it = 0; it < (PQ * PD) / 256; ++it)
+            q_next[it] = (q_src[it] && (it * 256 + tid) % PD < d) ? q_src[it][0] : 0.f;
+#pragma unroll
+        for (int it = 0; it < (PC * PD) / 256; ++it)
+            k_next[it] = (k_src[it] && (it * 256 + tid) % PD < d) ? k_src[it][0] : 0.f;
+
         for (int kc = 0; kc < d; kc += PD) {
             __syncthreads();
 #pragma unroll
             for (int it = 0; it < (PQ * PD) / 256; ++it) {
                 const int idx = it * 256 + tid, r = idx / PD, c = idx % PD;
-                const int qi = q_index[r];
-                qs[r][c] = (qi >= 0 && kc + c < d) ? (double)queries[(size_t)qi * d + kc + c] : 0.0;
+                qs[r][c] = (double)q_next[it];
             }
 #pragma unroll
             for (int it = 0; it < (PC * PD) / 256; ++it) {
                 const int idx = it * 256 + tid, r = idx / PD, c = idx % PD;
-                const long long col = c0 + r;
-                double v = 0.0;
-                if (col < ncols && kc + c < d) {
-                    const float *src = (col >= nslot_cols) ? queries + (size_t)(col - nslot_cols) * d
-                                       : keys + (size_t)(mode == 1 ? risk_slot[col] : col) * d;
-                    v = (double)src[kc + c];
-                }
-                ks[r][c] = v;
+                ks[r][c] = (double)k_next[it];
             }
             __syncthreads();
+            {
+                const int kn = kc + PD;
+#pragma unroll
+                for (int it = 0; it < (PQ * PD) / 256; ++it)
+                    q_next[it] = (q_src[it] && kn + (it * 256 + tid) % PD < d) ? q_src[it][kn] : 0.f;
+#pragma unroll
+                for (int it = 0; it < (PC * PD) / 256; ++it)
+                    k_next[it] = (k_src[it] && kn + (it * 256 + tid) % PD < d) ? k_src[it][kn] : 0.f;
+            }
 #pragma unroll 8
             for (int j = 0; j < PD; ++j) {
                 const double qa = qs[ty * 2][j], qb2 = qs[ty * 2 + 1][j];
