@@ -20,6 +20,7 @@ _SRC = os.path.join(_HERE, "prox_oracle.c")
 _LIB = os.path.join(_HERE, "_prox_oracle.so")
 
 LRU, FIFO = 0, 1
+L2SQ, COSINE = 0, 1
 
 
 def build(force: bool = False) -> str:
@@ -52,6 +53,11 @@ def lib():
                                         C.c_int32, C.c_int32]
         L.oracle_lsh_hash.restype = C.c_int64
         L.oracle_lsh_hash.argtypes = [fp, C.c_int32, C.c_int32, fp]
+        L.oracle_set_metric.restype = C.c_int
+        L.oracle_set_metric.argtypes = [C.c_void_p, C.c_int32]
+        L.oracle_cosdist.restype = C.c_double
+        L.oracle_cosdist.argtypes = [fp, fp, C.c_int32]
+        L.oracle_knn_batch_metric.argtypes = [C.c_int32, fp, C.c_int64, C.c_int32, fp, C.c_int64, C.c_int32, ip, dp]
         L.oracle_destroy.argtypes = [C.c_void_p]
         L.oracle_reset.argtypes = [C.c_void_p]
         L.oracle_counters.argtypes = [C.c_void_p, ip]
@@ -87,7 +93,14 @@ def sqdist(a, b) -> float:
     return float(lib().oracle_sqdist(_ptr(a, C.c_float), _ptr(b, C.c_float), a.size))
 
 
-def exact_topk(corpus, queries, k: int):
+def cosdist(a, b) -> float:
+    """Cosine distance 1 - cos(a, b) in fp64 over fp32 inputs (half the squared distance of the unit vectors)."""
+    a, b = _f32(a).ravel(), _f32(b).ravel()
+    assert a.shape == b.shape
+    return float(lib().oracle_cosdist(_ptr(a, C.c_float), _ptr(b, C.c_float), a.size))
+
+
+def exact_topk(corpus, queries, k: int, metric: int = L2SQ):
     """The database call alone: for each query the k nearest corpus rows, (ids[n,k], dists[n,k])."""
     X, Q = _f32(corpus), _f32(queries)
     if Q.ndim == 1:
@@ -96,8 +109,8 @@ def exact_topk(corpus, queries, k: int):
     assert X.shape[1] == d and 1 <= k <= X.shape[0]
     ids = np.empty((n, k), np.int64)
     dists = np.empty((n, k), np.float64)
-    lib().oracle_knn_batch(_ptr(X, C.c_float), X.shape[0], d, _ptr(Q, C.c_float), n, k,
-                           _ptr(ids, C.c_int64), _ptr(dists, C.c_double))
+    lib().oracle_knn_batch_metric(metric, _ptr(X, C.c_float), X.shape[0], d, _ptr(Q, C.c_float), n, k,
+                                  _ptr(ids, C.c_int64), _ptr(dists, C.c_double))
     return ids, dists
 
 
@@ -136,7 +149,7 @@ class Oracle:
     ``lsh_planes`` (L x d) with ``lsh_bucket`` = b switches to PROXIMITY-LSH: 2^L buckets of b entries."""
 
     def __init__(self, corpus, d: int, k: int, capacity: int, tau: float, policy: int, rho: int = 1,
-                 lsh_planes=None, lsh_bucket: int = 0):
+                 lsh_planes=None, lsh_bucket: int = 0, metric: int = L2SQ):
         self._X = None if corpus is None else _f32(corpus)
         N = 0 if self._X is None else self._X.shape[0]
         if self._X is not None:
@@ -155,6 +168,8 @@ class Oracle:
                                               float(tau), policy, self.rho)
         if not self._h:
             raise ValueError("oracle_create rejected the arguments")
+        if lib().oracle_set_metric(self._h, metric):
+            raise ValueError("unknown metric")
 
     def close(self):
         if self._h:

@@ -34,6 +34,10 @@
  *     measures the m stored rows against the CURRENT query and returns the k nearest (distance
  *     ascending, ties to the lower row id) with those distances.  rho = 1 is "no re-ranking"
  *     (Section 4): the stored list comes back as it is, as above;
+ *   - metric (Section 2.1: "typically L2, cosine, or inner-product, fixed before deployment"):
+ *     squared Euclidean by default; ORACLE_COSINE is the cosine distance 1 - cos(a, b), taken
+ *     as half the squared Euclidean distance of a/|a| and b/|b| (the same number, and exactly 0
+ *     for identical vectors so that tau = 0 stays exact matching); normalisation in fp64;
  *   - PROXIMITY-LSH (Section 3.2): L random hyperplanes through the origin, given by the caller
  *     as L normal vectors; bit l of the hash is (q . r_l >= 0), the dot product taken in fp64
  *     in index order; the 2^L buckets are PROXIMITY-FLAT caches of b entries each, every one
@@ -57,6 +61,7 @@
 #endif
 
 enum { ORACLE_LRU = 0, ORACLE_FIFO = 1 };
+enum { ORACLE_L2SQ = 0, ORACLE_COSINE = 1 };
 
 typedef struct {
     /* stored state of Algorithm 1: tau, c, the database D and the dict C */
@@ -64,6 +69,7 @@ typedef struct {
     int64_t N;
     int32_t d, k;
     int32_t rho, m;        /* re-ranking factor and m = rho * k entries per value list */
+    int32_t metric;        /* ORACLE_L2SQ or ORACLE_COSINE */
     int32_t lsh_L, lsh_b;  /* PROXIMITY-LSH: hyperplanes and bucket size; lsh_L < 0 = PROXIMITY-FLAT */
     float *planes;         /* lsh_L x d normal vectors (copy) */
     int64_t *bucket_count; /* 2^lsh_L */
@@ -103,6 +109,23 @@ double oracle_sqdist(const float *a, const float *b, int32_t d) {
     return acc;
 }
 
+/* Cosine distance 1 - cos(a, b) = |a/|a| - b/|b||^2 / 2, every step in fp64. */
+double oracle_cosdist(const float *a, const float *b, int32_t d) {
+    double na = 0.0, nb = 0.0;
+    for (int32_t j = 0; j < d; ++j) { na += (double)a[j] * (double)a[j]; nb += (double)b[j] * (double)b[j]; }
+    na = sqrt(na); nb = sqrt(nb);
+    double acc = 0.0;
+    for (int32_t j = 0; j < d; ++j) {
+        double diff = (double)a[j] / na - (double)b[j] / nb;
+        acc += diff * diff;
+    }
+    return 0.5 * acc;
+}
+
+static double oracle_dist(int32_t metric, const float *a, const float *b, int32_t d) {
+    return metric == ORACLE_COSINE ? oracle_cosdist(a, b, d) : oracle_sqdist(a, b, d);
+}
+
 /*
  * One pass of the selection behind retrieveDocumentIndices(q) over rows
  * [base_id, base_id + n) of the corpus (chunk points at row base_id).  The k
@@ -110,14 +133,14 @@ double oracle_sqdist(const float *a, const float *b, int32_t d) {
  * ascending, row id ascending); *have is how many are filled.  Chunks must be
  * fed in ascending row order so that equal distances keep the lower id first.
  */
-void oracle_topk_update(const float *chunk, int64_t n, int32_t d, int64_t base_id, const float *q,
-                        int32_t k, double *scratch, int64_t *out_ids, double *out_dists,
-                        int32_t *have_io) {
+void oracle_topk_update_metric(int32_t metric, const float *chunk, int64_t n, int32_t d, int64_t base_id,
+                               const float *q, int32_t k, double *scratch, int64_t *out_ids, double *out_dists,
+                               int32_t *have_io) {
     double *dist = scratch;
     int own = 0;
     if (!dist) { dist = (double *)malloc(sizeof(double) * (size_t)n); own = 1; }
 #pragma omp parallel for schedule(static)
-    for (int64_t i = 0; i < n; ++i) dist[i] = oracle_sqdist(q, chunk + i * (int64_t)d, d);
+    for (int64_t i = 0; i < n; ++i) dist[i] = oracle_dist(metric, q, chunk + i * (int64_t)d, d);
 
     int32_t have = *have_io;
     for (int64_t i = 0; i < n; ++i) {
@@ -137,15 +160,26 @@ void oracle_topk_update(const float *chunk, int64_t n, int32_t d, int64_t base_i
     if (own) free(dist);
 }
 
+void oracle_topk_update(const float *chunk, int64_t n, int32_t d, int64_t base_id, const float *q,
+                        int32_t k, double *scratch, int64_t *out_ids, double *out_dists,
+                        int32_t *have_io) {
+    oracle_topk_update_metric(ORACLE_L2SQ, chunk, n, d, base_id, q, k, scratch, out_ids, out_dists, have_io);
+}
+
 /*
  * retrieveDocumentIndices(q): the k rows of the corpus closest to q, as a list
  * sorted by (distance ascending, row id ascending).  Every row is measured.
  */
+void oracle_exact_topk_metric(int32_t metric, const float *corpus, int64_t N, int32_t d, const float *q, int32_t k,
+                              double *scratch, int64_t *out_ids, double *out_dists) {
+    int32_t have = 0;
+    oracle_topk_update_metric(metric, corpus, N, d, 0, q, k, scratch, out_ids, out_dists, &have);
+    for (int32_t r = have; r < k; ++r) { out_ids[r] = -1; out_dists[r] = INFINITY; }
+}
+
 void oracle_exact_topk(const float *corpus, int64_t N, int32_t d, const float *q, int32_t k,
                        double *scratch, int64_t *out_ids, double *out_dists) {
-    int32_t have = 0;
-    oracle_topk_update(corpus, N, d, 0, q, k, scratch, out_ids, out_dists, &have);
-    for (int32_t r = have; r < k; ++r) { out_ids[r] = -1; out_dists[r] = INFINITY; }
+    oracle_exact_topk_metric(ORACLE_L2SQ, corpus, N, d, q, k, scratch, out_ids, out_dists);
 }
 
 oracle_t *oracle_create_rho(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
@@ -204,6 +238,13 @@ void oracle_destroy(oracle_t *o) {
     free(o->origin); free(o->valid); free(o->scratch); free(o);
 }
 
+/* Chooses the distance of the cache keys and of the database (before the first query). */
+int oracle_set_metric(oracle_t *o, int32_t metric) {
+    if (metric != ORACLE_L2SQ && metric != ORACLE_COSINE) return 1;
+    o->metric = metric;
+    return 0;
+}
+
 void oracle_reset(oracle_t *o) {
     memset(o->valid, 0, (size_t)o->capacity);
     o->count = 0; o->clock = 0;
@@ -260,7 +301,7 @@ void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids,
     int64_t best_slot = -1;
     for (int64_t s = s_begin; s < s_end; ++s) {
         if (!o->valid[s]) continue;
-        double dist = oracle_sqdist(q, o->keys + s * d, d);
+        double dist = oracle_dist(o->metric, q, o->keys + s * d, d);
         o->probe_madds += d;
         if (dist < best) { second = best; best = dist; best_slot = s; }
         else if (dist < second) second = dist;
@@ -285,7 +326,7 @@ void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids,
             int32_t have = 0;
             for (int32_t r = 0; r < m; ++r) {
                 if (sid[r] < 0) continue;          /* the corpus had fewer than m rows */
-                const double v = oracle_sqdist(q, o->corpus + sid[r] * (int64_t)d, d);
+                const double v = oracle_dist(o->metric, q, o->corpus + sid[r] * (int64_t)d, d);
                 int32_t pos = have;
                 while (pos > 0 && (rd[pos - 1] > v || (rd[pos - 1] == v && rid[pos - 1] > sid[r]))) {
                     rd[pos] = rd[pos - 1]; rid[pos] = rid[pos - 1]; --pos;
@@ -306,7 +347,7 @@ void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids,
     /* line 6: I <- D.retrieveDocumentIndices(q) */
     int64_t *ids = (int64_t *)malloc(sizeof(int64_t) * m);
     double *dists = (double *)malloc(sizeof(double) * m);
-    if (o->corpus) oracle_exact_topk(o->corpus, o->N, d, q, m, o->scratch, ids, dists);   /* m = rho * k neighbours */
+    if (o->corpus) oracle_exact_topk_metric(o->metric, o->corpus, o->N, d, q, m, o->scratch, ids, dists);   /* m = rho * k neighbours */
     else for (int32_t r = 0; r < m; ++r) { ids[r] = -1; dists[r] = 0.0; }
 
     /* lines 7-8: if |C| >= c evict one entry (the smallest stamp; stamps are unique) */
@@ -349,12 +390,17 @@ void oracle_query_stream(oracle_t *o, const float *queries, int64_t n, const int
 }
 
 /* The database call alone for a set of queries (used to check sampled misses at large N). */
-void oracle_knn_batch(const float *corpus, int64_t N, int32_t d, const float *queries, int64_t n,
-                      int32_t k, int64_t *out_ids, double *out_dists) {
+void oracle_knn_batch_metric(int32_t metric, const float *corpus, int64_t N, int32_t d, const float *queries,
+                             int64_t n, int32_t k, int64_t *out_ids, double *out_dists) {
     double *scratch = (double *)malloc(sizeof(double) * (size_t)N);
     for (int64_t i = 0; i < n; ++i)
-        oracle_exact_topk(corpus, N, d, queries + i * d, k, scratch, out_ids + i * k, out_dists + i * k);
+        oracle_exact_topk_metric(metric, corpus, N, d, queries + i * d, k, scratch, out_ids + i * k, out_dists + i * k);
     free(scratch);
+}
+
+void oracle_knn_batch(const float *corpus, int64_t N, int32_t d, const float *queries, int64_t n,
+                      int32_t k, int64_t *out_ids, double *out_dists) {
+    oracle_knn_batch_metric(ORACLE_L2SQ, corpus, N, d, queries, n, k, out_ids, out_dists);
 }
 
 /* Read-only views for tests. */

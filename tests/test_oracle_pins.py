@@ -369,3 +369,50 @@ def test_lsh_operation_count_of_the_papers_example():
     before = o.counters()["probe_madds"]
     o.query(Q[b:])
     assert o.counters()["probe_madds"] - before == (L + b) * d == 23040
+
+
+# ---------------------------------------------------------------- cosine distance (Section 2.1)
+def test_cosine_closed_forms():
+    e = np.eye(6, dtype=np.float32)
+    assert oracle.cosdist(e[0], e[1]) == pytest.approx(1.0, abs=1e-15)           # orthogonal
+    assert oracle.cosdist(3 * e[2], 0.25 * e[2]) == 0.0                            # same direction, any length
+    assert oracle.cosdist(e[3], -7 * e[3]) == pytest.approx(2.0, abs=1e-15)       # opposite
+    a, b = unit_rows(2, 40, 12)
+    assert oracle.cosdist(5 * a, 0.1 * b) == pytest.approx(1.0 - float(a.astype(np.float64) @ b.astype(np.float64)), abs=1e-7)
+    assert oracle.cosdist(a, a) == 0.0 and oracle.cosdist(a, b) == oracle.cosdist(b, a)
+
+
+def test_cosine_topk_vs_numpy_and_scale_invariance():
+    rng = np.random.default_rng(13)
+    X = (rng.standard_normal((500, 24)) * rng.uniform(0.1, 9.0, (500, 1))).astype(np.float32)   # rows of very different length
+    Q = rng.standard_normal((7, 24)).astype(np.float32)
+    ids, dists = oracle.exact_topk(X, Q, 6, metric=oracle.COSINE)
+    Xn = X.astype(np.float64) / np.linalg.norm(X.astype(np.float64), axis=1, keepdims=True)
+    for i, q in enumerate(Q):
+        qn = q.astype(np.float64) / np.linalg.norm(q.astype(np.float64))
+        full = 1.0 - Xn @ qn
+        order = np.lexsort((np.arange(len(X)), full))[:6]
+        assert np.array_equal(ids[i], order) and np.allclose(dists[i], full[order], atol=1e-12)
+    l2_ids, _ = oracle.exact_topk(X, Q, 6)
+    assert (l2_ids != ids).any()                                                  # not the Euclidean neighbours here
+    ids2, dists2 = oracle.exact_topk(X * np.float32(4.0), Q * np.float32(0.5), 6, metric=oracle.COSINE)
+    assert np.array_equal(ids2, ids) and np.allclose(dists2, dists, atol=1e-12)    # powers of two scale exactly
+
+
+def test_cosine_cache_equals_the_l2_cache_on_unit_vectors():
+    """On unit vectors 1 - cos = |a - b|^2 / 2, so the cosine cache at tau must take the decisions
+    of the Euclidean cache at 2 tau and return the same lists with half the distances."""
+    X, Q, _ = small_workload(seed=14, N=500, nq=150)
+    d = X.shape[1]
+    c = oracle.Oracle(X, d, 5, 4, 0.25, oracle.LRU, metric=oracle.COSINE).query(Q)
+    e = oracle.Oracle(X, d, 5, 4, 0.5, oracle.LRU).query(Q)
+    assert 0.2 < c["hit"].mean() < 0.95
+    assert np.array_equal(c["hit"], e["hit"]) and np.array_equal(c["ids"], e["ids"]) and np.array_equal(c["slot"], e["slot"])
+    assert np.allclose(c["dists"], 0.5 * e["dists"], rtol=1e-5)
+
+
+def test_cosine_duplicate_hits_at_tau_zero_whatever_its_length():
+    X, Q, _ = small_workload(seed=15)
+    Q2 = np.concatenate([Q[:1], 2 * Q[:1], Q[1:2]])
+    r = oracle.Oracle(X, X.shape[1], 3, 4, 0.0, oracle.FIFO, metric=oracle.COSINE).query(Q2)
+    assert r["hit"].tolist() == [0, 1, 0]
