@@ -226,7 +226,7 @@ def run_ours(args):
             p = prox.Prox(corpus, k, (1 << args.lsh_bits) * args.lsh_bucket, tau, cfg.policy, rho=args.rho,
                           lsh_planes=planes, lsh_bucket=args.lsh_bucket)
         else:
-            p = prox.Prox(corpus, k, cfg.capacity, tau, cfg.policy, rho=args.rho)
+            p = prox.Prox(corpus, k, cfg.capacity, tau, cfg.policy, rho=args.rho, metric=args.metric)
         B = cfg.batch
         n_use = K * B
         ids = torch.empty(n_use, k, dtype=torch.int64, device=dev)
@@ -316,7 +316,7 @@ def run_ours(args):
         config=dict(workload=f"{cfg.name}: N={cfg.N} d={cfg.d} k={cfg.k} capacity={cfg.capacity} policy={cfg.policy} "
                              f"batch={cfg.batch} tau={head_tau} topics={cfg.n_topics} zipf={cfg.zipf_s} sigma={cfg.sigma}",
                     tau=head_tau, hit_rate=round(head["hit_rate"], 4), l2="inputs_exceed_l2" if cfg.N * cfg.d * 2 > 126e6 else "corpus_fits_l2",
-                    parallelism=f"replica x{world}", rho=args.rho,
+                    parallelism=f"replica x{world}", rho=args.rho, metric=args.metric,
                     cache="flat" if args.lsh_bits < 0 else f"lsh L={args.lsh_bits} b={args.lsh_bucket}", seed=args.seed, gen_seconds=round(t_gen, 1)),
         clocks=head["clocks"],
         e2e=dict(value=round(e2e, 1), unit=UNIT, h2d_bytes_per_step=head["h2d"], d2h_bytes_per_step=head["d2h"]),
@@ -515,6 +515,7 @@ def main():
     ap.add_argument("--rows", type=int, default=0, help="override the corpus size (profiling runs)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling runs)")
     ap.add_argument("--rho", type=int, default=1, help="re-ranking factor: rho * k rows fetched and stored per miss (1 = none)")
+    ap.add_argument("--metric", default="l2", choices=["l2", "cosine"], help="distance of the cache keys and of the corpus")
     ap.add_argument("--lsh-bits", type=int, default=-1, help="PROXIMITY-LSH with this many hyperplanes (-1: flat cache)")
     ap.add_argument("--lsh-bucket", type=int, default=20, help="entries per LSH bucket")
     ap.add_argument("--seed", type=int, default=0)

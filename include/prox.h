@@ -47,6 +47,8 @@ enum {
     PROX_MAX_K = 64,            /* largest k */
     PROX_MAX_FETCH = 128,       /* largest rho * k (neighbours fetched and stored per miss) */
     PROX_MAX_BATCH = 1024,      /* largest B of one call */
+    PROX_METRIC_L2SQ = 0,       /* prox_create_metric: squared Euclidean distance (the default everywhere else) */
+    PROX_METRIC_COSINE = 1,     /* prox_create_metric: cosine distance 1 - cos(a, b) */
     PROX_SCAN_AUTO = 0,         /* prox_set_scan_mode: tensor-core scan, two blocks per MMA (default) */
     PROX_SCAN_CUDA_CORE = 1,    /* prox_set_scan_mode: plain CUDA-core scan of the same bf16 scores */
     PROX_SCAN_TC_SINGLE = 2     /* prox_set_scan_mode: tensor-core scan, one block per MMA */
@@ -80,6 +82,19 @@ prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, int32_t k, i
  */
 prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
                              float tau, int32_t policy, int32_t rho);
+
+/*
+ * prox_create_metric -- prox_create_rho with the distance named (Section 2.1: the distance is
+ * "typically L2, cosine, or inner-product, fixed before deployment"; Section 3.1: the cache
+ * uses the database's distance).  PROX_METRIC_COSINE: keys and corpus rows are compared by
+ * 1 - cos(a, b), evaluated as half the squared Euclidean distance of a/|a| and b/|b| (identical
+ * vectors, of any length, are at distance exactly 0); tau applies to that value and out_dists
+ * hold it.  The library keeps its own unit-length fp32 copy of the corpus (N x d x 4 bytes
+ * more) and brings every query to unit length (norms in fp64) before the lookup.  Rows and
+ * queries must be non-zero.  Inner product is not offered.
+ */
+prox_handle *prox_create_metric(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
+                                float tau, int32_t policy, int32_t rho, int32_t metric);
 
 /*
  * prox_create_lsh -- PROXIMITY-LSH of Section 3.2: the cache is split into 2^L buckets of b

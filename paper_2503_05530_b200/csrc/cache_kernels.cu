@@ -825,6 +825,36 @@ static int probe_splits(const prox_handle *h, int B) {
     return (int)want;
 }
 
+// dst row = src row / |src row| (norm and quotient in fp64, rounded to fp32 once); one warp per row.
+// dst may be src.
+__global__ void __launch_bounds__(256)
+normalize_rows_kernel(const float *src, float *dst, long long n, int d) {
+    const long long r = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (r >= n) return;
+    const float *x = src + (size_t)r * d;
+    double acc = 0.0;
+    for (int j = lane; j < d; j += 32) acc += (double)x[j] * (double)x[j];
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, m);
+    const double nrm = sqrt(acc);
+    float *y = dst + (size_t)r * d;
+    for (int j = lane; j < d; j += 32) y[j] = (float)((double)x[j] / nrm);
+}
+
+__global__ void scale_kernel(float *v, long long n, float f) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) v[i] *= f;
+}
+
+void launch_normalize_rows(const float *src, float *dst, long long n, int d, cudaStream_t s) {
+    normalize_rows_kernel<<<(unsigned)((n + 7) / 8), 256, 0, s>>>(src, dst, n, d);
+}
+
+void launch_scale(float *v, long long n, float f, cudaStream_t s) {
+    scale_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(v, n, f);
+}
+
 void launch_risk_select(prox_handle *h, int B, cudaStream_t s) {
     // one block reads a small cache faster than four launches do
     if (h->C <= (1 << 16)) {

@@ -84,7 +84,7 @@ static bool dev_alloc(T *&p, size_t n) {
 }
 
 static void free_all(prox_handle *h) {
-    void *ptrs[] = {h->planes, h->bucket_count, h->lsh_code, h->lsh_order, h->lsh_seg, h->lsh_work, h->xb, h->xh, h->keys, h->val_ids, h->val_dists, h->stamp, h->risk_pos, h->st,
+    void *ptrs[] = {h->corpus_own, h->qn, h->planes, h->bucket_count, h->lsh_code, h->lsh_order, h->lsh_seg, h->lsh_work, h->xb, h->xh, h->keys, h->val_ids, h->val_dists, h->stamp, h->risk_pos, h->st,
                     h->risk_slot, h->risk_stamp, h->part_min, h->part_arg, h->d_risk, h->d_intra,
                     h->safe_min, h->safe_arg, h->cand_d, h->cand_code, h->n_cand, h->src, h->src_kind,
                     h->ins_slot, h->evt_slot, h->evt_dist, h->miss_list, h->miss_rank, h->qb, h->qbn,
@@ -205,6 +205,32 @@ extern "C" prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t 
     return h;
 }
 
+extern "C" prox_handle *prox_create_metric(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
+                                           float tau, int32_t policy, int32_t rho, int32_t metric) {
+    g_err[0] = 0;
+    if (metric == PROX_METRIC_L2SQ) return prox_create_rho(corpus, N, d, k, capacity, tau, policy, rho);
+    if (metric != PROX_METRIC_COSINE) { set_err("metric must be PROX_METRIC_L2SQ or PROX_METRIC_COSINE"); return nullptr; }
+    if (!corpus) { set_err("corpus is NULL"); return nullptr; }
+    if (N < 1 || N >= (1LL << 31) || d < 16 || d > 4096 || d % 16) { set_err("N or d out of range"); return nullptr; }
+    if (!(tau >= 0.f) || std::isinf(tau)) { set_err("tau must be finite and >= 0"); return nullptr; }
+    // 1 - cos(a, b) = |a/|a| - b/|b||^2 / 2: the Euclidean machinery on unit-length copies, at 2 tau
+    float *own = nullptr, *qn = nullptr;
+    if (!dev_alloc(own, (size_t)N * d) || !dev_alloc(qn, (size_t)kMaxBatch * d)) {
+        set_err("out of device memory for the unit-length copy of the corpus");
+        if (own) cudaFree(own);
+        return nullptr;
+    }
+    launch_normalize_rows(corpus, own, N, d, 0);
+    prox_handle *h = prox_create_rho(own, N, d, k, capacity, 2.f * tau, policy, rho);
+    if (!h) {
+        cudaFree(own);
+        cudaFree(qn);
+        return nullptr;
+    }
+    h->metric = PROX_METRIC_COSINE; h->corpus_own = own; h->qn = qn;
+    return h;
+}
+
 extern "C" prox_handle *prox_create_lsh(const float *corpus, int64_t N, int32_t d, int32_t k, int32_t L, int32_t b,
                                         const float *planes, float tau, int32_t policy, int32_t rho) {
     g_err[0] = 0;
@@ -293,6 +319,11 @@ extern "C" int32_t prox_query_batch(prox_handle *h, const float *queries, int32_
     if (rc) return rc;
     if (!out_ids || !out_dists || !out_hit) { set_err("an output pointer is NULL"); return PROX_ERR_INVALID_ARG; }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (h->metric == PROX_METRIC_COSINE) {                // unit-length copies stand in for the queries from here on
+        launch_normalize_rows(queries, h->qn, B, h->d, s);
+        h->launches++;
+        queries = h->qn;
+    }
 
     enqueue_probe_and_resolve(h, queries, B, out_hit, s);
     {
@@ -315,6 +346,10 @@ extern "C" int32_t prox_query_batch(prox_handle *h, const float *queries, int32_
         StageScope t(h, PROX_STAGE_SCATTER, s);
         if (h->rho > 1) launch_hit_rerank(h, queries, B, 2, out_ids, out_dists, s);   // hits on keys of this batch
         launch_scatter(h, queries, B, out_ids, out_dists, 1, s);
+    }
+    if (h->metric == PROX_METRIC_COSINE) {                // squared distance of unit vectors -> 1 - cos
+        launch_scale(out_dists, (long long)B * h->k_out, 0.5f, s);
+        h->launches++;
     }
     return check_launch("prox_query_batch");
 }
@@ -348,8 +383,17 @@ extern "C" int32_t prox_probe_batch(prox_handle *h, const float *queries, int32_
     if (rc) return rc;
     if (!out_hit) { set_err("out_hit is NULL"); return PROX_ERR_INVALID_ARG; }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (h->metric == PROX_METRIC_COSINE) {
+        launch_normalize_rows(queries, h->qn, B, h->d, s);
+        h->launches++;
+        queries = h->qn;
+    }
     enqueue_probe_and_resolve(h, queries, B, out_hit, s);
     if (out_slot || out_min_dist) launch_probe_outputs(h, B, out_slot, out_min_dist, s);
+    if (out_min_dist && h->metric == PROX_METRIC_COSINE) {
+        launch_scale(out_min_dist, B, 0.5f, s);
+        h->launches++;
+    }
     { StageScope t(h, PROX_STAGE_SCATTER, s); launch_scatter(h, queries, B, nullptr, nullptr, 0, s); }
     return check_launch("prox_probe_batch");
 }
@@ -368,6 +412,11 @@ extern "C" int32_t prox_cache_load(prox_handle *h, const float *keys, int64_t n,
     if (n < 0 || n > h->C) { set_err("n must be in [0, capacity]"); return PROX_ERR_INVALID_ARG; }
     if (n > 0 && !keys) { set_err("keys is NULL"); return PROX_ERR_INVALID_ARG; }
     if (h->lsh_L >= 0) { set_err("prox_cache_load is not available for a PROXIMITY-LSH handle"); return PROX_ERR_UNSUPPORTED; }
+    if (h->metric == PROX_METRIC_COSINE && n > 0) {       // the keys are stored at unit length
+        launch_normalize_rows(keys, h->keys, n, h->d, static_cast<cudaStream_t>(stream));
+        h->launches++;
+        keys = h->keys;
+    }
     launch_cache_load(h, keys, n, static_cast<cudaStream_t>(stream));
     return check_launch("prox_cache_load");
 }

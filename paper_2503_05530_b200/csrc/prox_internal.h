@@ -48,6 +48,10 @@ struct prox_handle {
     int64_t N;
     int32_t d, k, kp;         // k: entries of a value list (rho * k_out)
     int32_t k_out, rho;       // neighbours returned per query; re-ranking factor
+    // cosine distance: own unit-length copy of the corpus, unit-length copies of the batch queries
+    int32_t metric;
+    float *corpus_own;        // N x d (NULL for the Euclidean distance)
+    float *qn;                // kMaxBatch x d
     // PROXIMITY-LSH (lsh_L < 0: flat cache)
     int32_t lsh_L, lsh_b;
     float *planes;            // lsh_L x d normal vectors
@@ -148,6 +152,8 @@ void launch_hit_rerank(prox_handle *h, const float *q, int B, int kind, int64_t 
                        cudaStream_t s);   // rho > 1: hits of that kind (1 stored key, 2 key of this batch)
 void launch_scatter(prox_handle *h, const float *q, int B, int64_t *out_ids, float *out_dists,
                     int with_values, cudaStream_t s);
+void launch_normalize_rows(const float *src, float *dst, long long n, int d, cudaStream_t s);   // dst = src / |src| per row (may alias)
+void launch_scale(float *v, long long n, float f, cudaStream_t s);
 void launch_lsh_probe(prox_handle *h, const float *q, int B, uint8_t *out_hit, cudaStream_t s);   // hash, group, replay per bucket
 void launch_probe_outputs(prox_handle *h, int B, int32_t *out_slot, float *out_min_dist, cudaStream_t s);
 void launch_cache_load(prox_handle *h, const float *keys, int64_t n, cudaStream_t s);

@@ -21,6 +21,8 @@ SCAN_AUTO, SCAN_CUDA_CORE, SCAN_TC_SINGLE = 0, 1, 2
 STAGES = ("risk_select", "probe", "candidates", "resolve", "gather", "prep_miss", "scan", "merge",
           "rerank", "exact_pass", "scatter")
 _POLICY = {"lru": LRU, "fifo": FIFO, LRU: LRU, FIFO: FIFO}
+METRIC_L2SQ, METRIC_COSINE = 0, 1
+_METRIC = {"l2": METRIC_L2SQ, "cosine": METRIC_COSINE, METRIC_L2SQ: METRIC_L2SQ, METRIC_COSINE: METRIC_COSINE}
 
 
 class ProxError(RuntimeError):
@@ -53,6 +55,8 @@ def load_library():
     L.prox_create.argtypes = [vp, i64, i32, i32, i64, f32, i32]
     L.prox_create_rho.restype = vp
     L.prox_create_rho.argtypes = [vp, i64, i32, i32, i64, f32, i32, i32]
+    L.prox_create_metric.restype = vp
+    L.prox_create_metric.argtypes = [vp, i64, i32, i32, i64, f32, i32, i32, i32]
     L.prox_create_lsh.restype = vp
     L.prox_create_lsh.argtypes = [vp, i64, i32, i32, i32, i32, vp, f32, i32, i32]
     L.prox_query_batch.restype = i32
@@ -121,7 +125,7 @@ class Prox:
     """prox_create / prox_query_batch / prox_reset_cache / prox_destroy with tensors."""
 
     def __init__(self, corpus: torch.Tensor, k: int, capacity: int, tau: float, policy="lru", rho: int = 1,
-                 lsh_planes: torch.Tensor | None = None, lsh_bucket: int = 0):
+                 lsh_planes: torch.Tensor | None = None, lsh_bucket: int = 0, metric="l2"):
         self._lib = load_library()
         self._corpus = _dev_f32(corpus, "corpus")      # borrowed by the library: keep it alive
         self.N, self.d = corpus.shape
@@ -129,9 +133,12 @@ class Prox:
         self.policy = _POLICY[policy]
         self.rho = int(rho)                            # re-ranking factor (prox_create_rho); 1 = prox_create
         with torch.cuda.device(corpus.device):
+            self.metric = _METRIC[metric]
             if lsh_planes is None:
-                self._h = self._lib.prox_create_rho(corpus.data_ptr(), self.N, self.d, self.k, self.capacity,
-                                                    self.tau, self.policy, self.rho)
+                self._h = self._lib.prox_create_metric(corpus.data_ptr(), self.N, self.d, self.k, self.capacity,
+                                                       self.tau, self.policy, self.rho, self.metric)
+            elif self.metric != METRIC_L2SQ:
+                raise ProxError("PROXIMITY-LSH handles take the Euclidean distance only")
             else:
                 # PROXIMITY-LSH (prox_create_lsh): 2^L buckets of lsh_bucket entries; capacity = 2^L * lsh_bucket
                 P = _dev_f32(lsh_planes.reshape(-1, self.d), "lsh_planes")

@@ -17,10 +17,10 @@ REL_DIST = 1e-4
 
 
 def run_gpu(corpus_t, queries_t, k, capacity, tau, policy, batch, scan_mode=None, host_api=False, rho=1,
-            lsh_planes=None, lsh_bucket=0):
+            lsh_planes=None, lsh_bucket=0, metric="l2"):
     """corpus_t, queries_t: CUDA float32 tensors.  Returns numpy (ids, dists, hit) and the stats."""
     planes_t = None if lsh_planes is None else torch.as_tensor(lsh_planes).to(corpus_t.device)
-    p = prox.Prox(corpus_t, k, capacity, tau, policy, rho=rho, lsh_planes=planes_t, lsh_bucket=lsh_bucket)
+    p = prox.Prox(corpus_t, k, capacity, tau, policy, rho=rho, lsh_planes=planes_t, lsh_bucket=lsh_bucket, metric=metric)
     try:
         if scan_mode is not None:
             p.set_scan_mode(scan_mode)
@@ -48,7 +48,7 @@ def run_gpu(corpus_t, queries_t, k, capacity, tau, policy, batch, scan_mode=None
 
 
 def run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=None, max_forced=16, rho=1, lsh_planes=None,
-               lsh_bucket=0):
+               lsh_bucket=0, metric="l2"):
     """Oracle on the same bytes.  tau is rounded to float32 first, as the C ABI takes a float.
     If gpu_hit is given, queries whose decision ties with tau (rule (i)) adopt the GPU's
     decision so that both state machines stay in step; returns the list of such queries."""
@@ -57,7 +57,8 @@ def run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=None, max_forc
     force = np.full(len(queries), -1, np.int32)
     forced = []
     while True:
-        o = oracle.Oracle(corpus, d, k, capacity, tau32, POL[policy], rho=rho, lsh_planes=lsh_planes, lsh_bucket=lsh_bucket)
+        o = oracle.Oracle(corpus, d, k, capacity, tau32, POL[policy], rho=rho, lsh_planes=lsh_planes, lsh_bucket=lsh_bucket,
+                          metric=oracle.COSINE if metric == "cosine" else oracle.L2SQ)
         r = o.query(queries, force)
         o.close()
         if gpu_hit is None:
@@ -74,19 +75,20 @@ def run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=None, max_forc
         forced.append(i)
 
 
-def knn_tie_excused(corpus, q, k):
+def knn_tie_excused(corpus, q, k, metric="l2"):
     """Rule (ii): is there a tie to 1e-5 relative at the k/(k+1) boundary or inside the list?"""
     kk = min(k + 1, corpus.shape[0])
-    _, d = oracle.exact_topk(corpus, q, kk)
+    _, d = oracle.exact_topk(corpus, q, kk, metric=oracle.COSINE if metric == "cosine" else oracle.L2SQ)
     d = d[0]
     gaps = np.diff(d)
     return bool(np.any(gaps < REL_TIE * np.maximum(d[1:], 1e-300)))
 
 
-def compare(corpus, queries, k, capacity, tau, policy, gpu, max_excused_frac=1e-3, rho=1, lsh_planes=None, lsh_bucket=0):
+def compare(corpus, queries, k, capacity, tau, policy, gpu, max_excused_frac=1e-3, rho=1, lsh_planes=None, lsh_bucket=0,
+            metric="l2"):
     ids, dists, hit, stats = gpu
     ref, forced = run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=hit, rho=rho, lsh_planes=lsh_planes,
-                             lsh_bucket=lsh_bucket)
+                             lsh_bucket=lsh_bucket, metric=metric)
     n = len(queries)
     bad_hit = np.nonzero(ref["hit"] != hit)[0]
     assert len(bad_hit) == 0, f"hit/miss differs first at query {bad_hit[0]} (best={ref['best'][bad_hit[0]]}, tau={tau})"
@@ -95,7 +97,7 @@ def compare(corpus, queries, k, capacity, tau, policy, gpu, max_excused_frac=1e-
     for i in rows_bad:
         origin = int(ref["origin"][i])                       # the miss whose list is returned
         src = origin if origin >= 0 else i
-        tie = knn_tie_excused(corpus, queries[src], k * rho)
+        tie = knn_tie_excused(corpus, queries[src], k * rho, metric)
         if not tie and rho > 1 and src != i:                 # re-ranked hit: a tie among the stored rows for this query
             stored, _ = oracle.exact_topk(corpus, queries[src], k * rho)
             dd = np.sort(((queries[i].astype(np.float64)[None, :] - corpus[stored[0]].astype(np.float64)) ** 2).sum(1))

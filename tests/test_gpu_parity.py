@@ -22,7 +22,7 @@ def stream(N, d, comps, nq, topics, s, sigma, seed=0):
 def check(X, Q, k, cap, tau, policy, batch, **kw):
     gpu = run_gpu(X.to(DEV), Q.to(DEV), k, cap, tau, policy, batch, **kw)
     return compare(X.numpy(), Q.numpy(), k, cap, tau, policy, gpu, rho=kw.get("rho", 1),
-                   lsh_planes=kw.get("lsh_planes"), lsh_bucket=kw.get("lsh_bucket", 0)), gpu
+                   lsh_planes=kw.get("lsh_planes"), lsh_bucket=kw.get("lsh_bucket", 0), metric=kw.get("metric", "l2")), gpu
 
 
 # ------------------------------------------------------------------ hand-traced sequences
@@ -168,6 +168,41 @@ def test_reranking_factor_argument_checks():
     h = lib.prox_create_rho(Xd.data_ptr(), 500, 64, 32, 8, 0.5, 0, 4)
     assert h
     lib.prox_destroy(h)
+
+
+# ------------------------------------------------------------------ cosine distance (Section 2.1)
+@pytest.mark.parametrize("policy,batch,rho", [("lru", 64, 1), ("fifo", 1, 1), ("lru", 500, 2)])
+def test_cosine_distance_matches_the_oracle(policy, batch, rho):
+    """Rows and queries of very different lengths: the Euclidean neighbours are not the cosine ones."""
+    X, Q = stream(30011, 128, 48, 1500, 100, 1.0, 0.03, seed=51)
+    g = torch.Generator().manual_seed(52)
+    X = (X * (0.2 + 5.0 * torch.rand(X.shape[0], 1, generator=g))).contiguous()
+    Q = (Q * (0.5 + 3.0 * torch.rand(Q.shape[0], 1, generator=g))).contiguous()
+    res, gpu = check(X, Q, 10, 40, 0.12, policy, batch, rho=rho, metric="cosine")
+    assert 0.2 < res["hit_rate"] < 0.97
+    l2 = run_gpu(X.to(DEV), Q.to(DEV), 10, 40, 0.12, policy, batch, rho=rho)
+    miss = res["ref"]["hit"] == 0
+    assert (l2[0][miss] != gpu[0][miss]).any(axis=1).mean() > 0.5
+
+
+def test_cosine_probe_only_with_loaded_keys():
+    keys, centres = W.make_probe_keys(3000, 128, 256, seed=53)
+    keys = (keys * (0.3 + 4.0 * torch.rand(3000, 1, generator=torch.Generator().manual_seed(54)))).contiguous()
+    p = prox.Prox(keys[:64].contiguous().to(DEV), 1, 3000, 0.02, "lru", metric="cosine")
+    p.cache_load(keys.to(DEV))
+    o = oracle.Oracle(None, 128, 1, 3000, float(np.float32(0.02)), oracle.LRU, metric=oracle.COSINE)
+    o.cache_load(keys.numpy())
+    for b in range(2):
+        Q = W.make_probe_batch(keys / keys.norm(dim=1, keepdim=True), centres, 512, 0.015, 53, b) * 2.5
+        hit, slot, dist = p.probe_batch(Q.contiguous().to(DEV))
+        torch.cuda.synchronize()
+        r = o.query(Q.numpy())
+        assert np.array_equal(hit.cpu().numpy(), r["hit"]) and np.array_equal(slot.cpu().numpy(), r["slot"])
+        h = r["hit"] == 1
+        assert np.allclose(dist.cpu().numpy()[h], r["best"][h], rtol=1e-4, atol=1e-9)
+        assert 0.2 < r["hit"].mean() < 0.97
+    assert p.status() == prox.OK
+    p.close()
 
 
 # ------------------------------------------------------------------ PROXIMITY-LSH (Section 3.2)
