@@ -20,6 +20,7 @@
 #include <cuda.h>
 
 #include <new>
+#include <vector>
 
 #include "prox_internal.h"
 #include "scan_readout.cuh"
@@ -58,6 +59,8 @@ struct ScanArgs {
     long long N;
     int d, pass, kp;
     int ks;                 // 64-column groups per pipeline stage (1 or 2; the tensor maps' boxes match)
+    const float *w_in;      // speed of every pair (or block) as the previous launch measured it, tiles per ns
+    float *w_out;           // ... as this launch measures it
 };
 
 struct Control {
@@ -68,6 +71,7 @@ struct Control {
     uint32_t tmem_base;
     int abort_flag;                  // set by any thread whose wait ran out
     int done;                        // read-out warps that have finished (the bound warp stops at kReadWarps)
+    long long t_begin, t_end;        // row tiles of this pair (or block)
 };
 
 // One read-out warp owns, for every query column it reads, a private candidate list in global
@@ -95,7 +99,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     const int q0 = a.pass * kScanQ;
     int nq = *a.n_active - q0;
     if (nq > kScanQ) nq = kScanQ;
-    if (nq <= 0) return;                                  // nothing missed in this pass
+    if (nq <= 0) {                                        // nothing missed in this pass
+        if (blockIdx.x == 0)
+            for (int u = tid; u < n_units; u += kThreads) a.w_out[u] = a.w_in[u];
+        return;
+    }
     const int n_pad = nq <= 32 ? 32 : (nq <= 64 ? 64 : (nq <= 128 ? 128 : 256));
     const int q_rows = PAIR ? n_pad / 2 : n_pad;             // query rows this block stages (half of B in a pair)
     const CUtensorMap *tm_q = q_rows == 16 ? &tm_q16 : (q_rows == 32 ? &tm_q32 : (q_rows == 64 ? &tm_q64 : (q_rows == 128 ? &tm_q128 : &tm_q256)));
@@ -132,6 +140,32 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         mbar_init(smem_u32(&ctl.q_full), 1);
         ctl.abort_flag = 0;
         ctl.done = 0;
+        // Row tiles are dealt out in contiguous runs whose lengths follow the speeds that the
+        // previous launch measured (SMs differ by their place on the die: up to a quarter in
+        // tiles per second), so that all pairs end together.  Every block adds the same numbers
+        // in the same order and so arrives at the same split.
+        {
+            const long long nt = (a.N + kUnitRows - 1) / kUnitRows;
+            double mean = 0.0;
+            for (int u = 0; u < n_units; ++u) mean += (double)a.w_in[u];
+            mean /= n_units;
+            double total = 0.0, before = 0.0, upto = 0.0;
+            for (int u = 0; u < n_units; ++u) {
+                double w = (double)a.w_in[u];
+                if (!(w > 0.7 * mean)) w = 0.7 * mean;     // one odd measurement must not starve a pair
+                if (w > 1.4 * mean) w = 1.4 * mean;
+                if (u < unit) before += w;
+                if (u <= unit) upto += w;
+                total += w;
+            }
+            long long b0 = (long long)((double)nt * (before / total));
+            long long b1 = unit == n_units - 1 ? nt : (long long)((double)nt * (upto / total));
+            if (b0 > nt) b0 = nt;
+            if (b1 > nt) b1 = nt;
+            if (b1 < b0) b1 = b0;
+            ctl.t_begin = b0;
+            ctl.t_end = b1;
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -146,6 +180,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     if constexpr (PAIR) cluster_sync_all();               // both blocks' barriers exist before any remote signal
     tc_fence_after();
     const uint32_t tmem_base = ctl.tmem_base;
+    const long long t_begin = ctl.t_begin, t_end = ctl.t_end;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -160,12 +195,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             }
             uint32_t g = 0;
             bool ok = true;
-            for (long long tile = unit; ok && tile < ntiles; tile += n_units) {
+            for (long long tile = t_begin; ok && tile < t_end; ++tile) {
                 const int row0 = (int)(tile * kUnitRows) + (int)rank * kTileRows;
                 // the ring holds less than a tile, little to cover DRAM latency with: have the next
                 // tile's corpus rows brought into L2 while this one is consumed
-                if (tile + n_units < ntiles) {
-                    const int row_n = row0 + n_units * kUnitRows;
+                if (tile + 1 < t_end) {
+                    const int row_n = row0 + kUnitRows;
                     for (int st = 0; st < nst; ++st) tma_prefetch_l2_3d(&tm_x, 0, row_n, st * ks);
                 }
                 for (int st = 0; st < nst; ++st, ++g) {
@@ -194,7 +229,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             bool ok = true;
             if (resident) ok = mbar_wait(smem_u32(&ctl.q_full), 0, abort_flag);
             uint32_t g = 0, it = 0;
-            for (long long tile = unit; ok && tile < ntiles; tile += n_units, ++it) {
+            for (long long tile = t_begin; ok && tile < t_end; ++tile, ++it) {
                 const uint32_t b = it & 1u, bph = (it >> 1) & 1u;
                 if (!mbar_wait(smem_u32(&ctl.tmem_empty[b]), bph ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -290,16 +325,17 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         uint32_t published[kReadGroups];
 #pragma unroll
         for (int i = 0; i < kReadGroups; ++i) published[i] = 0u;
-        long long row = (long long)unit * kUnitRows + (long long)rank * kTileRows + quarter * 32 + lane;
-        float hn = (unit < ntiles && row < a.N) ? a.xh[row] : INFINITY;
+        long long row = t_begin * kUnitRows + (long long)rank * kTileRows + quarter * 32 + lane;
+        float hn = (t_begin < t_end && row < a.N) ? a.xh[row] : INFINITY;
+        const unsigned long long ns0 = global_ns();
         bool alive = true;
         const uint32_t empty_bar0 = PAIR ? map_to_rank(smem_u32(&ctl.tmem_empty[0]), 0) : smem_u32(&ctl.tmem_empty[0]);
         const uint32_t empty_bar1 = PAIR ? map_to_rank(smem_u32(&ctl.tmem_empty[1]), 0) : smem_u32(&ctl.tmem_empty[1]);
-        for (long long tile = unit; alive && tile < ntiles; tile += n_units, ++it) {
+        for (long long tile = t_begin; alive && tile < t_end; ++tile, ++it) {
             const uint32_t b = it & 1u, bph = (it >> 1) & 1u;
             // loads whose latency hides behind the wait and the read-out
-            const long long row_next = row + (long long)n_units * kUnitRows;
-            const float hn_next = (tile + n_units < ntiles && row_next < a.N) ? a.xh[row_next] : INFINITY;
+            const long long row_next = row + kUnitRows;
+            const float hn_next = (tile + 1 < t_end && row_next < a.N) ? a.xh[row_next] : INFINITY;
             uint32_t g_thr[kReadGroups];
 #pragma unroll
             for (int i = 0; i < kReadGroups; ++i) {
@@ -399,6 +435,13 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             row = row_next;
             hn = hn_next;
         }
+        // the speed of this pair (or block) for the next launch's split; kept when the launch was
+        // too short to tell (the same test in every block, so all keep or all renew)
+        if (rank == 0 && e == 0 && lane == 0) {
+            const unsigned long long ns = global_ns() - ns0;
+            const bool long_enough = ntiles >= 32LL * n_units;
+            a.w_out[unit] = (long_enough && alive && it > 0 && ns > 0) ? (float)((double)it / (double)ns) : a.w_in[unit];
+        }
         // the lists go to the merge as they are: it drops what the shared bound has ruled out
         __syncwarp();
         for (int lc = lane; lc < ncol; lc += 32) {
@@ -465,7 +508,11 @@ struct Maps {
     CUtensorMap x, q16, q32, q64, q128, q256;
     int ks = 1;
     bool ok = false;
+    float *speed = nullptr;        // device, 2 x kMaxUnits: the pairs' speeds, written by one launch, read by the next
+    int units = 0;                 // pairs (or blocks) the speeds were measured for
+    unsigned launch_no = 0;
 };
+constexpr int kMaxUnits = 256;
 
 }  // namespace
 
@@ -480,7 +527,8 @@ static int launch_scan_generic(prox_handle *h, void **state, const __nv_bfloat16
         *state = m;
         const uint32_t ks = ((h->d / kChunkK) % 2 == 0) ? 2 : 1;
         m->ks = (int)ks;
-        m->ok = make_map(&m->x, xb, (uint64_t)rows, (uint64_t)h->d, kTileRows, ks) &&
+        if (cudaMalloc(&m->speed, sizeof(float) * 2 * kMaxUnits) != cudaSuccess) { m->speed = nullptr; cudaGetLastError(); }
+        m->ok = m->speed != nullptr && make_map(&m->x, xb, (uint64_t)rows, (uint64_t)h->d, kTileRows, ks) &&
                 make_map(&m->q16, qb, kMaxBatch, (uint64_t)h->d, 16, ks) &&
                 make_map(&m->q32, qb, kMaxBatch, (uint64_t)h->d, 32, ks) &&
                 make_map(&m->q64, qb, kMaxBatch, (uint64_t)h->d, 64, ks) &&
@@ -498,6 +546,17 @@ static int launch_scan_generic(prox_handle *h, void **state, const __nv_bfloat16
     a.buf_cnt = h->buf_cnt; a.N = rows; a.d = h->d; a.pass = pass; a.kp = kp; a.ks = maps.ks;
     const bool pair = h->scan_mode != PROX_SCAN_TC_SINGLE && h->scan_ctas >= 2 && rows >= 2 * kTileRows;
     const int grid = pair ? (h->scan_ctas & ~1) : h->scan_ctas;
+    const int units = pair ? grid / 2 : grid;
+    if (units > kMaxUnits) return 1;
+    if (maps.units != units) {                            // first launch, or the launch shape changed: equal speeds
+        static const std::vector<float> ones(2 * kMaxUnits, 1.f);
+        if (cudaMemcpyAsync(maps.speed, ones.data(), sizeof(float) * 2 * kMaxUnits, cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return 1;
+        maps.units = units;
+    }
+    a.w_in = maps.speed + (maps.launch_no & 1u) * kMaxUnits;
+    a.w_out = maps.speed + ((maps.launch_no + 1u) & 1u) * kMaxUnits;
+    maps.launch_no++;
     h->scan_lists = 4 * grid;                             // one candidate list per read-out lane quarter
     h->scan_list_stride = h->tc_cap;
     cudaLaunchConfig_t cfg = {};
@@ -539,10 +598,12 @@ int launch_probe_scan_tc(prox_handle *h, int pass, cudaStream_t s) {
 }
 
 void free_scan_tc(prox_handle *h) {
-    delete static_cast<Maps *>(h->tc_state);
-    h->tc_state = nullptr;
-    delete static_cast<Maps *>(h->tc_state_keys);
-    h->tc_state_keys = nullptr;
+    for (void **st : {&h->tc_state, &h->tc_state_keys}) {
+        Maps *m = static_cast<Maps *>(*st);
+        if (m && m->speed) cudaFree(m->speed);
+        delete m;
+        *st = nullptr;
+    }
 }
 
 }  // namespace prox
