@@ -10,11 +10,13 @@
 //            N = padded query count, K = 16 per instruction, fp32 accumulators in tensor memory,
 //            two accumulator buffers so that the read-out of tile t overlaps the products of t+1);
 //   warp 2   keeps the score bounds that the blocks share fresh (see the bound warp below);
-//   warps 4-   read the accumulators (tcgen05.ld, one corpus row per thread, the warps of a
+//   warps 4-11 read the accumulators (tcgen05.ld, one corpus row per thread, the two warps of a
 //            tensor-memory lane quarter splitting the columns) into registers, hand the
 //            accumulator buffer back at once, then compare every score with the query's
 //            threshold and append survivors to warp-private candidate lists; a warp sorts and
 //            cuts a list of its own when it could overflow.
+// Row tiles are dealt to the pairs of blocks in contiguous runs whose lengths follow the speed
+// each pair showed in the previous launch.
 // Every wait on an mbarrier is bounded in time; on expiry the block latches PROX_ERR_TIMEOUT,
 // stops issuing work, lets copies in flight land, frees its tensor memory and returns.
 #include <cuda.h>

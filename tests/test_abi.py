@@ -37,6 +37,11 @@ def test_calls_without_handle_are_rejected_on_the_host():
     assert b"NULL" in lib.prox_last_error()
     lib.prox_destroy(None)
     assert not lib.prox_create(None, 10, 16, 1, 1, 0.5, 0)
+    # the wider constructors check their own arguments before they touch the device
+    assert not lib.prox_create_rho(None, 10, 16, 1, 1, 0.5, 0, 0) and b"rho" in lib.prox_last_error()
+    assert not lib.prox_create_metric(None, 10, 16, 1, 1, 0.5, 0, 1, 7) and b"metric" in lib.prox_last_error()
+    assert not lib.prox_create_lsh(None, 10, 16, 1, 25, 4, None, 0.5, 0, 1) and b"L must" in lib.prox_last_error()
+    assert not lib.prox_create_lsh(None, 10, 16, 1, 3, 0, None, 0.5, 0, 1) and b"bucket" in lib.prox_last_error()
 
 
 def test_binding_fails_loudly_without_the_library(monkeypatch):
