@@ -84,21 +84,45 @@ __device__ __forceinline__ float max_margin32(const uint32_t (&v)[32], const flo
     return fmaxf(m0, m1);
 }
 
+// Largest of 32 accumulator columns of this lane's row, thresholds aside.
+__device__ __forceinline__ float raw_max32(const uint32_t (&v)[32]) {
+    float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 32; j += 4) {
+        m0 = max3(m0, __uint_as_float(v[j]), __uint_as_float(v[j + 1]));
+        m1 = max3(m1, __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+    }
+    return fmaxf(m0, m1);
+}
+
 // Up to 64 accumulator columns (queries c0 .. c0+63; the second 32 only when `two`) of one corpus
 // row per lane, already in registers.  A column passes when acc - thr > half norm, i.e. score =
 // acc - half norm beats the threshold up to one rounding (the certificate's slack covers it).
-// One maximum per group and a single vote decide the common case that nothing passes.
+// Three levels, cheapest first:
+//   1. the row's largest accumulator of a group against the group's smallest threshold (tmin0 /
+//      tmin1: lower bounds of the thresholds of the 32 columns, held in registers): no row can
+//      pass a column if it does not pass this, and it needs no threshold from shared memory,
+//      whose load pipe all read-out warps share;
+//   2. for a group that some lane cannot rule out: the per-column margins, one vote;
+//   3. the appends.
 template <int CAP>
 __device__ __forceinline__ void readout64(const uint32_t (&v0)[32], const uint32_t (&v1)[32], bool two, int c0,
-                                          int lc0, float hn, int32_t row, const float *thr, int *wcnt,
-                                          uint32_t *best, u64 *lists, bool &need) {
-    const float m0 = max_margin32(v0, thr, c0);
-    const float m1 = two ? max_margin32(v1, thr, c0 + 32) : -INFINITY;
-    const unsigned any = __ballot_sync(0xffffffffu, fmaxf(m0, m1) > hn);
-    if (any == 0u) return;
-    if (__any_sync(0xffffffffu, m0 > hn)) append32<CAP>(v0, c0, lc0, hn, row, thr, wcnt, best, lists, need);
-    if (two && __any_sync(0xffffffffu, m1 > hn))
-        append32<CAP>(v1, c0 + 32, lc0 + 32, hn, row, thr, wcnt, best, lists, need);
+                                          int lc0, float hn, float tmin0, float tmin1, int32_t row,
+                                          const float *thr, int *wcnt, uint32_t *best, u64 *lists, bool &need) {
+    const bool c0p = raw_max32(v0) - tmin0 > hn;
+    const bool c1p = two && raw_max32(v1) - tmin1 > hn;
+    const unsigned maybe0 = __ballot_sync(0xffffffffu, c0p);
+    const unsigned maybe1 = __ballot_sync(0xffffffffu, c1p);
+    if ((maybe0 | maybe1) == 0u) return;
+    if (maybe0 != 0u) {
+        const float m0 = max_margin32(v0, thr, c0);
+        if (__any_sync(0xffffffffu, m0 > hn)) append32<CAP>(v0, c0, lc0, hn, row, thr, wcnt, best, lists, need);
+    }
+    if (maybe1 != 0u) {
+        const float m1 = max_margin32(v1, thr, c0 + 32);
+        if (__any_sync(0xffffffffu, m1 > hn))
+            append32<CAP>(v1, c0 + 32, lc0 + 32, hn, row, thr, wcnt, best, lists, need);
+    }
 }
 
 }  // namespace prox

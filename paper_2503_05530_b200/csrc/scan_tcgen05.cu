@@ -325,8 +325,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         int32_t *lists_cnt = a.buf_cnt + (size_t)(blockIdx.x * 4 + quarter) * kScanQ;
         uint32_t it = 0;
         uint32_t published[kReadGroups];
+        float tmin[kReadGroups];                                  // lower bound of the thresholds of each 32-column group
 #pragma unroll
-        for (int i = 0; i < kReadGroups; ++i) published[i] = 0u;
+        for (int i = 0; i < kReadGroups; ++i) { published[i] = 0u; tmin[i] = -INFINITY; }
         long long row = t_begin * kUnitRows + (long long)rank * kTileRows + quarter * 32 + lane;
         float hn = (t_begin < t_end && row < a.N) ? a.xh[row] : INFINITY;
         const unsigned long long ns0 = global_ns();
@@ -389,8 +390,13 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     }
                 }
                 if (active && c0 < cw)
-                    readout64<CAP>(v0, v1, c0 + 32 < cw, col_begin + c0, c0, hn, (int32_t)row, ctl.thr, wcnt, ctl.best[quarter],
-                                   lists, need);
+                {
+                    // (selected, not indexed: the array stays in registers)
+                    const float ta = c0 == 0 ? tmin[0] : tmin[kReadGroups > 2 ? 2 : 0];
+                    const float tb = c0 == 0 ? tmin[kReadGroups > 1 ? 1 : 0] : tmin[kReadGroups > 3 ? 3 : 0];
+                    readout64<CAP>(v0, v1, c0 + 32 < cw, col_begin + c0, c0, hn, ta, tb, (int32_t)row, ctl.thr, wcnt,
+                                   ctl.best[quarter], lists, need);
+                }
                 if (last) break;
             }
             if (!early) {
@@ -403,9 +409,18 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     }
                 }
             }
-            // the warp publishes the best score of its lane quarter for each of its columns (every
-            // tile at first, every fourth once the bounds move slowly)
+            // the warp publishes the best score of its lane quarter for each of its columns, and takes
+            // the smallest threshold of each of its column groups for the first level of the test
+            // (every tile at first, every fourth once the bounds move slowly; thresholds only rise,
+            // so an older minimum is still a lower bound)
             if (it < 16 || (it & 3u) == 0u) {
+#pragma unroll
+                for (int i = 0; i < kReadGroups; ++i) {
+                    float t = ctl.thr[col_begin + ((lane + 32 * i) < cw ? lane + 32 * i : 0)];
+#pragma unroll
+                    for (int m = 16; m > 0; m >>= 1) t = fminf(t, __shfl_xor_sync(0xffffffffu, t, m));
+                    tmin[i] = t;
+                }
 #pragma unroll
                 for (int i = 0; i < kReadGroups; ++i) {
                     const int lc = lane + 32 * i;
