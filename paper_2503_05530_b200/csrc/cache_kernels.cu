@@ -489,12 +489,27 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
     {
         const int i = tid;
         int n = 0;
+        bool settled = false;
         if (i < B) {
             n = n_cand[i];
-            sm.safe_min[i] = g_safe_min[i];
-            sm.safe_arg[i] = g_safe_arg[i];
+            const double sd = g_safe_min[i];
+            const int sa = g_safe_arg[i];
+            sm.safe_min[i] = sd;
+            sm.safe_arg[i] = sa;
             sm.b_slot[i] = -1;
             sm.b_stamp[i] = 0;
+            // A query with no at-risk or in-batch key within tau whose nearest safe key is within tau
+            // hits that key whatever the rest of the batch does (safe keys are not evicted in this
+            // batch, and touching one changes no eviction of this batch): settled here, in parallel.
+            if (n == 0 && sa >= 0 && sd <= tau) {
+                settled = true;
+                out_hit[i] = 1;
+                evt_slot[i] = sa;
+                evt_dist[i] = (float)sd;
+                miss_rank[i] = -1;
+                src_kind[i] = 1; src[i] = sa;
+                if (policy == PROX_LRU) atomicMax(&stamp[sa], (u64)(clock0 + i));     // the latest hit stays
+            }
         }
         if (i < R) {
             sm.r_slot[i] = risk_slot[i];
@@ -502,7 +517,7 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
             sm.r_alive[i] = 1;
             sm.r_touched[i] = 0;
         }
-        if (i < kMaxBatch) sm.ncand[i] = n;
+        if (i < kMaxBatch) sm.ncand[i] = settled ? -1 : n;
         // exclusive prefix sum of n over the block
         int x = n;
 #pragma unroll
@@ -544,6 +559,7 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
         for (int i = 0; i < B; ++i) {
             const u64 t = (u64)(clock0 + i);
             const int n = sm.ncand[i], o = sm.off[i];
+            if (n < 0) { ++n_hit; continue; }             // settled in the parallel pass
             const bool in_smem = (o + n <= kCsrCap);
             double bd = INFINITY;
             int bslot = 0x7fffffff, bcode = -1;
@@ -574,7 +590,7 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
                     miss_rank[i] = -1;
                     if (bcode == -2) {
                         src_kind[i] = 1; src[i] = bslot;
-                        if (policy == PROX_LRU) stamp[bslot] = t;
+                        if (policy == PROX_LRU) atomicMax(&stamp[bslot], t);   // a later query may have touched it in the parallel pass
                     } else if (bcode < kMaxBatch) {
                         src_kind[i] = 1; src[i] = bslot;
                         if (policy == PROX_LRU) { sm.r_stamp[bcode] = t; sm.r_touched[bcode] = 1; }
@@ -895,13 +911,12 @@ void launch_build_candidates(prox_handle *h, int B, cudaStream_t s) {
     h->launches++;
 }
 
+// Kernel attributes belong to a device: set when a handle is created there, not once per process.
+void set_cache_kernel_attributes() {
+    cudaFuncSetAttribute(resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ResolveSmem));
+}
+
 void launch_resolve(prox_handle *h, int B, uint8_t *out_hit, cudaStream_t s) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)sizeof(ResolveSmem));
-        attr_set = true;
-    }
     resolve_kernel<<<1, 1024, sizeof(ResolveSmem), s>>>(
         h->st, B, (long long)h->C, (double)h->tau, h->policy, h->stamp, h->risk_slot, h->risk_stamp,
         h->safe_min, h->safe_arg, h->cand_d, h->cand_code, h->n_cand, out_hit, h->src, h->src_kind,

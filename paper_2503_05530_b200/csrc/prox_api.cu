@@ -147,6 +147,8 @@ extern "C" prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t 
     }
     h->num_sms = prop.multiProcessorCount;
     h->scan_ctas = h->num_sms;
+    set_cache_kernel_attributes();
+    set_scan_kernel_attributes();
 
     const size_t MB = kMaxBatch, C = (size_t)capacity, P = (size_t)h->scan_ctas;
     bool ok = true;

@@ -687,11 +687,6 @@ void launch_merge_select(prox_handle *h, int pass, int B, int for_probe, cudaStr
     int nq = B - pass * kScanQ;
     if (nq > kScanQ) nq = kScanQ;
     if (nq <= 0) return;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(merge_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeStageMax * 8);
-        attr_set = true;
-    }
     // a scan of few rows never tightens its bounds, so every row may still be in the lists: stage them all
     const long long rows = for_probe ? (long long)h->C : (long long)h->N;
     const int stage_cap = rows <= kMergeStageMax ? (int)((rows + 1023) / 1024 * 1024) : kMergeStage;
@@ -704,15 +699,14 @@ void launch_merge_select(prox_handle *h, int pass, int B, int for_probe, cudaStr
 
 static size_t rerank_smem(int d) { return (size_t)kRerankMax * 12 + (size_t)d * 4; }
 
+// Kernel attributes belong to a device: set when a handle is created there, not once per process.
+void set_scan_kernel_attributes() {
+    cudaFuncSetAttribute(merge_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeStageMax * 8);
+    cudaFuncSetAttribute(rerank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rerank_smem(4096));
+    cudaFuncSetAttribute(fallback_collect_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFallbackGroup * 4096 * 4);
+}
+
 void launch_rerank(prox_handle *h, const float *q, int B, cudaStream_t s) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(rerank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)rerank_smem(4096));
-        cudaFuncSetAttribute(fallback_collect_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kFallbackGroup * 4096 * 4);
-        attr_set = true;
-    }
     rerank_kernel<<<B, 256, rerank_smem(h->d), s>>>(h->st, 0, h->corpus, q, h->d, h->k, (long long)h->N,
                                                     h->miss_list, h->cand_id, h->cand_n, h->cand_sk, h->qbn,
                                                     h->qerr, h->res_ids, h->res_dists, h->fail_list,
