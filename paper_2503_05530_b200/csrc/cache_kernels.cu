@@ -552,8 +552,71 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
         __syncthreads();
     }
 
+    // ---- no at-risk key and no query of the batch lies within tau of any query: the hits (all on
+    // safe keys) are settled, the others are misses that meet no one, so the replay has a closed
+    // form: the j-th miss takes the j-th free slot, then the j-th at-risk entry in stamp order
+    // (none of them was touched).  Taken when the evictions stay within the at-risk list.
+    bool closed_form = false;
+    if (sm.off[kMaxBatch] == 0) {
+        const int i = tid;
+        const int miss = (i < B && sm.ncand[i] == 0) ? 1 : 0;
+        int x = miss;
+#pragma unroll
+        for (int m = 1; m < 32; m <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, x, m);
+            if (lane >= m) x += y;
+        }
+        if (lane == 31) sm.warp_tot[warp] = x;
+        __syncthreads();
+        if (warp == 0) {
+            int w = sm.warp_tot[lane];
+#pragma unroll
+            for (int m = 1; m < 32; m <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, w, m);
+                if (lane >= m) w += y;
+            }
+            sm.warp_tot[lane] = w;
+        }
+        __syncthreads();
+        const int j = x + (warp > 0 ? sm.warp_tot[warp - 1] : 0) - 1;      // rank of this miss
+        const int n_miss = sm.warp_tot[31];
+        const long long free_slots = C > count0 ? C - count0 : 0;
+        const long long n_evict = n_miss > free_slots ? n_miss - free_slots : 0;
+        closed_form = n_evict <= (long long)R;
+        if (closed_form) {
+            if (miss) {
+                int slot;
+                if (j < free_slots) {
+                    slot = (int)(count0 + j);
+                } else {
+                    const int v = (int)(j - free_slots);
+                    slot = sm.r_slot[v];
+                    sm.r_alive[v] = 0;
+                }
+                out_hit[i] = 0;
+                src_kind[i] = 0; src[i] = -1;
+                evt_slot[i] = slot;
+                evt_dist[i] = INFINITY;
+                sm.b_slot[i] = slot;
+                sm.b_stamp[i] = (u64)(clock0 + i);
+                miss_list[j] = i;
+                miss_rank[i] = j;
+            }
+            if (tid == 0) {
+                st->count = count0 + n_miss - n_evict;
+                st->clock = clock0 + B;
+                st->n_miss = n_miss;
+                st->queries += B;
+                st->hits += B - n_miss;
+                st->misses += n_miss;
+                st->evictions += n_evict;
+            }
+        }
+        __syncthreads();
+    }
+
     // ---- sequential replay by warp 0
-    if (warp == 0) {
+    if (!closed_form && warp == 0) {
         long long cnt = count0;
         int p = 0, n_miss = 0, n_hit = 0, n_intra = 0, n_evict = 0;
         for (int i = 0; i < B; ++i) {
