@@ -84,7 +84,7 @@ static bool dev_alloc(T *&p, size_t n) {
 }
 
 static void free_all(prox_handle *h) {
-    void *ptrs[] = {h->corpus_own, h->qn, h->planes, h->bucket_count, h->lsh_code, h->lsh_order, h->lsh_seg, h->lsh_work, h->xb, h->xh, h->keys, h->val_ids, h->val_dists, h->stamp, h->risk_pos, h->st,
+    void *ptrs[] = {h->redo, h->corpus_own, h->qn, h->planes, h->bucket_count, h->lsh_code, h->lsh_order, h->lsh_seg, h->lsh_work, h->xb, h->xh, h->keys, h->val_ids, h->val_dists, h->stamp, h->risk_pos, h->st,
                     h->risk_slot, h->risk_stamp, h->part_min, h->part_arg, h->d_risk, h->d_intra,
                     h->safe_min, h->safe_arg, h->cand_d, h->cand_code, h->n_cand, h->src, h->src_kind,
                     h->ins_slot, h->evt_slot, h->evt_dist, h->miss_list, h->miss_rank, h->qb, h->qbn,
@@ -172,7 +172,7 @@ extern "C" prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t 
     ok = ok && dev_alloc(h->cand_n, MB) && dev_alloc(h->cand_sk, MB);
     ok = ok && dev_alloc(h->res_ids, MB * k) && dev_alloc(h->res_dists, MB * k);
     ok = ok && dev_alloc(h->fail_list, MB) && dev_alloc(h->fail_radius, MB);
-    ok = ok && dev_alloc(h->coll_id, MB * kCollectCap) && dev_alloc(h->coll_n, MB);
+    ok = ok && dev_alloc(h->coll_id, MB * kCollectCap) && dev_alloc(h->coll_n, MB) && dev_alloc(h->redo, MB + 1);
     // caches of a few thousand keys and more are probed on the tensor cores first (bf16 copies of the keys)
     h->probe_tc = (d % 64 == 0 && capacity >= 4096) ? 1 : 0;
     ok = ok && dev_alloc(h->use_partial, MB) && dev_alloc(h->pfail_list, MB);

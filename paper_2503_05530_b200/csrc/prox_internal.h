@@ -131,6 +131,7 @@ struct prox_handle {
     float *fail_radius;               // kMaxBatch: exact k-th distance among the candidates
     int32_t *coll_id;                 // kMaxBatch x kCollectCap (indexed by position in fail_list)
     int32_t *coll_n;                  // kMaxBatch
+    int32_t *redo;                    // kMaxBatch + 1: queries the fp32 sweep of the exact pass takes again; [kMaxBatch] any
 
     // staging for the host-buffer entry point
     float *stage_q;

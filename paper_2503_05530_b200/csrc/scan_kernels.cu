@@ -529,9 +529,86 @@ __device__ __forceinline__ void fallback_rows(const float *__restrict__ corpus, 
     }
 }
 
+// The same sweep over the bf16 copy of the corpus (half the bytes): |sqrt(coarse) - sqrt(exact)| is
+// at most the rounding error of the row, so the caller passes radii widened by that error and
+// every row within the exact radius is still collected (a few more with it).
+template <int NG>
+__device__ __forceinline__ void fallback_rows_bf16(const __nv_bfloat16 *__restrict__ xb, long long N, int d,
+                                                   long long warp, long long nwarps, const float *q_sm,
+                                                   const float *radius, float margin, int32_t *coll_id,
+                                                   int32_t *coll_n, int g0) {
+    constexpr int U = NG <= 2 ? 4 : 2;                 // rows in flight per warp: the sweep is bound by load latency
+    const int lane = threadIdx.x & 31;
+    for (long long r0 = warp; r0 < N; r0 += (long long)U * nwarps) {
+        float acc[U][NG];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int f = 0; f < NG; ++f) acc[u][f] = 0.f;
+        for (int j = lane; j < d / 8; j += 32) {
+            uint4 w[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const long long r = r0 + (long long)u * nwarps;
+                w[u] = r < N ? __ldcs(reinterpret_cast<const uint4 *>(xb + (size_t)r * d) + j) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int f = 0; f < NG; ++f) {
+                const float4 qa = *reinterpret_cast<const float4 *>(&q_sm[f * d + 8 * j]);
+                const float4 qb2 = *reinterpret_cast<const float4 *>(&q_sm[f * d + 8 * j + 4]);
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const uint32_t ww[4] = {w[u].x, w[u].y, w[u].z, w[u].w};   // eight bf16
+                    const float d0 = qa.x - __uint_as_float(ww[0] << 16), d1 = qa.y - __uint_as_float(ww[0] & 0xffff0000u);
+                    const float d2 = qa.z - __uint_as_float(ww[1] << 16), d3 = qa.w - __uint_as_float(ww[1] & 0xffff0000u);
+                    const float d4 = qb2.x - __uint_as_float(ww[2] << 16), d5 = qb2.y - __uint_as_float(ww[2] & 0xffff0000u);
+                    const float d6 = qb2.z - __uint_as_float(ww[3] << 16), d7 = qb2.w - __uint_as_float(ww[3] & 0xffff0000u);
+                    const float a = fmaf(d0, d0, fmaf(d1, d1, fmaf(d2, d2, fmaf(d3, d3, acc[u][f]))));
+                    acc[u][f] = fmaf(d4, d4, fmaf(d5, d5, fmaf(d6, d6, fmaf(d7, d7, a))));
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long r = r0 + (long long)u * nwarps;
+#pragma unroll
+            for (int f = 0; f < NG; ++f)
+#pragma unroll
+                for (int s = 16; s > 0; s >>= 1) acc[u][f] += __shfl_xor_sync(0xffffffffu, acc[u][f], s);
+            if (lane < NG && r < N) {
+                float mine = 0.f;
+#pragma unroll
+                for (int f = 0; f < NG; ++f)
+                    if (f == lane) mine = acc[u][f];
+                const float rad = radius[lane];                    // -1 for an empty place in the group
+                if (mine <= rad * (1.f + margin) + 1e-30f) {
+                    const int pos = atomicAdd(&coll_n[g0 + lane], 1);
+                    if (pos < kCollectCap) coll_id[(size_t)(g0 + lane) * kCollectCap + pos] = (int32_t)r;
+                }
+            }
+        }
+    }
+}
+
+// Between the two sweeps of the exact pass: a query whose widened radius over the bf16 copy took
+// in more rows than the collection holds is swept again over the fp32 rows with the exact radius.
+__global__ void __launch_bounds__(1024)
+fallback_mark_kernel(const DevState *st, int32_t *coll_n, int32_t *redo) {
+    __shared__ int any;
+    const int f = threadIdx.x;
+    if (f == 0) any = 0;
+    __syncthreads();
+    const bool over = f < st->n_fail && coll_n[f] > kCollectCap;
+    redo[f] = over ? 1 : 0;
+    if (over) { coll_n[f] = 0; any = 1; }
+    __syncthreads();
+    if (f == 0) redo[kMaxBatch] = any;
+}
+
 __global__ void __launch_bounds__(256)
-fallback_collect_kernel(DevState *st, const float *__restrict__ corpus, const float *__restrict__ queries,
-                        long long N, int d, const int32_t *__restrict__ miss_list,
+fallback_collect_kernel(DevState *st, const float *__restrict__ corpus, const __nv_bfloat16 *__restrict__ xb,
+                        const int32_t *__restrict__ redo,
+                        const float *__restrict__ queries, long long N, int d, const int32_t *__restrict__ miss_list,
                         const int32_t *__restrict__ fail_list, const float *__restrict__ fail_radius,
                         int32_t *coll_id, int32_t *coll_n) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -539,6 +616,7 @@ fallback_collect_kernel(DevState *st, const float *__restrict__ corpus, const fl
     __shared__ float radius[kFallbackGroup];
     const int n_fail = st->n_fail;
     if (n_fail == 0) return;
+    if (redo != nullptr && redo[kMaxBatch] == 0) return;                // second sweep: nothing overflowed
     const int tid = threadIdx.x;
     const long long warp = ((long long)blockIdx.x * blockDim.x + tid) >> 5;
     const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
@@ -551,8 +629,23 @@ fallback_collect_kernel(DevState *st, const float *__restrict__ corpus, const fl
             const int f = idx / d, j = idx - f * d;
             q_sm[idx] = (f < ng) ? queries[(size_t)miss_list[fail_list[g0 + f]] * d + j] : 0.f;
         }
-        if (tid < kFallbackGroup) radius[tid] = (tid < ng) ? fail_radius[g0 + tid] : -1.f;
+        if (tid < kFallbackGroup) {
+            float rad = (tid < ng) ? fail_radius[g0 + tid] : -1.f;
+            if (redo != nullptr && tid < ng && redo[g0 + tid] == 0) rad = -1.f;   // settled by the first sweep
+            if (xb != nullptr && rad >= 0.f) {                     // widened by the rows' rounding error, rounded up
+                const float w = sqrtf(rad) * (1.f + 2e-7f) + st->e_max * (1.f + 2e-7f);
+                rad = w * w * (1.f + 2e-7f);
+            }
+            radius[tid] = rad;
+        }
         __syncthreads();
+        if (xb != nullptr) {
+            if (ng == 1) fallback_rows_bf16<1>(xb, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
+            else if (ng == 2) fallback_rows_bf16<2>(xb, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
+            else if (ng <= 4) fallback_rows_bf16<4>(xb, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
+            else fallback_rows_bf16<8>(xb, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
+            continue;
+        }
         if (ng == 1) fallback_rows<1>(corpus, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
         else if (ng == 2) fallback_rows<2>(corpus, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
         else if (ng <= 4) fallback_rows<4>(corpus, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
@@ -724,9 +817,14 @@ void launch_hit_rerank(prox_handle *h, const float *q, int B, int kind, int64_t 
 
 void launch_fallback(prox_handle *h, const float *q, int B, cudaStream_t s) {
     fallback_collect_kernel<<<h->num_sms * 4, 256, (size_t)kFallbackGroup * h->d * 4, s>>>(
-        h->st, h->corpus, q, (long long)h->N, h->d, h->miss_list, h->fail_list, h->fail_radius, h->coll_id,
-        h->coll_n);
-    h->launches++;
+        h->st, h->corpus, h->xb, nullptr, q, (long long)h->N, h->d, h->miss_list, h->fail_list, h->fail_radius,
+        h->coll_id, h->coll_n);
+    // the bf16 sweep reads half the bytes; what it cannot hold is swept again in fp32
+    fallback_mark_kernel<<<1, 1024, 0, s>>>(h->st, h->coll_n, h->redo);
+    fallback_collect_kernel<<<h->num_sms * 4, 256, (size_t)kFallbackGroup * h->d * 4, s>>>(
+        h->st, h->corpus, nullptr, h->redo, q, (long long)h->N, h->d, h->miss_list, h->fail_list, h->fail_radius,
+        h->coll_id, h->coll_n);
+    h->launches += 3;
     rerank_kernel<<<B, 256, rerank_smem(h->d), s>>>(h->st, 1, h->corpus, q, h->d, h->k, (long long)h->N,
                                                     h->miss_list, h->cand_id, h->cand_n, h->cand_sk, h->qbn,
                                                     h->qerr, h->res_ids, h->res_dists, h->fail_list,
