@@ -38,7 +38,7 @@ namespace {
 #ifndef PROX_READ_WARPS
 #define PROX_READ_WARPS 8
 #endif
-constexpr int kReadWarps = PROX_READ_WARPS;          // 8, 12 or 16
+constexpr int kReadWarps = PROX_READ_WARPS;          // 4, 8, 12 or 16
 constexpr int kReadPerQuarter = kReadWarps / 4;      // warps that share a tensor-memory lane quarter
 constexpr int kReadGroups = (kScanQ / 32 + kReadPerQuarter - 1) / kReadPerQuarter;   // most 32-column groups of one warp
 constexpr int kReadCols = 32 * kReadGroups;          // most query columns one read-out warp takes
@@ -392,8 +392,10 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 if (active && c0 < cw)
                 {
                     // (selected, not indexed: the array stays in registers)
-                    const float ta = c0 == 0 ? tmin[0] : tmin[kReadGroups > 2 ? 2 : 0];
-                    const float tb = c0 == 0 ? tmin[kReadGroups > 1 ? 1 : 0] : tmin[kReadGroups > 3 ? 3 : 0];
+                    constexpr int G = kReadGroups;
+                    const int rd = c0 >> 6;                                   // 64-column round
+                    const float ta = rd == 0 ? tmin[0] : (rd == 1 ? tmin[G > 2 ? 2 : 0] : (rd == 2 ? tmin[G > 4 ? 4 : 0] : tmin[G > 6 ? 6 : 0]));
+                    const float tb = rd == 0 ? tmin[G > 1 ? 1 : 0] : (rd == 1 ? tmin[G > 3 ? 3 : 0] : (rd == 2 ? tmin[G > 5 ? 5 : 0] : tmin[G > 7 ? 7 : 0]));
                     readout64<CAP>(v0, v1, c0 + 32 < cw, col_begin + c0, c0, hn, ta, tb, (int32_t)row, ctl.thr, wcnt,
                                    ctl.best[quarter], lists, need);
                 }
