@@ -144,6 +144,63 @@ int32_t prox_query_batch(prox_handle *h, const float *queries, int32_t B, int64_
 int32_t prox_query_batch_host(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
                               float *out_dists, uint8_t *out_hit, void *stream);
 
+/* ---- a corpus split by rows over several GPUs -------------------------------------------- */
+
+/*
+ * The database call of Algorithm 1 (line 6) over a corpus too large for one GPU; the paper
+ * has no counterpart of this split, it is an addition of this library.  GPU g of G holds the
+ * rows [row_offset, row_offset + N) of the corpus; the cache and the queries are replicated:
+ * every GPU runs the same lookup on the same queries, so the G caches stay equal without any
+ * exchange.  Only the miss path differs: each GPU finds the k nearest rows of ITS shard
+ * (prox_shard_scan), the G lists of every miss are brought to every GPU by the caller (one
+ * all-gather of prox_shard_exchange_bytes bytes per GPU, any transport), and each GPU merges
+ * them into the k nearest of the whole corpus (prox_shard_merge; ties by lower id, so all GPUs
+ * arrive at the same bytes).  Row ids everywhere are ids of the whole corpus.
+ *
+ * prox_create_shard -- as prox_create_metric with rho = 1, for one shard.
+ *   corpus      DEVICE, N x d fp32: the shard's rows, borrowed.
+ *   N           rows of this shard, k <= N.
+ *   row_offset  id of the shard's first row; row_offset + N <= n_total.
+ *   n_total     rows of the whole corpus, < 2^31.
+ * A shard handle answers through prox_shard_scan / prox_shard_merge; prox_query_batch and
+ * prox_query_batch_host reject it.  prox_probe_batch, prox_cache_load, prox_reset_cache and the
+ * diagnostics work as usual.
+ */
+prox_handle *prox_create_shard(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
+                               float tau, int32_t policy, int32_t metric, int64_t row_offset,
+                               int64_t n_total);
+
+/*
+ * prox_shard_exchange_bytes -- size of one GPU's exchange record for a batch of B queries:
+ * B * k fp64 distances followed by B * k int64 row ids (16 * B * k bytes), miss j of the batch
+ * (in index order) at entries j*k .. j*k+k-1; the entries of places beyond the batch's number
+ * of misses hold distance +inf and id -1.  0 if an argument is out of range.
+ */
+int64_t prox_shard_exchange_bytes(const prox_handle *h, int32_t B);
+
+/*
+ * prox_shard_scan -- first half of LOOKUP for a batch: probe, threshold test, replay of the
+ * batch (hit flags, evictions, slots), the answers of hits on stored keys, and the exact k
+ * nearest rows of this shard for every miss.
+ *   queries, B, out_ids, out_dists, out_hit, stream: as in prox_query_batch; after this call
+ *             out_hit is final, out_ids / out_dists are final for hits on stored keys only.
+ *   xchg      DEVICE, prox_shard_exchange_bytes(h, B) bytes, 16-byte aligned: this GPU's record.
+ * Asynchronous.  Must be followed by prox_shard_merge for the same batch before the next batch.
+ */
+int32_t prox_shard_scan(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
+                        float *out_dists, uint8_t *out_hit, void *xchg, void *stream);
+
+/*
+ * prox_shard_merge -- second half: merges the G records, writes the answers of the misses and
+ * of the hits on keys of this batch, and inserts the batch's new keys with their lists.
+ *   gathered  DEVICE, G records back to back (any order of shards; every shard exactly once).
+ *   G         number of shards, 1 <= G <= 32.
+ *   queries, B, out_ids, out_dists: the arguments of the prox_shard_scan call this completes.
+ * Asynchronous.
+ */
+int32_t prox_shard_merge(prox_handle *h, const float *queries, int32_t B, const void *gathered, int32_t G,
+                         int64_t *out_ids, float *out_dists, void *stream);
+
 /* prox_reset_cache -- C = {} (count and clock to zero); the corpus stays.  Asynchronous on stream. */
 int32_t prox_reset_cache(prox_handle *h, void *stream);
 

@@ -315,12 +315,11 @@ static void enqueue_probe_and_resolve(prox_handle *h, const float *queries, int3
     { StageScope t(h, PROX_STAGE_RESOLVE, s); launch_resolve(h, B, out_hit, s); }
 }
 
-extern "C" int32_t prox_query_batch(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
-                                    float *out_dists, uint8_t *out_hit, void *stream) {
-    int rc = check_batch_args(h, queries, B);
-    if (rc) return rc;
-    if (!out_ids || !out_dists || !out_hit) { set_err("an output pointer is NULL"); return PROX_ERR_INVALID_ARG; }
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
+// First half of a batch: probe and replay, answers of hits on stored keys, and for every miss
+// the exact k nearest rows of the corpus held here (res_ids / res_dists).  Returns the queries
+// the rest of the batch works on (unit-length copies for the cosine distance).
+static const float *enqueue_lookup_and_scan(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
+                                            float *out_dists, uint8_t *out_hit, cudaStream_t s) {
     if (h->metric == PROX_METRIC_COSINE) {                // unit-length copies stand in for the queries from here on
         launch_normalize_rows(queries, h->qn, B, h->d, s);
         h->launches++;
@@ -344,6 +343,13 @@ extern "C" int32_t prox_query_batch(prox_handle *h, const float *queries, int32_
     }
     { StageScope t(h, PROX_STAGE_RERANK, s); launch_rerank(h, queries, B, s); }
     { StageScope t(h, PROX_STAGE_EXACT_PASS, s); launch_fallback(h, queries, B, s); }
+    return queries;
+}
+
+// Second half: answers of the misses and of the hits on keys of this batch, insertion of the
+// batch's new keys with their lists (from res_ids / res_dists).
+static void enqueue_answers_and_inserts(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
+                                        float *out_dists, cudaStream_t s) {
     {
         StageScope t(h, PROX_STAGE_SCATTER, s);
         if (h->rho > 1) launch_hit_rerank(h, queries, B, 2, out_ids, out_dists, s);   // hits on keys of this batch
@@ -353,7 +359,73 @@ extern "C" int32_t prox_query_batch(prox_handle *h, const float *queries, int32_
         launch_scale(out_dists, (long long)B * h->k_out, 0.5f, s);
         h->launches++;
     }
+}
+
+extern "C" int32_t prox_query_batch(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
+                                    float *out_dists, uint8_t *out_hit, void *stream) {
+    int rc = check_batch_args(h, queries, B);
+    if (rc) return rc;
+    if (!out_ids || !out_dists || !out_hit) { set_err("an output pointer is NULL"); return PROX_ERR_INVALID_ARG; }
+    if (h->sharded) {
+        set_err("this handle holds one shard of a corpus: use prox_shard_scan and prox_shard_merge");
+        return PROX_ERR_INVALID_ARG;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    queries = enqueue_lookup_and_scan(h, queries, B, out_ids, out_dists, out_hit, s);
+    enqueue_answers_and_inserts(h, queries, B, out_ids, out_dists, s);
     return check_launch("prox_query_batch");
+}
+
+extern "C" prox_handle *prox_create_shard(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
+                                          float tau, int32_t policy, int32_t metric, int64_t row_offset,
+                                          int64_t n_total) {
+    g_err[0] = 0;
+    if (n_total < 1 || n_total >= (1LL << 31)) { set_err("n_total must be in [1, 2^31)"); return nullptr; }
+    if (row_offset < 0 || N < 1 || row_offset > n_total - N) {
+        set_err("the shard's rows [row_offset, row_offset + N) must lie within [0, n_total)");
+        return nullptr;
+    }
+    prox_handle *h = prox_create_metric(corpus, N, d, k, capacity, tau, policy, 1, metric);
+    if (!h) return nullptr;
+    h->sharded = 1; h->row_offset = row_offset; h->n_total = n_total;
+    return h;
+}
+
+extern "C" int64_t prox_shard_exchange_bytes(const prox_handle *h, int32_t B) {
+    if (!h || B < 1 || B > kMaxBatch) return 0;
+    return (int64_t)16 * B * h->k;
+}
+
+extern "C" int32_t prox_shard_scan(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
+                                   float *out_dists, uint8_t *out_hit, void *xchg, void *stream) {
+    int rc = check_batch_args(h, queries, B);
+    if (rc) return rc;
+    if (!out_ids || !out_dists || !out_hit || !xchg) { set_err("an output pointer is NULL"); return PROX_ERR_INVALID_ARG; }
+    if (!h->sharded) { set_err("not a shard handle (prox_create_shard)"); return PROX_ERR_INVALID_ARG; }
+    if (reinterpret_cast<uintptr_t>(xchg) % 16) { set_err("xchg must be 16-byte aligned"); return PROX_ERR_INVALID_ARG; }
+    if (h->shard_pending) { set_err("the previous prox_shard_scan was not completed by prox_shard_merge"); return PROX_ERR_INVALID_ARG; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    enqueue_lookup_and_scan(h, queries, B, out_ids, out_dists, out_hit, s);
+    { StageScope t(h, PROX_STAGE_SCATTER, s); launch_shard_pack(h, B, xchg, s); }
+    h->shard_pending = B;
+    return check_launch("prox_shard_scan");
+}
+
+extern "C" int32_t prox_shard_merge(prox_handle *h, const float *queries, int32_t B, const void *gathered, int32_t G,
+                                    int64_t *out_ids, float *out_dists, void *stream) {
+    int rc = check_batch_args(h, queries, B);
+    if (rc) return rc;
+    if (!out_ids || !out_dists || !gathered) { set_err("a pointer is NULL"); return PROX_ERR_INVALID_ARG; }
+    if (!h->sharded) { set_err("not a shard handle (prox_create_shard)"); return PROX_ERR_INVALID_ARG; }
+    if (G < 1 || G > 32) { set_err("G must be in [1, 32]"); return PROX_ERR_INVALID_ARG; }
+    if (reinterpret_cast<uintptr_t>(gathered) % 16) { set_err("gathered must be 16-byte aligned"); return PROX_ERR_INVALID_ARG; }
+    if (h->shard_pending != B) { set_err("no prox_shard_scan of %d queries is waiting for its merge", B); return PROX_ERR_INVALID_ARG; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (h->metric == PROX_METRIC_COSINE) queries = h->qn;  // the unit-length copies made by prox_shard_scan
+    { StageScope t(h, PROX_STAGE_MERGE, s); launch_shard_merge(h, B, gathered, G, s); }
+    enqueue_answers_and_inserts(h, queries, B, out_ids, out_dists, s);
+    h->shard_pending = 0;
+    return check_launch("prox_shard_merge");
 }
 
 extern "C" int32_t prox_query_batch_host(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
@@ -404,6 +476,7 @@ extern "C" int32_t prox_reset_cache(prox_handle *h, void *stream) {
     g_err[0] = 0;
     if (!h) { set_err("handle is NULL"); return PROX_ERR_INVALID_ARG; }
     launch_reset(h, static_cast<cudaStream_t>(stream));
+    h->shard_pending = 0;
     if (h->lsh_L >= 0) cudaMemsetAsync(h->bucket_count, 0, sizeof(int32_t) << h->lsh_L, static_cast<cudaStream_t>(stream));
     return check_launch("prox_reset_cache");
 }

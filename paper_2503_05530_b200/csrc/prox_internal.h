@@ -60,6 +60,11 @@ struct prox_handle {
     int32_t *lsh_order;       // kMaxBatch: batch queries sorted by (bucket, index)
     int32_t *lsh_seg;         // kMaxBatch + 1: where each bucket's run starts in lsh_order
     int32_t *lsh_work;        // [0] number of runs, [1] evictions, [2] hits on keys of this batch
+    // a corpus split by rows over several GPUs (sharded = 0: the whole corpus is here)
+    int32_t sharded;
+    int64_t row_offset;       // id of this shard's first row
+    int64_t n_total;          // rows of the whole corpus
+    int32_t shard_pending;    // batch size of a prox_shard_scan that prox_shard_merge has not completed, else 0
     int64_t C;
     float tau;
     int32_t policy;
@@ -173,4 +178,7 @@ void free_scan_tc(prox_handle *h);
 void launch_merge_select(prox_handle *h, int pass, int B, int for_probe, cudaStream_t s);
 void launch_rerank(prox_handle *h, const float *q, int B, cudaStream_t s);
 void launch_fallback(prox_handle *h, const float *q, int B, cudaStream_t s);
+// row shards
+void launch_shard_pack(prox_handle *h, int B, void *xchg, cudaStream_t s);       // this shard's exchange record
+void launch_shard_merge(prox_handle *h, int B, const void *gathered, int G, cudaStream_t s);   // G records -> res_ids / res_dists
 }  // namespace prox

@@ -61,6 +61,14 @@ def load_library():
     L.prox_create_lsh.argtypes = [vp, i64, i32, i32, i32, i32, vp, f32, i32, i32]
     L.prox_query_batch.restype = i32
     L.prox_query_batch.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    L.prox_create_shard.restype = vp
+    L.prox_create_shard.argtypes = [vp, i64, i32, i32, i64, f32, i32, i32, i64, i64]
+    L.prox_shard_exchange_bytes.restype = i64
+    L.prox_shard_exchange_bytes.argtypes = [vp, i32]
+    L.prox_shard_scan.restype = i32
+    L.prox_shard_scan.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]
+    L.prox_shard_merge.restype = i32
+    L.prox_shard_merge.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp]
     L.prox_query_batch_host.restype = i32
     L.prox_query_batch_host.argtypes = [vp, vp, i32, vp, vp, vp, vp]
     L.prox_reset_cache.restype = i32
@@ -243,3 +251,83 @@ class Prox:
         n = (C.c_int64 * len(STAGES))()
         _check(self._lib.prox_profile_read(self._h, ms, n, _stream_ptr(stream)))
         return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(STAGES)}
+
+
+def shard_rows(n_total: int, n_shards: int, shard: int) -> tuple[int, int]:
+    """Rows [first, first + count) of shard `shard` when n_total rows are dealt to n_shards GPUs in
+    contiguous runs whose lengths differ by at most one (the longer runs first)."""
+    if not (0 <= shard < n_shards):
+        raise ProxError("shard index out of range")
+    base, extra = divmod(int(n_total), int(n_shards))
+    first = shard * base + min(shard, extra)
+    return first, base + (1 if shard < extra else 0)
+
+
+def all_gather_records(record: torch.Tensor, group=None) -> torch.Tensor:
+    """The one exchange step of a row-sharded lookup: every rank contributes its exchange record
+    (a 1-d uint8 tensor of equal length on every rank) and receives all of them back to back, in
+    rank order.  Without an initialised process group (or with a group of one) the record is its
+    own gathering."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:
+        return record
+    G = dist.get_world_size(group)
+    out = torch.empty(G * record.numel(), dtype=record.dtype, device=record.device)
+    dist.all_gather_into_tensor(out, record, group=group)
+    return out
+
+
+class ProxShard(Prox):
+    """One row shard of a corpus split over several GPUs (prox_create_shard / prox_shard_scan /
+    prox_shard_merge).  Every rank holds the rows shard_rows(n_total, G, rank) and calls
+    query_batch with the same queries; the cache is replicated and needs no exchange."""
+
+    def __init__(self, corpus_shard: torch.Tensor, row_offset: int, n_total: int, k: int, capacity: int, tau: float,
+                 policy="lru", metric="l2", group=None):
+        self._lib = load_library()
+        self._corpus = _dev_f32(corpus_shard, "corpus_shard")
+        self.N, self.d = corpus_shard.shape
+        self.k, self.capacity, self.tau = int(k), int(capacity), float(tau)
+        self.policy, self.rho, self.metric = _POLICY[policy], 1, _METRIC[metric]
+        self.row_offset, self.n_total, self.group = int(row_offset), int(n_total), group
+        with torch.cuda.device(corpus_shard.device):
+            self._h = self._lib.prox_create_shard(corpus_shard.data_ptr(), self.N, self.d, self.k, self.capacity,
+                                                  self.tau, self.policy, self.metric, self.row_offset, self.n_total)
+        if not self._h:
+            raise ProxError(f"prox_create_shard failed: {last_error()}")
+        self.device = corpus_shard.device
+
+    def exchange_bytes(self, B: int) -> int:
+        return int(self._lib.prox_shard_exchange_bytes(self._h, B))
+
+    def shard_scan(self, queries: torch.Tensor, out_ids, out_dists, out_hit, record: torch.Tensor, stream=None):
+        q = _dev_f32(queries, "queries")
+        if q.shape[1] != self.d or record.numel() * record.element_size() < self.exchange_bytes(q.shape[0]):
+            raise ProxError("queries have the wrong dimension or the record is too small")
+        _check(self._lib.prox_shard_scan(self._h, q.data_ptr(), q.shape[0], out_ids.data_ptr(), out_dists.data_ptr(),
+                                         out_hit.data_ptr(), record.data_ptr(), _stream_ptr(stream)))
+
+    def shard_merge(self, queries: torch.Tensor, gathered: torch.Tensor, n_shards: int, out_ids, out_dists, stream=None):
+        B = queries.shape[0]
+        if gathered.numel() * gathered.element_size() < n_shards * self.exchange_bytes(B):
+            raise ProxError("gathered holds fewer than n_shards records")
+        _check(self._lib.prox_shard_merge(self._h, queries.data_ptr(), B, gathered.data_ptr(), int(n_shards),
+                                          out_ids.data_ptr(), out_dists.data_ptr(), _stream_ptr(stream)))
+
+    def query_batch(self, queries: torch.Tensor, out_ids=None, out_dists=None, out_hit=None, stream=None):
+        """Scan of this shard, all-gather of the records over the process group, merge."""
+        B = queries.shape[0]
+        if out_ids is None:
+            out_ids = torch.empty(B, self.k, dtype=torch.int64, device=self.device)
+        if out_dists is None:
+            out_dists = torch.empty(B, self.k, dtype=torch.float32, device=self.device)
+        if out_hit is None:
+            out_hit = torch.empty(B, dtype=torch.uint8, device=self.device)
+        record = torch.empty(self.exchange_bytes(B), dtype=torch.uint8, device=self.device)
+        self.shard_scan(queries, out_ids, out_dists, out_hit, record, stream)
+        gathered = all_gather_records(record, self.group)
+        self.shard_merge(queries, gathered, gathered.numel() // record.numel(), out_ids, out_dists, stream)
+        return out_ids, out_dists, out_hit
+
+    def query_batch_host(self, *a, **kw):
+        raise ProxError("a shard handle takes device tensors (query_batch)")
