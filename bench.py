@@ -202,7 +202,8 @@ def run_ours(args):
                          name=cfg.name + "-cut", n_components=max(1, cfg.n_components * (args.rows or cfg.N) // cfg.N),
                          n_topics=min(cfg.n_topics, (args.rows or cfg.N) // 4))
     peaks = load_peaks()
-    seed = stream_seed(args.seed, rank)
+    sharded = bool(args.shard_rows)                          # one corpus dealt to the ranks by rows, one query stream
+    seed = args.seed if sharded else stream_seed(args.seed, rank)
     K, Wm = args.steps, args.warmup
     n_batches_total = (cfg.n_queries + cfg.batch - 1) // cfg.batch
     if K <= 0:
@@ -210,8 +211,19 @@ def run_ours(args):
     nq = min(cfg.n_queries, (K + Wm) * cfg.batch)
 
     t_gen = time.time()
-    corpus = W.make_corpus(cfg.N, cfg.d, cfg.n_components, args.seed, dev)     # the index is the same on every rank
-    queries, _, _ = W.make_query_stream(corpus, max(nq, cfg.batch), cfg.n_topics, cfg.zipf_s, cfg.sigma, seed)
+    n_total = cfg.N
+    if sharded:
+        if args.rho != 1 or args.lsh_bits >= 0:
+            raise SystemExit("--shard-rows goes with the flat cache and rho = 1")
+        first, count = prox.shard_rows(n_total, world, rank)
+        topic_rows = W.pick_topics(n_total, cfg.n_topics, seed, dev)
+        corpus, topic_data = W.make_corpus_shard(n_total, cfg.d, cfg.n_components, args.seed, dev, first, count, topic_rows)
+        queries = W.make_query_stream_from_topics(topic_data, max(nq, cfg.batch), cfg.zipf_s, cfg.sigma, seed)
+        cfg = cfg.scaled(N=count)                              # what this rank scans
+        del topic_data
+    else:
+        corpus = W.make_corpus(cfg.N, cfg.d, cfg.n_components, args.seed, dev)     # the index is the same on every rank
+        queries, _, _ = W.make_query_stream(corpus, max(nq, cfg.batch), cfg.n_topics, cfg.zipf_s, cfg.sigma, seed)
     torch.cuda.synchronize()
     t_gen = time.time() - t_gen
 
@@ -221,7 +233,9 @@ def run_ours(args):
     results = {}
     handle_args = None
     for tau in taus:
-        if args.lsh_bits >= 0:                                 # PROXIMITY-LSH: 2^L buckets of b entries
+        if sharded:
+            p = prox.ProxShard(corpus, first, n_total, k, cfg.capacity, tau, cfg.policy, metric=args.metric)
+        elif args.lsh_bits >= 0:                               # PROXIMITY-LSH: 2^L buckets of b entries
             planes = torch.randn(args.lsh_bits, cfg.d, device=dev, generator=torch.Generator(device=dev).manual_seed(args.seed + 77))
             p = prox.Prox(corpus, k, (1 << args.lsh_bits) * args.lsh_bucket, tau, cfg.policy, rho=args.rho,
                           lsh_planes=planes, lsh_bucket=args.lsh_bucket)
@@ -282,11 +296,13 @@ def run_ours(args):
     head = results[head_tau]
     ms, total_q = aggregate_over_ranks(head["ms"], K * cfg.batch, dist, dev)
     ms_e2e, _ = aggregate_over_ranks(head["ms_e2e"], K * cfg.batch, dist, dev)
+    if sharded:
+        total_q = K * cfg.batch                              # every rank answered the same queries
     value = total_q / (ms * 1e-3)
     e2e = total_q / (ms_e2e * 1e-3)
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not sharded:
         cpu = cpu_baseline(cfg, corpus, queries, head_tau, budget_s=args.cpu_seconds)
     if rank != 0:
         if dist:
@@ -311,12 +327,12 @@ def run_ours(args):
                           unresolved=r["stats"]["unresolved"]))
     line = dict(
         metric=METRIC, value=round(value, 1), unit=UNIT, n_gpus=world, steps=K, warmup=Wm,
-        ms_per_step=round(ms / K, 4), higher_is_better=True, scaling="weak", vs_baseline=None,
+        ms_per_step=round(ms / K, 4), higher_is_better=True, scaling="strong" if sharded else "weak", vs_baseline=None,
         dtype="bf16 scan + f64 rerank/probe", data="synthetic",
-        config=dict(workload=f"{cfg.name}: N={cfg.N} d={cfg.d} k={cfg.k} capacity={cfg.capacity} policy={cfg.policy} "
+        config=dict(workload=f"{cfg.name}: N={n_total} d={cfg.d} k={cfg.k} capacity={cfg.capacity} policy={cfg.policy} "
                              f"batch={cfg.batch} tau={head_tau} topics={cfg.n_topics} zipf={cfg.zipf_s} sigma={cfg.sigma}",
                     tau=head_tau, hit_rate=round(head["hit_rate"], 4), l2="inputs_exceed_l2" if cfg.N * cfg.d * 2 > 126e6 else "corpus_fits_l2",
-                    parallelism=f"replica x{world}", rho=args.rho, metric=args.metric,
+                    parallelism=f"row shards x{world} ({cfg.N} rows each), cache replicated" if sharded else f"replica x{world}", rho=args.rho, metric=args.metric,
                     cache="flat" if args.lsh_bits < 0 else f"lsh L={args.lsh_bits} b={args.lsh_bucket}", seed=args.seed, gen_seconds=round(t_gen, 1)),
         clocks=head["clocks"],
         e2e=dict(value=round(e2e, 1), unit=UNIT, h2d_bytes_per_step=head["h2d"], d2h_bytes_per_step=head["d2h"]),
@@ -518,6 +534,8 @@ def main():
     ap.add_argument("--metric", default="l2", choices=["l2", "cosine"], help="distance of the cache keys and of the corpus")
     ap.add_argument("--lsh-bits", type=int, default=-1, help="PROXIMITY-LSH with this many hyperplanes (-1: flat cache)")
     ap.add_argument("--lsh-bucket", type=int, default=20, help="entries per LSH bucket")
+    ap.add_argument("--shard-rows", action="store_true", help="deal the rows of ONE corpus to the ranks (every rank answers the same "
+                    "queries; one all-gather per batch) instead of running independent replicas")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--default-steps", type=int, default=800, help="cap of the timed batches when --steps is 0 (a whole query stream if it is shorter)")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)

@@ -329,5 +329,26 @@ class ProxShard(Prox):
         self.shard_merge(queries, gathered, gathered.numel() // record.numel(), out_ids, out_dists, stream)
         return out_ids, out_dists, out_hit
 
-    def query_batch_host(self, *a, **kw):
-        raise ProxError("a shard handle takes device tensors (query_batch)")
+    def query_batch_host(self, queries: torch.Tensor, out_ids: torch.Tensor, out_dists: torch.Tensor,
+                         out_hit: torch.Tensor, stream=None):
+        """Host tensors in and out (pinned for speed): copies on the current stream around
+        query_batch, then synchronises.  Every rank passes the same queries."""
+        B = queries.shape[0]
+        for t in (queries, out_ids, out_dists, out_hit):
+            if t.is_cuda or not t.is_contiguous():
+                raise ProxError("query_batch_host takes contiguous host tensors")
+        if getattr(self, "_stage", None) is None:
+            MB = MAX_BATCH
+            self._stage = (torch.empty(MB, self.d, dtype=torch.float32, device=self.device),
+                           torch.empty(MB, self.k, dtype=torch.int64, device=self.device),
+                           torch.empty(MB, self.k, dtype=torch.float32, device=self.device),
+                           torch.empty(MB, dtype=torch.uint8, device=self.device))
+        q, ids, dists, hit = (t[:B] for t in self._stage)
+        with torch.cuda.stream(stream if stream is not None else torch.cuda.current_stream()):
+            q.copy_(queries, non_blocking=True)
+            self.query_batch(q, ids, dists, hit)
+            out_ids.copy_(ids, non_blocking=True)
+            out_dists.copy_(dists, non_blocking=True)
+            out_hit.copy_(hit, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+        return out_ids, out_dists, out_hit

@@ -70,6 +70,34 @@ def make_corpus(N: int, d: int, n_components: int, seed: int = 0, device="cpu",
     return mixture_rows(N, centres, seed, chunk_rows=chunk_rows)
 
 
+def make_corpus_shard(N: int, d: int, n_components: int, seed: int, device, first: int, count: int,
+                      keep_rows: torch.Tensor | None = None, chunk_rows: int = 1 << 18):
+    """Rows [first, first + count) of make_corpus(N, ...) without holding the whole corpus: every
+    chunk is drawn as make_corpus draws it, the shard's part is kept.  With keep_rows (int64 row
+    ids of the whole corpus) the second result holds those rows too (the topics of a query
+    stream may live in any shard)."""
+    centres = mixture_centres(n_components, d, seed, device)
+    shard = torch.empty(count, d, device=device, dtype=torch.float32)
+    kept = None if keep_rows is None else torch.empty(keep_rows.numel(), d, device=device, dtype=torch.float32)
+    for ci, r0 in enumerate(range(0, N, chunk_rows)):
+        r1 = min(N, r0 + chunk_rows)
+        a, b = max(r0, first), min(r1, first + count)
+        sel = None
+        if keep_rows is not None:
+            sel = torch.nonzero((keep_rows >= r0) & (keep_rows < r1)).flatten()
+        if a >= b and (sel is None or sel.numel() == 0):
+            continue
+        g = _gen(device, seed, _STREAM_CORPUS, ci)
+        comp = torch.randint(0, centres.shape[0], (r1 - r0,), generator=g, device=device)
+        x = torch.randn(r1 - r0, d, generator=g, device=device, dtype=torch.float32)
+        x = _normalize_(x.mul_(0.3).add_(centres[comp]))
+        if a < b:
+            shard[a - first:b - first] = x[a - r0:b - r0]
+        if sel is not None and sel.numel():
+            kept[sel] = x[keep_rows[sel] - r0]
+    return shard, kept
+
+
 def pick_topics(N: int, T: int, seed: int = 0, device="cpu") -> torch.Tensor:
     """T distinct row indices (int64), in the order that defines the Zipf ranks."""
     assert T <= N
@@ -117,6 +145,14 @@ def make_query_stream(corpus: torch.Tensor, n_queries: int, n_topics: int, zipf_
     ranks = zipf_ranks(n_topics, zipf_s, n_queries, seed, device)
     q = noisy_copies(corpus[topic_rows[ranks]], sigma, seed)
     return q, ranks, topic_rows
+
+
+def make_query_stream_from_topics(topic_data: torch.Tensor, n_queries: int, zipf_s: float, sigma: float,
+                                  seed: int = 0) -> torch.Tensor:
+    """The queries of make_query_stream when only the topics' rows are at hand: topic_data =
+    corpus[pick_topics(N, T, seed)]."""
+    ranks = zipf_ranks(topic_data.shape[0], zipf_s, n_queries, seed, topic_data.device)
+    return noisy_copies(topic_data[ranks], sigma, seed)
 
 
 def make_probe_keys(C: int, d: int, n_components: int, seed: int = 0, device="cpu"):

@@ -94,3 +94,15 @@ def test_all_gather_without_a_process_group_is_the_record_itself():
     from paper_2503_05530_b200 import prox
     r = torch.arange(32, dtype=torch.uint8)
     assert prox.all_gather_records(r) is r
+
+
+def test_shard_generator_draws_the_rows_of_the_whole_corpus():
+    from paper_2503_05530_b200 import prox, workloads as W
+    N, d = 1003, 16
+    X = W.make_corpus(N, d, 8, 3, "cpu", chunk_rows=100)
+    Q, _, rows = W.make_query_stream(X, 60, 25, 1.0, 0.05, 3)
+    for g in range(3):
+        first, cnt = prox.shard_rows(N, 3, g)
+        shard, kept = W.make_corpus_shard(N, d, 8, 3, "cpu", first, cnt, rows, chunk_rows=100)
+        assert torch.equal(shard, X[first:first + cnt]) and torch.equal(kept, X[rows])
+        assert torch.equal(W.make_query_stream_from_topics(kept, 60, 1.0, 0.05, 3), Q)
