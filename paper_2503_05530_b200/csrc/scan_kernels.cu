@@ -239,7 +239,7 @@ struct MergeSrc {
     }
 };
 
-__global__ void __launch_bounds__(1024)
+__global__ void __launch_bounds__(1024, 2)
 merge_select_kernel(const int *__restrict__ n_active, int pass, int n_lists, int stride, int kp, int stage_cap,
                     const u64 *__restrict__ buf, const int32_t *__restrict__ buf_cnt,
                     const uint32_t *__restrict__ thr_g, int32_t *cand_id, float *cand_score, int32_t *cand_n,
@@ -256,26 +256,43 @@ merge_select_kernel(const int *__restrict__ n_active, int pass, int n_lists, int
     if (tid == 0) { s_total = 0; s_gt = 0; s_eq = 0; }
     __syncthreads();
     const uint32_t g0 = thr_g[m];
-    // warp w takes the lists w, w + 32, ...: their counts come in with one load per 32 lists
+    // warp w takes the lists w, w + 32, ...: their counts come in with one load per 32 lists.  The
+    // entries are few per list and scattered over many lists, so the staging is bound by load
+    // latency: two lists at a time, up to 64 entries of each in flight per round (two blocks of 1024
+    // threads share an SM, which leaves 32 registers a thread).
     for (int p0 = warp; p0 < n_lists; p0 += 32 * 32) {
         int my_c = 0;
         if (p0 + 32 * lane < n_lists) {
             my_c = buf_cnt[(size_t)(p0 + 32 * lane) * kScanQ + q];
             if (my_c > stride) my_c = stride;
         }
-        for (int i = 0; i < 32 && p0 + 32 * i < n_lists; ++i) {
-            const int p = p0 + 32 * i;
-            const int c = __shfl_sync(0xffffffffu, my_c, i);
-            const u64 *list = buf + ((size_t)p * kScanQ + q) * stride;
-            for (int e0 = 0; e0 < c; e0 += 32) {
-                const u64 ent = (e0 + lane < c) ? list[e0 + lane] : 0ull;
-                const bool keep = ent != 0ull && (uint32_t)(ent >> 32) >= g0;
-                const unsigned mask = __ballot_sync(0xffffffffu, keep);
-                if (mask == 0u) continue;
-                int base = 0;
-                if (lane == 0) base = atomicAdd(&s_total, __popc(mask));
-                base = __shfl_sync(0xffffffffu, base, 0) + __popc(mask & ((1u << lane) - 1u));
-                if (keep && base < stage_cap) stage[base] = ent;
+        for (int i = 0; i < 32 && p0 + 32 * i < n_lists; i += 2) {
+            const int ca = __shfl_sync(0xffffffffu, my_c, i);
+            const int cb = __shfl_sync(0xffffffffu, my_c, (i + 1) & 31);
+            const bool two = i + 1 < 32 && p0 + 32 * (i + 1) < n_lists;
+            const int c0 = ca, c1 = two ? cb : 0;
+            const u64 *list0 = buf + ((size_t)(p0 + 32 * i) * kScanQ + q) * stride;
+            const u64 *list1 = list0 + (size_t)32 * kScanQ * stride;          // list p + 32 (read only when two)
+            const int cmax = c0 > c1 ? c0 : c1;
+            for (int e0 = 0; e0 < cmax; e0 += 64) {
+                u64 ent[4];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int idx = e0 + 32 * u + lane;
+                    ent[u] = idx < c0 ? list0[idx] : 0ull;
+                    ent[2 + u] = idx < c1 ? list1[idx] : 0ull;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (e0 + 32 * (u & 1) >= (u < 2 ? c0 : c1)) continue;      // warp-uniform: nothing was loaded
+                    const bool keep = ent[u] != 0ull && (uint32_t)(ent[u] >> 32) >= g0;
+                    const unsigned mask = __ballot_sync(0xffffffffu, keep);
+                    if (mask == 0u) continue;
+                    int base = 0;
+                    if (lane == 0) base = atomicAdd(&s_total, __popc(mask));
+                    base = __shfl_sync(0xffffffffu, base, 0) + __popc(mask & ((1u << lane) - 1u));
+                    if (keep && base < stage_cap) stage[base] = ent[u];
+                }
             }
         }
     }

@@ -39,6 +39,34 @@ __device__ __forceinline__ void append32(const uint32_t (&v)[32], int c0, int lc
         pass |= (__uint_as_float(v[4 * j4 + 3]) - t4.w > hn) ? (8u << (4 * j4)) : 0u;
     }
     bool full = false;
+    // While the thresholds are still open (the first tiles of a launch) every row of the quarter
+    // passes the same columns.  Then the 32 rows of a column go to 32 consecutive places of its
+    // list with one store, the count moves once and the best score is one warp reduction: no
+    // per-entry atomics, no register selection, and nothing that orders one column after another.
+    const uint32_t pass0 = __shfl_sync(0xffffffffu, pass, 0);
+    if (__all_sync(0xffffffffu, pass == pass0) && __popc(pass0) >= 8) {
+        const int lane = threadIdx.x & 31;
+        const bool mine = (pass0 >> lane) & 1u;                   // lane l keeps the books of column l of the group
+        const int base_mine = wcnt[lc0 + lane];
+        uint32_t top_mine = 0u;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            if ((pass0 >> j) & 1u) {                             // warp-uniform
+                const u64 ent = pack_entry(__uint_as_float(v[j]) - hn, row);
+                const uint32_t top = __reduce_max_sync(0xffffffffu, (uint32_t)(ent >> 32));
+                if (lane == j) top_mine = top;
+                const int base = __shfl_sync(0xffffffffu, base_mine, j);
+                if (base + lane < CAP) lists[(size_t)(c0 + j) * CAP + base + lane] = ent;
+            }
+        }
+        if (mine) {                                              // the warp's columns are its own: plain updates
+            wcnt[lc0 + lane] = base_mine + 32;
+            if (top_mine > best[c0 + lane]) best[c0 + lane] = top_mine;
+        }
+        __syncwarp();
+        if (__any_sync(0xffffffffu, mine && base_mine + 32 > CAP - 33)) need = true;
+        return;
+    }
 #pragma unroll 1
     while (pass) {
         const int j = __ffs(pass) - 1;

@@ -73,6 +73,7 @@ struct Control {
     uint32_t tmem_base;
     int abort_flag;                  // set by any thread whose wait ran out
     int done;                        // read-out warps that have finished (the bound warp stops at kReadWarps)
+    int first_pub;                   // read-out warps that have published the bests of their first tile
     long long t_begin, t_end;        // row tiles of this pair (or block)
 };
 
@@ -142,6 +143,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         mbar_init(smem_u32(&ctl.q_full), 1);
         ctl.abort_flag = 0;
         ctl.done = 0;
+        ctl.first_pub = 0;
         // Row tiles are dealt out in contiguous runs whose lengths follow the speeds that the
         // previous launch measured (SMs differ by their place on the die: up to a quarter in
         // tiles per second), so that all pairs end together.  Every block adds the same numbers
@@ -274,6 +276,13 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         if (a.kp <= P && P <= 1024) {
             volatile int *done = &ctl.done;
             int jq = blockIdx.x, jobs = 0;
+            // The first bounds are worth the most (until they arrive every row passes), and there is
+            // nothing to select from before the first tile has been read out: the blocks start in
+            // step, so this block's own first publication tells when the others' are due.
+            {
+                volatile int *first_pub = &ctl.first_pub;
+                while (*first_pub < kReadWarps && *done < kReadWarps && !*abort_flag) __nanosleep(200);
+            }
             while (*done < kReadWarps && !*abort_flag) {
                 if (jq >= nq) jq = blockIdx.x;
                 if (jq < nq) {
@@ -284,9 +293,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                         t[i8] = (eidx < P) ? __ldcg(&top1[(size_t)jq * P + eidx]) : 0u;
                     }
                     // the k'-th largest of them, bit by bit: the largest value that at least k' reach
+                    // (the first rounds stop at 16 bits: a bound 2^-7 below the exact one, in half the time)
                     uint32_t rth = 0u;
+                    const int low_bit = jobs < 6 ? 16 : 0;
 #pragma unroll 1
-                    for (int bit = 31; bit >= 0; --bit) {
+                    for (int bit = 31; bit >= low_bit; --bit) {
                         const uint32_t cand = rth | (1u << bit);
                         int n_ge = 0;
 #pragma unroll
@@ -301,7 +312,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 // shares an issue port with read-out warps, so it backs off once they have settled
                 // (in short naps, so that the block does not outlive its read-out by a long one)
                 const int naps = ++jobs < 48 ? 1 : 10;
-                for (int n = 0; n < naps && *done < kReadWarps; ++n) __nanosleep(2000);
+                if (jobs < 6) __nanosleep(300);                 // the first rounds follow one another closely
+                else
+                    for (int n = 0; n < naps && *done < kReadWarps; ++n) __nanosleep(2000);
             }
         }
     } else if (warp >= 4) {
@@ -434,6 +447,10 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                             published[i] = bq;
                         }
                     }
+                }
+                if (it == 0) {
+                    __syncwarp();
+                    if (lane == 0) atomicAdd(&ctl.first_pub, 1);
                 }
             }
             if (need) {                                           // warp-uniform
