@@ -241,14 +241,20 @@ risk_finish_kernel(DevState *st, RiskWork *w, int32_t *risk_pos, int32_t *risk_s
 // ------------------------------------------------------------------------------------------
 // Probe: squared distances, in fp64 over the fp32 values and in difference form (so that a
 // bitwise duplicate is at distance exactly 0), from each query to every valid key and to
-// every earlier query of the batch.  Tile: 32 queries x 64 columns per block, d in chunks of 32.
+// every earlier query of the batch.  Tile: 32 queries x 64 (or 32) columns per block, d in chunks of 32 (or 64).
 //   mode 0  columns = slots [0, count) then the batch [count, count + B): everything in fp64.
 //   mode 1  columns = the R at-risk slots then the batch: what the resolve needs as full rows
 //           when the safe slots are handled by the coarse tensor-core probe.
 //   mode 2  queries = those the coarse probe could not certify (pfail_list), columns = slots.
 // ------------------------------------------------------------------------------------------
-constexpr int PQ = 32, PC = 64, PD = 32;
+constexpr int PQ = 32;
+constexpr int kProbeColsWide = 64, kProbeColsNarrow = 32;
 
+// PC = columns per block tile, PD = dimensions per step: 64 x 32, or 32 x 64 for a small cache,
+// where the wide tiles leave most SMs without a block and the time goes into the chain of steps
+// (a barrier and a load latency each): narrower tiles give twice the blocks, deeper steps half
+// the chain with twice the loads in flight.
+template <int PC, int PD>
 __global__ void __launch_bounds__(256)
 probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
              const float *__restrict__ queries, const int32_t *__restrict__ risk_pos, int B, int d,
@@ -280,11 +286,11 @@ probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
 
     for (long long t = t_begin; t < t_end; ++t) {
         const long long c0 = t * PC;
-        double acc[2][4];
+        double acc[2][PC / 16];
 #pragma unroll
         for (int a = 0; a < 2; ++a)
 #pragma unroll
-            for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+            for (int b = 0; b < PC / 16; ++b) acc[a][b] = 0.0;
 
         // operands of the next 32 dimensions are fetched into registers while the current ones are
         // multiplied: small problems (few blocks per SM) are bound by this latency, not by the fp64 rate
@@ -339,7 +345,7 @@ probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
             for (int j = 0; j < PD; ++j) {
                 const double qa = qs[ty * 2][j], qb2 = qs[ty * 2 + 1][j];
 #pragma unroll
-                for (int b = 0; b < 4; ++b) {
+                for (int b = 0; b < PC / 16; ++b) {
                     const double kv = ks[tx + 16 * b][j];
                     const double d0 = qa - kv, d1 = qb2 - kv;
                     acc[0][b] = fma(d0, d0, acc[0][b]);
@@ -352,7 +358,7 @@ probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
             const int i = q_index[ty * 2 + a];
             if (i < 0) continue;
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
+            for (int b = 0; b < PC / 16; ++b) {
                 const long long col = c0 + tx + 16 * b;
                 if (col >= ncols) continue;
                 const double v = acc[a][b];
@@ -894,7 +900,15 @@ __global__ void cache_load_kernel(long long n, int d, int k, const float *__rest
 // ------------------------------------------------------------------------------------------
 // Launchers
 // ------------------------------------------------------------------------------------------
+// Columns per tile of the fp64 probe: narrow tiles when wide ones would not give every SM two blocks.
+static int probe_cols(const prox_handle *h, int B) {
+    const long long wide = (h->C + B + kProbeColsWide - 1) / kProbeColsWide;
+    const int qtiles = (B + PQ - 1) / PQ;
+    return wide * qtiles < 2LL * h->num_sms ? kProbeColsNarrow : kProbeColsWide;
+}
+
 static int probe_splits(const prox_handle *h, int B) {
+    const int PC = probe_cols(h, B);
     const long long ntiles = (h->C + B + PC - 1) / PC;
     const int qtiles = (B + PQ - 1) / PQ;
     long long want = (4LL * h->num_sms + qtiles - 1) / qtiles;     // about four blocks per SM
@@ -956,13 +970,18 @@ void launch_risk_select(prox_handle *h, int B, cudaStream_t s) {
 
 void launch_probe(prox_handle *h, const float *q, int B, int mode, cudaStream_t s) {
     int splits = probe_splits(h, B);
+    const int PC = probe_cols(h, B);
     if (mode == 1) {                                      // at most 2 * kMaxBatch columns
         const int tiles = (2 * B + PC - 1) / PC;
         if (splits > tiles) splits = tiles;
     }
     dim3 grid((B + PQ - 1) / PQ, splits);
-    probe_kernel<<<grid, 256, 0, s>>>(h->st, h->keys, q, h->risk_pos, B, h->d, h->part_min, h->part_arg,
-                                      h->d_risk, h->d_intra, mode, h->risk_slot, h->pfail_list);
+    if (PC == kProbeColsNarrow)
+        probe_kernel<kProbeColsNarrow, 64><<<grid, 256, 0, s>>>(h->st, h->keys, q, h->risk_pos, B, h->d, h->part_min, h->part_arg,
+                                                            h->d_risk, h->d_intra, mode, h->risk_slot, h->pfail_list);
+    else
+        probe_kernel<kProbeColsWide, 32><<<grid, 256, 0, s>>>(h->st, h->keys, q, h->risk_pos, B, h->d, h->part_min, h->part_arg,
+                                                          h->d_risk, h->d_intra, mode, h->risk_slot, h->pfail_list);
     h->launches++;
 }
 
