@@ -113,10 +113,10 @@ def pick_workload(name: str, free_bytes: int) -> W.Config:
 
 
 # DRAM bytes per algorithmic byte of one scan launch, from one ncu capture of scan_tc_kernel on a 4 M x 768 cut
-# of the "large" workload (dram__bytes_read.sum + dram__bytes_write.sum = 7.80 GB against 6.16 GB); the extra
+# of the "large" workload (dram__bytes_read.sum + dram__bytes_write.sum = 7.78 GB against 6.16 GB); the extra
 # bytes grow with the row tiles like the algorithmic ones, so the ratio carries over to a full launch.
 # Valid for d = 768 and 256 misses per launch only; set to None when the kernel changes.
-SCAN_TRAFFIC_RATIO_D768_M256 = 1.266
+SCAN_TRAFFIC_RATIO_D768_M256 = 1.263
 
 
 def roofline_of_scan(cfg, mean_misses, scan_ms_per_launch, peaks, traffic=None):
