@@ -384,7 +384,7 @@ __device__ __forceinline__ double exact_sqdist_warp(const float *__restrict__ q_
 constexpr int kRerankMax = kCollectCap;            // entries the sort buffers hold
 
 // mode 0: candidates of the coarse scan (+ certificate); mode 1: rows collected by the exact pass
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 rerank_kernel(DevState *st, int mode, const float *__restrict__ corpus, const float *__restrict__ queries,
               int d, int k, long long N, const int32_t *__restrict__ miss_list,
               const int32_t *__restrict__ cand_id, const int32_t *__restrict__ cand_n,
@@ -422,7 +422,8 @@ rerank_kernel(DevState *st, int mode, const float *__restrict__ corpus, const fl
     while (n2 < n) n2 <<= 1;
     for (int e = tid; e < n2; e += blockDim.x) { sd[e] = INFINITY; sid[e] = 0x7fffffff; }
     __syncthreads();
-    for (int c = warp; c < n; c += 8) {
+    // one candidate row per warp at a time: the gathers are bound by latency, so the block is wide
+    for (int c = warp; c < n; c += (int)(blockDim.x >> 5)) {
         const int row = ids[c];
         const double v = exact_sqdist_warp(q_sm, corpus + (size_t)row * d, d);
         if (lane == 0) { sd[c] = v; sid[c] = row; }
@@ -817,7 +818,7 @@ void set_scan_kernel_attributes() {
 }
 
 void launch_rerank(prox_handle *h, const float *q, int B, cudaStream_t s) {
-    rerank_kernel<<<B, 256, rerank_smem(h->d), s>>>(h->st, 0, h->corpus, q, h->d, h->k, (long long)h->N,
+    rerank_kernel<<<B, 1024, rerank_smem(h->d), s>>>(h->st, 0, h->corpus, q, h->d, h->k, (long long)h->N,
                                                     h->miss_list, h->cand_id, h->cand_n, h->cand_sk, h->qbn,
                                                     h->qerr, h->res_ids, h->res_dists, h->fail_list,
                                                     h->fail_radius, h->coll_id, h->coll_n);
@@ -842,7 +843,7 @@ void launch_fallback(prox_handle *h, const float *q, int B, cudaStream_t s) {
         h->st, h->corpus, nullptr, h->redo, q, (long long)h->N, h->d, h->miss_list, h->fail_list, h->fail_radius,
         h->coll_id, h->coll_n);
     h->launches += 3;
-    rerank_kernel<<<B, 256, rerank_smem(h->d), s>>>(h->st, 1, h->corpus, q, h->d, h->k, (long long)h->N,
+    rerank_kernel<<<B, 1024, rerank_smem(h->d), s>>>(h->st, 1, h->corpus, q, h->d, h->k, (long long)h->N,
                                                     h->miss_list, h->cand_id, h->cand_n, h->cand_sk, h->qbn,
                                                     h->qerr, h->res_ids, h->res_dists, h->fail_list,
                                                     h->fail_radius, h->coll_id, h->coll_n);
