@@ -289,9 +289,9 @@ static void enqueue_probe_and_resolve(prox_handle *h, const float *queries, int3
     { StageScope t(h, PROX_STAGE_RISK_SELECT, s); launch_risk_select(h, B, s); }
     {
         StageScope t(h, PROX_STAGE_PROBE, s);
-        // the coarse pass has a fixed cost of a few launches: it pays off from about three million
+        // the coarse pass has a fixed cost of a few launches: it pays off from about two million
         // query-key pairs per batch on
-        bool coarse = h->probe_tc && h->scan_mode != PROX_SCAN_CUDA_CORE && (long long)B * h->C >= 3LL * (1 << 20);
+        bool coarse = h->probe_tc && h->scan_mode != PROX_SCAN_CUDA_CORE && (long long)B * h->C >= 2LL * (1 << 20);
         if (coarse) {
             // safe slots: coarse scores on the tensor cores, exact recheck of the best few;
             // at-risk slots and the batch itself: full fp64 rows; uncertified queries: fp64 over all slots
