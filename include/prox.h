@@ -64,7 +64,7 @@ enum {
  *   k        neighbours per query, 1 <= k <= min(N, PROX_MAX_K).
  *   capacity c of Section 3.3.1, >= 1 (c = 0 is rejected: Algorithm 1 would evict from an empty store).
  *   tau      tolerance of Section 3.3.3 on the squared distance, >= 0 and not NaN;
- *            a key matches when distance <= tau (Algorithm 1, line 4).
+ *            a key matches when distance <= tau (the threshold test of Algorithm 1).
  *   policy   PROX_LRU or PROX_FIFO.
  * Returns NULL on failure (see prox_last_error).  Allocates with cudaMalloc on
  * the current device and synchronises that device before returning.
@@ -84,9 +84,9 @@ prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t d, int32_t 
                              float tau, int32_t policy, int32_t rho);
 
 /*
- * prox_create_metric -- prox_create_rho with the distance named (Section 2.1: the distance is
- * "typically L2, cosine, or inner-product, fixed before deployment"; Section 3.1: the cache
- * uses the database's distance).  PROX_METRIC_COSINE: keys and corpus rows are compared by
+ * prox_create_metric -- prox_create_rho with the distance named (Section 2.2, Vector search: the
+ * distance function is chosen once, before deployment; Section 3.1: the cache uses the
+ * database's distance).  PROX_METRIC_COSINE: keys and corpus rows are compared by
  * 1 - cos(a, b), evaluated as half the squared Euclidean distance of a/|a| and b/|b| (identical
  * vectors, of any length, are at distance exactly 0); tau applies to that value and out_dists
  * hold it.  The library keeps its own unit-length fp32 copy of the corpus (N x d x 4 bytes
@@ -126,10 +126,10 @@ prox_handle *prox_create_lsh(const float *corpus, int64_t N, int32_t d, int32_t 
  *             are the distances stored with the key, i.e. those of the key's own query.
  *             (With rho > 1, see prox_create_rho: a hit returns the k stored rows nearest
  *             to this query with their distances to this query.)
- *   out_hit   DEVICE, B bytes: 1 = cache hit (Algorithm 1, line 5), 0 = miss (lines 6-10).
+ *   out_hit   DEVICE, B bytes: 1 = cache hit (the stored list is returned), 0 = miss (the database is asked and the result inserted).
  *   stream    a cudaStream_t (NULL = the default stream).
  * Misses are answered by an exact k-nearest-neighbour search over the whole corpus
- * (Algorithm 1, line 6, with a flat exact index as in Section 4.2.1).
+ * (the database call of Algorithm 1, with a flat exact index as in Section 4.2.1).
  * Asynchronous; no device-to-host copy and no synchronisation happens inside.
  * Errors found on the device are latched and reported by prox_status.
  */
@@ -147,7 +147,7 @@ int32_t prox_query_batch_host(prox_handle *h, const float *queries, int32_t B, i
 /* ---- a corpus split by rows over several GPUs -------------------------------------------- */
 
 /*
- * The database call of Algorithm 1 (line 6) over a corpus too large for one GPU; the paper
+ * The database call of Algorithm 1 over a corpus too large for one GPU; the paper
  * has no counterpart of this split, it is an addition of this library.  GPU g of G holds the
  * rows [row_offset, row_offset + N) of the corpus; the cache and the queries are replicated:
  * every GPU runs the same lookup on the same queries, so the G caches stay equal without any
@@ -216,12 +216,12 @@ const char *prox_last_error(void);
  * prox_cache_load -- fill slots 0..n-1 with the given keys (DEVICE, n x d fp32), stamps
  * 0..n-1 and empty value lists (ids -1, distances 0); count = clock = n.  Stands in for
  * n earlier misses when only the probe is measured (the lookup-time experiment of
- * Section 4.4.1).  n <= capacity.  Asynchronous on stream.
+ * Section 4.5.1, lookup times for increasing cache occupancies).  n <= capacity.  Asynchronous on stream.
  */
 int32_t prox_cache_load(prox_handle *h, const float *keys, int64_t n, void *stream);
 
 /*
- * prox_probe_batch -- lines 2-4 and 7-9 of Algorithm 1 only: probe, threshold test,
+ * prox_probe_batch -- Algorithm 1 without its database call: probe, threshold test,
  * LRU touch, eviction and insertion of the query as a key, with an empty value list in
  * place of the database call.
  *   out_hit      DEVICE, B bytes.
@@ -286,8 +286,7 @@ enum {
 
 /*
  * prox_nearest_key_static -- for every query the nearest of n_keys keys and its squared distance
- * (the argmin of Algorithm 1's lines 2-3; the paper has no counterpart of this entry point, it is
- * an addition of this library).  It is meant for callers that cannot allocate device memory at
+ * (the paper has no counterpart of this entry point, it is an addition of this library).  It is meant for callers that cannot allocate device memory at
  * the time of the call: code embedded in an application that owns all GPU memory and forbids
  * further allocations, code running with a fixed memory budget, a thread that must not touch the
  * allocator.  The call needs no handle, calls no cudaMalloc / cudaFree and no allocating library
@@ -300,7 +299,9 @@ enum {
  * Sizes beyond these limits are rejected with PROX_ERR_INVALID_ARG and a text in prox_last_error();
  * nothing is launched then.  Asynchronous on stream.
  * The first call on a GPU looks up the device address of the built-in array (once per GPU, with
- * that GPU current); make that first call outside any stream capture.
+ * that GPU current); make that first call outside any stream capture.  The address is kept for
+ * the life of the process: it does not survive a cudaDeviceReset of that GPU, after which this
+ * entry point must not be called again in the same process.
  * All calls on one GPU share the array, which keeps the last call's contents (the call clears the
  * counters it needs at zero itself): calls that could run at the same time on one GPU race with
  * each other, so order them on one stream.

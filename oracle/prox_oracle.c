@@ -14,7 +14,7 @@
  *     state it), the database call on a miss, eviction when |C| >= c, insert.
  *   - Section 3.3.2 (eviction policy): FIFO evicts the oldest inserted entry
  *     whatever its use; LRU evicts the entry unused for the longest time.
- *   - Section 2.1 / Section 3 (retrieveDocumentIndices): the database call is
+ *   - Section 2.2 (Vector search) / Section 3 (retrieveDocumentIndices): the database call is
  *     the exact k nearest rows of the corpus, returned as a list sorted by
  *     increasing distance (the FAISS-Flat case of Section 4.2.1).
  *
@@ -34,7 +34,7 @@
  *     measures the m stored rows against the CURRENT query and returns the k nearest (distance
  *     ascending, ties to the lower row id) with those distances.  rho = 1 is "no re-ranking"
  *     (Section 4): the stored list comes back as it is, as above;
- *   - metric (Section 2.1: "typically L2, cosine, or inner-product, fixed before deployment"):
+ *   - metric (Section 2.2, Vector search: the distance function is chosen once, before deployment):
  *     squared Euclidean by default; ORACLE_COSINE is the cosine distance 1 - cos(a, b), taken
  *     as half the squared Euclidean distance of a/|a| and b/|b| (the same number, and exactly 0
  *     for identical vectors so that tau = 0 stays exact matching); normalisation in fp64;
@@ -289,7 +289,7 @@ void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids,
     const int32_t d = o->d, k = o->k, m = o->m;
     const int64_t t = o->clock++;                 /* this query's time stamp */
 
-    /* lines 2-3 of Algorithm 1: all key distances, then the minimum (first minimum in slot order) */
+    /* Algorithm 1, the distances and their minimum: every valid key is measured, the first minimum in slot order wins */
     /* PROXIMITY-LSH: only the bucket that the hash names is looked at and updated */
     int64_t s_begin = 0, s_end = o->capacity, bucket = -1;
     if (o->lsh_L >= 0) {
@@ -308,11 +308,11 @@ void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids,
     }
     if (dtrace) { dtrace[0] = best; dtrace[1] = second; }
 
-    int hit = (best_slot >= 0 && best <= o->tau);  /* line 4: min_dist <= tau */
+    int hit = (best_slot >= 0 && best <= o->tau);  /* the threshold test of Algorithm 1, inclusive */
     if (force == 0) hit = 0;
     if (force == 1 && best_slot >= 0) hit = 1;
 
-    if (hit) {                                     /* line 5: return C[key] */
+    if (hit) {                                     /* hit: the value stored under the matched key */
         if (o->policy == ORACLE_LRU) o->stamp[best_slot] = t;   /* a hit is a use (LRU only) */
         const int64_t *sid = o->val_ids + best_slot * m;
         if (o->rho == 1 || !o->corpus) {           /* no re-ranking: the stored list, as it is */
@@ -344,13 +344,13 @@ void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids,
         return;
     }
 
-    /* line 6: I <- D.retrieveDocumentIndices(q) */
+    /* miss: the database is asked (retrieveDocumentIndices) */
     int64_t *ids = (int64_t *)malloc(sizeof(int64_t) * m);
     double *dists = (double *)malloc(sizeof(double) * m);
     if (o->corpus) oracle_exact_topk_metric(o->metric, o->corpus, o->N, d, q, m, o->scratch, ids, dists);   /* m = rho * k neighbours */
     else for (int32_t r = 0; r < m; ++r) { ids[r] = -1; dists[r] = 0.0; }
 
-    /* lines 7-8: if |C| >= c evict one entry (the smallest stamp; stamps are unique) */
+    /* a full cache (|C| >= c) gives up one entry first: the smallest stamp (stamps are unique) */
     int64_t slot, evicted = -1;
     const int64_t held = bucket >= 0 ? o->bucket_count[bucket] : o->count;      /* |C| of this (bucket's) cache */
     if (held >= s_end - s_begin) {
@@ -364,7 +364,7 @@ void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids,
         slot = s_begin + held;                     /* slots fill in index order */
     }
 
-    /* line 9: C[q] <- I */
+    /* the query becomes a key, the fetched list its value */
     memcpy(o->keys + slot * d, q, sizeof(float) * d);
     memcpy(o->val_ids + slot * m, ids, sizeof(int64_t) * m);
     memcpy(o->val_dists + slot * m, dists, sizeof(double) * m);
@@ -372,7 +372,7 @@ void oracle_lookup(oracle_t *o, const float *q, int32_t force, int64_t *out_ids,
     if (bucket >= 0) o->bucket_count[bucket]++;
     o->n_misses++;
 
-    /* line 10: return I (its k nearest when more were fetched) */
+    /* the fetched list is returned (its k nearest when more were fetched) */
     if (out_ids) memcpy(out_ids, ids, sizeof(int64_t) * k);
     if (out_dists) memcpy(out_dists, dists, sizeof(double) * k);
     if (trace) { trace[0] = 0; trace[1] = slot; trace[2] = t; trace[3] = evicted; }

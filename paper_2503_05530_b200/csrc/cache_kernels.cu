@@ -1,5 +1,5 @@
-// Cache-side kernels: the probe (lines 2-3 of Algorithm 1 for a whole batch), the
-// sequential-order resolve (lines 4-9), and the copies that read and write the value slots.
+// Cache-side kernels: the probe (the key distances and their minimum in Algorithm 1, for a whole batch), the
+// sequential-order resolve (threshold test, eviction, insertion), and the copies that read and write the value slots.
 //
 // How a batch is made to behave like B sequential lookups.  During one batch the only
 // pre-batch entries that can be evicted are the R = min(B, |C|) entries that come first in
@@ -396,7 +396,7 @@ probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
 
 // ------------------------------------------------------------------------------------------
 // Per query: reduce the partial safe minima; list the at-risk and in-batch keys within tau
-// (Algorithm 1, line 4, inclusive).  code < kMaxBatch: at-risk position; else kMaxBatch + j.
+// (the threshold test of Algorithm 1, inclusive).  code < kMaxBatch: at-risk position; else kMaxBatch + j.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(128)
 build_candidates_kernel(const DevState *__restrict__ st, int B, int S, double tau,
@@ -446,7 +446,7 @@ build_candidates_kernel(const DevState *__restrict__ st, int B, int S, double ta
 }
 
 // ------------------------------------------------------------------------------------------
-// Resolve: replay queries 0..B-1 in order (Algorithm 1, lines 4-9) on the candidate lists.
+// Resolve: replay queries 0..B-1 in order (Algorithm 1 from the threshold test to the insertion) on the candidate lists.
 // One block; warp 0 walks the batch, the other warps only help to load and store.
 // ------------------------------------------------------------------------------------------
 constexpr int kCsrCap = 8192;
@@ -752,7 +752,7 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
 // ------------------------------------------------------------------------------------------
 // Value-slot traffic.
 // ------------------------------------------------------------------------------------------
-// Hits on a key that was resident before the batch: copy its stored list (Algorithm 1, line 5).
+// Hits on a key that was resident before the batch: copy its stored list (the hit branch of Algorithm 1).
 // Runs before any slot is overwritten by this batch.
 __global__ void gather_hits_kernel(int B, int k, const int32_t *__restrict__ src,
                                    const int32_t *__restrict__ src_kind,
@@ -768,8 +768,8 @@ __global__ void gather_hits_kernel(int B, int k, const int32_t *__restrict__ src
     }
 }
 
-// Misses return their fresh list (line 10); hits on a key inserted earlier in the batch return
-// that query's list; entries that own a slot at batch end are written (line 9).
+// Misses return their fresh list (the end of Algorithm 1); hits on a key inserted earlier in the batch return
+// that query's list; entries that own a slot at batch end are written (the insertion of Algorithm 1).
 __global__ void scatter_kernel(int B, int d, int k, int k_out, int with_values, const float *__restrict__ queries,
                                const int32_t *__restrict__ src, const int32_t *__restrict__ src_kind,
                                const int32_t *__restrict__ ins_slot,

@@ -101,7 +101,7 @@ lsh_resolve_kernel(const DevState *st, int B, int d, int b, double tau, int poli
         const int i = order[r];
         const float *q = queries + (size_t)i * d;
         const int cnt = s_cnt;
-        // distances to the resident keys of the bucket (Algorithm 1, line 2), difference form in fp64
+        // distances to the resident keys of the bucket (Algorithm 1), difference form in fp64
         for (int s = warp; s < cnt; s += 8) {
             const float *key = keys + (size_t)(slot0 + s) * d;
             double acc = 0.0;
@@ -119,7 +119,7 @@ lsh_resolve_kernel(const DevState *st, int B, int d, int b, double tau, int poli
             for (int s = 0; s < cnt; ++s)
                 if (s_dist[s] < best) { best = s_dist[s]; bs = s; }          // the lowest slot wins a tie
             const u64 t = (u64)(clock0 + i);                                  // one stamp per query
-            if (bs >= 0 && best <= tau) {                                     // line 4
+            if (bs >= 0 && best <= tau) {                                     // threshold test
                 out_hit[i] = 1;
                 if (policy == PROX_LRU) s_stamp[bs] = t;
                 const int own = s_owner[bs];
@@ -130,7 +130,7 @@ lsh_resolve_kernel(const DevState *st, int B, int d, int b, double tau, int poli
                 evt_dist[i] = (float)best;
                 ins_slot[i] = -1;
                 s_slot = -1;
-            } else {                                                          // lines 6-9
+            } else {                                                          // miss: evict if full, insert
                 int s;
                 if (cnt < b) {
                     s = cnt;

@@ -2,7 +2,7 @@
 //
 // Who needs this: code that is not allowed to call cudaMalloc when it wants a lookup -- a plugin
 // running inside a host application that owns the memory pool and forbids outside allocations,
-// a thread that is in the middle of capturing a stream, a service with a frozen memory budget.
+// a service with a frozen memory budget.
 // Such a caller passes the keys, the queries and the outputs (all memory it already owns); the
 // partial results that the blocks exchange live in an array that is part of the library image.
 //
@@ -35,7 +35,7 @@ struct NaScratch {
 // Lives in the library image on every GPU that loads it (about 192 KB) until the process exits.
 static __device__ __align__(256) unsigned char g_na_scratch[sizeof(NaScratch)];
 
-// Squared distances in fp64 over the fp32 values, difference form (Algorithm 1, lines 2-3, for
+// Squared distances in fp64 over the fp32 values, difference form (the distances and argmin of Algorithm 1, for
 // a batch): each block scans a range of keys for 32 queries; the block that finishes last for
 // a query tile reduces the partial minima (ties go to the lowest slot) and writes the outputs.
 __global__ void __launch_bounds__(256)

@@ -197,6 +197,7 @@ extern "C" prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t 
     cudaMemset(h->buf_cnt, 0, 4 * P * kScanQ * sizeof(int32_t));
     launch_convert_corpus(h, 0);
     launch_reset(h, 0);
+    init_scan_tc(h);
     const cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         set_err("set-up kernels failed: %s", cudaGetErrorString(e));

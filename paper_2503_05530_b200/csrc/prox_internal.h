@@ -174,6 +174,7 @@ int launch_probe_scan_tc(prox_handle *h, int pass, cudaStream_t s);    // coarse
 void launch_probe_exact(prox_handle *h, const float *q, int B, cudaStream_t s);
 void launch_scan_pass(prox_handle *h, int pass, cudaStream_t s);       // CUDA-core scan
 int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s);     // tcgen05 scan; nonzero = not available
+void init_scan_tc(prox_handle *h);                                      // tensor maps, at prox_create
 void free_scan_tc(prox_handle *h);
 void launch_merge_select(prox_handle *h, int pass, int B, int for_probe, cudaStream_t s);
 void launch_rerank(prox_handle *h, const float *q, int B, cudaStream_t s);

@@ -1,4 +1,4 @@
-// Miss path: exact k nearest corpus rows for the queries that missed (Algorithm 1, line 6,
+// Miss path: exact k nearest corpus rows for the queries that missed (the database call of Algorithm 1,
 // with an exact flat index as in Section 4.2.1).
 //
 // Route to the exact answer:
@@ -672,7 +672,7 @@ fallback_collect_kernel(DevState *st, const float *__restrict__ corpus, const __
 }
 
 // ------------------------------------------------------------------------------------------
-// Coarse tensor-core probe (Algorithm 1, lines 2-3, for large caches): the scan kernel run over
+// Coarse tensor-core probe (the key distances of Algorithm 1, for large caches): the scan kernel run over
 // the bf16 copies of the keys gives, per query, the kProbeKp slots with the best coarse scores;
 // here their exact fp64 distances give the nearest safe slot, with the same kind of
 // certificate as the corpus scan.  At-risk slots are left out (the fp64 probe measures them as

@@ -1,6 +1,6 @@
 // Tensor-core corpus scan for sm_100a: coarse scores s = bf16(q).bf16(x) - |bf16(x)|^2 / 2 for
 // every corpus row and up to 256 miss queries per pass, with the per-query best-k' selection
-// fused into the accumulator read-out (Algorithm 1, line 6: the database call of the misses).
+// fused into the accumulator read-out (Algorithm 1: the database call of the misses).
 //
 // One persistent block per SM, 4 + 8 warps:
 //   warp 0   one lane issues TMA loads (cp.async.bulk.tensor, no multicast) of 128-row x 64-col
@@ -22,7 +22,6 @@
 #include <cuda.h>
 
 #include <new>
-#include <vector>
 
 #include "prox_internal.h"
 #include "scan_readout.cuh"
@@ -550,31 +549,48 @@ struct Maps {
 };
 constexpr int kMaxUnits = 256;
 
+// Equal speeds for every pair: the state before the first measurement.
+__global__ void speed_init_kernel(float *speed) {
+    for (int i = threadIdx.x; i < 2 * kMaxUnits; i += blockDim.x) speed[i] = 1.f;
+}
+
 }  // namespace
+
+// Tensor maps and the speed table of one scanned matrix: made once, at prox_create, so that the
+// batch calls neither allocate nor copy.
+static void ensure_maps(prox_handle *h, void **state, const __nv_bfloat16 *xb, long long rows,
+                        const __nv_bfloat16 *qb) {
+    if (*state) return;
+    Maps *m = new (std::nothrow) Maps();
+    if (!m) return;
+    *state = m;
+    const uint32_t ks = ((h->d / kChunkK) % 2 == 0) ? 2 : 1;
+    m->ks = (int)ks;
+    if (cudaMalloc(&m->speed, sizeof(float) * 2 * kMaxUnits) != cudaSuccess) { m->speed = nullptr; cudaGetLastError(); }
+    m->ok = m->speed != nullptr && make_map(&m->x, xb, (uint64_t)rows, (uint64_t)h->d, kTileRows, ks) &&
+            make_map(&m->q16, qb, kMaxBatch, (uint64_t)h->d, 16, ks) &&
+            make_map(&m->q32, qb, kMaxBatch, (uint64_t)h->d, 32, ks) &&
+            make_map(&m->q64, qb, kMaxBatch, (uint64_t)h->d, 64, ks) &&
+            make_map(&m->q128, qb, kMaxBatch, (uint64_t)h->d, 128, ks) &&
+            make_map(&m->q256, qb, kMaxBatch, (uint64_t)h->d, 256, ks);
+    cudaFuncSetAttribute(scan_tc_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
+    cudaFuncSetAttribute(scan_tc_kernel<512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
+    cudaFuncSetAttribute(scan_tc_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
+    cudaFuncSetAttribute(scan_tc_kernel<512, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
+}
+
+void init_scan_tc(prox_handle *h) {
+    if (h->d % kChunkK) return;
+    if (h->N >= kTileRows) ensure_maps(h, &h->tc_state, h->xb, (long long)h->N, h->qb);
+    if (h->probe_tc) ensure_maps(h, &h->tc_state_keys, h->keys_b, (long long)h->C, h->pqb);
+}
 
 // One pass of the tensor-core scan of `rows` bf16 rows (xb, half norms xh) against the bf16 query
 // block qb.  Returns nonzero when the tensor-core path cannot run (no tensor-map encoder in the
 // driver, out of memory for the maps); the caller then falls back.
 static int launch_scan_generic(prox_handle *h, void **state, const __nv_bfloat16 *xb, const float *xh, long long rows,
                                const __nv_bfloat16 *qb, const int *n_active, int kp, int pass, cudaStream_t s) {
-    if (!*state) {
-        Maps *m = new (std::nothrow) Maps();
-        if (!m) return 1;
-        *state = m;
-        const uint32_t ks = ((h->d / kChunkK) % 2 == 0) ? 2 : 1;
-        m->ks = (int)ks;
-        if (cudaMalloc(&m->speed, sizeof(float) * 2 * kMaxUnits) != cudaSuccess) { m->speed = nullptr; cudaGetLastError(); }
-        m->ok = m->speed != nullptr && make_map(&m->x, xb, (uint64_t)rows, (uint64_t)h->d, kTileRows, ks) &&
-                make_map(&m->q16, qb, kMaxBatch, (uint64_t)h->d, 16, ks) &&
-                make_map(&m->q32, qb, kMaxBatch, (uint64_t)h->d, 32, ks) &&
-                make_map(&m->q64, qb, kMaxBatch, (uint64_t)h->d, 64, ks) &&
-                make_map(&m->q128, qb, kMaxBatch, (uint64_t)h->d, 128, ks) &&
-                make_map(&m->q256, qb, kMaxBatch, (uint64_t)h->d, 256, ks);
-        cudaFuncSetAttribute(scan_tc_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
-        cudaFuncSetAttribute(scan_tc_kernel<512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
-        cudaFuncSetAttribute(scan_tc_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
-        cudaFuncSetAttribute(scan_tc_kernel<512, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
-    }
+    if (!*state) return 1;
     Maps &maps = *static_cast<Maps *>(*state);
     if (!maps.ok) return 1;
     ScanArgs a;
@@ -585,14 +601,11 @@ static int launch_scan_generic(prox_handle *h, void **state, const __nv_bfloat16
     const int units = pair ? grid / 2 : grid;
     if (units > kMaxUnits) return 1;
     if (maps.units != units) {                            // first launch, or the launch shape changed: equal speeds
-        static const std::vector<float> ones(2 * kMaxUnits, 1.f);
-        if (cudaMemcpyAsync(maps.speed, ones.data(), sizeof(float) * 2 * kMaxUnits, cudaMemcpyHostToDevice, s) != cudaSuccess)
-            return 1;
+        speed_init_kernel<<<1, 256, 0, s>>>(maps.speed);
         maps.units = units;
     }
     a.w_in = maps.speed + (maps.launch_no & 1u) * kMaxUnits;
     a.w_out = maps.speed + ((maps.launch_no + 1u) & 1u) * kMaxUnits;
-    maps.launch_no++;
     h->scan_lists = 4 * grid;                             // one candidate list per read-out lane quarter
     h->scan_list_stride = h->tc_cap;
     cudaLaunchConfig_t cfg = {};
@@ -614,7 +627,11 @@ static int launch_scan_generic(prox_handle *h, void **state, const __nv_bfloat16
     else
         e = h->tc_cap == 256 ? cudaLaunchKernelEx(&cfg, scan_tc_kernel<256, false>, maps.x, maps.q16, maps.q32, maps.q64, maps.q128, maps.q256, a)
                              : cudaLaunchKernelEx(&cfg, scan_tc_kernel<512, false>, maps.x, maps.q16, maps.q32, maps.q64, maps.q128, maps.q256, a);
-    if (e != cudaSuccess) return 1;
+    if (e != cudaSuccess) {                               // the caller falls back: leave no error behind, keep the speeds' turn
+        cudaGetLastError();
+        return 1;
+    }
+    maps.launch_no++;
     h->launches++;
     return 0;
 }

@@ -1,6 +1,6 @@
 // A corpus split by rows over several GPUs: the exchange record of one shard's miss results and
 // the merge of all shards' records into the k nearest rows of the whole corpus (the database
-// call of Algorithm 1, line 6, answered by G shards).
+// call of Algorithm 1, answered by G shards).
 #include "prox_internal.h"
 
 namespace prox {

@@ -24,11 +24,21 @@ def load_trace(path, d=16):
     corpus[:, 0] = np.arange(n_pts)
     queries = np.zeros((len(rows), d), np.float32)
     queries[:, 0] = [r[0] for r in rows]
+    preload = None
+    if "preload" in params:                                   # keys bulk-loaded before the first query
+        vals = [float(x) for x in params["preload"].split(",")]
+        preload = np.zeros((len(vals), d), np.float32)
+        preload[:, 0] = vals
     return dict(name=os.path.basename(path), policy=params["policy"], capacity=int(params["capacity"]), k=k,
-                tau=float(params["tau"]), corpus=corpus, queries=queries,
+                tau=float(params["tau"]), corpus=corpus, queries=queries, preload=preload,
                 hit=np.array([r[1] for r in rows], np.uint8), slot=np.array([r[2] for r in rows]),
                 evicted=np.array([r[3] for r in rows]), ids=np.array([r[4] for r in rows], np.int64))
 
 
 def all_traces(d=16):
     return [load_trace(p, d) for p in sorted(glob.glob(os.path.join(GOLDEN_DIR, "trace_*.txt")))]
+
+
+def all_load_traces(d=16):
+    """Traces that start from a bulk-loaded cache (`preload=` in the header line)."""
+    return [load_trace(p, d) for p in sorted(glob.glob(os.path.join(GOLDEN_DIR, "load_*.txt")))]

@@ -4,7 +4,8 @@ oracle on the same bytes, and compare under the stated rule.
 Rule: hit flags and returned ids equal; distances within 1e-4 relative.  A query may differ only
 if (i) its nearest-key distance ties with tau to 1e-5 relative (never when that distance is 0),
 or (ii) its k-th and (k+1)-th neighbour distances, or two neighbours inside the list, tie to 1e-5
-relative.  Such queries are counted and must stay below 0.1 % of the stream."""
+relative, and the ids that differ are exactly the tied ones.  Such queries are counted and must
+stay below 0.1 % of the stream; unless a test says otherwise none is accepted at all."""
 import numpy as np
 import torch
 
@@ -75,17 +76,30 @@ def run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=None, max_forc
         forced.append(i)
 
 
-def knn_tie_excused(corpus, q, k, metric="l2"):
-    """Rule (ii): is there a tie to 1e-5 relative at the k/(k+1) boundary or inside the list?"""
-    kk = min(k + 1, corpus.shape[0])
-    _, d = oracle.exact_topk(corpus, q, kk, metric=oracle.COSINE if metric == "cosine" else oracle.L2SQ)
-    d = d[0]
-    gaps = np.diff(d)
-    return bool(np.any(gaps < REL_TIE * np.maximum(d[1:], 1e-300)))
+def ids_differ_only_within_ties(corpus, q, gpu_ids, ref_ids, ref_dists, metric="l2"):
+    """Rule (ii), applied to the positions that differ and to nothing else: wherever the library's
+    list names another row than the oracle's, that row's exact distance to the query must tie with
+    the oracle's distance at the same position to 1e-5 relative (two rows swapped inside the
+    list, or another row of a tie group at the k / k+1 boundary), and the library's list must not
+    name a row twice.  A tie somewhere else in the list excuses nothing."""
+    if len(set(int(x) for x in gpu_ids)) != len(gpu_ids):
+        return False
+    dist = oracle.cosdist if metric == "cosine" else oracle.sqdist
+    for p in np.nonzero(np.asarray(gpu_ids) != np.asarray(ref_ids))[0]:
+        g = int(gpu_ids[p])
+        if g < 0 or g >= corpus.shape[0]:
+            return False
+        dg, dr = dist(q, corpus[g]), float(ref_dists[p])
+        if not abs(dg - dr) < REL_TIE * max(dr, dg, 1e-300):
+            return False
+    return True
 
 
 def compare(corpus, queries, k, capacity, tau, policy, gpu, max_excused_frac=1e-3, rho=1, lsh_planes=None, lsh_bucket=0,
-            metric="l2"):
+            metric="l2", allow_excused=False):
+    """allow_excused=False (the default): the exemptions exist but no query may need one -- probe,
+    threshold test and rerank run in fp64 like the oracle, so none has ever been needed; a test
+    whose inputs are built to tie passes allow_excused=True and stays under max_excused_frac."""
     ids, dists, hit, stats = gpu
     ref, forced = run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=hit, rho=rho, lsh_planes=lsh_planes,
                              lsh_bucket=lsh_bucket, metric=metric)
@@ -97,11 +111,9 @@ def compare(corpus, queries, k, capacity, tau, policy, gpu, max_excused_frac=1e-
     for i in rows_bad:
         origin = int(ref["origin"][i])                       # the miss whose list is returned
         src = origin if origin >= 0 else i
-        tie = knn_tie_excused(corpus, queries[src], k * rho, metric)
-        if not tie and rho > 1 and src != i:                 # re-ranked hit: a tie among the stored rows for this query
-            stored, _ = oracle.exact_topk(corpus, queries[src], k * rho)
-            dd = np.sort(((queries[i].astype(np.float64)[None, :] - corpus[stored[0]].astype(np.float64)) ** 2).sum(1))
-            tie = bool(np.any(np.diff(dd) < REL_TIE * np.maximum(dd[1:], 1e-300)))
+        # a re-ranked hit is measured against the current query, everything else against the query of the list
+        q_eval = queries[i] if (rho > 1 and src != i) else queries[src]
+        tie = ids_differ_only_within_ties(corpus, q_eval, ids[i], ref["ids"][i], ref["dists"][i], metric)
         assert tie, f"ids differ at query {i} (list of query {src}): oracle {ref['ids'][i]} gpu {ids[i]}"
         excused.add(int(i))
     ok_rows = np.setdiff1d(np.arange(n), rows_bad)
@@ -111,5 +123,6 @@ def compare(corpus, queries, k, capacity, tau, policy, gpu, max_excused_frac=1e-
     assert np.all(err <= tol), f"distance error {err.max()} (relative {np.max(err / np.maximum(np.abs(rd), 1e-30))})"
     assert len(excused) <= max(max_excused_frac * n, 0) or len(excused) == 0 or len(excused) / n < max_excused_frac, \
         f"{len(excused)} of {n} queries needed the tie exemption"
+    assert allow_excused or len(excused) == 0, f"queries {sorted(excused)[:8]} needed a tie exemption"
     assert stats["hits"] == int(ref["hit"].sum()) and stats["misses"] == n - int(ref["hit"].sum())
     return dict(ref=ref, excused=len(excused), hit_rate=float(ref["hit"].mean()))

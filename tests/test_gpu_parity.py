@@ -6,7 +6,8 @@ import torch
 
 import oracle
 from paper_2503_05530_b200 import prox, workloads as W
-from golden_traces import all_traces
+from golden_traces import all_load_traces, all_traces
+import oracle_workers
 from parity import compare, run_gpu, run_oracle
 
 pytestmark = pytest.mark.gpu
@@ -44,6 +45,35 @@ def test_golden_trace_slots_via_probe():
         torch.cuda.synchronize()
         assert np.array_equal(hit.cpu().numpy(), tr["hit"]) and np.array_equal(slot.cpu().numpy(), tr["slot"])
         p.close()
+
+
+@pytest.mark.parametrize("tr", all_load_traces(), ids=lambda t: t["name"])
+@pytest.mark.parametrize("batch", [1, 4, 64])
+def test_golden_traces_from_a_loaded_cache_on_gpu(tr, batch):
+    """A bulk-loaded cache: which slot leaves first afterwards (hand-traced fixtures)."""
+    X, Q = torch.from_numpy(tr["corpus"]).to(DEV), torch.from_numpy(tr["queries"]).to(DEV)
+    for probe_only in (False, True):
+        p = prox.Prox(X, tr["k"], tr["capacity"], tr["tau"], tr["policy"])
+        p.cache_load(torch.from_numpy(tr["preload"]).to(DEV))
+        hits, slots, ids = [], [], []
+        for a in range(0, Q.shape[0], batch):
+            if probe_only:
+                h, s_, _ = p.probe_batch(Q[a:a + batch])
+                slots.append(s_.clone())
+            else:
+                i_, _, h = p.query_batch(Q[a:a + batch])
+                ids.append(i_.clone())
+            hits.append(h.clone())
+        torch.cuda.synchronize()
+        assert p.status() == prox.OK
+        st = p.stats()
+        p.close()
+        assert np.array_equal(torch.cat(hits).cpu().numpy(), tr["hit"])
+        assert st["evictions"] == int((tr["evicted"] >= 0).sum())
+        if probe_only:
+            assert np.array_equal(torch.cat(slots).cpu().numpy(), tr["slot"])
+        else:
+            assert np.array_equal(torch.cat(ids).cpu().numpy(), tr["ids"])
 
 
 # ------------------------------------------------------------------ the small sequential configuration
@@ -170,7 +200,7 @@ def test_reranking_factor_argument_checks():
     lib.prox_destroy(h)
 
 
-# ------------------------------------------------------------------ cosine distance (Section 2.1)
+# ------------------------------------------------------------------ cosine distance (Section 2.2)
 @pytest.mark.parametrize("policy,batch,rho", [("lru", 64, 1), ("fifo", 1, 1), ("lru", 500, 2)])
 def test_cosine_distance_matches_the_oracle(policy, batch, rho):
     """Rows and queries of very different lengths: the Euclidean neighbours are not the cosine ones."""
@@ -286,6 +316,52 @@ def test_probe_only_cache_above_the_multi_block_risk_selection(policy):
     assert 100 < misses < 3900
     assert p.status() == prox.OK
     p.close()
+
+
+@pytest.mark.parametrize("n_keys,n_batches,batch,policies", [(1 << 17, 2, 1024, ("lru", "fifo")), (1 << 20, 1, 256, ("lru",))])
+def test_probe_only_at_the_benchmarked_cache_sizes(n_keys, n_batches, batch, policies):
+    """The probe-only workload at the sizes the benchmark reports (2^17 and 2^20 keys of 768
+    dimensions, full cache, tau = 0.5): every flag, matched or written slot and hit distance against
+    the oracle.  The oracle walks all keys for every query on one core (a minute or two per batch),
+    so its runs go to worker processes and overlap the GPU side and one another; the cache state is
+    sequential, so a batch cannot be sampled: at 2^20 keys one batch of 256 queries is replayed."""
+    d, tau = 768, 0.5
+    keys, centres = W.make_probe_keys(n_keys, d, 4096, seed=8)
+    Qs = torch.stack([W.make_probe_batch(keys, centres, batch, 0.02, 8, b) for b in range(n_batches)])
+    kb, kdesc = oracle_workers.share(keys.numpy())
+    qb, qdesc = oracle_workers.share(Qs.numpy())
+    try:
+        with oracle_workers.pool(len(policies)) as pool:
+            jobs = [pool.apply_async(oracle_workers.probe_trace_worker, (kdesc, qdesc, tau, pol)) for pol in policies]
+            keys_d, got = keys.to(DEV), {}
+            for pol in policies:
+                p = prox.Prox(keys_d[:64].contiguous(), 1, n_keys, tau, pol)
+                p.cache_load(keys_d)
+                got[pol] = []
+                for b in range(n_batches):
+                    hit, slot, dist = p.probe_batch(Qs[b].to(DEV))
+                    got[pol].append((hit.cpu().numpy(), slot.cpu().numpy(), dist.cpu().numpy()))
+                torch.cuda.synchronize()
+                assert p.status() == prox.OK, prox.last_error()
+                got[pol].append(p.stats())
+                p.close()
+            for pol, job in zip(policies, jobs):
+                ref = job.get(timeout=900)
+                evictions = 0
+                for b in range(n_batches):
+                    hit, slot, dist = got[pol][b]
+                    r = ref[b]
+                    assert np.array_equal(hit, r["hit"]), f"{pol} batch {b}: first differing flag at {np.nonzero(hit != r['hit'])[0][:1]}"
+                    assert np.array_equal(slot, r["slot"]), f"{pol} batch {b}: first differing slot at {np.nonzero(slot != r['slot'])[0][:1]}"
+                    h = r["hit"] == 1
+                    assert np.allclose(dist[h], r["best"][h], rtol=1e-6)
+                    assert 0.3 < r["hit"].mean() < 0.97
+                    evictions += int((r["evicted"] >= 0).sum())
+                assert got[pol][n_batches]["evictions"] == evictions > 0
+    finally:
+        for blk in (kb, qb):
+            blk.close()
+            blk.unlink()
 
 
 def test_large_cache_stream_with_coarse_probe():

@@ -99,7 +99,7 @@ def test_duplicate_rows_across_shards_keep_the_lower_id():
     got = ids[miss]
     assert np.array_equal(got[:, 1] - got[:, 0], np.full(miss.sum(), 4000))
     assert np.array_equal(got[:, 2] - got[:, 1], np.full(miss.sum(), 4000))
-    compare(X.numpy(), Q.numpy(), 6, 32, 0.0, "lru", (ids, dists, hit, _), max_excused_frac=1.0)
+    compare(X.numpy(), Q.numpy(), 6, 32, 0.0, "lru", (ids, dists, hit, _))
 
 
 def test_shard_argument_checks():

@@ -7,7 +7,7 @@ import torch
 
 import oracle
 from paper_2503_05530_b200 import workloads as W
-from golden_traces import all_traces
+from golden_traces import all_load_traces, all_traces
 
 POL = {"lru": oracle.LRU, "fifo": oracle.FIFO}
 
@@ -17,7 +17,7 @@ def unit_rows(n, d, seed):
     return (r / np.linalg.norm(r, axis=1, keepdims=True)).astype(np.float32)
 
 
-# ---------------------------------------------------------------- distance (Algorithm 1, line 2)
+# ---------------------------------------------------------------- distance (Algorithm 1, distance(q, k))
 def test_sqdist_closed_forms():
     assert oracle.sqdist([1, 2, 3], [4, 6, 8]) == 50.0           # 9 + 16 + 25
     e = np.eye(8, dtype=np.float32)
@@ -37,7 +37,7 @@ def test_sqdist_closed_forms():
     assert oracle.sqdist([-1, -1], [1, 1]) == 8.0
 
 
-# ---------------------------------------------------------------- database call (Algorithm 1, line 6)
+# ---------------------------------------------------------------- database call (Algorithm 1, retrieveDocumentIndices)
 @pytest.mark.parametrize("n,d,k,seed", [(50, 3, 5, 0), (1000, 16, 10, 1), (777, 128, 32, 2), (64, 768, 64, 3)])
 def test_exact_topk_vs_numpy_bruteforce(n, d, k, seed):
     X = unit_rows(n, d, seed)
@@ -197,6 +197,42 @@ def test_golden_traces(tr):
     assert np.array_equal(r["slot"], tr["slot"])
     assert np.array_equal(r["evicted"], tr["evicted"])
     assert np.array_equal(r["ids"], tr["ids"])
+
+
+@pytest.mark.parametrize("tr", all_load_traces(), ids=lambda t: t["name"])
+def test_golden_traces_from_a_loaded_cache(tr):
+    """Bulk load: which entry leaves first afterwards (hand-traced, Section 3.3.2)."""
+    o = oracle.Oracle(tr["corpus"], tr["corpus"].shape[1], tr["k"], tr["capacity"], tr["tau"], POL[tr["policy"]])
+    o.cache_load(tr["preload"])
+    assert o.counters()["count"] == len(tr["preload"])
+    r = o.query(tr["queries"])
+    assert np.array_equal(r["hit"], tr["hit"])
+    assert np.array_equal(r["slot"], tr["slot"])
+    assert np.array_equal(r["evicted"], tr["evicted"])
+    assert np.array_equal(r["ids"], tr["ids"])
+
+
+@pytest.mark.parametrize("policy", ["lru", "fifo"])
+def test_loaded_cache_equals_the_same_keys_inserted_by_misses(policy):
+    """A bulk load of n distinct keys must leave the cache as n misses on those keys would (tau = 0:
+    no hits): same slots, same eviction order afterwards, whatever the policy."""
+    X, Q, _ = small_workload(8, nq=90)
+    n, cap = 12, 12
+    a = oracle.Oracle(None, X.shape[1], 1, cap, 0.05, POL[policy])
+    a.cache_load(Q[:n])
+    b = oracle.Oracle(None, X.shape[1], 1, cap, 0.0, POL[policy])
+    rb0 = b.query(Q[:n])
+    assert rb0["hit"].sum() == 0 and np.array_equal(rb0["slot"], np.arange(n))
+    b.close()
+    # same tolerance from here on: rebuild b at tau = 0.05 by forcing the first n queries to miss
+    b = oracle.Oracle(None, X.shape[1], 1, cap, 0.05, POL[policy])
+    force = np.full(len(Q), -1, np.int32)
+    force[:n] = 0
+    rb = b.query(Q, force)
+    ra = a.query(Q[n:])
+    for key in ("hit", "slot", "evicted", "best"):
+        assert np.array_equal(ra[key], rb[key][n:]), key
+    assert ra["evicted"].max() >= 0 and 0 < ra["hit"].sum() < len(ra["hit"])
 
 
 def test_fifo_and_lru_traces_differ():
@@ -371,7 +407,7 @@ def test_lsh_operation_count_of_the_papers_example():
     assert o.counters()["probe_madds"] - before == (L + b) * d == 23040
 
 
-# ---------------------------------------------------------------- cosine distance (Section 2.1)
+# ---------------------------------------------------------------- cosine distance (Section 2.2)
 def test_cosine_closed_forms():
     e = np.eye(6, dtype=np.float32)
     assert oracle.cosdist(e[0], e[1]) == pytest.approx(1.0, abs=1e-15)           # orthogonal
