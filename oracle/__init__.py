@@ -20,7 +20,7 @@ _SRC = os.path.join(_HERE, "prox_oracle.c")
 _LIB = os.path.join(_HERE, "_prox_oracle.so")
 
 LRU, FIFO = 0, 1
-L2SQ, COSINE = 0, 1
+L2SQ, COSINE, IP = 0, 1, 2
 
 
 def build(force: bool = False) -> str:
@@ -57,6 +57,8 @@ def lib():
         L.oracle_set_metric.argtypes = [C.c_void_p, C.c_int32]
         L.oracle_cosdist.restype = C.c_double
         L.oracle_cosdist.argtypes = [fp, fp, C.c_int32]
+        L.oracle_ipdist.restype = C.c_double
+        L.oracle_ipdist.argtypes = [fp, fp, C.c_int32]
         L.oracle_knn_batch_metric.argtypes = [C.c_int32, fp, C.c_int64, C.c_int32, fp, C.c_int64, C.c_int32, ip, dp]
         L.oracle_destroy.argtypes = [C.c_void_p]
         L.oracle_reset.argtypes = [C.c_void_p]
@@ -98,6 +100,13 @@ def cosdist(a, b) -> float:
     a, b = _f32(a).ravel(), _f32(b).ravel()
     assert a.shape == b.shape
     return float(lib().oracle_cosdist(_ptr(a, C.c_float), _ptr(b, C.c_float), a.size))
+
+
+def ipdist(a, b) -> float:
+    """Inner product as a distance, -(a . b), in fp64 over fp32 inputs."""
+    a, b = _f32(a).ravel(), _f32(b).ravel()
+    assert a.shape == b.shape
+    return float(lib().oracle_ipdist(_ptr(a, C.c_float), _ptr(b, C.c_float), a.size))
 
 
 def exact_topk(corpus, queries, k: int, metric: int = L2SQ):
@@ -169,7 +178,9 @@ class Oracle:
         if not self._h:
             raise ValueError("oracle_create rejected the arguments")
         if lib().oracle_set_metric(self._h, metric):
-            raise ValueError("unknown metric")
+            self.close()
+            raise ValueError("metric unknown, or not available with these arguments (a negative tolerance goes with the "
+                             "inner product only; PROXIMITY-LSH does not take the inner product)")
 
     def close(self):
         if self._h:

@@ -38,6 +38,12 @@
  *     squared Euclidean by default; ORACLE_COSINE is the cosine distance 1 - cos(a, b), taken
  *     as half the squared Euclidean distance of a/|a| and b/|b| (the same number, and exactly 0
  *     for identical vectors so that tau = 0 stays exact matching); normalisation in fp64;
+ *     ORACLE_IP is the inner product turned into a distance, -(a . b): the nearest key or row is
+ *     the one with the largest inner product, and a key matches when -(q . key) <= tau, i.e. when
+ *     q . key >= -tau.  For this metric tau may be any finite number (on unit vectors -1 <= -a.b
+ *     <= 1), and tau = 0 is not exact matching: it accepts every key that is not on the far side
+ *     of the query (inner product >= 0).  A vector is in general not its own nearest neighbour
+ *     (a longer vector in the same direction scores higher);
  *   - PROXIMITY-LSH (Section 3.2): L random hyperplanes through the origin, given by the caller
  *     as L normal vectors; bit l of the hash is (q . r_l >= 0), the dot product taken in fp64
  *     in index order; the 2^L buckets are PROXIMITY-FLAT caches of b entries each, every one
@@ -61,7 +67,7 @@
 #endif
 
 enum { ORACLE_LRU = 0, ORACLE_FIFO = 1 };
-enum { ORACLE_L2SQ = 0, ORACLE_COSINE = 1 };
+enum { ORACLE_L2SQ = 0, ORACLE_COSINE = 1, ORACLE_IP = 2 };
 
 typedef struct {
     /* stored state of Algorithm 1: tau, c, the database D and the dict C */
@@ -122,7 +128,15 @@ double oracle_cosdist(const float *a, const float *b, int32_t d) {
     return 0.5 * acc;
 }
 
+/* Inner product as a distance: -(a . b), the sum taken in fp64 in index order. */
+double oracle_ipdist(const float *a, const float *b, int32_t d) {
+    double acc = 0.0;
+    for (int32_t j = 0; j < d; ++j) acc += (double)a[j] * (double)b[j];
+    return -acc;
+}
+
 static double oracle_dist(int32_t metric, const float *a, const float *b, int32_t d) {
+    if (metric == ORACLE_IP) return oracle_ipdist(a, b, d);
     return metric == ORACLE_COSINE ? oracle_cosdist(a, b, d) : oracle_sqdist(a, b, d);
 }
 
@@ -184,7 +198,7 @@ void oracle_exact_topk(const float *corpus, int64_t N, int32_t d, const float *q
 
 oracle_t *oracle_create_rho(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
                             double tau, int32_t policy, int32_t rho) {
-    if (d < 1 || k < 1 || capacity < 1 || rho < 1 || !(tau >= 0.0)) return NULL;
+    if (d < 1 || k < 1 || capacity < 1 || rho < 1 || !(tau == tau) || isinf(tau)) return NULL;   /* the sign of tau: oracle_set_metric */
     if (policy != ORACLE_LRU && policy != ORACLE_FIFO) return NULL;
     const int32_t m = rho * k;
     if (corpus && (N < 1 || m > N)) return NULL;
@@ -238,9 +252,13 @@ void oracle_destroy(oracle_t *o) {
     free(o->origin); free(o->valid); free(o->scratch); free(o);
 }
 
-/* Chooses the distance of the cache keys and of the database (before the first query). */
+/* Chooses the distance of the cache keys and of the database (before the first query).  Squared
+   Euclidean and cosine distances are never negative, so a negative tolerance is refused there;
+   the inner-product distance takes any finite tolerance. */
 int oracle_set_metric(oracle_t *o, int32_t metric) {
-    if (metric != ORACLE_L2SQ && metric != ORACLE_COSINE) return 1;
+    if (metric != ORACLE_L2SQ && metric != ORACLE_COSINE && metric != ORACLE_IP) return 1;
+    if (metric != ORACLE_IP && !(o->tau >= 0.0)) return 1;
+    if (metric == ORACLE_IP && o->lsh_L >= 0) return 1;    /* hyperplane buckets go with angles, not with inner products */
     o->metric = metric;
     return 0;
 }

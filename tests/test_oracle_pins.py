@@ -452,3 +452,101 @@ def test_cosine_duplicate_hits_at_tau_zero_whatever_its_length():
     Q2 = np.concatenate([Q[:1], 2 * Q[:1], Q[1:2]])
     r = oracle.Oracle(X, X.shape[1], 3, 4, 0.0, oracle.FIFO, metric=oracle.COSINE).query(Q2)
     assert r["hit"].tolist() == [0, 1, 0]
+
+
+# ---------------------------------------------------------------- inner product (Section 2.2)
+def test_inner_product_closed_forms():
+    assert oracle.ipdist([1, 2, 3], [4, 5, 6]) == -32.0
+    e = np.eye(5, dtype=np.float32)
+    for i in range(5):
+        for j in range(5):
+            assert oracle.ipdist(e[i], e[j]) == (-1.0 if i == j else 0.0)
+    a, b = unit_rows(2, 64, 21)
+    assert oracle.ipdist(a, b) == oracle.ipdist(b, a)
+    assert oracle.ipdist(a, -a) == pytest.approx(1.0, abs=1e-6) and oracle.ipdist(a, -a) > 0      # opposite: the farthest
+    assert oracle.ipdist(2 * a, b) == pytest.approx(2 * oracle.ipdist(a, b), rel=1e-15)           # linear, unlike a true distance
+    assert oracle.ipdist([3, 0], [0, 4]) == 0.0 and oracle.sqdist([3, 0], [0, 4]) == 25.0          # not the Euclidean value
+
+
+def test_inner_product_topk_vs_numpy():
+    rng = np.random.default_rng(22)
+    X = (rng.standard_normal((600, 40)) * rng.uniform(0.2, 3.0, (600, 1))).astype(np.float32)
+    Q = rng.standard_normal((6, 40)).astype(np.float32)
+    X[77] = X[12]                                                     # equal inner products: the lower id first
+    ids, dists = oracle.exact_topk(X, Q, 600, metric=oracle.IP)
+    for i, q in enumerate(Q):
+        full = -(X.astype(np.float64) @ q.astype(np.float64))
+        order = np.lexsort((np.arange(len(X)), full))
+        p12, p77 = np.where(ids[i] == 12)[0][0], np.where(ids[i] == 77)[0][0]
+        assert p77 == p12 + 1
+        assert np.array_equal(ids[i][:10], order[:10]) and np.allclose(dists[i], np.sort(full), rtol=0, atol=1e-12)
+        assert np.all(np.diff(dists[i]) >= 0) and dists[i][0] < 0    # most similar first
+    l2_ids, _ = oracle.exact_topk(X, Q, 10)
+    assert (l2_ids != ids[:, :10]).any()                              # rows of unequal length: not the Euclidean neighbours
+
+
+def test_inner_product_equals_euclidean_neighbours_on_unit_vectors():
+    """|q - x|^2 = |q|^2 + |x|^2 - 2 q.x: with all lengths equal the two rankings agree."""
+    X, Q = unit_rows(800, 48, 23), unit_rows(9, 48, 24)
+    ip_ids, ip_d = oracle.exact_topk(X, Q, 12, metric=oracle.IP)
+    l2_ids, l2_d = oracle.exact_topk(X, Q, 12)
+    assert np.array_equal(ip_ids, l2_ids)
+    assert np.allclose(ip_d, (l2_d - 2.0) / 2.0, atol=2e-7)
+
+
+def test_inner_product_cache_follows_algorithm_1():
+    """Independent replay with -q.k as the distance; the tolerance is negative here (a key matches
+    when q.k >= 0.9), which only this metric allows."""
+    X, Q, _ = small_workload(16, nq=200)
+    cap, tau = 6, -0.9
+    r = oracle.Oracle(X, X.shape[1], 3, cap, tau, oracle.LRU, metric=oracle.IP).query(Q)
+    keys, stamp = {}, {}
+    Q64 = Q.astype(np.float64)
+    for i in range(len(Q)):
+        dist = {s: -float(Q64[i] @ Q64[j]) for s, j in keys.items()}
+        best = min(dist, key=lambda s: (dist[s], s)) if dist else None
+        if best is not None and dist[best] <= tau:
+            assert r["hit"][i] == 1 and r["slot"][i] == best and r["origin"][i] == keys[best]
+            assert r["best"][i] == pytest.approx(dist[best], abs=1e-12)
+            stamp[best] = i
+        else:
+            assert r["hit"][i] == 0
+            if len(keys) >= cap:
+                victim = min(stamp, key=stamp.get)
+                assert r["evicted"][i] == victim
+                del keys[victim], stamp[victim]
+                slot = victim
+            else:
+                slot = len(keys)
+            assert r["slot"][i] == slot
+            keys[slot], stamp[slot] = i, i
+    assert 0.1 < r["hit"].mean() < 0.95 and (r["evicted"] >= 0).any()
+    ids, dists = oracle.exact_topk(X, Q, 3, metric=oracle.IP)
+    miss = r["hit"] == 0
+    assert np.array_equal(r["ids"][miss], ids[miss]) and np.array_equal(r["dists"][miss], dists[miss])
+
+
+def test_inner_product_prefers_the_longer_key_and_tau_zero_is_a_half_space():
+    e = np.eye(4, dtype=np.float32)
+    keys = np.stack([e[0], 3 * e[0], -e[0]])
+    o = oracle.Oracle(None, 4, 1, 3, 0.0, oracle.FIFO, metric=oracle.IP)
+    o.cache_load(keys)
+    r = o.query(np.stack([e[0], e[1], -e[0] + e[1]]))
+    assert r["slot"].tolist()[0] == 1 and r["best"][0] == -3.0      # not its own duplicate in slot 0
+    assert r["hit"].tolist() == [1, 1, 1]                           # e1 is orthogonal to every key: -0 <= 0 matches (slot 0)
+    assert r["slot"].tolist()[1] == 0 and r["slot"].tolist()[2] == 2
+    o2 = oracle.Oracle(None, 4, 1, 3, -0.5, oracle.FIFO, metric=oracle.IP)
+    o2.cache_load(keys)
+    assert o2.query(np.stack([e[1]]))["hit"].tolist() == [0]        # inner product 0 < 0.5
+
+
+def test_negative_tolerance_goes_with_the_inner_product_only():
+    with pytest.raises(ValueError):
+        oracle.Oracle(None, 8, 1, 4, -0.1, oracle.LRU)
+    with pytest.raises(ValueError):
+        oracle.Oracle(None, 8, 1, 4, -0.1, oracle.LRU, metric=oracle.COSINE)
+    with pytest.raises(ValueError):
+        oracle.Oracle(None, 8, 1, 4, float("nan"), oracle.LRU, metric=oracle.IP)
+    with pytest.raises(ValueError):                                   # hyperplane buckets are for angles
+        oracle.Oracle(None, 8, 1, 8, 0.5, oracle.LRU, lsh_planes=np.zeros((1, 8), np.float32), lsh_bucket=4, metric=oracle.IP)
+    oracle.Oracle(None, 8, 1, 4, -0.1, oracle.LRU, metric=oracle.IP).close()
