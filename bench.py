@@ -531,7 +531,7 @@ def main():
     ap.add_argument("--rows", type=int, default=0, help="override the corpus size (profiling runs)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling runs)")
     ap.add_argument("--rho", type=int, default=1, help="re-ranking factor: rho * k rows fetched and stored per miss (1 = none)")
-    ap.add_argument("--metric", default="l2", choices=["l2", "cosine"], help="distance of the cache keys and of the corpus")
+    ap.add_argument("--metric", default="l2", choices=["l2", "cosine", "ip"], help="distance of the cache keys and of the corpus")
     ap.add_argument("--lsh-bits", type=int, default=-1, help="PROXIMITY-LSH with this many hyperplanes (-1: flat cache)")
     ap.add_argument("--lsh-bucket", type=int, default=20, help="entries per LSH bucket")
     ap.add_argument("--shard-rows", action="store_true", help="deal the rows of ONE corpus to the ranks (every rank answers the same "

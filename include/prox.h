@@ -49,6 +49,7 @@ enum {
     PROX_MAX_BATCH = 1024,      /* largest B of one call */
     PROX_METRIC_L2SQ = 0,       /* prox_create_metric: squared Euclidean distance (the default everywhere else) */
     PROX_METRIC_COSINE = 1,     /* prox_create_metric: cosine distance 1 - cos(a, b) */
+    PROX_METRIC_IP = 2,         /* prox_create_metric: inner product as a distance, -(a . b) */
     PROX_SCAN_AUTO = 0,         /* prox_set_scan_mode: tensor-core scan, two blocks per MMA (default) */
     PROX_SCAN_CUDA_CORE = 1,    /* prox_set_scan_mode: plain CUDA-core scan of the same bf16 scores */
     PROX_SCAN_TC_SINGLE = 2     /* prox_set_scan_mode: tensor-core scan, one block per MMA */
@@ -91,7 +92,14 @@ prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t d, int32_t 
  * vectors, of any length, are at distance exactly 0); tau applies to that value and out_dists
  * hold it.  The library keeps its own unit-length fp32 copy of the corpus (N x d x 4 bytes
  * more) and brings every query to unit length (norms in fp64) before the lookup.  Rows and
- * queries must be non-zero.  Inner product is not offered.
+ * queries must be non-zero.
+ * PROX_METRIC_IP: the inner product turned into a distance, -(a . b): the nearest key or row is
+ * the one with the largest inner product with the query, a key matches when -(q . key) <= tau
+ * (q . key >= -tau), and out_dists hold -(q . row), most similar first.  For this metric tau may
+ * be any finite number, negative ones included (on unit vectors the value lies in [-1, 1]); tau = 0
+ * is not exact matching here, it accepts every key whose inner product with the query is >= 0,
+ * and a query is in general not its own nearest key (a longer key in the same direction scores
+ * higher).  Not offered for PROXIMITY-LSH handles; large caches are probed in fp64 only.
  */
 prox_handle *prox_create_metric(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
                                 float tau, int32_t policy, int32_t rho, int32_t metric);

@@ -241,7 +241,8 @@ risk_finish_kernel(DevState *st, RiskWork *w, int32_t *risk_pos, int32_t *risk_s
 // ------------------------------------------------------------------------------------------
 // Probe: squared distances, in fp64 over the fp32 values and in difference form (so that a
 // bitwise duplicate is at distance exactly 0), from each query to every valid key and to
-// every earlier query of the batch.  Tile: 32 queries x 64 (or 32) columns per block, d in chunks of 32 (or 64).
+// every earlier query of the batch.  IP = true: the inner product as a distance, -(q . key),
+// an fp64 sum of the products.  Tile: 32 queries x 64 (or 32) columns per block, d in chunks of 32 (or 64).
 //   mode 0  columns = slots [0, count) then the batch [count, count + B): everything in fp64.
 //   mode 1  columns = the R at-risk slots then the batch: what the resolve needs as full rows
 //           when the safe slots are handled by the coarse tensor-core probe.
@@ -254,7 +255,7 @@ constexpr int kProbeColsWide = 64, kProbeColsNarrow = 32;
 // where the wide tiles leave most SMs without a block and the time goes into the chain of steps
 // (a barrier and a load latency each): narrower tiles give twice the blocks, deeper steps half
 // the chain with twice the loads in flight.
-template <int PC, int PD>
+template <int PC, int PD, bool IP>
 __global__ void __launch_bounds__(256)
 probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
              const float *__restrict__ queries, const int32_t *__restrict__ risk_pos, int B, int d,
@@ -347,9 +348,14 @@ probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
 #pragma unroll
                 for (int b = 0; b < PC / 16; ++b) {
                     const double kv = ks[tx + 16 * b][j];
-                    const double d0 = qa - kv, d1 = qb2 - kv;
-                    acc[0][b] = fma(d0, d0, acc[0][b]);
-                    acc[1][b] = fma(d1, d1, acc[1][b]);
+                    if constexpr (IP) {
+                        acc[0][b] = fma(-qa, kv, acc[0][b]);
+                        acc[1][b] = fma(-qb2, kv, acc[1][b]);
+                    } else {
+                        const double d0 = qa - kv, d1 = qb2 - kv;
+                        acc[0][b] = fma(d0, d0, acc[0][b]);
+                        acc[1][b] = fma(d1, d1, acc[1][b]);
+                    }
                 }
             }
         }
@@ -976,12 +982,10 @@ void launch_probe(prox_handle *h, const float *q, int B, int mode, cudaStream_t 
         if (splits > tiles) splits = tiles;
     }
     dim3 grid((B + PQ - 1) / PQ, splits);
-    if (PC == kProbeColsNarrow)
-        probe_kernel<kProbeColsNarrow, 64><<<grid, 256, 0, s>>>(h->st, h->keys, q, h->risk_pos, B, h->d, h->part_min, h->part_arg,
-                                                            h->d_risk, h->d_intra, mode, h->risk_slot, h->pfail_list);
-    else
-        probe_kernel<kProbeColsWide, 32><<<grid, 256, 0, s>>>(h->st, h->keys, q, h->risk_pos, B, h->d, h->part_min, h->part_arg,
-                                                          h->d_risk, h->d_intra, mode, h->risk_slot, h->pfail_list);
+    auto kern = PC == kProbeColsNarrow ? (metric_is_ip(h) ? probe_kernel<kProbeColsNarrow, 64, true> : probe_kernel<kProbeColsNarrow, 64, false>)
+                                       : (metric_is_ip(h) ? probe_kernel<kProbeColsWide, 32, true> : probe_kernel<kProbeColsWide, 32, false>);
+    kern<<<grid, 256, 0, s>>>(h->st, h->keys, q, h->risk_pos, B, h->d, h->part_min, h->part_arg, h->d_risk, h->d_intra, mode,
+                              h->risk_slot, h->pfail_list);
     h->launches++;
 }
 

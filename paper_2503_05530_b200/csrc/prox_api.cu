@@ -84,7 +84,7 @@ static bool dev_alloc(T *&p, size_t n) {
 }
 
 static void free_all(prox_handle *h) {
-    void *ptrs[] = {h->redo, h->corpus_own, h->qn, h->planes, h->bucket_count, h->lsh_code, h->lsh_order, h->lsh_seg, h->lsh_work, h->xb, h->xh, h->keys, h->val_ids, h->val_dists, h->stamp, h->risk_pos, h->st,
+    void *ptrs[] = {h->over_list, h->over_d, h->over_id, h->over_ticket, h->redo, h->corpus_own, h->qn, h->planes, h->bucket_count, h->lsh_code, h->lsh_order, h->lsh_seg, h->lsh_work, h->xb, h->xh, h->keys, h->val_ids, h->val_dists, h->stamp, h->risk_pos, h->st,
                     h->risk_slot, h->risk_stamp, h->part_min, h->part_arg, h->d_risk, h->d_intra,
                     h->safe_min, h->safe_arg, h->cand_d, h->cand_code, h->n_cand, h->src, h->src_kind,
                     h->ins_slot, h->evt_slot, h->evt_dist, h->miss_list, h->miss_rank, h->qb, h->qbn,
@@ -110,8 +110,17 @@ extern "C" prox_handle *prox_create(const float *corpus, int64_t N, int32_t d, i
     return prox_create_rho(corpus, N, d, k, capacity, tau, policy, 1);
 }
 
+static prox_handle *create_handle(const float *corpus, int64_t N, int32_t d, int32_t k_out, int64_t capacity, float tau,
+                                  int32_t policy, int32_t rho, int32_t metric);
+
 extern "C" prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t d, int32_t k_out,
                                         int64_t capacity, float tau, int32_t policy, int32_t rho) {
+    return create_handle(corpus, N, d, k_out, capacity, tau, policy, rho, PROX_METRIC_L2SQ);
+}
+
+// metric: PROX_METRIC_L2SQ (also the machinery under the cosine distance) or PROX_METRIC_IP.
+static prox_handle *create_handle(const float *corpus, int64_t N, int32_t d, int32_t k_out, int64_t capacity, float tau,
+                                  int32_t policy, int32_t rho, int32_t metric) {
     g_err[0] = 0;
     if (rho < 1) { set_err("rho must be >= 1"); return nullptr; }
     if (k_out < 1 || k_out > kMaxK || k_out > N) { set_err("k must be in [1, min(N, %d)]", kMaxK); return nullptr; }
@@ -124,13 +133,18 @@ extern "C" prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t 
     if (N < 1 || N >= (1LL << 31)) { set_err("N must be in [1, 2^31)"); return nullptr; }
     if (d < 16 || d > 4096 || d % 16) { set_err("d must be a multiple of 16 in [16, 4096]"); return nullptr; }
     if (capacity < 1 || capacity >= (1LL << 31)) { set_err("capacity must be in [1, 2^31)"); return nullptr; }
-    if (!(tau >= 0.f) || std::isinf(tau)) { set_err("tau must be finite and >= 0"); return nullptr; }
+    if (metric == PROX_METRIC_IP) {
+        if (std::isnan(tau) || std::isinf(tau)) { set_err("tau must be finite"); return nullptr; }
+    } else if (!(tau >= 0.f) || std::isinf(tau)) {
+        set_err("tau must be finite and >= 0");
+        return nullptr;
+    }
     if (policy != PROX_LRU && policy != PROX_FIFO) { set_err("policy must be PROX_LRU or PROX_FIFO"); return nullptr; }
 
     prox_handle *h = new (std::nothrow) prox_handle();
     if (!h) { set_err("out of host memory"); return nullptr; }
     std::memset(h, 0, sizeof(*h));
-    h->corpus = corpus; h->N = N; h->d = d; h->k = k; h->k_out = k_out; h->rho = rho; h->lsh_L = -1; h->C = capacity; h->tau = tau; h->policy = policy;
+    h->corpus = corpus; h->N = N; h->d = d; h->k = k; h->k_out = k_out; h->rho = rho; h->lsh_L = -1; h->C = capacity; h->tau = tau; h->policy = policy; h->metric = metric;
     h->kp = 4 * k < 64 ? 64 : (4 * k > kMaxKp ? kMaxKp : 4 * k);
     h->scan_mode = PROX_SCAN_AUTO;
     cudaDeviceProp prop;
@@ -173,8 +187,11 @@ extern "C" prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t 
     ok = ok && dev_alloc(h->res_ids, MB * k) && dev_alloc(h->res_dists, MB * k);
     ok = ok && dev_alloc(h->fail_list, MB) && dev_alloc(h->fail_radius, MB);
     ok = ok && dev_alloc(h->coll_id, MB * kCollectCap) && dev_alloc(h->coll_n, MB) && dev_alloc(h->redo, MB + 1);
+    ok = ok && dev_alloc(h->over_list, MB) && dev_alloc(h->over_d, (size_t)kOverMax * P * k) &&
+         dev_alloc(h->over_id, (size_t)kOverMax * P * k) && dev_alloc(h->over_ticket, (size_t)kOverMax);
     // caches of a few thousand keys and more are probed on the tensor cores first (bf16 copies of the keys)
-    h->probe_tc = (d % 64 == 0 && capacity >= 4096) ? 1 : 0;
+    // (the coarse probe's certificate is written for the Euclidean distance)
+    h->probe_tc = (d % 64 == 0 && capacity >= 4096 && metric != PROX_METRIC_IP) ? 1 : 0;
     ok = ok && dev_alloc(h->use_partial, MB) && dev_alloc(h->pfail_list, MB);
     if (h->probe_tc) {
         ok = ok && dev_alloc(h->keys_b, C * d) && dev_alloc(h->kh, C);
@@ -195,6 +212,7 @@ extern "C" prox_handle *prox_create_rho(const float *corpus, int64_t N, int32_t 
         cudaMemset(h->keys_b, 0, C * d * sizeof(__nv_bfloat16));
     }
     cudaMemset(h->buf_cnt, 0, 4 * P * kScanQ * sizeof(int32_t));
+    cudaMemset(h->over_ticket, 0, kOverMax * sizeof(unsigned));
     launch_convert_corpus(h, 0);
     launch_reset(h, 0);
     init_scan_tc(h);
@@ -212,7 +230,8 @@ extern "C" prox_handle *prox_create_metric(const float *corpus, int64_t N, int32
                                            float tau, int32_t policy, int32_t rho, int32_t metric) {
     g_err[0] = 0;
     if (metric == PROX_METRIC_L2SQ) return prox_create_rho(corpus, N, d, k, capacity, tau, policy, rho);
-    if (metric != PROX_METRIC_COSINE) { set_err("metric must be PROX_METRIC_L2SQ or PROX_METRIC_COSINE"); return nullptr; }
+    if (metric == PROX_METRIC_IP) return create_handle(corpus, N, d, k, capacity, tau, policy, rho, PROX_METRIC_IP);
+    if (metric != PROX_METRIC_COSINE) { set_err("metric must be PROX_METRIC_L2SQ, PROX_METRIC_COSINE or PROX_METRIC_IP"); return nullptr; }
     if (!corpus) { set_err("corpus is NULL"); return nullptr; }
     if (N < 1 || N >= (1LL << 31) || d < 16 || d > 4096 || d % 16) { set_err("N or d out of range"); return nullptr; }
     if (!(tau >= 0.f) || std::isinf(tau)) { set_err("tau must be finite and >= 0"); return nullptr; }

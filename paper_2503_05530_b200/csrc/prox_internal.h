@@ -16,6 +16,7 @@ constexpr int kScanQ = 256;                  // queries per scan pass (MMA N dim
 constexpr int kTileRows = 128;               // corpus rows per scan tile (MMA M dimension)
 constexpr int kBufCap = 512;                 // entries of one (CTA, query) candidate buffer
 constexpr int kCollectCap = 2048;            // rows the exact pass may collect per query
+constexpr int kOverMax = 64;                 // queries per batch whose collection may overflow and still be answered exactly
 constexpr int kProbeSplitMax = 64;           // column splits of the probe grid
 constexpr int kProbeKp = 64;                 // slots per query the coarse probe keeps for the exact recheck
 
@@ -33,6 +34,7 @@ struct DevState {
     float kn_max;             // upper bound of |bf16(key)| over those keys
     int n_probe;              // queries of the current batch (read by the coarse probe's kernels)
     int n_pfail;              // queries whose coarse probe was not certified
+    int n_over;               // queries whose exact pass collected more rows than it can hold
     // statistics
     long long queries, hits, misses, intra_hits, evictions, scan_batches, uncertified,
         fallback_rows, unresolved, probe_uncertified;
@@ -137,6 +139,10 @@ struct prox_handle {
     int32_t *coll_id;                 // kMaxBatch x kCollectCap (indexed by position in fail_list)
     int32_t *coll_n;                  // kMaxBatch
     int32_t *redo;                    // kMaxBatch + 1: queries the fp32 sweep of the exact pass takes again; [kMaxBatch] any
+    int32_t *over_list;               // kMaxBatch: places in fail_list of the queries whose collection overflowed
+    double *over_d;                   // kOverMax x blocks x k: every block's nearest rows of its share of the corpus
+    int32_t *over_id;                 // kOverMax x blocks x k
+    unsigned *over_ticket;            // kOverMax: blocks that have delivered their list (back to 0 after the merge)
 
     // staging for the host-buffer entry point
     float *stage_q;
@@ -151,6 +157,7 @@ void set_cache_kernel_attributes();
 void set_scan_kernel_attributes();
 // create-time kernels
 void launch_convert_corpus(prox_handle *h, cudaStream_t s);
+inline bool metric_is_ip(const prox_handle *h) { return h->metric == PROX_METRIC_IP; }
 // cache kernels
 void launch_risk_select(prox_handle *h, int B, cudaStream_t s);
 void launch_probe(prox_handle *h, const float *q, int B, int mode, cudaStream_t s);   // 0 all slots, 1 at-risk + batch, 2 failed queries

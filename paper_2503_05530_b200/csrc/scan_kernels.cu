@@ -29,7 +29,7 @@ namespace prox {
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 convert_corpus_kernel(const float *__restrict__ x, long long N, int d, __nv_bfloat16 *__restrict__ xb,
-                      float *__restrict__ xh, DevState *st) {
+                      float *__restrict__ xh, DevState *st, int ip) {
     const int lane = threadIdx.x & 31;
     const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
@@ -57,7 +57,7 @@ convert_corpus_kernel(const float *__restrict__ x, long long N, int d, __nv_bflo
             nn += __shfl_xor_sync(0xffffffffu, nn, m);
             ee += __shfl_xor_sync(0xffffffffu, ee, m);
         }
-        if (lane == 0) xh[r] = 0.5f * nn;
+        if (lane == 0) xh[r] = ip ? 0.f : 0.5f * nn;      // inner product: the coarse score is the product alone
         emax = fmaxf(emax, ee);
         nmax = fmaxf(nmax, nn);
     }
@@ -86,6 +86,7 @@ prep_miss_kernel(DevState *st, const float *__restrict__ queries, int B, int d,
         }
         if (tid == 0) {
             st->n_fail = 0;
+            st->n_over = 0;
             if (n_miss > 0) st->scan_batches++;
         }
     }
@@ -381,6 +382,18 @@ __device__ __forceinline__ double exact_sqdist_warp(const float *__restrict__ q_
     return acc;
 }
 
+// The distance of the handle's metric in fp64: squared Euclidean, or -(q . x) for the inner product.
+__device__ __forceinline__ double exact_dist_warp(const float *__restrict__ q_sm, const float *__restrict__ x, int d,
+                                                  int ip) {
+    if (!ip) return exact_sqdist_warp(q_sm, x, d);
+    const int lane = threadIdx.x & 31;
+    double acc = 0.0;
+    for (int j = lane; j < d; j += 32) acc = fma((double)q_sm[j], (double)x[j], acc);
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, m);
+    return -acc;
+}
+
 constexpr int kRerankMax = kCollectCap;            // entries the sort buffers hold
 
 // mode 0: candidates of the coarse scan (+ certificate); mode 1: rows collected by the exact pass
@@ -390,7 +403,8 @@ rerank_kernel(DevState *st, int mode, const float *__restrict__ corpus, const fl
               const int32_t *__restrict__ cand_id, const int32_t *__restrict__ cand_n,
               const float *__restrict__ cand_sk, const float *__restrict__ qbn,
               const float *__restrict__ qerr, int32_t *res_ids, double *res_dists, int32_t *fail_list,
-              float *fail_radius, const int32_t *__restrict__ coll_id, const int32_t *__restrict__ coll_n) {
+              float *fail_radius, const int32_t *__restrict__ coll_id, const int32_t *__restrict__ coll_n, int ip,
+              int32_t *over_list) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *sd = reinterpret_cast<double *>(smem_raw);                 // kRerankMax
     int *sid = reinterpret_cast<int *>(sd + kRerankMax);               // kRerankMax
@@ -409,9 +423,9 @@ rerank_kernel(DevState *st, int mode, const float *__restrict__ corpus, const fl
         if (f >= st->n_fail) return;
         m = fail_list[f];
         n = coll_n[f];
-        if (n > kCollectCap) {
-            n = kCollectCap;
-            if (tid == 0) atomicAdd((u64 *)&st->unresolved, 1ull);
+        if (n > kCollectCap) {                     // more rows inside the radius than the collection holds:
+            if (tid == 0) over_list[atomicAdd(&st->n_over, 1)] = f;      // answered by the streaming pass below
+            return;
         }
         if (tid == 0) atomicAdd((u64 *)&st->fallback_rows, (u64)n);
         ids = coll_id + (size_t)f * kCollectCap;
@@ -425,7 +439,7 @@ rerank_kernel(DevState *st, int mode, const float *__restrict__ corpus, const fl
     // one candidate row per warp at a time: the gathers are bound by latency, so the block is wide
     for (int c = warp; c < n; c += (int)(blockDim.x >> 5)) {
         const int row = ids[c];
-        const double v = exact_sqdist_warp(q_sm, corpus + (size_t)row * d, d);
+        const double v = exact_dist_warp(q_sm, corpus + (size_t)row * d, d, ip);
         if (lane == 0) { sd[c] = v; sid[c] = row; }
     }
     block_sort_asc(sd, sid, n2);
@@ -446,16 +460,25 @@ rerank_kernel(DevState *st, int mode, const float *__restrict__ corpus, const fl
             const double qn = sqrt((double)qbn[m]), xn = (double)st->xn_max;
             const double slack = 4.0 * (double)(d + 16) * 5.9604644775390625e-08 *
                                  (2.0 * qn * xn + xn * xn + qn * qn);
-            const double cprime = (double)qbn[m] - 2.0 * (double)sk - slack;
-            const double g = (double)qerr[m] + (double)st->e_max;
-            const double root = cprime > 0.0 ? sqrt(cprime) : 0.0;
-            const double lower = root > g ? (root - g) * (root - g) : 0.0;
-            certified = sd[k - 1] < lower;
+            if (ip) {
+                // inner product: q.x = bf16(q).bf16(x) + (q - bf16 q).x + bf16(q).(x - bf16 x), and no
+                // outside row has a coarse product above sk: q.x <= sk + a |x| + |bf16 q| e + slack
+                const double a = (double)qerr[m], e = (double)st->e_max;
+                const double upper = (double)sk + a * (xn + e) + qn * e + slack;
+                certified = sd[k - 1] < -upper;
+            } else {
+                const double cprime = (double)qbn[m] - 2.0 * (double)sk - slack;
+                const double g = (double)qerr[m] + (double)st->e_max;
+                const double root = cprime > 0.0 ? sqrt(cprime) : 0.0;
+                const double lower = root > g ? (root - g) * (root - g) : 0.0;
+                certified = sd[k - 1] < lower;
+            }
         }
         if (!certified) {
             const int f = atomicAdd(&st->n_fail, 1);
             fail_list[f] = m;
-            fail_radius[f] = (float)sd[k - 1] * (1.f + 1e-6f) + 1e-30f;   // rounded up
+            const float rk = (float)sd[k - 1];
+            fail_radius[f] = rk + fabsf(rk) * 1e-6f + 1e-30f;             // rounded up (the value may be negative)
             atomicAdd((u64 *)&st->uncertified, 1ull);
         }
     }
@@ -473,7 +496,7 @@ hit_rerank_kernel(int B, int d, int k, int k_out, int kind, const float *__restr
                   const float *__restrict__ queries, const int32_t *__restrict__ src,
                   const int32_t *__restrict__ src_kind, const int32_t *__restrict__ miss_rank,
                   const int32_t *__restrict__ val_ids, const int32_t *__restrict__ res_ids, int64_t *out_ids,
-                  float *out_dists) {
+                  float *out_dists, int ip) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *sd = reinterpret_cast<double *>(smem_raw);                 // kMaxFetch
     int *sid = reinterpret_cast<int *>(sd + kMaxFetch);                // kMaxFetch
@@ -489,7 +512,7 @@ hit_rerank_kernel(int B, int d, int k, int k_out, int kind, const float *__restr
     for (int c = warp; c < k; c += 8) {
         const int row = ids[c];
         if (row < 0) continue;
-        const double v = exact_sqdist_warp(q_sm, corpus + (size_t)row * d, d);
+        const double v = exact_dist_warp(q_sm, corpus + (size_t)row * d, d, ip);
         if (lane == 0) { sd[c] = v; sid[c] = row; }
     }
     block_sort_asc(sd, sid, n2);
@@ -502,17 +525,19 @@ hit_rerank_kernel(int B, int d, int k, int k_out, int kind, const float *__restr
 
 // ------------------------------------------------------------------------------------------
 // Exact pass for uncertified queries: every corpus row within the radius (the exact k-th
-// candidate distance) in fp32 difference form, with the fp32 rounding margin on top.
-// Eight queries per sweep of the corpus; one warp per row.
+// candidate distance) in fp32 difference form (inner product: fp32 sum of products, negated),
+// with the fp32 rounding margin on top.  Eight queries per sweep of the corpus; one warp per row.
+// `limit` holds, per query of the group, the largest fp32 value that is still collected (radius
+// and margins folded in by the caller; -inf for an empty place in the group).
 // ------------------------------------------------------------------------------------------
 constexpr int kFallbackGroup = 8;
 
 // Rows warp, warp + nwarps, ... of the corpus against NG queries held in shared memory (NG is the
 // number of queries actually in the group, rounded up to 1, 2, 4 or 8, so that a lone failing
 // query costs one query's arithmetic and the pass stays bound by the corpus read).
-template <int NG>
+template <int NG, bool IP>
 __device__ __forceinline__ void fallback_rows(const float *__restrict__ corpus, long long N, int d, long long warp,
-                                              long long nwarps, const float *q_sm, const float *radius, float margin,
+                                              long long nwarps, const float *q_sm, const float *limit,
                                               int32_t *coll_id, int32_t *coll_n, int g0) {
     const int lane = threadIdx.x & 31;
     for (long long r = warp; r < N; r += nwarps) {
@@ -525,8 +550,12 @@ __device__ __forceinline__ void fallback_rows(const float *__restrict__ corpus, 
 #pragma unroll
             for (int f = 0; f < NG; ++f) {
                 const float4 qv = *reinterpret_cast<const float4 *>(&q_sm[f * d + 4 * j]);
-                const float d0 = qv.x - xv.x, d1 = qv.y - xv.y, d2 = qv.z - xv.z, d3 = qv.w - xv.w;
-                acc[f] = fmaf(d0, d0, fmaf(d1, d1, fmaf(d2, d2, fmaf(d3, d3, acc[f]))));
+                if constexpr (IP) {
+                    acc[f] = fmaf(-qv.x, xv.x, fmaf(-qv.y, xv.y, fmaf(-qv.z, xv.z, fmaf(-qv.w, xv.w, acc[f]))));
+                } else {
+                    const float d0 = qv.x - xv.x, d1 = qv.y - xv.y, d2 = qv.z - xv.z, d3 = qv.w - xv.w;
+                    acc[f] = fmaf(d0, d0, fmaf(d1, d1, fmaf(d2, d2, fmaf(d3, d3, acc[f]))));
+                }
             }
         }
 #pragma unroll
@@ -538,8 +567,7 @@ __device__ __forceinline__ void fallback_rows(const float *__restrict__ corpus, 
 #pragma unroll
             for (int f = 0; f < NG; ++f)
                 if (f == lane) mine = acc[f];
-            const float rad = radius[lane];                        // -1 for an empty place in the group
-            if (mine <= rad * (1.f + margin) + 1e-30f) {
+            if (mine <= limit[lane]) {
                 const int pos = atomicAdd(&coll_n[g0 + lane], 1);
                 if (pos < kCollectCap) coll_id[(size_t)(g0 + lane) * kCollectCap + pos] = (int32_t)r;
             }
@@ -550,10 +578,10 @@ __device__ __forceinline__ void fallback_rows(const float *__restrict__ corpus, 
 // The same sweep over the bf16 copy of the corpus (half the bytes): |sqrt(coarse) - sqrt(exact)| is
 // at most the rounding error of the row, so the caller passes radii widened by that error and
 // every row within the exact radius is still collected (a few more with it).
-template <int NG>
+template <int NG, bool IP>
 __device__ __forceinline__ void fallback_rows_bf16(const __nv_bfloat16 *__restrict__ xb, long long N, int d,
                                                    long long warp, long long nwarps, const float *q_sm,
-                                                   const float *radius, float margin, int32_t *coll_id,
+                                                   const float *limit, int32_t *coll_id,
                                                    int32_t *coll_n, int g0) {
     constexpr int U = NG <= 2 ? 4 : 2;                 // rows in flight per warp: the sweep is bound by load latency
     const int lane = threadIdx.x & 31;
@@ -577,12 +605,19 @@ __device__ __forceinline__ void fallback_rows_bf16(const __nv_bfloat16 *__restri
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     const uint32_t ww[4] = {w[u].x, w[u].y, w[u].z, w[u].w};   // eight bf16
-                    const float d0 = qa.x - __uint_as_float(ww[0] << 16), d1 = qa.y - __uint_as_float(ww[0] & 0xffff0000u);
-                    const float d2 = qa.z - __uint_as_float(ww[1] << 16), d3 = qa.w - __uint_as_float(ww[1] & 0xffff0000u);
-                    const float d4 = qb2.x - __uint_as_float(ww[2] << 16), d5 = qb2.y - __uint_as_float(ww[2] & 0xffff0000u);
-                    const float d6 = qb2.z - __uint_as_float(ww[3] << 16), d7 = qb2.w - __uint_as_float(ww[3] & 0xffff0000u);
-                    const float a = fmaf(d0, d0, fmaf(d1, d1, fmaf(d2, d2, fmaf(d3, d3, acc[u][f]))));
-                    acc[u][f] = fmaf(d4, d4, fmaf(d5, d5, fmaf(d6, d6, fmaf(d7, d7, a))));
+                    const float x0 = __uint_as_float(ww[0] << 16), x1 = __uint_as_float(ww[0] & 0xffff0000u);
+                    const float x2 = __uint_as_float(ww[1] << 16), x3 = __uint_as_float(ww[1] & 0xffff0000u);
+                    const float x4 = __uint_as_float(ww[2] << 16), x5 = __uint_as_float(ww[2] & 0xffff0000u);
+                    const float x6 = __uint_as_float(ww[3] << 16), x7 = __uint_as_float(ww[3] & 0xffff0000u);
+                    if constexpr (IP) {
+                        const float a = fmaf(-qa.x, x0, fmaf(-qa.y, x1, fmaf(-qa.z, x2, fmaf(-qa.w, x3, acc[u][f]))));
+                        acc[u][f] = fmaf(-qb2.x, x4, fmaf(-qb2.y, x5, fmaf(-qb2.z, x6, fmaf(-qb2.w, x7, a))));
+                    } else {
+                        const float d0 = qa.x - x0, d1 = qa.y - x1, d2 = qa.z - x2, d3 = qa.w - x3;
+                        const float d4 = qb2.x - x4, d5 = qb2.y - x5, d6 = qb2.z - x6, d7 = qb2.w - x7;
+                        const float a = fmaf(d0, d0, fmaf(d1, d1, fmaf(d2, d2, fmaf(d3, d3, acc[u][f]))));
+                        acc[u][f] = fmaf(d4, d4, fmaf(d5, d5, fmaf(d6, d6, fmaf(d7, d7, a))));
+                    }
                 }
             }
         }
@@ -598,8 +633,7 @@ __device__ __forceinline__ void fallback_rows_bf16(const __nv_bfloat16 *__restri
 #pragma unroll
                 for (int f = 0; f < NG; ++f)
                     if (f == lane) mine = acc[u][f];
-                const float rad = radius[lane];                    // -1 for an empty place in the group
-                if (mine <= rad * (1.f + margin) + 1e-30f) {
+                if (mine <= limit[lane]) {
                     const int pos = atomicAdd(&coll_n[g0 + lane], 1);
                     if (pos < kCollectCap) coll_id[(size_t)(g0 + lane) * kCollectCap + pos] = (int32_t)r;
                 }
@@ -623,15 +657,25 @@ fallback_mark_kernel(const DevState *st, int32_t *coll_n, int32_t *redo) {
     if (f == 0) redo[kMaxBatch] = any;
 }
 
+template <int NG, bool IP>
+__device__ __forceinline__ void fallback_sweep(const float *__restrict__ corpus, const __nv_bfloat16 *__restrict__ xb,
+                                               long long N, int d, long long warp, long long nwarps, const float *q_sm,
+                                               const float *limit, int32_t *coll_id, int32_t *coll_n, int g0) {
+    if (xb != nullptr) fallback_rows_bf16<NG, IP>(xb, N, d, warp, nwarps, q_sm, limit, coll_id, coll_n, g0);
+    else fallback_rows<NG, IP>(corpus, N, d, warp, nwarps, q_sm, limit, coll_id, coll_n, g0);
+}
+
+template <bool IP>
 __global__ void __launch_bounds__(256)
 fallback_collect_kernel(DevState *st, const float *__restrict__ corpus, const __nv_bfloat16 *__restrict__ xb,
                         const int32_t *__restrict__ redo,
                         const float *__restrict__ queries, long long N, int d, const int32_t *__restrict__ miss_list,
                         const int32_t *__restrict__ fail_list, const float *__restrict__ fail_radius,
+                        const float *__restrict__ qbn, const float *__restrict__ qerr,
                         int32_t *coll_id, int32_t *coll_n) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *q_sm = reinterpret_cast<float *>(smem_raw);                  // kFallbackGroup x d
-    __shared__ float radius[kFallbackGroup];
+    __shared__ float limit[kFallbackGroup];
     const int n_fail = st->n_fail;
     if (n_fail == 0) return;
     if (redo != nullptr && redo[kMaxBatch] == 0) return;                // second sweep: nothing overflowed
@@ -648,26 +692,148 @@ fallback_collect_kernel(DevState *st, const float *__restrict__ corpus, const __
             q_sm[idx] = (f < ng) ? queries[(size_t)miss_list[fail_list[g0 + f]] * d + j] : 0.f;
         }
         if (tid < kFallbackGroup) {
-            float rad = (tid < ng) ? fail_radius[g0 + tid] : -1.f;
-            if (redo != nullptr && tid < ng && redo[g0 + tid] == 0) rad = -1.f;   // settled by the first sweep
-            if (xb != nullptr && rad >= 0.f) {                     // widened by the rows' rounding error, rounded up
-                const float w = sqrtf(rad) * (1.f + 2e-7f) + st->e_max * (1.f + 2e-7f);
-                rad = w * w * (1.f + 2e-7f);
+            bool live = tid < ng;
+            if (redo != nullptr && live && redo[g0 + tid] == 0) live = false;   // settled by the first sweep
+            float lim = -INFINITY;
+            if (live) {
+                const float rad = fail_radius[g0 + tid];
+                if constexpr (IP) {
+                    // |q| (|x| + e) bounds the sum of |q_j x_j|: margin times it covers the fp32 sum; over the
+                    // bf16 copy the row's rounding error moves the product by at most |q| e_max more
+                    const int m = fail_list[g0 + tid];
+                    const float qn = (sqrtf(qbn[m]) + qerr[m]) * (1.f + 2e-7f);
+                    const float xn = (st->xn_max + st->e_max) * (1.f + 2e-7f);
+                    lim = rad + margin * qn * xn * (1.f + 2e-7f) + 1e-30f;
+                    if (xb != nullptr) lim += qn * st->e_max * (1.f + 4e-7f);
+                } else if (xb != nullptr) {                        // widened by the rows' rounding error, rounded up
+                    const float w = sqrtf(rad) * (1.f + 2e-7f) + st->e_max * (1.f + 2e-7f);
+                    lim = w * w * (1.f + 2e-7f) * (1.f + margin) + 1e-30f;
+                } else {
+                    lim = rad * (1.f + margin) + 1e-30f;
+                }
             }
-            radius[tid] = rad;
+            limit[tid] = lim;
         }
         __syncthreads();
-        if (xb != nullptr) {
-            if (ng == 1) fallback_rows_bf16<1>(xb, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
-            else if (ng == 2) fallback_rows_bf16<2>(xb, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
-            else if (ng <= 4) fallback_rows_bf16<4>(xb, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
-            else fallback_rows_bf16<8>(xb, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
-            continue;
+        if (ng == 1) fallback_sweep<1, IP>(corpus, xb, N, d, warp, nwarps, q_sm, limit, coll_id, coll_n, g0);
+        else if (ng == 2) fallback_sweep<2, IP>(corpus, xb, N, d, warp, nwarps, q_sm, limit, coll_id, coll_n, g0);
+        else if (ng <= 4) fallback_sweep<4, IP>(corpus, xb, N, d, warp, nwarps, q_sm, limit, coll_id, coll_n, g0);
+        else fallback_sweep<8, IP>(corpus, xb, N, d, warp, nwarps, q_sm, limit, coll_id, coll_n, g0);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Last resort of the exact pass: a query with more rows inside its radius than the collection
+// holds (thousands of copies of one row next to the query, say).  Every block walks its own
+// contiguous share of the corpus, measures every row exactly (fp64) and keeps the rows that are
+// still among its k nearest by (distance, row id) in a shared-memory buffer that is sorted and
+// cut to k whenever it fills up; the block that delivers its list last merges all lists the same
+// way and writes the answer.  No row is ever dropped unseen, so the result is exact whatever the
+// number of ties.  Queries are taken one after the other (up to kOverMax per batch); the pass
+// costs one reading of the fp32 corpus per query and runs for pathological inputs only.
+// ------------------------------------------------------------------------------------------
+constexpr int kOverBuf = 4096;
+
+// Sorts the n entries of the buffer by (distance, row) and keeps the first k; returns how many stay.
+__device__ int over_compact(double *bd, int *bid, int n, int k) {
+    for (int e = n + threadIdx.x; e < kOverBuf; e += blockDim.x) { bd[e] = INFINITY; bid[e] = 0x7fffffff; }
+    block_sort_asc(bd, bid, kOverBuf);
+    return n < k ? n : k;
+}
+
+template <bool IP>
+__global__ void __launch_bounds__(1024)
+overflow_topk_kernel(DevState *st, const float *__restrict__ corpus, const float *__restrict__ queries, long long N,
+                     int d, int k, const int32_t *__restrict__ miss_list, const int32_t *__restrict__ fail_list,
+                     const float *__restrict__ fail_radius, const int32_t *__restrict__ over_list, double *over_d,
+                     int32_t *over_id, unsigned *over_ticket, int32_t *res_ids, double *res_dists) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *bd = reinterpret_cast<double *>(smem_raw);                 // kOverBuf
+    int *bid = reinterpret_cast<int *>(bd + kOverBuf);                 // kOverBuf
+    float *q_sm = reinterpret_cast<float *>(bid + kOverBuf);           // d
+    __shared__ int s_cnt;
+    __shared__ unsigned s_last;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    int n_over = st->n_over;
+    if (n_over == 0) return;
+    if (n_over > kOverMax) {                   // beyond what the lists hold: those queries stay unanswered, and say so
+        if (blockIdx.x == 0 && tid == 0) {
+            atomicAdd((u64 *)&st->unresolved, (u64)(n_over - kOverMax));
+            atomicCAS(&st->error, 0, PROX_ERR_INTERNAL);
         }
-        if (ng == 1) fallback_rows<1>(corpus, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
-        else if (ng == 2) fallback_rows<2>(corpus, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
-        else if (ng <= 4) fallback_rows<4>(corpus, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
-        else fallback_rows<8>(corpus, N, d, warp, nwarps, q_sm, radius, margin, coll_id, coll_n, g0);
+        n_over = kOverMax;
+    }
+    const long long per = (N + gridDim.x - 1) / gridDim.x;
+    const long long r0 = (long long)blockIdx.x * per, r1 = r0 + per < N ? r0 + per : N;
+
+    for (int o = 0; o < n_over; ++o) {
+        const int f = over_list[o], m = fail_list[f];
+        __syncthreads();
+        for (int j = tid; j < d; j += blockDim.x) q_sm[j] = queries[(size_t)miss_list[m] * d + j];
+        if (tid == 0) s_cnt = 0;
+        // a row counts while (distance, row) <= (bound_d, bound_id): first the radius, then the block's k-th nearest
+        double bound_d = (double)fail_radius[f];
+        int bound_id = 0x7fffffff;
+        __syncthreads();
+        for (long long base = r0; base < r1; base += nwarps) {
+            const long long row = base + warp;
+            if (row < r1) {
+                const double v = exact_dist_warp(q_sm, corpus + (size_t)row * d, d, IP ? 1 : 0);
+                if (lane == 0 && (v < bound_d || (v == bound_d && (int)row <= bound_id))) {
+                    const int pos = atomicAdd(&s_cnt, 1);
+                    bd[pos] = v;
+                    bid[pos] = (int)row;
+                }
+            }
+            __syncthreads();
+            const int n = s_cnt;
+            if (n > kOverBuf - nwarps) {       // the next round could overflow: sort, keep k, tighten the bound
+                const int keep = over_compact(bd, bid, n, k);
+                if (keep == k) { bound_d = bd[k - 1]; bound_id = bid[k - 1]; }
+                __syncthreads();
+                if (tid == 0) s_cnt = keep;
+                __syncthreads();
+            }
+        }
+        const int mine = over_compact(bd, bid, s_cnt, k);
+        double *my_d = over_d + ((size_t)o * gridDim.x + blockIdx.x) * k;
+        int32_t *my_id = over_id + ((size_t)o * gridDim.x + blockIdx.x) * k;
+        for (int e = tid; e < k; e += blockDim.x) {
+            my_d[e] = e < mine ? bd[e] : INFINITY;
+            my_id[e] = e < mine ? bid[e] : -1;
+        }
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) s_last = (atomicAdd(&over_ticket[o], 1u) == gridDim.x - 1) ? 1u : 0u;
+        __syncthreads();
+        if (s_last) {                          // every block's list is in memory: merge them the same way
+            __threadfence();
+            int n = 0;
+            const int total = (int)gridDim.x * k;
+            for (int e0 = 0; e0 < total; e0 += kOverBuf - k) {
+                const int chunk = total - e0 < kOverBuf - k ? total - e0 : kOverBuf - k;
+                for (int e = tid; e < chunk; e += blockDim.x) {
+                    bd[n + e] = __ldcg(over_d + (size_t)o * total + e0 + e);
+                    const int id = __ldcg(over_id + (size_t)o * total + e0 + e);
+                    bid[n + e] = id < 0 ? 0x7fffffff : id;
+                }
+                __syncthreads();
+                n = over_compact(bd, bid, n + chunk, k);
+                __syncthreads();
+            }
+            if (n < k || bid[k - 1] == 0x7fffffff) {     // cannot happen: at least k rows lie inside the radius
+                if (tid == 0) atomicCAS(&st->error, 0, PROX_ERR_INTERNAL);
+            } else {
+                for (int r = tid; r < k; r += blockDim.x) {
+                    res_ids[(size_t)m * k + r] = bid[r];
+                    res_dists[(size_t)m * k + r] = bd[r];
+                }
+            }
+            if (tid == 0) {
+                over_ticket[o] = 0u;           // ready for the next batch
+                atomicAdd((u64 *)&st->fallback_rows, (u64)N);
+            }
+        }
     }
 }
 
@@ -774,7 +940,7 @@ probe_exact_kernel(DevState *st, const float *__restrict__ keys, const float *__
 // ------------------------------------------------------------------------------------------
 void launch_convert_corpus(prox_handle *h, cudaStream_t s) {
     convert_corpus_kernel<<<h->num_sms * 8, 256, 0, s>>>(h->corpus, (long long)h->N, h->d, h->xb, h->xh,
-                                                         h->st);
+                                                         h->st, metric_is_ip(h) ? 1 : 0);
     h->launches++;
 }
 
@@ -814,14 +980,17 @@ static size_t rerank_smem(int d) { return (size_t)kRerankMax * 12 + (size_t)d * 
 void set_scan_kernel_attributes() {
     cudaFuncSetAttribute(merge_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeStageMax * 8);
     cudaFuncSetAttribute(rerank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rerank_smem(4096));
-    cudaFuncSetAttribute(fallback_collect_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFallbackGroup * 4096 * 4);
+    cudaFuncSetAttribute(fallback_collect_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFallbackGroup * 4096 * 4);
+    cudaFuncSetAttribute(fallback_collect_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFallbackGroup * 4096 * 4);
+    cudaFuncSetAttribute(overflow_topk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOverBuf * 12 + 4096 * 4);
+    cudaFuncSetAttribute(overflow_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOverBuf * 12 + 4096 * 4);
 }
 
 void launch_rerank(prox_handle *h, const float *q, int B, cudaStream_t s) {
     rerank_kernel<<<B, 1024, rerank_smem(h->d), s>>>(h->st, 0, h->corpus, q, h->d, h->k, (long long)h->N,
                                                     h->miss_list, h->cand_id, h->cand_n, h->cand_sk, h->qbn,
                                                     h->qerr, h->res_ids, h->res_dists, h->fail_list,
-                                                    h->fail_radius, h->coll_id, h->coll_n);
+                                                    h->fail_radius, h->coll_id, h->coll_n, metric_is_ip(h) ? 1 : 0, h->over_list);
     h->launches++;
 }
 
@@ -829,24 +998,32 @@ void launch_hit_rerank(prox_handle *h, const float *q, int B, int kind, int64_t 
                        cudaStream_t s) {
     const size_t smem = (size_t)kMaxFetch * 12 + (size_t)h->d * 4;
     hit_rerank_kernel<<<B, 256, smem, s>>>(B, h->d, h->k, h->k_out, kind, h->corpus, q, h->src, h->src_kind,
-                                           h->miss_rank, h->val_ids, h->res_ids, out_ids, out_dists);
+                                           h->miss_rank, h->val_ids, h->res_ids, out_ids, out_dists,
+                                           metric_is_ip(h) ? 1 : 0);
     h->launches++;
 }
 
 void launch_fallback(prox_handle *h, const float *q, int B, cudaStream_t s) {
-    fallback_collect_kernel<<<h->num_sms * 4, 256, (size_t)kFallbackGroup * h->d * 4, s>>>(
+    auto collect = metric_is_ip(h) ? fallback_collect_kernel<true> : fallback_collect_kernel<false>;
+    collect<<<h->num_sms * 4, 256, (size_t)kFallbackGroup * h->d * 4, s>>>(
         h->st, h->corpus, h->xb, nullptr, q, (long long)h->N, h->d, h->miss_list, h->fail_list, h->fail_radius,
-        h->coll_id, h->coll_n);
+        h->qbn, h->qerr, h->coll_id, h->coll_n);
     // the bf16 sweep reads half the bytes; what it cannot hold is swept again in fp32
     fallback_mark_kernel<<<1, 1024, 0, s>>>(h->st, h->coll_n, h->redo);
-    fallback_collect_kernel<<<h->num_sms * 4, 256, (size_t)kFallbackGroup * h->d * 4, s>>>(
+    collect<<<h->num_sms * 4, 256, (size_t)kFallbackGroup * h->d * 4, s>>>(
         h->st, h->corpus, nullptr, h->redo, q, (long long)h->N, h->d, h->miss_list, h->fail_list, h->fail_radius,
-        h->coll_id, h->coll_n);
+        h->qbn, h->qerr, h->coll_id, h->coll_n);
     h->launches += 3;
     rerank_kernel<<<B, 1024, rerank_smem(h->d), s>>>(h->st, 1, h->corpus, q, h->d, h->k, (long long)h->N,
                                                     h->miss_list, h->cand_id, h->cand_n, h->cand_sk, h->qbn,
                                                     h->qerr, h->res_ids, h->res_dists, h->fail_list,
-                                                    h->fail_radius, h->coll_id, h->coll_n);
+                                                    h->fail_radius, h->coll_id, h->coll_n, metric_is_ip(h) ? 1 : 0, h->over_list);
+    h->launches++;
+    // queries whose collection overflowed even in the fp32 sweep (returns at once when there is none)
+    auto over = metric_is_ip(h) ? overflow_topk_kernel<true> : overflow_topk_kernel<false>;
+    over<<<h->scan_ctas, 1024, (size_t)kOverBuf * 12 + (size_t)h->d * 4, s>>>(
+        h->st, h->corpus, q, (long long)h->N, h->d, h->k, h->miss_list, h->fail_list, h->fail_radius, h->over_list,
+        h->over_d, h->over_id, h->over_ticket, h->res_ids, h->res_dists);
     h->launches++;
 }
 

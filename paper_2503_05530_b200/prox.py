@@ -21,8 +21,9 @@ SCAN_AUTO, SCAN_CUDA_CORE, SCAN_TC_SINGLE = 0, 1, 2
 STAGES = ("risk_select", "probe", "candidates", "resolve", "gather", "prep_miss", "scan", "merge",
           "rerank", "exact_pass", "scatter")
 _POLICY = {"lru": LRU, "fifo": FIFO, LRU: LRU, FIFO: FIFO}
-METRIC_L2SQ, METRIC_COSINE = 0, 1
-_METRIC = {"l2": METRIC_L2SQ, "cosine": METRIC_COSINE, METRIC_L2SQ: METRIC_L2SQ, METRIC_COSINE: METRIC_COSINE}
+METRIC_L2SQ, METRIC_COSINE, METRIC_IP = 0, 1, 2
+_METRIC = {"l2": METRIC_L2SQ, "cosine": METRIC_COSINE, "ip": METRIC_IP, METRIC_L2SQ: METRIC_L2SQ,
+           METRIC_COSINE: METRIC_COSINE, METRIC_IP: METRIC_IP}
 
 
 class ProxError(RuntimeError):

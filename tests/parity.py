@@ -13,6 +13,7 @@ import oracle
 from paper_2503_05530_b200 import prox
 
 POL = {"lru": oracle.LRU, "fifo": oracle.FIFO}
+ORACLE_METRIC = {"l2": oracle.L2SQ, "cosine": oracle.COSINE, "ip": oracle.IP}
 REL_TIE = 1e-5
 REL_DIST = 1e-4
 
@@ -59,7 +60,7 @@ def run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=None, max_forc
     forced = []
     while True:
         o = oracle.Oracle(corpus, d, k, capacity, tau32, POL[policy], rho=rho, lsh_planes=lsh_planes, lsh_bucket=lsh_bucket,
-                          metric=oracle.COSINE if metric == "cosine" else oracle.L2SQ)
+                          metric=ORACLE_METRIC[metric])
         r = o.query(queries, force)
         o.close()
         if gpu_hit is None:
@@ -69,7 +70,7 @@ def run_oracle(corpus, queries, k, capacity, tau, policy, gpu_hit=None, max_forc
             return r, forced
         i = int(diff[0])
         best = r["best"][i]
-        tie = best != 0.0 and np.isfinite(best) and abs(best - tau32) < REL_TIE * max(tau32, best)
+        tie = best != 0.0 and np.isfinite(best) and abs(best - tau32) < REL_TIE * max(abs(tau32), abs(best))
         if not tie:
             return r, forced
         force[i] = int(gpu_hit[i])
@@ -84,13 +85,13 @@ def ids_differ_only_within_ties(corpus, q, gpu_ids, ref_ids, ref_dists, metric="
     name a row twice.  A tie somewhere else in the list excuses nothing."""
     if len(set(int(x) for x in gpu_ids)) != len(gpu_ids):
         return False
-    dist = oracle.cosdist if metric == "cosine" else oracle.sqdist
+    dist = {"cosine": oracle.cosdist, "ip": oracle.ipdist}.get(metric, oracle.sqdist)
     for p in np.nonzero(np.asarray(gpu_ids) != np.asarray(ref_ids))[0]:
         g = int(gpu_ids[p])
         if g < 0 or g >= corpus.shape[0]:
             return False
         dg, dr = dist(q, corpus[g]), float(ref_dists[p])
-        if not abs(dg - dr) < REL_TIE * max(dr, dg, 1e-300):
+        if not abs(dg - dr) < REL_TIE * max(abs(dr), abs(dg), 1e-300):
             return False
     return True
 

@@ -8,6 +8,7 @@ import oracle
 from paper_2503_05530_b200 import prox, workloads as W
 from golden_traces import all_load_traces, all_traces
 import oracle_workers
+import parity
 from parity import compare, run_gpu, run_oracle
 
 pytestmark = pytest.mark.gpu
@@ -172,6 +173,32 @@ def test_uncertified_queries_take_the_exact_pass():
     assert np.allclose(gpu[1], dists, rtol=1e-4, atol=1e-12)
 
 
+@pytest.mark.parametrize("metric", ["l2", "ip"])
+def test_thousands_of_copies_of_one_row_are_still_answered_exactly(metric):
+    """More rows tie at the k-th distance than the exact pass can collect (3000 copies of the row
+    nearest to the query, scattered over the corpus): the answer is still the oracle's, the copies
+    in id order, through the streaming pass that keeps every row it sees or proves it out."""
+    g = torch.Generator().manual_seed(71)
+    X = W.make_corpus(20000, 128, 16, seed=71)
+    Q, _, _ = W.make_query_stream(X, 12, 3, 1.0, 0.02, seed=71)
+    where = torch.randperm(20000, generator=g)[:3000]
+    X = X.clone()
+    X[where] = X[int(where[0])].clone()                               # 3000 identical rows
+    Q = Q.clone()
+    Q[:6] = (X[int(where[0])] + 0.01 * torch.randn(6, 128, generator=g))    # queries next to the copies
+    Q = (Q / Q.norm(dim=1, keepdim=True)).contiguous()
+    k = 10
+    tau = 0.0 if metric == "l2" else -2.0
+    gpu = run_gpu(X.to(DEV), Q.to(DEV), k, 16, tau, "lru", 4, metric=metric)
+    ids, dists = oracle.exact_topk(X.numpy(), Q.numpy(), k, metric=parity.ORACLE_METRIC[metric])
+    assert gpu[3]["unresolved"] == 0 and gpu[3]["hits"] == 0
+    assert np.array_equal(gpu[0], ids)
+    assert np.allclose(gpu[1], dists, rtol=1e-4, atol=1e-12)
+    first_copies = np.sort(where.numpy())[:k]
+    assert np.array_equal(gpu[0][0], first_copies)                     # ties come back in id order
+    assert gpu[3]["uncertified"] >= 6
+
+
 # ------------------------------------------------------------------ re-ranking factor (Section 3.3)
 @pytest.mark.parametrize("policy,batch,rho,k", [("lru", 64, 4, 10), ("fifo", 1, 2, 5), ("lru", 200, 2, 32),
                                                 ("fifo", 1024, 4, 32)])
@@ -233,6 +260,70 @@ def test_cosine_probe_only_with_loaded_keys():
         assert 0.2 < r["hit"].mean() < 0.97
     assert p.status() == prox.OK
     p.close()
+
+
+# ------------------------------------------------------------------ inner product (Section 2.2)
+@pytest.mark.parametrize("policy,batch,rho,d,tau", [("lru", 64, 1, 128, -0.9), ("fifo", 1, 1, 128, -0.9), ("lru", 500, 2, 128, -0.9),
+                                                    ("fifo", 256, 1, 768, -0.95), ("lru", 100, 1, 80, -0.9)])
+def test_inner_product_matches_the_oracle(policy, batch, rho, d, tau):
+    """Rows of very different lengths, so that the rows with the largest inner products are not the
+    Euclidean neighbours; the tolerance is negative (a key matches when q.key >= 0.9 or 0.95).
+    d = 80 is not a multiple of 64: that handle scans on the CUDA cores."""
+    X, Q = stream(30011, d, 48, 1500, 100, 1.0, 0.03, seed=61)
+    g = torch.Generator().manual_seed(62)
+    X = (X * (0.5 + 1.5 * torch.rand(X.shape[0], 1, generator=g))).contiguous()
+    res, gpu = check(X, Q, 10, 40, tau, policy, batch, rho=rho, metric="ip")
+    assert 0.2 < res["hit_rate"] < 0.97
+    assert (gpu[1] < 0).all()                                           # -(q.x) of the most similar rows
+    l2 = run_gpu(X.to(DEV), Q.to(DEV), 10, 40, 0.3, policy, batch, rho=rho)
+    miss = res["ref"]["hit"] == 0
+    assert (l2[0][miss] != gpu[0][miss]).any(axis=1).mean() > 0.5
+
+
+def test_inner_product_uncertified_queries_take_the_exact_pass():
+    """Rows packed so tightly that the bf16 products cannot separate them: both sweeps of the
+    exact pass run with the inner product's margins."""
+    g = torch.Generator().manual_seed(63)
+    c = torch.randn(256, generator=g)
+    X = c + 2e-4 * torch.randn(6000, 256, generator=g)
+    X = (X / X.norm(dim=1, keepdim=True)).contiguous()
+    Q = X[:40] + 1e-4 * torch.randn(40, 256, generator=g)
+    Q = (Q / Q.norm(dim=1, keepdim=True)).contiguous()
+    gpu = run_gpu(X.to(DEV), Q.to(DEV), 10, 16, -2.0, "lru", 8, metric="ip")          # -q.x <= -2 never holds: all miss
+    assert gpu[3]["uncertified"] > 0 and gpu[3]["unresolved"] == 0 and gpu[3]["hits"] == 0
+    ids, dists = oracle.exact_topk(X.numpy(), Q.numpy(), 10, metric=oracle.IP)
+    assert np.array_equal(gpu[0], ids)
+    assert np.allclose(gpu[1], dists, rtol=1e-4, atol=1e-12)
+
+
+def test_inner_product_probe_only_and_argument_checks():
+    keys, centres = W.make_probe_keys(3000, 128, 256, seed=64)
+    keys = (keys * (0.5 + 1.5 * torch.rand(3000, 1, generator=torch.Generator().manual_seed(65)))).contiguous()
+    tau = -1.2
+    p = prox.Prox(keys[:64].contiguous().to(DEV), 1, 3000, tau, "lru", metric="ip")
+    p.cache_load(keys.to(DEV))
+    o = oracle.Oracle(None, 128, 1, 3000, float(np.float32(tau)), oracle.LRU, metric=oracle.IP)
+    o.cache_load(keys.numpy())
+    for b in range(2):
+        Q = W.make_probe_batch(keys / keys.norm(dim=1, keepdim=True), centres, 512, 0.015, 64, b)
+        hit, slot, dist = p.probe_batch(Q.contiguous().to(DEV))
+        torch.cuda.synchronize()
+        r = o.query(Q.numpy())
+        assert np.array_equal(hit.cpu().numpy(), r["hit"]) and np.array_equal(slot.cpu().numpy(), r["slot"])
+        h = r["hit"] == 1
+        assert np.allclose(dist.cpu().numpy()[h], r["best"][h], rtol=1e-6)
+        assert 0.1 < r["hit"].mean() < 0.97
+    assert p.status() == prox.OK
+    p.close()
+    lib = prox.load_library()
+    Xd = keys.to(DEV)
+    assert not lib.prox_create_metric(Xd.data_ptr(), 3000, 128, 4, 8, -0.5, 0, 1, prox.METRIC_L2SQ)       # negative tau: inner product only
+    assert not lib.prox_create_metric(Xd.data_ptr(), 3000, 128, 4, 8, -0.5, 0, 1, prox.METRIC_COSINE)
+    assert not lib.prox_create_metric(Xd.data_ptr(), 3000, 128, 4, 8, float("nan"), 0, 1, prox.METRIC_IP)
+    assert not lib.prox_create_metric(Xd.data_ptr(), 3000, 128, 4, 8, 0.5, 0, 1, 3)
+    h = lib.prox_create_metric(Xd.data_ptr(), 3000, 128, 4, 8, -0.5, 0, 1, prox.METRIC_IP)
+    assert h
+    lib.prox_destroy(h)
 
 
 # ------------------------------------------------------------------ PROXIMITY-LSH (Section 3.2)
@@ -326,7 +417,9 @@ def test_probe_only_at_the_benchmarked_cache_sizes(n_keys, n_batches, batch, pol
     so its runs go to worker processes and overlap the GPU side and one another; the cache state is
     sequential, so a batch cannot be sampled: at 2^20 keys one batch of 256 queries is replayed."""
     d, tau = 768, 0.5
-    keys, centres = W.make_probe_keys(n_keys, d, 4096, seed=8)
+    # two keys per mixture component on average: about one fresh draw in seven finds no key of its
+    # component in the cache and misses, so every batch also evicts and inserts
+    keys, centres = W.make_probe_keys(n_keys, d, n_keys // 2, seed=8)
     Qs = torch.stack([W.make_probe_batch(keys, centres, batch, 0.02, 8, b) for b in range(n_batches)])
     kb, kdesc = oracle_workers.share(keys.numpy())
     qb, qdesc = oracle_workers.share(Qs.numpy())
@@ -355,7 +448,7 @@ def test_probe_only_at_the_benchmarked_cache_sizes(n_keys, n_batches, batch, pol
                     assert np.array_equal(slot, r["slot"]), f"{pol} batch {b}: first differing slot at {np.nonzero(slot != r['slot'])[0][:1]}"
                     h = r["hit"] == 1
                     assert np.allclose(dist[h], r["best"][h], rtol=1e-6)
-                    assert 0.3 < r["hit"].mean() < 0.97
+                    assert 0.3 < r["hit"].mean() < 0.99
                     evictions += int((r["evicted"] >= 0).sum())
                 assert got[pol][n_batches]["evictions"] == evictions > 0
     finally:

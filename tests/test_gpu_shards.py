@@ -88,6 +88,15 @@ def test_row_shards_cosine_distance():
     assert 0.05 < r["hit_rate"] < 0.98
 
 
+def test_row_shards_inner_product():
+    X = W.make_corpus(24001, 64, 32, 12)
+    Q, _, _ = W.make_query_stream(X, 900, 120, 1.0, 0.04, 12)
+    X = (X * (0.5 + 1.5 * torch.rand(X.shape[0], 1, generator=torch.Generator().manual_seed(13)))).contiguous()
+    gpu = run_shards(X, Q, 8, 64, -0.9, "lru", 100, 4, metric="ip")
+    r = compare(X.numpy(), Q.numpy(), 8, 64, -0.9, "lru", gpu, metric="ip")
+    assert 0.05 < r["hit_rate"] < 0.98
+
+
 def test_duplicate_rows_across_shards_keep_the_lower_id():
     base = W.make_corpus(4000, 64, 16, 8)
     X = torch.cat([base, base, base])                          # every row three times, one copy per shard
