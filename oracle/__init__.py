@@ -42,6 +42,7 @@ def lib():
         fp, ip, dp, i32p = (C.POINTER(C.c_float), C.POINTER(C.c_int64), C.POINTER(C.c_double),
                             C.POINTER(C.c_int32))
         L.oracle_num_threads.restype = C.c_int
+        L.oracle_set_threads.argtypes = [C.c_int]
         L.oracle_sqdist.restype = C.c_double
         L.oracle_sqdist.argtypes = [fp, fp, C.c_int32]
         L.oracle_create.restype = C.c_void_p
@@ -86,6 +87,11 @@ def _ptr(a: np.ndarray, ctype):
 
 def num_threads() -> int:
     return int(lib().oracle_num_threads())
+
+
+def set_threads(n: int) -> None:
+    """Threads the row loops of the database call use from now on (the arithmetic does not depend on it)."""
+    lib().oracle_set_threads(int(n))
 
 
 def sqdist(a, b) -> float:

@@ -105,6 +105,15 @@ int oracle_num_threads(void) {
 #endif
 }
 
+/* Threads that the row loops of the database call may use from now on (timing runs: one core, all cores). */
+void oracle_set_threads(int n) {
+#ifdef _OPENMP
+    if (n >= 1) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 /* Squared Euclidean distance, Algorithm 1 "distance(q, k)": sum_j (a_j - b_j)^2 in fp64. */
 double oracle_sqdist(const float *a, const float *b, int32_t d) {
     double acc = 0.0;

@@ -324,10 +324,13 @@ class ProxShard(Prox):
             out_dists = torch.empty(B, self.k, dtype=torch.float32, device=self.device)
         if out_hit is None:
             out_hit = torch.empty(B, dtype=torch.uint8, device=self.device)
-        record = torch.empty(self.exchange_bytes(B), dtype=torch.uint8, device=self.device)
-        self.shard_scan(queries, out_ids, out_dists, out_hit, record, stream)
-        gathered = all_gather_records(record, self.group)
-        self.shard_merge(queries, gathered, gathered.numel() // record.numel(), out_ids, out_dists, stream)
+        # the exchange is ordered on the stream the two library calls use: torch orders a collective after
+        # the work already queued on the CURRENT stream and makes that stream wait for its result
+        with torch.cuda.stream(stream if stream is not None else torch.cuda.current_stream()):
+            record = torch.empty(self.exchange_bytes(B), dtype=torch.uint8, device=self.device)
+            self.shard_scan(queries, out_ids, out_dists, out_hit, record, stream)
+            gathered = all_gather_records(record, self.group)
+            self.shard_merge(queries, gathered, gathered.numel() // record.numel(), out_ids, out_dists, stream)
         return out_ids, out_dists, out_hit
 
     def query_batch_host(self, queries: torch.Tensor, out_ids: torch.Tensor, out_dists: torch.Tensor,

@@ -264,10 +264,10 @@ def test_cosine_probe_only_with_loaded_keys():
 
 # ------------------------------------------------------------------ inner product (Section 2.2)
 @pytest.mark.parametrize("policy,batch,rho,d,tau", [("lru", 64, 1, 128, -0.9), ("fifo", 1, 1, 128, -0.9), ("lru", 500, 2, 128, -0.9),
-                                                    ("fifo", 256, 1, 768, -0.95), ("lru", 100, 1, 80, -0.9)])
+                                                    ("fifo", 256, 1, 768, -0.55), ("lru", 100, 1, 80, -0.9)])
 def test_inner_product_matches_the_oracle(policy, batch, rho, d, tau):
     """Rows of very different lengths, so that the rows with the largest inner products are not the
-    Euclidean neighbours; the tolerance is negative (a key matches when q.key >= 0.9 or 0.95).
+    Euclidean neighbours; the tolerance is negative (a key matches when q.key >= 0.9 or 0.55).
     d = 80 is not a multiple of 64: that handle scans on the CUDA cores."""
     X, Q = stream(30011, d, 48, 1500, 100, 1.0, 0.03, seed=61)
     g = torch.Generator().manual_seed(62)
@@ -299,7 +299,7 @@ def test_inner_product_uncertified_queries_take_the_exact_pass():
 def test_inner_product_probe_only_and_argument_checks():
     keys, centres = W.make_probe_keys(3000, 128, 256, seed=64)
     keys = (keys * (0.5 + 1.5 * torch.rand(3000, 1, generator=torch.Generator().manual_seed(65)))).contiguous()
-    tau = -1.2
+    tau = -1.7                                                          # only the longer keys of a component match
     p = prox.Prox(keys[:64].contiguous().to(DEV), 1, 3000, tau, "lru", metric="ip")
     p.cache_load(keys.to(DEV))
     o = oracle.Oracle(None, 128, 1, 3000, float(np.float32(tau)), oracle.LRU, metric=oracle.IP)

@@ -80,6 +80,66 @@ def test_two_shards_exchange_and_merge_to_the_whole_corpus_result():
     assert rows0 == (0, 501)
 
 
+def _rank_stream(rank, world, port, out):
+    """A stream of several batches: the cache is replicated (its decisions depend on the queries
+    alone, so every rank replays the same trace without talking to anyone), each batch's misses
+    are answered from the shards' own nearest rows through one exchange, and the merged lists
+    are what later hits return."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import oracle
+    from paper_2503_05530_b200 import prox, workloads as W
+    N, d, k, B, n, cap, tau = 1503, 32, 5, 16, 112, 6, 0.3
+    X = W.make_corpus(N, d, 8, 4, "cpu")
+    X[700:710] = X[20:30]                                     # equal rows in different shards
+    Q, _, _ = W.make_query_stream(X, n, 40, 1.0, 0.05, 4)
+    Xn, Qn = X.numpy(), Q.numpy()
+    first, cnt = prox.shard_rows(N, world, rank)
+    trace = oracle.Oracle(None, d, k, cap, float(np.float32(tau)), oracle.LRU)
+    lists, out_ids, out_hit = {}, np.empty((n, k), np.int64), np.empty(n, np.uint8)
+    for a in range(0, n, B):
+        r = trace.query(Qn[a:a + B])
+        miss = np.nonzero(r["hit"] == 0)[0]
+        if len(miss):
+            ids, dists = oracle.exact_topk(Xn[first:first + cnt], Qn[a:a + B][miss], k)
+        else:
+            ids, dists = np.empty((0, k), np.int64), np.empty((0, k), np.float64)
+        record = torch.from_numpy(make_record(ids + first, dists, B, k, len(miss)))
+        gathered = prox.all_gather_records(record)            # the one exchange of the batch
+        got_i, _ = merge_records(gathered.numpy(), world, B, k, len(miss))
+        for j, m in enumerate(miss):
+            lists[a + int(m)] = got_i[j]
+        for i in range(B):
+            out_ids[a + i] = lists[int(r["origin"][i])]        # a hit returns the list of the miss that made its key
+            out_hit[a + i] = r["hit"][i]
+    whole = oracle.Oracle(Xn, d, k, cap, float(np.float32(tau)), oracle.LRU).query(Qn)
+    same = bool(np.array_equal(out_ids, whole["ids"]) and np.array_equal(out_hit, whole["hit"]))
+    digest = torch.tensor([float(out_ids.sum()), float(out_hit.sum())], dtype=torch.float64)
+    both = [torch.zeros(2, dtype=torch.float64) for _ in range(world)]
+    dist.all_gather(both, digest)
+    if rank == 0:
+        out.put((same, [b.tolist() for b in both], float(whole["hit"].mean()), int((whole["evicted"] >= 0).sum())))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_shards_carry_a_stream_of_batches():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = 33500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_rank_stream, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    same, digests, hit_rate, evictions = out.get(timeout=180)
+    for p in procs:
+        p.join(timeout=120)
+        assert p.exitcode == 0
+    assert same, "the sharded stream differs from the oracle on the whole corpus"
+    assert digests[0] == digests[1], "both ranks must end with the same lists and flags"
+    assert 0.2 < hit_rate < 0.95 and evictions > 0
+
+
 def test_shard_rows_cover_the_corpus_once():
     from paper_2503_05530_b200 import prox
     for n, g in [(10, 3), (7, 7), (24_000_000, 8), (5, 1), (100, 32)]:
