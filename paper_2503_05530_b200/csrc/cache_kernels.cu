@@ -402,7 +402,9 @@ probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
 
 // ------------------------------------------------------------------------------------------
 // Per query: reduce the partial safe minima; list the at-risk and in-batch keys within tau
-// (the threshold test of Algorithm 1, inclusive).  code < kMaxBatch: at-risk position; else kMaxBatch + j.
+// (the threshold test of Algorithm 1, inclusive), nearest first.  code < kMaxBatch: at-risk
+// position; else kMaxBatch + j.  The list is sorted by (distance, code) so that the replay only
+// has to find the first entry that is still resident.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(128)
 build_candidates_kernel(const DevState *__restrict__ st, int B, int S, double tau,
@@ -411,6 +413,8 @@ build_candidates_kernel(const DevState *__restrict__ st, int B, int S, double ta
                         double *safe_min, int32_t *safe_arg, double *cand_d, int32_t *cand_code,
                         int32_t *n_cand, const int32_t *__restrict__ use_partial) {
     __shared__ int s_n;
+    __shared__ double s_d[2 * kMaxBatch];
+    __shared__ int s_code[2 * kMaxBatch];
     const int i = blockIdx.x, tid = threadIdx.x;
     if (i >= B) return;
     if (tid == 0) s_n = 0;
@@ -435,7 +439,6 @@ build_candidates_kernel(const DevState *__restrict__ st, int B, int S, double ta
         }
     }
     const int R = st->n_risk;
-    const size_t base = (size_t)i * (2 * kMaxBatch);
     for (int e = tid; e < R + i; e += blockDim.x) {
         double v;
         int code;
@@ -443,17 +446,40 @@ build_candidates_kernel(const DevState *__restrict__ st, int B, int S, double ta
         else { v = d_intra[(size_t)i * kMaxBatch + (e - R)]; code = kMaxBatch + (e - R); }
         if (v <= tau) {
             const int pos = atomicAdd(&s_n, 1);
-            cand_d[base + pos] = v;
-            cand_code[base + pos] = code;
+            s_d[pos] = v;
+            s_code[pos] = code;
         }
     }
     __syncthreads();
-    if (tid == 0) n_cand[i] = s_n;
+    const int n = s_n;
+    if (n > 1) {                                          // (block-uniform)
+        int n2 = 2;
+        while (n2 < n) n2 <<= 1;
+        for (int e = n + tid; e < n2; e += blockDim.x) { s_d[e] = INFINITY; s_code[e] = 0x7fffffff; }
+        block_sort_asc(s_d, s_code, n2);
+    }
+    const size_t base = (size_t)i * (2 * kMaxBatch);
+    for (int e = tid; e < n; e += blockDim.x) {
+        cand_d[base + e] = s_d[e];
+        cand_code[base + e] = s_code[e];
+    }
+    if (tid == 0) n_cand[i] = n;
 }
 
 // ------------------------------------------------------------------------------------------
-// Resolve: replay queries 0..B-1 in order (Algorithm 1 from the threshold test to the insertion) on the candidate lists.
-// One block; warp 0 walks the batch, the other warps only help to load and store.
+// Resolve: replay queries 0..B-1 in order (Algorithm 1 from the threshold test to the insertion).
+// One block.  Three kinds of query:
+//   settled     no at-risk or in-batch key within tau, nearest safe key within tau: a hit on that
+//               key whatever the rest of the batch does; answered in parallel while loading;
+//   plain miss  no key of any kind within tau: a miss for certain; it only has to take its slot
+//               in order;
+//   entangled   some at-risk or in-batch key within tau: hit or miss depends on which of them are
+//               still resident when its turn comes.
+// Warp 0 walks the entangled queries in order; the plain misses between two of them are settled
+// 32 at a time (free slots first, then the next at-risk entries that nobody touched, found by
+// one vote per 32 entries).  An entangled query finds the first resident entry of its sorted list
+// with one vote per 32 entries.  Only when the at-risk list is used up (a capacity below the
+// batch size) does a miss search all refreshed and in-batch entries for the oldest stamp.
 // ------------------------------------------------------------------------------------------
 constexpr int kCsrCap = 8192;
 
@@ -468,18 +494,106 @@ struct ResolveSmem {
     int safe_arg[kMaxBatch];
     int ncand[kMaxBatch];
     int off[kMaxBatch + 1];
-    int warp_tot[32];
+    int plain_list[kMaxBatch];         // the plain misses in index order
+    int ent_list[kMaxBatch];           // the entangled queries in index order
+    int plain_before[kMaxBatch];       // per entangled query (by its place in ent_list): plain misses before it
+    int warp_tot[3][32];
+    int one[1];
     unsigned char r_alive[kMaxBatch];
     unsigned char r_touched[kMaxBatch];
 };
 
-__device__ __forceinline__ void lexmin_shfl(double &d, int &slot, int &code) {
+struct ReplayState {
+    long long cnt;                     // |C| so far
+    int p;                             // first at-risk position that may still be untouched and resident
+    int n_miss, n_evict;
+};
+
+struct ResolveOut {
+    uint8_t *out_hit;
+    int32_t *src, *src_kind, *evt_slot, *miss_list, *miss_rank;
+    float *evt_dist;
+};
+
+// The misses list[a .. b) (query indices, ascending) take their slots in order.  Whole warp.
+__device__ void settle_misses(ResolveSmem &sm, ReplayState &rs, const int *list, int a, int b, int R, long long C,
+                              long long clock0, DevState *st, const ResolveOut &o) {
+    const int lane = threadIdx.x & 31;
+    for (int base = a; base < b; base += 32) {
+        const int m = b - base < 32 ? b - base : 32;
+        const int i = lane < m ? list[base + lane] : -1;
+        const long long free_now = C - rs.cnt;
+        const int n_free = free_now <= 0 ? 0 : (free_now < m ? (int)free_now : m);
+        int slot = -1;
+        if (lane < n_free) slot = (int)(rs.cnt + lane);
+        rs.cnt += n_free;
+        const int need = m - n_free;
+        int got = 0;
+        while (got < need && rs.p < R) {                   // the next 32 at-risk entries
+            const int e = rs.p + lane;
+            const bool ok = e < R && sm.r_alive[e] && !sm.r_touched[e];
+            const unsigned mask = __ballot_sync(0xffffffffu, ok);
+            const int avail = __popc(mask);
+            const int use = avail < need - got ? avail : need - got;
+            const int t = lane - n_free - got;             // this lane's turn among the evicting misses
+            if (t >= 0 && t < use) slot = sm.r_slot[rs.p + (int)__fns(mask, 0, t + 1)];
+            if (ok && __popc(mask & ((1u << lane) - 1u)) < use) sm.r_alive[e] = 0;
+            got += use;
+            rs.p = (use == avail) ? rs.p + 32 : rs.p + (int)__fns(mask, 0, use) + 1;
+            __syncwarp();
+        }
+        if (rs.p > R) rs.p = R;
+        rs.n_evict += got;
+        const int n_fast = n_free + got;
+        if (lane < n_fast) {
+            const int rank = rs.n_miss + lane;
+            o.out_hit[i] = 0; o.src_kind[i] = 0; o.src[i] = -1;
+            o.evt_slot[i] = slot; o.evt_dist[i] = INFINITY;
+            sm.b_slot[i] = slot; sm.b_stamp[i] = (u64)(clock0 + i);
+            o.miss_list[rank] = i; o.miss_rank[i] = rank;
+        }
+        __syncwarp();
+        // the at-risk list is used up: each remaining miss evicts the oldest of the refreshed at-risk
+        // entries and of the entries this batch inserted before it
+        for (int t = n_fast; t < m; ++t) {
+            const int ii = __shfl_sync(0xffffffffu, i, t);
+            u64 bs = ~0ull;
+            int bc = -1;
+            for (int e = lane; e < R + ii; e += 32) {
+                u64 v;
+                bool ok;
+                if (e < R) { ok = sm.r_alive[e] != 0; v = sm.r_stamp[e]; }
+                else { ok = sm.b_slot[e - R] >= 0; v = sm.b_stamp[e - R]; }
+                if (ok && v < bs) { bs = v; bc = e; }
+            }
 #pragma unroll
-    for (int m = 1; m < 32; m <<= 1) {
-        const double od = __shfl_xor_sync(0xffffffffu, d, m);
-        const int os = __shfl_xor_sync(0xffffffffu, slot, m);
-        const int oc = __shfl_xor_sync(0xffffffffu, code, m);
-        if (od < d || (od == d && os < slot)) { d = od; slot = os; code = oc; }
+            for (int mm = 1; mm < 32; mm <<= 1) {
+                const u64 ov = __shfl_xor_sync(0xffffffffu, bs, mm);
+                const int oc = __shfl_xor_sync(0xffffffffu, bc, mm);
+                if (ov < bs) { bs = ov; bc = oc; }
+            }
+            int vslot = 0;
+            if (bc < 0) {                                  // cannot happen with capacity >= 1
+                if (lane == 0) atomicCAS(&st->error, 0, PROX_ERR_INTERNAL);
+            } else if (bc < R) {
+                vslot = sm.r_slot[bc];
+                if (lane == 0) sm.r_alive[bc] = 0;
+            } else {
+                vslot = sm.b_slot[bc - R];
+                if (lane == 0) sm.b_slot[bc - R] = -1;
+            }
+            __syncwarp();
+            if (lane == 0) {
+                const int rank = rs.n_miss + t;
+                o.out_hit[ii] = 0; o.src_kind[ii] = 0; o.src[ii] = -1;
+                o.evt_slot[ii] = vslot; o.evt_dist[ii] = INFINITY;
+                sm.b_slot[ii] = vslot; sm.b_stamp[ii] = (u64)(clock0 + ii);
+                o.miss_list[rank] = ii; o.miss_rank[ii] = rank;
+            }
+            rs.n_evict++;
+            __syncwarp();
+        }
+        rs.n_miss += m;
     }
 }
 
@@ -496,12 +610,13 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int R = st->n_risk;
     const long long count0 = st->count, clock0 = st->clock;
+    ResolveOut o{out_hit, src, src_kind, evt_slot, miss_list, miss_rank, evt_dist};
 
-    // ---- load
+    // ---- load, classify, three prefix sums (candidates, plain misses, entangled queries)
+    int n_plain = 0, n_ent = 0, n_settled = 0;
     {
         const int i = tid;
-        int n = 0;
-        bool settled = false;
+        int n = 0, kind = 0;                               // 1 settled, 2 plain miss, 3 entangled
         if (i < B) {
             n = n_cand[i];
             const double sd = g_safe_min[i];
@@ -510,11 +625,12 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
             sm.safe_arg[i] = sa;
             sm.b_slot[i] = -1;
             sm.b_stamp[i] = 0;
+            const bool safe_hit = sa >= 0 && sd <= tau;
+            kind = n > 0 ? 3 : (safe_hit ? 1 : 2);
             // A query with no at-risk or in-batch key within tau whose nearest safe key is within tau
             // hits that key whatever the rest of the batch does (safe keys are not evicted in this
             // batch, and touching one changes no eviction of this batch): settled here, in parallel.
-            if (n == 0 && sa >= 0 && sd <= tau) {
-                settled = true;
+            if (kind == 1) {
                 out_hit[i] = 1;
                 evt_slot[i] = sa;
                 evt_dist[i] = (float)sd;
@@ -529,134 +645,113 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
             sm.r_alive[i] = 1;
             sm.r_touched[i] = 0;
         }
-        if (i < kMaxBatch) sm.ncand[i] = settled ? -1 : n;
-        // exclusive prefix sum of n over the block
-        int x = n;
+        if (i < kMaxBatch) sm.ncand[i] = n;
+        int x[3] = {n, kind == 2 ? 1 : 0, kind == 3 ? 1 : 0};
 #pragma unroll
         for (int m = 1; m < 32; m <<= 1) {
-            const int y = __shfl_up_sync(0xffffffffu, x, m);
-            if (lane >= m) x += y;
+#pragma unroll
+            for (int c = 0; c < 3; ++c) {
+                const int y = __shfl_up_sync(0xffffffffu, x[c], m);
+                if (lane >= m) x[c] += y;
+            }
         }
-        if (lane == 31) sm.warp_tot[warp] = x;
+        if (lane == 31) { sm.warp_tot[0][warp] = x[0]; sm.warp_tot[1][warp] = x[1]; sm.warp_tot[2][warp] = x[2]; }
         __syncthreads();
-        if (warp == 0) {
-            int w = sm.warp_tot[lane];
+        if (warp < 3) {
+            int w = sm.warp_tot[warp][lane];
 #pragma unroll
             for (int m = 1; m < 32; m <<= 1) {
                 const int y = __shfl_up_sync(0xffffffffu, w, m);
                 if (lane >= m) w += y;
             }
-            sm.warp_tot[lane] = w;
+            sm.warp_tot[warp][lane] = w;
         }
         __syncthreads();
-        const int incl = x + (warp > 0 ? sm.warp_tot[warp - 1] : 0);
-        if (i < kMaxBatch) sm.off[i] = incl - n;
-        if (i == kMaxBatch - 1) sm.off[kMaxBatch] = incl;
+        const int incl_n = x[0] + (warp > 0 ? sm.warp_tot[0][warp - 1] : 0);
+        const int excl_plain = x[1] + (warp > 0 ? sm.warp_tot[1][warp - 1] : 0) - (kind == 2 ? 1 : 0);
+        const int excl_ent = x[2] + (warp > 0 ? sm.warp_tot[2][warp - 1] : 0) - (kind == 3 ? 1 : 0);
+        if (i < kMaxBatch) sm.off[i] = incl_n - n;
+        if (i == kMaxBatch - 1) sm.off[kMaxBatch] = incl_n;
+        if (kind == 2) sm.plain_list[excl_plain] = i;
+        if (kind == 3) { sm.ent_list[excl_ent] = i; sm.plain_before[excl_ent] = excl_plain; }
+        n_plain = sm.warp_tot[1][31];
+        n_ent = sm.warp_tot[2][31];
+        n_settled = B - n_plain - n_ent;
         __syncthreads();
         for (int row = warp; row < B; row += 32) {
-            const int o = sm.off[row], nn = sm.ncand[row];
-            if (o + nn <= kCsrCap)
+            const int off = sm.off[row], nn = sm.ncand[row];
+            if (off + nn <= kCsrCap)
                 for (int e = lane; e < nn; e += 32) {
-                    sm.csr_d[o + e] = cand_d[(size_t)row * (2 * kMaxBatch) + e];
-                    sm.csr_code[o + e] = cand_code[(size_t)row * (2 * kMaxBatch) + e];
+                    sm.csr_d[off + e] = cand_d[(size_t)row * (2 * kMaxBatch) + e];
+                    sm.csr_code[off + e] = cand_code[(size_t)row * (2 * kMaxBatch) + e];
                 }
         }
         __syncthreads();
     }
 
-    // ---- no at-risk key and no query of the batch lies within tau of any query: the hits (all on
-    // safe keys) are settled, the others are misses that meet no one, so the replay has a closed
-    // form: the j-th miss takes the j-th free slot, then the j-th at-risk entry in stamp order
-    // (none of them was touched).  Taken when the evictions stay within the at-risk list.
-    bool closed_form = false;
-    if (sm.off[kMaxBatch] == 0) {
-        const int i = tid;
-        const int miss = (i < B && sm.ncand[i] == 0) ? 1 : 0;
-        int x = miss;
-#pragma unroll
-        for (int m = 1; m < 32; m <<= 1) {
-            const int y = __shfl_up_sync(0xffffffffu, x, m);
-            if (lane >= m) x += y;
-        }
-        if (lane == 31) sm.warp_tot[warp] = x;
-        __syncthreads();
-        if (warp == 0) {
-            int w = sm.warp_tot[lane];
-#pragma unroll
-            for (int m = 1; m < 32; m <<= 1) {
-                const int y = __shfl_up_sync(0xffffffffu, w, m);
-                if (lane >= m) w += y;
+    // ---- replay by warp 0
+    if (warp == 0) {
+        ReplayState rs{count0, 0, 0, 0};
+        int n_hit = n_settled, n_intra = 0, done_plain = 0;
+        for (int k = 0; k < n_ent; ++k) {
+            const int i = sm.ent_list[k];
+            const int upto = sm.plain_before[k];
+            if (upto > done_plain) {
+                settle_misses(sm, rs, sm.plain_list, done_plain, upto, R, C, clock0, st, o);
+                done_plain = upto;
             }
-            sm.warp_tot[lane] = w;
-        }
-        __syncthreads();
-        const int j = x + (warp > 0 ? sm.warp_tot[warp - 1] : 0) - 1;      // rank of this miss
-        const int n_miss = sm.warp_tot[31];
-        const long long free_slots = C > count0 ? C - count0 : 0;
-        const long long n_evict = n_miss > free_slots ? n_miss - free_slots : 0;
-        closed_form = n_evict <= (long long)R;
-        if (closed_form) {
-            if (miss) {
-                int slot;
-                if (j < free_slots) {
-                    slot = (int)(count0 + j);
-                } else {
-                    const int v = (int)(j - free_slots);
-                    slot = sm.r_slot[v];
-                    sm.r_alive[v] = 0;
-                }
-                out_hit[i] = 0;
-                src_kind[i] = 0; src[i] = -1;
-                evt_slot[i] = slot;
-                evt_dist[i] = INFINITY;
-                sm.b_slot[i] = slot;
-                sm.b_stamp[i] = (u64)(clock0 + i);
-                miss_list[j] = i;
-                miss_rank[i] = j;
-            }
-            if (tid == 0) {
-                st->count = count0 + n_miss - n_evict;
-                st->clock = clock0 + B;
-                st->n_miss = n_miss;
-                st->queries += B;
-                st->hits += B - n_miss;
-                st->misses += n_miss;
-                st->evictions += n_evict;
-            }
-        }
-        __syncthreads();
-    }
-
-    // ---- sequential replay by warp 0
-    if (!closed_form && warp == 0) {
-        long long cnt = count0;
-        int p = 0, n_miss = 0, n_hit = 0, n_intra = 0, n_evict = 0;
-        for (int i = 0; i < B; ++i) {
             const u64 t = (u64)(clock0 + i);
-            const int n = sm.ncand[i], o = sm.off[i];
-            if (n < 0) { ++n_hit; continue; }             // settled in the parallel pass
-            const bool in_smem = (o + n <= kCsrCap);
+            const int n = sm.ncand[i], off = sm.off[i];
+            const bool in_smem = (off + n <= kCsrCap);
+            const double *ld = in_smem ? sm.csr_d + off : cand_d + (size_t)i * (2 * kMaxBatch);
+            const int *lc = in_smem ? sm.csr_code + off : cand_code + (size_t)i * (2 * kMaxBatch);
+            // the nearest entry of the sorted list that is still resident; among entries at exactly
+            // the same distance the lowest slot
             double bd = INFINITY;
             int bslot = 0x7fffffff, bcode = -1;
-            for (int e = lane; e < n; e += 32) {
-                double v;
-                int code;
-                if (in_smem) { v = sm.csr_d[o + e]; code = sm.csr_code[o + e]; }
-                else { v = cand_d[(size_t)i * (2 * kMaxBatch) + e]; code = cand_code[(size_t)i * (2 * kMaxBatch) + e]; }
-                int slot;
-                bool valid;
-                if (code < kMaxBatch) { valid = sm.r_alive[code] != 0; slot = sm.r_slot[code]; }
-                else { slot = sm.b_slot[code - kMaxBatch]; valid = slot >= 0; }
-                if (valid && (v < bd || (v == bd && slot < bslot))) { bd = v; bslot = slot; bcode = code; }
+            for (int e0 = 0; e0 < n && bcode == -1; e0 += 32) {
+                const int e = e0 + lane;
+                int code = -1, slot = -1;
+                bool valid = false;
+                if (e < n) {
+                    code = lc[e];
+                    if (code < kMaxBatch) { valid = sm.r_alive[code] != 0; slot = sm.r_slot[code]; }
+                    else { slot = sm.b_slot[code - kMaxBatch]; valid = slot >= 0; }
+                }
+                const unsigned mask = __ballot_sync(0xffffffffu, valid);
+                if (mask == 0u) continue;
+                const int first = __ffs(mask) - 1;
+                bd = ld[e0 + first];
+                bslot = __shfl_sync(0xffffffffu, slot, first);
+                bcode = __shfl_sync(0xffffffffu, code, first);
+                // entries at the same distance (in this group of 32 or beyond it)
+                for (int f0 = e0; f0 < n; f0 += 32) {
+                    const int f = f0 + lane;
+                    bool same = false;
+                    int fcode = -1, fslot = 0x7fffffff;
+                    if (f < n && f > e0 + first && ld[f] == bd) {
+                        fcode = lc[f];
+                        if (fcode < kMaxBatch) { same = sm.r_alive[fcode] != 0; fslot = sm.r_slot[fcode]; }
+                        else { fslot = sm.b_slot[fcode - kMaxBatch]; same = fslot >= 0; }
+                    }
+                    const bool past = f < n && ld[f] > bd;     // sorted: nothing equal follows
+                    unsigned smask = __ballot_sync(0xffffffffu, same);
+                    while (smask) {
+                        const int l = __ffs(smask) - 1;
+                        smask &= smask - 1;
+                        const int os = __shfl_sync(0xffffffffu, fslot, l);
+                        const int oc = __shfl_sync(0xffffffffu, fcode, l);
+                        if (os < bslot) { bslot = os; bcode = oc; }
+                    }
+                    if (__any_sync(0xffffffffu, past)) break;
+                }
             }
-            if (lane == 0) {
+            {
                 const double sd = sm.safe_min[i];
                 const int sa = sm.safe_arg[i];
                 if (sa >= 0 && sd <= tau && (sd < bd || (sd == bd && sa < bslot))) { bd = sd; bslot = sa; bcode = -2; }
             }
-            lexmin_shfl(bd, bslot, bcode);
-            const bool hit = (bcode != -1);
-            if (hit) {
+            if (bcode != -1) {                             // hit
                 ++n_hit;
                 if (lane == 0) {
                     out_hit[i] = 1;
@@ -675,72 +770,23 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
                     }
                 }
                 if (bcode >= kMaxBatch) ++n_intra;
-            } else {
-                int slot;
-                if (cnt < C) {
-                    slot = (int)cnt;
-                    ++cnt;
-                } else {
-                    // victim: the first at-risk entry in stamp order that is still there and untouched
-                    while (p < R && (sm.r_touched[p] || !sm.r_alive[p])) ++p;
-                    __syncwarp();                           // every lane has read before lane 0 writes
-                    if (p < R) {
-                        slot = sm.r_slot[p];
-                        if (lane == 0) sm.r_alive[p] = 0;
-                        ++p;
-                    } else {
-                        // only refreshed entries and entries of this batch are left: smallest stamp
-                        u64 bs = ~0ull;
-                        int bc = -1;
-                        for (int e = lane; e < R + i; e += 32) {
-                            u64 v;
-                            bool ok;
-                            if (e < R) { ok = sm.r_alive[e] != 0; v = sm.r_stamp[e]; }
-                            else { ok = sm.b_slot[e - R] >= 0; v = sm.b_stamp[e - R]; }
-                            if (ok && v < bs) { bs = v; bc = e; }
-                        }
-#pragma unroll
-                        for (int m = 1; m < 32; m <<= 1) {
-                            const u64 ov = __shfl_xor_sync(0xffffffffu, bs, m);
-                            const int oc = __shfl_xor_sync(0xffffffffu, bc, m);
-                            if (ov < bs) { bs = ov; bc = oc; }
-                        }
-                        if (bc < 0) {                       // cannot happen with capacity >= 1
-                            if (lane == 0) atomicCAS(&st->error, 0, PROX_ERR_INTERNAL);
-                            slot = 0;
-                        } else if (bc < R) {
-                            slot = sm.r_slot[bc];
-                            if (lane == 0) sm.r_alive[bc] = 0;
-                        } else {
-                            slot = sm.b_slot[bc - R];
-                            if (lane == 0) sm.b_slot[bc - R] = -1;
-                        }
-                    }
-                    ++n_evict;
-                }
-                if (lane == 0) {
-                    out_hit[i] = 0;
-                    src_kind[i] = 0; src[i] = -1;
-                    evt_slot[i] = slot;
-                    evt_dist[i] = INFINITY;
-                    sm.b_slot[i] = slot;
-                    sm.b_stamp[i] = t;
-                    miss_list[n_miss] = i;
-                    miss_rank[i] = n_miss;
-                }
-                ++n_miss;
+                __syncwarp();
+            } else {                                       // every key within tau has left: a miss after all
+                if (lane == 0) sm.one[0] = i;
+                __syncwarp();
+                settle_misses(sm, rs, sm.one, 0, 1, R, C, clock0, st, o);
             }
-            __syncwarp();
         }
+        if (n_plain > done_plain) settle_misses(sm, rs, sm.plain_list, done_plain, n_plain, R, C, clock0, st, o);
         if (lane == 0) {
-            st->count = cnt;
+            st->count = rs.cnt;
             st->clock = clock0 + B;
-            st->n_miss = n_miss;
+            st->n_miss = rs.n_miss;
             st->queries += B;
             st->hits += n_hit;
-            st->misses += n_miss;
+            st->misses += rs.n_miss;
             st->intra_hits += n_intra;
-            st->evictions += n_evict;
+            st->evictions += rs.n_evict;
         }
     }
     __syncthreads();
