@@ -247,6 +247,9 @@ risk_finish_kernel(DevState *st, RiskWork *w, int32_t *risk_pos, int32_t *risk_s
 //   mode 1  columns = the R at-risk slots then the batch: what the resolve needs as full rows
 //           when the safe slots are handled by the coarse tensor-core probe.
 //   mode 2  queries = those the coarse probe could not certify (pfail_list), columns = slots.
+//   mode 3  columns = slots only, the at-risk ones left out: the safe minimum alone (the at-risk
+//           slots and the batch go through the tensor-core pass of probe_side.cu).
+//   mode 4  mode 1, but only if that pass listed more pairs than it can hold (else return at once).
 // ------------------------------------------------------------------------------------------
 constexpr int PQ = 32;
 constexpr int kProbeColsWide = 64, kProbeColsNarrow = 32;
@@ -266,12 +269,16 @@ probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
     __shared__ double ks[PC][PD + 1];
     __shared__ int q_index[PQ];
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    if (mode == 4) {
+        if (!st->side_overflow) return;
+        mode = 1;
+    }
     const long long count = st->count;
     const int R = st->n_risk;
     const int nq = mode == 2 ? st->n_pfail : B;            // queries this launch serves
     if ((int)blockIdx.x * PQ >= nq) return;
     const long long nslot_cols = mode == 1 ? R : count;      // columns that are cached keys
-    const long long ncols = mode == 2 ? count : nslot_cols + B;
+    const long long ncols = (mode == 2 || mode == 3) ? count : nslot_cols + B;
     if (tid < PQ) {
         const int r = blockIdx.x * PQ + tid;
         q_index[tid] = r < nq ? (mode == 2 ? pfail_list[r] : r) : -1;
@@ -371,7 +378,7 @@ probe_kernel(const DevState *__restrict__ st, const float *__restrict__ keys,
                 if (col < nslot_cols) {
                     const int rp = mode == 1 ? (int)col : risk_pos[col];
                     if (rp >= 0) {
-                        if (mode != 2) d_risk[(size_t)i * kMaxBatch + rp] = v;
+                        if (mode < 2) d_risk[(size_t)i * kMaxBatch + rp] = v;
                     } else if (v < best_d[a] || (v == best_d[a] && (int)col < best_s[a])) {
                         best_d[a] = v;
                         best_s[a] = (int)col;
@@ -411,7 +418,7 @@ build_candidates_kernel(const DevState *__restrict__ st, int B, int S, double ta
                         const double *__restrict__ part_min, const int32_t *__restrict__ part_arg,
                         const double *__restrict__ d_risk, const double *__restrict__ d_intra,
                         double *safe_min, int32_t *safe_arg, double *cand_d, int32_t *cand_code,
-                        int32_t *n_cand, const int32_t *__restrict__ use_partial) {
+                        int32_t *n_cand, const int32_t *__restrict__ use_partial, int lists_ready) {
     __shared__ int s_n;
     __shared__ double s_d[2 * kMaxBatch];
     __shared__ int s_code[2 * kMaxBatch];
@@ -439,15 +446,22 @@ build_candidates_kernel(const DevState *__restrict__ st, int B, int S, double ta
         }
     }
     const int R = st->n_risk;
-    for (int e = tid; e < R + i; e += blockDim.x) {
-        double v;
-        int code;
-        if (e < R) { v = d_risk[(size_t)i * kMaxBatch + e]; code = e; }
-        else { v = d_intra[(size_t)i * kMaxBatch + (e - R)]; code = kMaxBatch + (e - R); }
-        if (v <= tau) {
-            const int pos = atomicAdd(&s_n, 1);
-            s_d[pos] = v;
-            s_code[pos] = code;
+    const size_t base = (size_t)i * (2 * kMaxBatch);
+    if (lists_ready && !st->side_overflow) {              // the pairs within tau are listed already: only sort them
+        const int nl = n_cand[i];
+        for (int e = tid; e < nl; e += blockDim.x) { s_d[e] = cand_d[base + e]; s_code[e] = cand_code[base + e]; }
+        if (tid == 0) s_n = nl;
+    } else {
+        for (int e = tid; e < R + i; e += blockDim.x) {
+            double v;
+            int code;
+            if (e < R) { v = d_risk[(size_t)i * kMaxBatch + e]; code = e; }
+            else { v = d_intra[(size_t)i * kMaxBatch + (e - R)]; code = kMaxBatch + (e - R); }
+            if (v <= tau) {
+                const int pos = atomicAdd(&s_n, 1);
+                s_d[pos] = v;
+                s_code[pos] = code;
+            }
         }
     }
     __syncthreads();
@@ -458,7 +472,6 @@ build_candidates_kernel(const DevState *__restrict__ st, int B, int S, double ta
         for (int e = n + tid; e < n2; e += blockDim.x) { s_d[e] = INFINITY; s_code[e] = 0x7fffffff; }
         block_sort_asc(s_d, s_code, n2);
     }
-    const size_t base = (size_t)i * (2 * kMaxBatch);
     for (int e = tid; e < n; e += blockDim.x) {
         cand_d[base + e] = s_d[e];
         cand_code[base + e] = s_code[e];
@@ -1023,7 +1036,7 @@ void launch_risk_select(prox_handle *h, int B, cudaStream_t s) {
 void launch_probe(prox_handle *h, const float *q, int B, int mode, cudaStream_t s) {
     int splits = probe_splits(h, B);
     const int PC = probe_cols(h, B);
-    if (mode == 1) {                                      // at most 2 * kMaxBatch columns
+    if (mode == 1 || mode == 4) {                         // at most 2 * kMaxBatch columns
         const int tiles = (2 * B + PC - 1) / PC;
         if (splits > tiles) splits = tiles;
     }
@@ -1035,11 +1048,11 @@ void launch_probe(prox_handle *h, const float *q, int B, int mode, cudaStream_t 
     h->launches++;
 }
 
-void launch_build_candidates(prox_handle *h, int B, cudaStream_t s) {
-    build_candidates_kernel<<<B, 128, 0, s>>>(h->st, B, probe_splits(h, B), (double)h->tau, h->part_min,
+void launch_build_candidates(prox_handle *h, int B, int splits, int lists_ready, cudaStream_t s) {
+    build_candidates_kernel<<<B, 128, 0, s>>>(h->st, B, splits < 0 ? probe_splits(h, B) : splits, (double)h->tau, h->part_min,
                                               h->part_arg, h->d_risk, h->d_intra, h->safe_min,
                                               h->safe_arg, h->cand_d, h->cand_code, h->n_cand,
-                                              h->probe_tc ? h->use_partial : nullptr);
+                                              h->probe_tc ? h->use_partial : nullptr, lists_ready);
     h->launches++;
 }
 
@@ -1066,7 +1079,7 @@ void launch_scatter(prox_handle *h, const float *q, int B, int64_t *out_ids, flo
                     int with_values, cudaStream_t s) {
     scatter_kernel<<<B, 128, 0, s>>>(B, h->d, h->k, h->k_out, with_values, q, h->src, h->src_kind, h->ins_slot,
                                      h->miss_rank, h->res_ids, h->res_dists, h->keys, h->val_ids,
-                                     h->val_dists, out_ids, out_dists, h->probe_tc ? h->keys_b : nullptr, h->kh,
+                                     h->val_dists, out_ids, out_dists, h->key_copies ? h->keys_b : nullptr, h->kh,
                                      h->st);
     h->launches++;
 }
@@ -1079,17 +1092,17 @@ void launch_probe_outputs(prox_handle *h, int B, int32_t *out_slot, float *out_m
 
 void launch_reset(prox_handle *h, cudaStream_t s) {
     const long long C = h->C;
-    reset_kernel<<<(unsigned)((C + 255) / 256), 256, 0, s>>>(h->st, h->risk_pos, C, 0, h->probe_tc ? h->kh : nullptr);
+    reset_kernel<<<(unsigned)((C + 255) / 256), 256, 0, s>>>(h->st, h->risk_pos, C, 0, h->key_copies ? h->kh : nullptr);
     h->launches++;
 }
 
 void launch_cache_load(prox_handle *h, const float *keys, int64_t n, cudaStream_t s) {
     const long long C = h->C;
-    reset_kernel<<<(unsigned)((C + 255) / 256), 256, 0, s>>>(h->st, h->risk_pos, C, (long long)n, h->probe_tc ? h->kh : nullptr);
+    reset_kernel<<<(unsigned)((C + 255) / 256), 256, 0, s>>>(h->st, h->risk_pos, C, (long long)n, h->key_copies ? h->kh : nullptr);
     h->launches++;
     if (n > 0) {
         cache_load_kernel<<<(unsigned)n, 128, 0, s>>>((long long)n, h->d, h->k, keys, h->keys, h->val_ids,
-                                                      h->val_dists, h->stamp, h->probe_tc ? h->keys_b : nullptr,
+                                                      h->val_dists, h->stamp, h->key_copies ? h->keys_b : nullptr,
                                                       h->kh, h->st);
         h->launches++;
     }

@@ -91,7 +91,7 @@ static void free_all(prox_handle *h) {
                     h->qerr, h->thr_g, h->top1, h->buf, h->buf_cnt, h->cand_id, h->cand_score, h->cand_n,
                     h->cand_sk, h->res_ids, h->res_dists, h->fail_list, h->fail_radius, h->coll_id,
                     h->coll_n, h->stage_q, h->stage_ids, h->stage_dists, h->stage_hit, h->keys_b, h->kh, h->pqb,
-                    h->pqbn, h->pqerr, h->use_partial, h->pfail_list};
+                    h->pqbn, h->pqerr, h->use_partial, h->pfail_list, h->side_pairs};
     for (void *p : ptrs)
         if (p) cudaFree(p);
 }
@@ -180,8 +180,11 @@ static prox_handle *create_handle(const float *corpus, int64_t N, int32_t d, int
     ok = ok && dev_alloc(h->qb, MB * d) && dev_alloc(h->qbn, MB) && dev_alloc(h->qerr, MB) && dev_alloc(h->thr_g, MB);
     ok = ok && dev_alloc(h->top1, MB * 4 * P);          // per query: best score of every block's lane quarter
     h->tc_cap = h->kp <= 128 ? 256 : 512;               // four warp-private lists per block in the tensor-core scan
-    const size_t buf_entries = P * kScanQ * (size_t)(4 * h->tc_cap > kBufCap ? 4 * h->tc_cap : kBufCap);
-    ok = ok && dev_alloc(h->buf, buf_entries) && dev_alloc(h->buf_cnt, 4 * P * kScanQ);
+    // every pass of a batch (kScanQ queries each) keeps its lists until the one merge at the end
+    constexpr size_t kPasses = kMaxBatch / kScanQ;
+    h->buf_pass_stride = P * kScanQ * (size_t)(4 * h->tc_cap > kBufCap ? 4 * h->tc_cap : kBufCap);
+    h->cnt_pass_stride = 4 * P * kScanQ;
+    ok = ok && dev_alloc(h->buf, kPasses * h->buf_pass_stride) && dev_alloc(h->buf_cnt, kPasses * h->cnt_pass_stride);
     ok = ok && dev_alloc(h->cand_id, MB * kMaxKp) && dev_alloc(h->cand_score, MB * kMaxKp);
     ok = ok && dev_alloc(h->cand_n, MB) && dev_alloc(h->cand_sk, MB);
     ok = ok && dev_alloc(h->res_ids, MB * k) && dev_alloc(h->res_dists, MB * k);
@@ -193,9 +196,13 @@ static prox_handle *create_handle(const float *corpus, int64_t N, int32_t d, int
     // (the coarse probe's certificate is written for the Euclidean distance)
     h->probe_tc = (d % 64 == 0 && capacity >= 4096 && metric != PROX_METRIC_IP) ? 1 : 0;
     ok = ok && dev_alloc(h->use_partial, MB) && dev_alloc(h->pfail_list, MB);
-    if (h->probe_tc) {
+    // bf16 copies of the keys and of the batch: for the coarse probe of large caches and for the
+    // tensor-core pass over the at-risk slots and the batch itself (large batches)
+    h->key_copies = metric != PROX_METRIC_IP ? 1 : 0;
+    if (h->key_copies) {
         ok = ok && dev_alloc(h->keys_b, C * d) && dev_alloc(h->kh, C);
         ok = ok && dev_alloc(h->pqb, MB * d) && dev_alloc(h->pqbn, MB) && dev_alloc(h->pqerr, MB);
+        ok = ok && dev_alloc(h->side_pairs, (size_t)kPairCap);
     }
     ok = ok && dev_alloc(h->stage_q, MB * d) && dev_alloc(h->stage_ids, MB * k);
     ok = ok && dev_alloc(h->stage_dists, MB * k) && dev_alloc(h->stage_hit, MB);
@@ -207,11 +214,11 @@ static prox_handle *create_handle(const float *corpus, int64_t N, int32_t d, int
     }
     cudaMemset(h->st, 0, sizeof(DevState));
     cudaMemset(h->qb, 0, MB * d * sizeof(__nv_bfloat16));
-    if (h->probe_tc) {
+    if (h->key_copies) {
         cudaMemset(h->pqb, 0, MB * d * sizeof(__nv_bfloat16));
         cudaMemset(h->keys_b, 0, C * d * sizeof(__nv_bfloat16));
     }
-    cudaMemset(h->buf_cnt, 0, 4 * P * kScanQ * sizeof(int32_t));
+    cudaMemset(h->buf_cnt, 0, kPasses * h->cnt_pass_stride * sizeof(int32_t));
     cudaMemset(h->over_ticket, 0, kOverMax * sizeof(unsigned));
     launch_convert_corpus(h, 0);
     launch_reset(h, 0);
@@ -263,7 +270,7 @@ extern "C" prox_handle *prox_create_lsh(const float *corpus, int64_t N, int32_t 
     prox_handle *h = prox_create_rho(corpus, N, d, k, (int64_t)b << L, tau, policy, rho);
     if (!h) return nullptr;
     h->lsh_L = L; h->lsh_b = b;
-    h->probe_tc = 0;                                      // buckets are probed directly; no bf16 key copies
+    h->probe_tc = 0; h->key_copies = 0;                   // buckets are probed directly; no bf16 key copies are kept
     const size_t MB = kMaxBatch;
     bool ok = dev_alloc(h->planes, (size_t)(L > 0 ? L : 1) * d) && dev_alloc(h->bucket_count, (size_t)1 << L) &&
               dev_alloc(h->lsh_code, MB) && dev_alloc(h->lsh_order, MB) && dev_alloc(h->lsh_seg, MB + 1) &&
@@ -307,31 +314,43 @@ static void enqueue_probe_and_resolve(prox_handle *h, const float *queries, int3
         return;
     }
     { StageScope t(h, PROX_STAGE_RISK_SELECT, s); launch_risk_select(h, B, s); }
+    // large batches: the at-risk slots and the batch itself on the tensor cores, exact recheck of the
+    // pairs that could lie within tau (instead of B x 2B fp64 rows)
+    const bool side = h->key_copies && h->scan_mode != PROX_SCAN_CUDA_CORE && B >= kSideMinBatch;
+    int splits = -1;
     {
         StageScope t(h, PROX_STAGE_PROBE, s);
         // the coarse pass has a fixed cost of a few launches: it pays off from about two million
         // query-key pairs per batch on
         bool coarse = h->probe_tc && h->scan_mode != PROX_SCAN_CUDA_CORE && (long long)B * h->C >= 2LL * (1 << 20);
+        if (coarse || side) launch_prep_probe(h, queries, B, s);
         if (coarse) {
             // safe slots: coarse scores on the tensor cores, exact recheck of the best few;
-            // at-risk slots and the batch itself: full fp64 rows; uncertified queries: fp64 over all slots
-            launch_prep_probe(h, queries, B, s);
+            // at-risk slots and the batch itself: full fp64 rows (or the pass above); uncertified
+            // queries: fp64 over all slots
             const int passes = (B + kScanQ - 1) / kScanQ;
-            for (int p = 0; p < passes && coarse; ++p) {
-                if (launch_probe_scan_tc(h, p, s) != 0) { coarse = false; break; }
-                launch_merge_select(h, p, B, 1, s);
-            }
+            for (int p = 0; p < passes && coarse; ++p)
+                if (launch_probe_scan_tc(h, p, s) != 0) coarse = false;
+            if (coarse) launch_merge_select(h, B, 1, s);
         }
+        if (side) launch_probe_side(h, queries, B, s);
         if (coarse) {
             launch_probe_exact(h, queries, B, s);
-            launch_probe(h, queries, B, 1, s);
+            launch_probe(h, queries, B, side ? 4 : 1, s);
             launch_probe(h, queries, B, 2, s);
         } else {
             if (h->probe_tc) cudaMemsetAsync(h->use_partial, 0xff, sizeof(int32_t) * kMaxBatch, s);   // all from partials
-            launch_probe(h, queries, B, 0, s);
+            if (side) {
+                // a capacity within the batch size: every stored key is at risk, there is no safe slot to scan
+                if (h->C > B) launch_probe(h, queries, B, 3, s);
+                else splits = 0;
+                launch_probe(h, queries, B, 4, s);
+            } else {
+                launch_probe(h, queries, B, 0, s);
+            }
         }
     }
-    { StageScope t(h, PROX_STAGE_CANDIDATES, s); launch_build_candidates(h, B, s); }
+    { StageScope t(h, PROX_STAGE_CANDIDATES, s); launch_build_candidates(h, B, splits, side ? 1 : 0, s); }
     { StageScope t(h, PROX_STAGE_RESOLVE, s); launch_resolve(h, B, out_hit, s); }
 }
 
@@ -354,13 +373,20 @@ static const float *enqueue_lookup_and_scan(prox_handle *h, const float *queries
     }
     { StageScope t(h, PROX_STAGE_PREP_MISS, s); launch_prep_miss(h, queries, B, s); }
     const int passes = (B + kScanQ - 1) / kScanQ;
-    for (int p = 0; p < passes; ++p) {
-        {
-            StageScope t(h, PROX_STAGE_SCAN, s);
-            if (h->scan_mode == PROX_SCAN_CUDA_CORE || launch_scan_pass_tc(h, p, s) != 0) launch_scan_pass(h, p, s);
+    {
+        StageScope t(h, PROX_STAGE_SCAN, s);
+        // one kind of scan for all passes of a batch: the merge reads every pass's lists in one layout
+        bool tc = h->scan_mode != PROX_SCAN_CUDA_CORE;
+        for (int p = 0; p < passes; ++p) {
+            if (tc && launch_scan_pass_tc(h, p, s) != 0) {
+                tc = false;
+                p = -1;                                    // (before the first pass has run: start again on the CUDA cores)
+                continue;
+            }
+            if (!tc) launch_scan_pass(h, p, s);
         }
-        { StageScope t(h, PROX_STAGE_MERGE, s); launch_merge_select(h, p, B, 0, s); }
     }
+    { StageScope t(h, PROX_STAGE_MERGE, s); launch_merge_select(h, B, 0, s); }
     { StageScope t(h, PROX_STAGE_RERANK, s); launch_rerank(h, queries, B, s); }
     { StageScope t(h, PROX_STAGE_EXACT_PASS, s); launch_fallback(h, queries, B, s); }
     return queries;

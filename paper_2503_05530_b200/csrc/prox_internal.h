@@ -18,6 +18,8 @@ constexpr int kBufCap = 512;                 // entries of one (CTA, query) cand
 constexpr int kCollectCap = 2048;            // rows the exact pass may collect per query
 constexpr int kOverMax = 64;                 // queries per batch whose collection may overflow and still be answered exactly
 constexpr int kProbeSplitMax = 64;           // column splits of the probe grid
+constexpr int kPairCap = 1 << 20;             // query-key pairs the tensor-core pass over at-risk slots and batch may hand on
+constexpr int kSideMinBatch = 512;            // batches from this size on take that pass instead of fp64 rows
 constexpr int kProbeKp = 64;                 // slots per query the coarse probe keeps for the exact recheck
 
 // Device-resident scalars of a handle.
@@ -35,6 +37,8 @@ struct DevState {
     int n_probe;              // queries of the current batch (read by the coarse probe's kernels)
     int n_pfail;              // queries whose coarse probe was not certified
     int n_over;               // queries whose exact pass collected more rows than it can hold
+    int n_pairs;              // pairs listed by the tensor-core pass over the at-risk slots and the batch
+    int side_overflow;        // 1 = more such pairs than the list holds: the fp64 rows are used instead
     // statistics
     long long queries, hits, misses, intra_hits, evictions, scan_batches, uncertified,
         fallback_rows, unresolved, probe_uncertified;
@@ -113,6 +117,8 @@ struct prox_handle {
     int32_t *use_partial;             // kMaxBatch: 1 = the safe minimum comes from the fp64 probe's partial minima
     int32_t *pfail_list;              // kMaxBatch: queries that take the exact fp64 probe
     int32_t probe_tc;                 // 1 = coarse tensor-core probe in use for this handle
+    int32_t key_copies;               // 1 = bf16 copies of the keys are kept (coarse probe, tensor-core pass over at-risk slots)
+    uint32_t *side_pairs;             // kPairCap: (query << 16 | code) of the pairs that pass
     void *tc_state_keys;              // tensor maps of the coarse probe
     int32_t *miss_list;               // kMaxBatch
     int32_t *miss_rank;               // kMaxBatch
@@ -125,6 +131,8 @@ struct prox_handle {
     unsigned long long *buf;          // candidate lists of the scan blocks (layout set by the scan that ran)
     int32_t *buf_cnt;                 // entries per list
     int32_t scan_ctas;                // P
+    size_t buf_pass_stride;           // entries of `buf` that one scan pass (up to kScanQ queries) owns
+    size_t cnt_pass_stride;           // entries of `buf_cnt` that one scan pass owns
     int32_t scan_lists;               // lists per query written by the last scan pass
     int32_t scan_list_stride;         // entries between consecutive (list, query) buffers
     int32_t tc_cap;                   // entries per (warp, query) buffer of the tensor-core scan
@@ -160,8 +168,8 @@ void launch_convert_corpus(prox_handle *h, cudaStream_t s);
 inline bool metric_is_ip(const prox_handle *h) { return h->metric == PROX_METRIC_IP; }
 // cache kernels
 void launch_risk_select(prox_handle *h, int B, cudaStream_t s);
-void launch_probe(prox_handle *h, const float *q, int B, int mode, cudaStream_t s);   // 0 all slots, 1 at-risk + batch, 2 failed queries
-void launch_build_candidates(prox_handle *h, int B, cudaStream_t s);
+void launch_probe(prox_handle *h, const float *q, int B, int mode, cudaStream_t s);   // 0 all slots + batch, 1 at-risk + batch, 2 failed queries, 3 safe slots only, 4 = 1 if the pair list overflowed
+void launch_build_candidates(prox_handle *h, int B, int splits, int lists_ready, cudaStream_t s);   // splits < 0: as the probe used
 void launch_resolve(prox_handle *h, int B, uint8_t *out_hit, cudaStream_t s);
 void launch_gather_hits(prox_handle *h, int B, int64_t *out_ids, float *out_dists, cudaStream_t s);
 void launch_hit_rerank(prox_handle *h, const float *q, int B, int kind, int64_t *out_ids, float *out_dists,
@@ -179,11 +187,12 @@ void launch_prep_miss(prox_handle *h, const float *q, int B, cudaStream_t s);
 void launch_prep_probe(prox_handle *h, const float *q, int B, cudaStream_t s);
 int launch_probe_scan_tc(prox_handle *h, int pass, cudaStream_t s);    // coarse probe over the bf16 keys; nonzero = not available
 void launch_probe_exact(prox_handle *h, const float *q, int B, cudaStream_t s);
+void launch_probe_side(prox_handle *h, const float *q, int B, cudaStream_t s);   // at-risk slots and batch on the tensor cores -> candidate lists
 void launch_scan_pass(prox_handle *h, int pass, cudaStream_t s);       // CUDA-core scan
 int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s);     // tcgen05 scan; nonzero = not available
 void init_scan_tc(prox_handle *h);                                      // tensor maps, at prox_create
 void free_scan_tc(prox_handle *h);
-void launch_merge_select(prox_handle *h, int pass, int B, int for_probe, cudaStream_t s);
+void launch_merge_select(prox_handle *h, int B, int for_probe, cudaStream_t s);   // all passes of the batch at once
 void launch_rerank(prox_handle *h, const float *q, int B, cudaStream_t s);
 void launch_fallback(prox_handle *h, const float *q, int B, cudaStream_t s);
 // row shards

@@ -241,18 +241,20 @@ struct MergeSrc {
 };
 
 __global__ void __launch_bounds__(1024, 2)
-merge_select_kernel(const int *__restrict__ n_active, int pass, int n_lists, int stride, int kp, int stage_cap,
-                    const u64 *__restrict__ buf, const int32_t *__restrict__ buf_cnt,
-                    const uint32_t *__restrict__ thr_g, int32_t *cand_id, float *cand_score, int32_t *cand_n,
-                    float *cand_sk) {
+merge_select_kernel(const int *__restrict__ n_active, int n_lists, int stride, int kp, int stage_cap,
+                    const u64 *__restrict__ buf, const int32_t *__restrict__ buf_cnt, size_t buf_pass_stride,
+                    size_t cnt_pass_stride, const uint32_t *__restrict__ thr_g, int32_t *cand_id, float *cand_score,
+                    int32_t *cand_n, float *cand_sk) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     u64 *stage = reinterpret_cast<u64 *>(smem_raw);
     __shared__ unsigned hist[256];
     __shared__ uint32_t s_prefix, s_mask;
     __shared__ int s_remaining, s_total, s_gt, s_eq;
-    const int q = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int m = pass * kScanQ + q;
+    const int m = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (m >= *n_active) return;
+    const int pass = m / kScanQ, q = m - pass * kScanQ;    // every pass of the batch has its own lists
+    buf += (size_t)pass * buf_pass_stride;
+    buf_cnt += (size_t)pass * cnt_pass_stride;
 
     if (tid == 0) { s_total = 0; s_gt = 0; s_eq = 0; }
     __syncthreads();
@@ -362,7 +364,9 @@ merge_select_kernel(const int *__restrict__ n_active, int pass, int n_lists, int
     }
     if (tid == 0) {
         cand_n[m] = keep;
-        cand_sk[m] = (total >= kp) ? o2f(T) : -INFINITY;
+        // fewer than k' entries: no row outside them scored above the bound the scan started from
+        // (-inf for the corpus scan: every row is a candidate; the tolerance's bound for the probe)
+        cand_sk[m] = (total >= kp) ? o2f(T) : o2f(g0);
     }
 }
 
@@ -848,21 +852,28 @@ overflow_topk_kernel(DevState *st, const float *__restrict__ corpus, const float
 //   - no slot outside the candidates can be within tau.
 // Otherwise the query is handed to the exact fp64 probe over all slots.
 // ------------------------------------------------------------------------------------------
+// Largest coarse squared distance that a pair whose true squared distance is at most tau can show:
+// rounding to bf16 moves either vector by at most a resp. e, the fp32 sum and norms by the slack.
+__device__ __forceinline__ double coarse_bound(double tau, double a, double e, double qn, double kn, int d) {
+    const double slack = 4.0 * (double)(d + 16) * 5.9604644775390625e-08 * (2.0 * qn * kn + kn * kn + qn * qn);
+    const double r = sqrt(tau) + a + e;
+    return r * r * (1.0 + 1e-6) + slack * (1.0 + 1e-6) + 4e-7 * (qn * qn + kn * kn) + 1e-30;
+}
+
 __global__ void __launch_bounds__(128)
-prep_probe_kernel(DevState *st, const float *__restrict__ queries, int B, int d, __nv_bfloat16 *pqb, float *pqbn,
-                  float *pqerr, uint32_t *thr_g, uint32_t *top1, int n_blocks, int32_t *use_partial) {
+prep_probe_kernel(DevState *st, const float *__restrict__ queries, int B, int d, double tau, __nv_bfloat16 *pqb,
+                  float *pqbn, float *pqerr, uint32_t *thr_g, uint32_t *top1, int n_blocks, int32_t *use_partial,
+                  int32_t *n_cand) {
     __shared__ float red[2][4];
     const int m = blockIdx.x, tid = threadIdx.x;
-    if (m == 0) {
-        for (int i = tid; i < kMaxBatch; i += blockDim.x) thr_g[i] = f2o(-INFINITY);
-        if (tid == 0) { st->n_probe = B; st->n_pfail = 0; }
-    }
+    if (m == 0 && tid == 0) { st->n_probe = B; st->n_pfail = 0; st->n_pairs = 0; st->side_overflow = 0; }
     for (int i = tid; i < n_blocks; i += blockDim.x) top1[(size_t)m * n_blocks + i] = 0u;
     if (m >= B) {
+        if (tid == 0) thr_g[m] = f2o(-INFINITY);
         for (int j = tid; j < d; j += blockDim.x) pqb[(size_t)m * d + j] = __float2bfloat16_rn(0.f);
         return;
     }
-    if (tid == 0) use_partial[m] = 0;
+    if (tid == 0) { use_partial[m] = 0; n_cand[m] = 0; }
     const float *src = queries + (size_t)m * d;
     float nn = 0.f, ee = 0.f;
     for (int j = tid; j < d; j += blockDim.x) {
@@ -881,8 +892,15 @@ prep_probe_kernel(DevState *st, const float *__restrict__ queries, int B, int d,
     if ((tid & 31) == 0) { red[0][tid >> 5] = nn; red[1][tid >> 5] = ee; }
     __syncthreads();
     if (tid == 0) {
-        pqbn[m] = red[0][0] + red[0][1] + red[0][2] + red[0][3];
-        pqerr[m] = sqrtf(red[1][0] + red[1][1] + red[1][2] + red[1][3]) * 1.0001f;
+        const float n2 = red[0][0] + red[0][1] + red[0][2] + red[0][3];
+        const float err = sqrtf(red[1][0] + red[1][1] + red[1][2] + red[1][3]) * 1.0001f;
+        pqbn[m] = n2;
+        pqerr[m] = err;
+        // The scan starts from the tolerance's bound instead of an open threshold: a key whose coarse
+        // score is below it cannot lie within tau, and only a key within tau matters to the lookup.
+        // score = (|bf16 q|^2 - coarse distance) / 2, rounded down.
+        const double T = coarse_bound(tau, (double)err, (double)st->ke_max, sqrt((double)n2), (double)st->kn_max, d);
+        thr_g[m] = f2o(__double2float_rd(0.5 * ((double)n2 - T)));
     }
 }
 
@@ -956,21 +974,19 @@ void launch_scan_pass(prox_handle *h, int pass, cudaStream_t s) {
     h->scan_lists = h->scan_ctas;                         // one candidate list per block and query
     h->scan_list_stride = kBufCap;
     scan_cc_kernel<<<h->scan_ctas, 256, 0, s>>>(h->st, h->xb, h->xh, h->qb, (long long)h->N, h->d, pass,
-                                                h->kp, h->thr_g, h->top1, h->buf, h->buf_cnt);
+                                                h->kp, h->thr_g, h->top1, h->buf + (size_t)pass * h->buf_pass_stride,
+                                                h->buf_cnt + (size_t)pass * h->cnt_pass_stride);
     h->launches++;
 }
 
-void launch_merge_select(prox_handle *h, int pass, int B, int for_probe, cudaStream_t s) {
-    int nq = B - pass * kScanQ;
-    if (nq > kScanQ) nq = kScanQ;
-    if (nq <= 0) return;
+void launch_merge_select(prox_handle *h, int B, int for_probe, cudaStream_t s) {
     // a scan of few rows never tightens its bounds, so every row may still be in the lists: stage them all
     const long long rows = for_probe ? (long long)h->C : (long long)h->N;
     const int stage_cap = rows <= kMergeStageMax ? (int)((rows + 1023) / 1024 * 1024) : kMergeStage;
-    merge_select_kernel<<<nq, 1024, (size_t)stage_cap * 8, s>>>(for_probe ? &h->st->n_probe : &h->st->n_miss, pass,
-                                                          h->scan_lists, h->scan_list_stride, for_probe ? kProbeKp : h->kp, stage_cap,
-                                                          h->buf, h->buf_cnt, h->thr_g, h->cand_id, h->cand_score,
-                                                          h->cand_n, h->cand_sk);
+    merge_select_kernel<<<B, 1024, (size_t)stage_cap * 8, s>>>(for_probe ? &h->st->n_probe : &h->st->n_miss,
+                                                         h->scan_lists, h->scan_list_stride, for_probe ? kProbeKp : h->kp, stage_cap,
+                                                         h->buf, h->buf_cnt, h->buf_pass_stride, h->cnt_pass_stride, h->thr_g,
+                                                         h->cand_id, h->cand_score, h->cand_n, h->cand_sk);
     h->launches++;
 }
 
@@ -1033,8 +1049,8 @@ namespace prox {
 void launch_prep_probe(prox_handle *h, const float *q, int B, cudaStream_t s) {
     int rows = ((B + kScanQ - 1) / kScanQ) * kScanQ;
     if (rows > kMaxBatch) rows = kMaxBatch;
-    prep_probe_kernel<<<rows, 128, 0, s>>>(h->st, q, B, h->d, h->pqb, h->pqbn, h->pqerr, h->thr_g, h->top1,
-                                           4 * h->scan_ctas, h->use_partial);
+    prep_probe_kernel<<<rows, 128, 0, s>>>(h->st, q, B, h->d, (double)h->tau, h->pqb, h->pqbn, h->pqerr, h->thr_g, h->top1,
+                                           4 * h->scan_ctas, h->use_partial, h->n_cand);
     h->launches++;
 }
 

@@ -590,8 +590,8 @@ static int launch_scan_generic(prox_handle *h, void **state, const __nv_bfloat16
     Maps &maps = *static_cast<Maps *>(*state);
     if (!maps.ok) return 1;
     ScanArgs a;
-    a.st = h->st; a.n_active = n_active; a.xh = xh; a.thr_g = h->thr_g; a.top1 = h->top1; a.buf = h->buf;
-    a.buf_cnt = h->buf_cnt; a.N = rows; a.d = h->d; a.pass = pass; a.kp = kp; a.ks = maps.ks;
+    a.st = h->st; a.n_active = n_active; a.xh = xh; a.thr_g = h->thr_g; a.top1 = h->top1; a.buf = h->buf + (size_t)pass * h->buf_pass_stride;
+    a.buf_cnt = h->buf_cnt + (size_t)pass * h->cnt_pass_stride; a.N = rows; a.d = h->d; a.pass = pass; a.kp = kp; a.ks = maps.ks;
     const bool pair = h->scan_mode != PROX_SCAN_TC_SINGLE && h->scan_ctas >= 2 && rows >= 2 * kTileRows;
     const int grid = pair ? (h->scan_ctas & ~1) : h->scan_ctas;
     const int units = pair ? grid / 2 : grid;
