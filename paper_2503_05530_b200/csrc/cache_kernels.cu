@@ -512,6 +512,8 @@ struct ResolveSmem {
     int plain_before[kMaxBatch];       // per entangled query (by its place in ent_list): plain misses before it
     int warp_tot[3][32];
     int one[1];
+    int head[kMaxBatch];               // first entry of the query's list that may still be a resident key
+    unsigned char kind[kMaxBatch];     // 1 settled (hits a safe key), 2 plain miss, 3 entangled
     unsigned char r_alive[kMaxBatch];
     unsigned char r_touched[kMaxBatch];
 };
@@ -625,32 +627,24 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
     const long long count0 = st->count, clock0 = st->clock;
     ResolveOut o{out_hit, src, src_kind, evt_slot, miss_list, miss_rank, evt_dist};
 
-    // ---- load, classify, three prefix sums (candidates, plain misses, entangled queries)
+    // ---- load and classify
     int n_plain = 0, n_ent = 0, n_settled = 0;
     {
         const int i = tid;
         int n = 0, kind = 0;                               // 1 settled, 2 plain miss, 3 entangled
+        double sd = INFINITY;
+        int sa = -1;
+        bool safe_hit = false;
         if (i < B) {
             n = n_cand[i];
-            const double sd = g_safe_min[i];
-            const int sa = g_safe_arg[i];
+            sd = g_safe_min[i];
+            sa = g_safe_arg[i];
             sm.safe_min[i] = sd;
             sm.safe_arg[i] = sa;
             sm.b_slot[i] = -1;
             sm.b_stamp[i] = 0;
-            const bool safe_hit = sa >= 0 && sd <= tau;
+            safe_hit = sa >= 0 && sd <= tau;
             kind = n > 0 ? 3 : (safe_hit ? 1 : 2);
-            // A query with no at-risk or in-batch key within tau whose nearest safe key is within tau
-            // hits that key whatever the rest of the batch does (safe keys are not evicted in this
-            // batch, and touching one changes no eviction of this batch): settled here, in parallel.
-            if (kind == 1) {
-                out_hit[i] = 1;
-                evt_slot[i] = sa;
-                evt_dist[i] = (float)sd;
-                miss_rank[i] = -1;
-                src_kind[i] = 1; src[i] = sa;
-                if (policy == PROX_LRU) atomicMax(&stamp[sa], (u64)(clock0 + i));     // the latest hit stays
-            }
         }
         if (i < R) {
             sm.r_slot[i] = risk_slot[i];
@@ -658,38 +652,29 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
             sm.r_alive[i] = 1;
             sm.r_touched[i] = 0;
         }
-        if (i < kMaxBatch) sm.ncand[i] = n;
-        int x[3] = {n, kind == 2 ? 1 : 0, kind == 3 ? 1 : 0};
+        if (i < kMaxBatch) { sm.ncand[i] = n; sm.kind[i] = (unsigned char)kind; sm.head[i] = 0; }
+        // exclusive prefix sum of the list lengths: where each list sits in the shared copy
+        int x = n;
 #pragma unroll
         for (int m = 1; m < 32; m <<= 1) {
-#pragma unroll
-            for (int c = 0; c < 3; ++c) {
-                const int y = __shfl_up_sync(0xffffffffu, x[c], m);
-                if (lane >= m) x[c] += y;
-            }
+            const int y = __shfl_up_sync(0xffffffffu, x, m);
+            if (lane >= m) x += y;
         }
-        if (lane == 31) { sm.warp_tot[0][warp] = x[0]; sm.warp_tot[1][warp] = x[1]; sm.warp_tot[2][warp] = x[2]; }
+        if (lane == 31) sm.warp_tot[0][warp] = x;
         __syncthreads();
-        if (warp < 3) {
-            int w = sm.warp_tot[warp][lane];
+        if (warp == 0) {
+            int w = sm.warp_tot[0][lane];
 #pragma unroll
             for (int m = 1; m < 32; m <<= 1) {
                 const int y = __shfl_up_sync(0xffffffffu, w, m);
                 if (lane >= m) w += y;
             }
-            sm.warp_tot[warp][lane] = w;
+            sm.warp_tot[0][lane] = w;
         }
         __syncthreads();
-        const int incl_n = x[0] + (warp > 0 ? sm.warp_tot[0][warp - 1] : 0);
-        const int excl_plain = x[1] + (warp > 0 ? sm.warp_tot[1][warp - 1] : 0) - (kind == 2 ? 1 : 0);
-        const int excl_ent = x[2] + (warp > 0 ? sm.warp_tot[2][warp - 1] : 0) - (kind == 3 ? 1 : 0);
+        const int incl_n = x + (warp > 0 ? sm.warp_tot[0][warp - 1] : 0);
         if (i < kMaxBatch) sm.off[i] = incl_n - n;
         if (i == kMaxBatch - 1) sm.off[kMaxBatch] = incl_n;
-        if (kind == 2) sm.plain_list[excl_plain] = i;
-        if (kind == 3) { sm.ent_list[excl_ent] = i; sm.plain_before[excl_ent] = excl_plain; }
-        n_plain = sm.warp_tot[1][31];
-        n_ent = sm.warp_tot[2][31];
-        n_settled = B - n_plain - n_ent;
         __syncthreads();
         for (int row = warp; row < B; row += 32) {
             const int off = sm.off[row], nn = sm.ncand[row];
@@ -699,6 +684,74 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
                     sm.csr_code[off + e] = cand_code[(size_t)row * (2 * kMaxBatch) + e];
                 }
         }
+        __syncthreads();
+
+        // Most queries with a listed key can still be decided without the others.  A listed query of
+        // the batch that is known to hit was never inserted: it cannot be anyone's key, so it drops
+        // off the front of the lists; and when the nearest safe key is strictly nearer than the first
+        // listed key that could still be resident, the query hits that safe key whatever happens to
+        // the listed ones.  A few rounds, each one settling what the round before made decidable.
+        for (int round = 0; round < 4; ++round) {
+            bool changed = false;
+            if (i < B && kind == 3) {
+                const int off = sm.off[i];
+                const bool in_smem = off + n <= kCsrCap;
+                const int *lc = in_smem ? sm.csr_code + off : cand_code + (size_t)i * (2 * kMaxBatch);
+                const double *ld = in_smem ? sm.csr_d + off : cand_d + (size_t)i * (2 * kMaxBatch);
+                int hd = sm.head[i];
+                while (hd < n) {
+                    const int code = lc[hd];
+                    if (code >= kMaxBatch && sm.kind[code - kMaxBatch] == 1) ++hd;
+                    else break;
+                }
+                sm.head[i] = hd;
+                if (hd == n) { kind = safe_hit ? 1 : 2; changed = true; }
+                else if (safe_hit && sd < ld[hd]) { kind = 1; changed = true; }
+            }
+            __syncthreads();                               // everyone has read the kinds of this round
+            if (changed) sm.kind[i] = (unsigned char)kind;
+            if (!__syncthreads_or(changed ? 1 : 0)) break;
+        }
+        // a settled query hits its nearest safe key: safe keys are not evicted in this batch, and
+        // touching one changes no eviction of this batch
+        if (i < B && kind == 1) {
+            out_hit[i] = 1;
+            evt_slot[i] = sa;
+            evt_dist[i] = (float)sd;
+            miss_rank[i] = -1;
+            src_kind[i] = 1; src[i] = sa;
+            if (policy == PROX_LRU) atomicMax(&stamp[sa], (u64)(clock0 + i));     // the latest hit stays
+        }
+
+        // plain misses and entangled queries, each in index order
+        int y2[2] = {kind == 2 ? 1 : 0, kind == 3 ? 1 : 0};
+#pragma unroll
+        for (int m = 1; m < 32; m <<= 1) {
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                const int y = __shfl_up_sync(0xffffffffu, y2[c], m);
+                if (lane >= m) y2[c] += y;
+            }
+        }
+        if (lane == 31) { sm.warp_tot[1][warp] = y2[0]; sm.warp_tot[2][warp] = y2[1]; }
+        __syncthreads();
+        if (warp == 1 || warp == 2) {
+            int w = sm.warp_tot[warp][lane];
+#pragma unroll
+            for (int m = 1; m < 32; m <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, w, m);
+                if (lane >= m) w += y;
+            }
+            sm.warp_tot[warp][lane] = w;
+        }
+        __syncthreads();
+        const int excl_plain = y2[0] + (warp > 0 ? sm.warp_tot[1][warp - 1] : 0) - (kind == 2 ? 1 : 0);
+        const int excl_ent = y2[1] + (warp > 0 ? sm.warp_tot[2][warp - 1] : 0) - (kind == 3 ? 1 : 0);
+        if (kind == 2) sm.plain_list[excl_plain] = i;
+        if (kind == 3) { sm.ent_list[excl_ent] = i; sm.plain_before[excl_ent] = excl_plain; }
+        n_plain = sm.warp_tot[1][31];
+        n_ent = sm.warp_tot[2][31];
+        n_settled = B - n_plain - n_ent;
         __syncthreads();
     }
 
@@ -722,7 +775,19 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
             // the same distance the lowest slot
             double bd = INFINITY;
             int bslot = 0x7fffffff, bcode = -1;
-            for (int e0 = 0; e0 < n && bcode == -1; e0 += 32) {
+            const int h0 = sm.head[i];
+            {
+                // common case, without a vote: the first listed entry is resident and no other entry is
+                // exactly as near
+                const int code = lc[h0];
+                int slot;
+                bool valid;
+                if (code < kMaxBatch) { valid = sm.r_alive[code] != 0; slot = sm.r_slot[code]; }
+                else { slot = sm.b_slot[code - kMaxBatch]; valid = slot >= 0; }
+                const double d0 = ld[h0];
+                if (valid && (h0 + 1 >= n || ld[h0 + 1] > d0)) { bd = d0; bslot = slot; bcode = code; }
+            }
+            for (int e0 = h0; e0 < n && bcode == -1; e0 += 32) {
                 const int e = e0 + lane;
                 int code = -1, slot = -1;
                 bool valid = false;

@@ -328,9 +328,7 @@ static void enqueue_probe_and_resolve(prox_handle *h, const float *queries, int3
             // safe slots: coarse scores on the tensor cores, exact recheck of the best few;
             // at-risk slots and the batch itself: full fp64 rows (or the pass above); uncertified
             // queries: fp64 over all slots
-            const int passes = (B + kScanQ - 1) / kScanQ;
-            for (int p = 0; p < passes && coarse; ++p)
-                if (launch_probe_scan_tc(h, p, s) != 0) coarse = false;
+            if (launch_probe_scan_tc(h, s) != 0) coarse = false;
             if (coarse) launch_merge_select(h, B, 1, s);
         }
         if (side) launch_probe_side(h, queries, B, s);
@@ -375,16 +373,9 @@ static const float *enqueue_lookup_and_scan(prox_handle *h, const float *queries
     const int passes = (B + kScanQ - 1) / kScanQ;
     {
         StageScope t(h, PROX_STAGE_SCAN, s);
-        // one kind of scan for all passes of a batch: the merge reads every pass's lists in one layout
-        bool tc = h->scan_mode != PROX_SCAN_CUDA_CORE;
-        for (int p = 0; p < passes; ++p) {
-            if (tc && launch_scan_pass_tc(h, p, s) != 0) {
-                tc = false;
-                p = -1;                                    // (before the first pass has run: start again on the CUDA cores)
-                continue;
-            }
-            if (!tc) launch_scan_pass(h, p, s);
-        }
+        // the tensor-core scan takes all passes of the batch in one launch, its CUDA-core twin one by one
+        if (h->scan_mode == PROX_SCAN_CUDA_CORE || launch_scan_tc(h, s) != 0)
+            for (int p = 0; p < passes; ++p) launch_scan_pass(h, p, s);
     }
     { StageScope t(h, PROX_STAGE_MERGE, s); launch_merge_select(h, B, 0, s); }
     { StageScope t(h, PROX_STAGE_RERANK, s); launch_rerank(h, queries, B, s); }

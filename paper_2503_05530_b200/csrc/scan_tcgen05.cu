@@ -57,8 +57,9 @@ struct ScanArgs {
     uint32_t *top1;
     u64 *buf;
     int32_t *buf_cnt;
+    size_t buf_pass_stride, cnt_pass_stride;   // entries of buf / buf_cnt that belong to one pass
     long long N;
-    int d, pass, kp;
+    int d, kp;
     int ks;                 // 64-column groups per pipeline stage (1 or 2; the tensor maps' boxes match)
     const float *w_in;      // speed of every pair (or block) as the previous launch measured it, tiles per ns
     float *w_out;           // ... as this launch measures it
@@ -98,14 +99,25 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     const int n_units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     constexpr int kUnitRows = PAIR ? 2 * kTileRows : kTileRows;            // corpus rows per tile of a unit
 
-    const int q0 = a.pass * kScanQ;
-    int nq = *a.n_active - q0;
-    if (nq > kScanQ) nq = kScanQ;
-    if (nq <= 0) {                                        // nothing missed in this pass
+    // The queries are taken in passes of up to kScanQ; the pairs (or blocks) are dealt to the passes
+    // round robin and each pass's pairs split the row tiles among themselves, so that one launch
+    // serves the whole batch and a small matrix is not walked four times by idle-starting blocks.
+    const int n_act = *a.n_active;
+    const int n_pass = (n_act + kScanQ - 1) / kScanQ;
+    if (n_pass <= 0) {                                    // nothing to scan for
         if (blockIdx.x == 0)
             for (int u = tid; u < n_units; u += kThreads) a.w_out[u] = a.w_in[u];
         return;
     }
+    const int pass = unit % n_pass;
+    const int sub = unit / n_pass, n_sub = (n_units - pass + n_pass - 1) / n_pass;    // place among the pass's pairs
+    const int q0 = pass * kScanQ;
+    const int nq = n_act - q0 < kScanQ ? n_act - q0 : kScanQ;
+    // lists of the other passes that this block will not write must read as empty
+    for (int p2 = 0; p2 < n_pass; ++p2)
+        if (p2 != pass)
+            for (int idx = tid; idx < 4 * kScanQ; idx += kThreads)
+                a.buf_cnt[(size_t)p2 * a.cnt_pass_stride + (size_t)blockIdx.x * 4 * kScanQ + idx] = 0;
     const int n_pad = nq <= 32 ? 32 : (nq <= 64 ? 64 : (nq <= 128 ? 128 : 256));
     const int q_rows = PAIR ? n_pad / 2 : n_pad;             // query rows this block stages (half of B in a pair)
     const CUtensorMap *tm_q = q_rows == 16 ? &tm_q16 : (q_rows == 32 ? &tm_q32 : (q_rows == 64 ? &tm_q64 : (q_rows == 128 ? &tm_q128 : &tm_q256)));
@@ -150,19 +162,19 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         {
             const long long nt = (a.N + kUnitRows - 1) / kUnitRows;
             double mean = 0.0;
-            for (int u = 0; u < n_units; ++u) mean += (double)a.w_in[u];
-            mean /= n_units;
+            for (int j = 0; j < n_sub; ++j) mean += (double)a.w_in[pass + j * n_pass];
+            mean /= n_sub;
             double total = 0.0, before = 0.0, upto = 0.0;
-            for (int u = 0; u < n_units; ++u) {
-                double w = (double)a.w_in[u];
+            for (int j = 0; j < n_sub; ++j) {
+                double w = (double)a.w_in[pass + j * n_pass];
                 if (!(w > 0.7 * mean)) w = 0.7 * mean;     // one odd measurement must not starve a pair
                 if (w > 1.4 * mean) w = 1.4 * mean;
-                if (u < unit) before += w;
-                if (u <= unit) upto += w;
+                if (j < sub) before += w;
+                if (j <= sub) upto += w;
                 total += w;
             }
             long long b0 = (long long)((double)nt * (before / total));
-            long long b1 = unit == n_units - 1 ? nt : (long long)((double)nt * (upto / total));
+            long long b1 = sub == n_sub - 1 ? nt : (long long)((double)nt * (upto / total));
             if (b0 > nt) b0 = nt;
             if (b1 > nt) b1 = nt;
             if (b1 < b0) b1 = b0;
@@ -268,9 +280,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         // The rows of a block split further into its four lane quarters, so there are four times
         // as many disjoint row sets as blocks: a tighter bound, and one that exists for k' up to that.
         const int P = 4 * gridDim.x;
-        if (a.kp <= P && P <= 1024) {
+        const int my = PAIR ? 2 * sub + (int)rank : sub;        // this block among the blocks of its pass
+        const int nb = PAIR ? 2 * n_sub : n_sub;
+        if (a.kp <= 4 * nb && P <= 1024) {
             volatile int *done = &ctl.done;
-            int jq = blockIdx.x, jobs = 0;
+            int jq = my, jobs = 0;
             // The first bounds are worth the most (until they arrive every row passes), and there is
             // nothing to select from before the first tile has been read out: the blocks start in
             // step, so this block's own first publication tells when the others' are due.
@@ -279,7 +293,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 while (*first_pub < kReadWarps && *done < kReadWarps && !*abort_flag) __nanosleep(200);
             }
             while (*done < kReadWarps && !*abort_flag) {
-                if (jq >= nq) jq = blockIdx.x;
+                if (jq >= nq) jq = my;
                 if (jq < nq) {
                     uint32_t t[32];
 #pragma unroll
@@ -302,7 +316,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     }
                     if (lane == 0 && rth != 0u) atomicMax(&thr_g[jq], rth);
                 }
-                jq += gridDim.x;
+                jq += nb;
                 // bounds move fast while the first tiles come in and slowly afterwards; this warp
                 // shares an issue port with read-out warps, so it backs off once they have settled
                 // (in short naps, so that the block does not outlive its read-out by a long one)
@@ -329,8 +343,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         const int ncol = active ? (nq - col_begin < cw ? (nq - col_begin > 0 ? nq - col_begin : 0) : cw) : 0;
         int *wcnt = ctl.wcnt[e];
         // lists of this warp: [(block * 4 + quarter) * kScanQ + query] * CAP
-        u64 *lists = a.buf + ((size_t)(blockIdx.x * 4 + quarter) * kScanQ) * CAP;
-        int32_t *lists_cnt = a.buf_cnt + (size_t)(blockIdx.x * 4 + quarter) * kScanQ;
+        u64 *lists = a.buf + (size_t)pass * a.buf_pass_stride + ((size_t)(blockIdx.x * 4 + quarter) * kScanQ) * CAP;
+        int32_t *lists_cnt = a.buf_cnt + (size_t)pass * a.cnt_pass_stride + (size_t)(blockIdx.x * 4 + quarter) * kScanQ;
         uint32_t it = 0;
         uint32_t published[kReadGroups];
         float tmin[kReadGroups];                                  // lower bound of the thresholds of each 32-column group
@@ -470,7 +484,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         // too short to tell (the same test in every block, so all keep or all renew)
         if (rank == 0 && e == 0 && lane == 0) {
             const unsigned long long ns = global_ns() - ns0;
-            const bool long_enough = ntiles >= 32LL * n_units;
+            const bool long_enough = ntiles >= 32LL * n_sub;
             a.w_out[unit] = (long_enough && alive && it > 0 && ns > 0) ? (float)((double)it / (double)ns) : a.w_in[unit];
         }
         // the lists go to the merge as they are: it drops what the shared bound has ruled out
@@ -585,13 +599,14 @@ void init_scan_tc(prox_handle *h) {
 // block qb.  Returns nonzero when the tensor-core path cannot run (no tensor-map encoder in the
 // driver, out of memory for the maps); the caller then falls back.
 static int launch_scan_generic(prox_handle *h, void **state, const __nv_bfloat16 *xb, const float *xh, long long rows,
-                               const __nv_bfloat16 *qb, const int *n_active, int kp, int pass, cudaStream_t s) {
+                               const __nv_bfloat16 *qb, const int *n_active, int kp, cudaStream_t s) {
     if (!*state) return 1;
     Maps &maps = *static_cast<Maps *>(*state);
     if (!maps.ok) return 1;
     ScanArgs a;
-    a.st = h->st; a.n_active = n_active; a.xh = xh; a.thr_g = h->thr_g; a.top1 = h->top1; a.buf = h->buf + (size_t)pass * h->buf_pass_stride;
-    a.buf_cnt = h->buf_cnt + (size_t)pass * h->cnt_pass_stride; a.N = rows; a.d = h->d; a.pass = pass; a.kp = kp; a.ks = maps.ks;
+    a.st = h->st; a.n_active = n_active; a.xh = xh; a.thr_g = h->thr_g; a.top1 = h->top1; a.buf = h->buf;
+    a.buf_cnt = h->buf_cnt; a.buf_pass_stride = h->buf_pass_stride; a.cnt_pass_stride = h->cnt_pass_stride;
+    a.N = rows; a.d = h->d; a.kp = kp; a.ks = maps.ks;
     const bool pair = h->scan_mode != PROX_SCAN_TC_SINGLE && h->scan_ctas >= 2 && rows >= 2 * kTileRows;
     const int grid = pair ? (h->scan_ctas & ~1) : h->scan_ctas;
     const int units = pair ? grid / 2 : grid;
@@ -632,18 +647,19 @@ static int launch_scan_generic(prox_handle *h, void **state, const __nv_bfloat16
     return 0;
 }
 
-// The corpus scan of the misses.  Nonzero: the handle cannot take the tensor-core path (d not a
-// multiple of 64, fewer corpus rows than one tile); the caller then runs the CUDA-core scan.
-int launch_scan_pass_tc(prox_handle *h, int pass, cudaStream_t s) {
+// The corpus scan of the misses, all passes of the batch in one launch.  Nonzero: the handle cannot
+// take the tensor-core path (d not a multiple of 64, fewer corpus rows than one tile); the caller
+// then runs the CUDA-core scan.
+int launch_scan_tc(prox_handle *h, cudaStream_t s) {
     if (h->d % kChunkK || h->N < kTileRows) return 1;
-    return launch_scan_generic(h, &h->tc_state, h->xb, h->xh, (long long)h->N, h->qb, &h->st->n_miss, h->kp, pass, s);
+    return launch_scan_generic(h, &h->tc_state, h->xb, h->xh, (long long)h->N, h->qb, &h->st->n_miss, h->kp, s);
 }
 
 // The coarse probe: the same scan over the bf16 copies of the cached keys, all batch queries,
 // keeping the kProbeKp best slots per query.
-int launch_probe_scan_tc(prox_handle *h, int pass, cudaStream_t s) {
+int launch_probe_scan_tc(prox_handle *h, cudaStream_t s) {
     return launch_scan_generic(h, &h->tc_state_keys, h->keys_b, h->kh, (long long)h->C, h->pqb, &h->st->n_probe,
-                               kProbeKp, pass, s);
+                               kProbeKp, s);
 }
 
 void free_scan_tc(prox_handle *h) {
