@@ -163,18 +163,36 @@ risk_pick_kernel(const DevState *st, RiskWork *w, int B, long long C) {
         if (tid == 0) w->bin = kRiskBins;                // every entry (or none) is at risk
         return;
     }
+    // sums of 64 consecutive bins, one group per warp at a time (coalesced), then the group and the
+    // bin inside it where the running count reaches R
     constexpr int per = kRiskBins / 1024;
-    unsigned sum = 0;
-    for (int i = 0; i < per; ++i) sum += w->hist[tid * per + i];
-    part[tid] = sum;
+    static_assert(per == 64, "two coalesced loads per lane cover one group");
+    __shared__ unsigned fine[per];
+    __shared__ unsigned s_acc;
+    __shared__ int s_group;
+    const int lane = tid & 31, warp = tid >> 5;
+    for (int g = warp; g < 1024; g += 32) {
+        unsigned v = w->hist[g * per + lane] + w->hist[g * per + 32 + lane];
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+        if (lane == 0) part[g] = v;
+    }
     __syncthreads();
     if (tid == 0) {
         unsigned acc = 0;
         int t = 0;
         while (t < 1023 && acc + part[t] < (unsigned)R) { acc += part[t]; ++t; }
-        int b = t * per;
-        while (b < kRiskBins - 1 && acc + w->hist[b] < (unsigned)R) { acc += w->hist[b]; ++b; }
-        w->bin = b;
+        s_acc = acc;
+        s_group = t;
+    }
+    __syncthreads();
+    if (tid < per) fine[tid] = w->hist[s_group * per + tid];
+    __syncthreads();
+    if (tid == 0) {
+        unsigned acc = s_acc;
+        int i = 0;
+        while (i < per - 1 && acc + fine[i] < (unsigned)R) { acc += fine[i]; ++i; }
+        w->bin = s_group * per + i;
     }
 }
 
@@ -236,6 +254,27 @@ risk_finish_kernel(DevState *st, RiskWork *w, int32_t *risk_pos, int32_t *risk_s
     if (tid < n_sure) { s_key[found + tid] = w->sure_key[tid]; s_val[found + tid] = w->sure_val[tid]; }
     __syncthreads();
     publish_risk_list(st, R, s_key, s_val, risk_pos, risk_slot, risk_stamp);
+}
+
+// FIFO needs no selection: slots fill in index order and a victim's slot is reused by the entry
+// that replaces it, so the stored entries form a ring in insertion order, and the R oldest are the
+// R slots from the ring's head on (Section 3.3.2: FIFO evicts the oldest inserted entry).
+__global__ void __launch_bounds__(1024)
+risk_ring_kernel(DevState *st, const u64 *__restrict__ stamp, int32_t *risk_pos, int32_t *risk_slot,
+                 u64 *risk_stamp, int B, long long C) {
+    const int tid = threadIdx.x;
+    const int prev = st->n_risk;
+    for (int r = tid; r < prev; r += blockDim.x) risk_pos[risk_slot[r]] = -1;
+    const long long count = st->count, head = st->fifo_head;
+    __syncthreads();
+    const int R = risk_count(count, B, C);
+    if (tid < R) {
+        const long long slot = (head + tid) % count;
+        risk_slot[tid] = (int32_t)slot;
+        risk_stamp[tid] = stamp[slot];
+        risk_pos[slot] = tid;
+    }
+    if (tid == 0) st->n_risk = R;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -612,16 +651,14 @@ __device__ void settle_misses(ResolveSmem &sm, ReplayState &rs, const int *list,
     }
 }
 
-__global__ void __launch_bounds__(1024)
-resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *stamp,
-               const int32_t *__restrict__ risk_slot, const u64 *__restrict__ risk_stamp,
-               const double *__restrict__ g_safe_min, const int32_t *__restrict__ g_safe_arg,
-               const double *__restrict__ cand_d, const int32_t *__restrict__ cand_code,
-               const int32_t *__restrict__ n_cand, uint8_t *out_hit, int32_t *src, int32_t *src_kind,
-               int32_t *ins_slot, int32_t *evt_slot, float *evt_dist, int32_t *miss_list,
-               int32_t *miss_rank) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    ResolveSmem &sm = *reinterpret_cast<ResolveSmem *>(smem_raw);
+// The whole replay, for a block of 1024 threads (sm: the block's ResolveSmem).
+__device__ void resolve_block(ResolveSmem &sm, DevState *st, int B, long long C, double tau, int policy, u64 *stamp,
+                              const int32_t *risk_slot, const u64 *risk_stamp,
+                              const double *g_safe_min, const int32_t *g_safe_arg,
+                              const double *cand_d, const int32_t *cand_code,
+                              const int32_t *n_cand, uint8_t *out_hit, int32_t *src, int32_t *src_kind,
+                              int32_t *ins_slot, int32_t *evt_slot, float *evt_dist, int32_t *miss_list,
+                              int32_t *miss_rank) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int R = st->n_risk;
     const long long count0 = st->count, clock0 = st->clock;
@@ -858,6 +895,7 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
         if (n_plain > done_plain) settle_misses(sm, rs, sm.plain_list, done_plain, n_plain, R, C, clock0, st, o);
         if (lane == 0) {
             st->count = rs.cnt;
+            if (policy == PROX_FIFO) st->fifo_head = (st->fifo_head + rs.n_evict) % C;   // the ring turns by one per eviction
             st->clock = clock0 + B;
             st->n_miss = rs.n_miss;
             st->queries += B;
@@ -876,6 +914,170 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
         const int s = sm.b_slot[j];
         ins_slot[j] = s;
         if (s >= 0) stamp[s] = sm.b_stamp[j];
+    }
+}
+
+__global__ void __launch_bounds__(1024)
+resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *stamp,
+               const int32_t *__restrict__ risk_slot, const u64 *__restrict__ risk_stamp,
+               const double *__restrict__ g_safe_min, const int32_t *__restrict__ g_safe_arg,
+               const double *__restrict__ cand_d, const int32_t *__restrict__ cand_code,
+               const int32_t *__restrict__ n_cand, uint8_t *out_hit, int32_t *src, int32_t *src_kind,
+               int32_t *ins_slot, int32_t *evt_slot, float *evt_dist, int32_t *miss_list,
+               int32_t *miss_rank) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    ResolveSmem &sm = *reinterpret_cast<ResolveSmem *>(smem_raw);
+    resolve_block(sm, st, B, C, tau, policy, stamp, risk_slot, risk_stamp, g_safe_min, g_safe_arg, cand_d, cand_code,
+                  n_cand, out_hit, src, src_kind, ins_slot, evt_slot, evt_dist, miss_list, miss_rank);
+}
+
+// ------------------------------------------------------------------------------------------
+// Small batches against a small cache (a query at a time, a few hundred keys): the work is a few
+// microseconds, the cost is the chain of launches.  Two launches instead of five: all distances
+// (every query against every stored key and every earlier query of the batch, fp64), then one
+// block that picks the at-risk entries, finds the nearest safe key and the listed keys of every
+// query, replays the batch and copies the stored lists of the hits.
+// ------------------------------------------------------------------------------------------
+constexpr int kSmallBatch = 4;                       // largest B of this path
+constexpr int kSmallCapacity = 2048;                 // largest capacity of this path
+
+template <bool IP>
+__global__ void __launch_bounds__(256)
+small_dist_kernel(const DevState *__restrict__ st, const float *__restrict__ keys, const float *__restrict__ queries,
+                  int B, int d, int ld, double *__restrict__ d_all) {
+    const long long count = st->count;
+    const int lane = threadIdx.x & 31;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    for (long long col = warp; col < count + B; col += nwarps) {
+        const float *x = col < count ? keys + (size_t)col * d : queries + (size_t)(col - count) * d;
+        double acc[kSmallBatch];
+#pragma unroll
+        for (int i = 0; i < kSmallBatch; ++i) acc[i] = 0.0;
+        for (int j = lane; j < d; j += 32) {
+            const double xv = (double)x[j];
+#pragma unroll
+            for (int i = 0; i < kSmallBatch; ++i) {
+                if (i < B) {
+                    const double qv = (double)queries[(size_t)i * d + j];
+                    if constexpr (IP) acc[i] = fma(-qv, xv, acc[i]);
+                    else { const double df = qv - xv; acc[i] = fma(df, df, acc[i]); }
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kSmallBatch; ++i) {
+#pragma unroll
+            for (int m = 16; m > 0; m >>= 1) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], m);
+            if (lane == 0 && i < B) d_all[(size_t)i * ld + col] = acc[i];
+        }
+    }
+}
+
+__global__ void __launch_bounds__(1024)
+small_resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *stamp, int32_t *risk_pos,
+                     int32_t *risk_slot, u64 *risk_stamp, const double *__restrict__ d_all, int ld, double *safe_min,
+                     int32_t *safe_arg, double *cand_d, int32_t *cand_code, int32_t *n_cand, uint8_t *out_hit,
+                     int32_t *src, int32_t *src_kind, int32_t *ins_slot, int32_t *evt_slot, float *evt_dist,
+                     int32_t *miss_list, int32_t *miss_rank, int k, const int32_t *__restrict__ val_ids,
+                     const float *__restrict__ val_dists, int64_t *out_ids, float *out_dists) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    ResolveSmem &sm = *reinterpret_cast<ResolveSmem *>(smem_raw);
+    __shared__ unsigned hist[256];
+    __shared__ u64 s_key[1024];
+    __shared__ int s_val[1024];
+    __shared__ u64 s_prefix, s_mask;
+    __shared__ int s_remaining, s_n;
+    __shared__ double s_d[4 * kSmallBatch];            // at most R + B - 1 <= 2 B - 1 listed keys per query
+    __shared__ int s_code[4 * kSmallBatch];
+    __shared__ double w_d[32];
+    __shared__ int w_s[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // ---- the at-risk entries of this batch
+    const int prev = st->n_risk;
+    for (int r = tid; r < prev; r += blockDim.x) risk_pos[risk_slot[r]] = -1;
+    const long long count = st->count, clock = st->clock;
+    __syncthreads();
+    const int R = risk_count(count, B, C);
+    if (R > 0) {
+        const int found = select_smallest(stamp, nullptr, count, R, clock, hist, s_key, s_val, &s_prefix, &s_mask,
+                                          &s_remaining, &s_n);
+        if (found != R) {                    // stamps must be unique; anything else is a broken state
+            if (tid == 0) { atomicCAS(&st->error, 0, PROX_ERR_INTERNAL); st->n_risk = 0; }
+            return;
+        }
+        publish_risk_list(st, R, s_key, s_val, risk_pos, risk_slot, risk_stamp);
+    } else if (tid == 0) {
+        st->n_risk = 0;
+    }
+    __syncthreads();
+
+    // ---- per query: the nearest safe key, and the at-risk and in-batch keys within tau, nearest first
+    for (int i = 0; i < B; ++i) {
+        const double *row = d_all + (size_t)i * ld;
+        double bd = INFINITY;
+        int bs = 0x7fffffff;
+        for (long long c = tid; c < count; c += blockDim.x) {
+            if (risk_pos[c] >= 0) continue;
+            const double v = row[c];
+            if (v < bd || (v == bd && (int)c < bs)) { bd = v; bs = (int)c; }
+        }
+#pragma unroll
+        for (int m = 1; m < 32; m <<= 1) {
+            const double od = __shfl_xor_sync(0xffffffffu, bd, m);
+            const int os = __shfl_xor_sync(0xffffffffu, bs, m);
+            if (od < bd || (od == bd && os < bs)) { bd = od; bs = os; }
+        }
+        if (lane == 0) { w_d[warp] = bd; w_s[warp] = bs; }
+        if (tid == 0) s_n = 0;
+        __syncthreads();
+        if (warp == 0) {
+            bd = w_d[lane]; bs = w_s[lane];
+#pragma unroll
+            for (int m = 1; m < 32; m <<= 1) {
+                const double od = __shfl_xor_sync(0xffffffffu, bd, m);
+                const int os = __shfl_xor_sync(0xffffffffu, bs, m);
+                if (od < bd || (od == bd && os < bs)) { bd = od; bs = os; }
+            }
+            if (lane == 0) { safe_min[i] = bd; safe_arg[i] = bs == 0x7fffffff ? -1 : bs; }
+        }
+        for (int e = tid; e < R + i; e += blockDim.x) {
+            const double v = e < R ? row[risk_slot[e]] : row[count + (e - R)];
+            if (v <= tau) {
+                const int pos = atomicAdd(&s_n, 1);
+                s_d[pos] = v;
+                s_code[pos] = e < R ? e : kMaxBatch + (e - R);
+            }
+        }
+        __syncthreads();
+        const int n = s_n;
+        if (n > 1) {
+            int n2 = 2;
+            while (n2 < n) n2 <<= 1;
+            for (int e = n + tid; e < n2; e += blockDim.x) { s_d[e] = INFINITY; s_code[e] = 0x7fffffff; }
+            block_sort_asc(s_d, s_code, n2);
+        }
+        for (int e = tid; e < n; e += blockDim.x) {
+            cand_d[(size_t)i * (2 * kMaxBatch) + e] = s_d[e];
+            cand_code[(size_t)i * (2 * kMaxBatch) + e] = s_code[e];
+        }
+        if (tid == 0) n_cand[i] = n;
+        __syncthreads();
+    }
+
+    // ---- replay, then the stored lists of the hits on keys that were there before the batch
+    resolve_block(sm, st, B, C, tau, policy, stamp, risk_slot, risk_stamp, safe_min, safe_arg, cand_d, cand_code, n_cand,
+                  out_hit, src, src_kind, ins_slot, evt_slot, evt_dist, miss_list, miss_rank);
+    if (out_ids != nullptr) {
+        __syncthreads();
+        for (int i = 0; i < B; ++i) {
+            if (src_kind[i] != 1) continue;
+            const int sl = src[i];
+            for (int r = tid; r < k; r += blockDim.x) {
+                out_ids[(size_t)i * k + r] = (int64_t)val_ids[(size_t)sl * k + r];
+                out_dists[(size_t)i * k + r] = val_dists[(size_t)sl * k + r];
+            }
+        }
     }
 }
 
@@ -1079,6 +1281,11 @@ void launch_scale(float *v, long long n, float f, cudaStream_t s) {
 }
 
 void launch_risk_select(prox_handle *h, int B, cudaStream_t s) {
+    if (h->policy == PROX_FIFO) {
+        risk_ring_kernel<<<1, 1024, 0, s>>>(h->st, h->stamp, h->risk_pos, h->risk_slot, h->risk_stamp, B, (long long)h->C);
+        h->launches++;
+        return;
+    }
     // one block reads a small cache faster than four launches do
     if (h->C <= (1 << 16)) {
         risk_select_kernel<<<1, 1024, 0, s>>>(h->st, h->stamp, h->risk_pos, h->risk_slot, h->risk_stamp, B,
@@ -1124,6 +1331,7 @@ void launch_build_candidates(prox_handle *h, int B, int splits, int lists_ready,
 // Kernel attributes belong to a device: set when a handle is created there, not once per process.
 void set_cache_kernel_attributes() {
     cudaFuncSetAttribute(resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ResolveSmem));
+    cudaFuncSetAttribute(small_resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ResolveSmem));
 }
 
 void launch_resolve(prox_handle *h, int B, uint8_t *out_hit, cudaStream_t s) {
@@ -1132,6 +1340,23 @@ void launch_resolve(prox_handle *h, int B, uint8_t *out_hit, cudaStream_t s) {
         h->safe_min, h->safe_arg, h->cand_d, h->cand_code, h->n_cand, out_hit, h->src, h->src_kind,
         h->ins_slot, h->evt_slot, h->evt_dist, h->miss_list, h->miss_rank);
     h->launches++;
+}
+
+// B and capacity small enough for the two-launch path (the handle's own distance; any policy).
+bool small_lookup_fits(const prox_handle *h, int B) { return B <= kSmallBatch && h->C <= kSmallCapacity && h->lsh_L < 0; }
+
+// Probe, at-risk selection, candidates, replay and (with out_ids) the gather of the hits' stored lists.
+void launch_small_lookup(prox_handle *h, const float *q, int B, uint8_t *out_hit, int64_t *out_ids, float *out_dists,
+                         cudaStream_t s) {
+    const int ld = (int)h->C + B;
+    const int blocks = (ld + 7) / 8;
+    if (metric_is_ip(h)) small_dist_kernel<true><<<blocks, 256, 0, s>>>(h->st, h->keys, q, B, h->d, ld, h->d_risk);
+    else small_dist_kernel<false><<<blocks, 256, 0, s>>>(h->st, h->keys, q, B, h->d, ld, h->d_risk);
+    small_resolve_kernel<<<1, 1024, sizeof(ResolveSmem), s>>>(
+        h->st, B, (long long)h->C, (double)h->tau, h->policy, h->stamp, h->risk_pos, h->risk_slot, h->risk_stamp, h->d_risk,
+        ld, h->safe_min, h->safe_arg, h->cand_d, h->cand_code, h->n_cand, out_hit, h->src, h->src_kind, h->ins_slot,
+        h->evt_slot, h->evt_dist, h->miss_list, h->miss_rank, h->k, h->val_ids, h->val_dists, out_ids, out_dists);
+    h->launches += 2;
 }
 
 void launch_gather_hits(prox_handle *h, int B, int64_t *out_ids, float *out_dists, cudaStream_t s) {

@@ -306,12 +306,19 @@ static int check_batch_args(prox_handle *h, const void *queries, int32_t B) {
     return PROX_OK;
 }
 
-static void enqueue_probe_and_resolve(prox_handle *h, const float *queries, int32_t B, uint8_t *out_hit,
-                                      cudaStream_t s) {
+// gather_ids / gather_dists: where the stored lists of hits on pre-batch keys may be copied to in
+// the same pass (NULL: the caller does it).  Returns true when that copy has been done.
+static bool enqueue_probe_and_resolve(prox_handle *h, const float *queries, int32_t B, uint8_t *out_hit,
+                                      int64_t *gather_ids, float *gather_dists, cudaStream_t s) {
     if (h->lsh_L >= 0) {                                  // PROXIMITY-LSH: the query's bucket only
         StageScope t(h, PROX_STAGE_PROBE, s);
         launch_lsh_probe(h, queries, B, out_hit, s);
-        return;
+        return false;
+    }
+    if (small_lookup_fits(h, B) && h->scan_mode != PROX_SCAN_CUDA_CORE) {   // a few queries, a small cache: two launches
+        StageScope t(h, PROX_STAGE_PROBE, s);
+        launch_small_lookup(h, queries, B, out_hit, gather_ids, gather_dists, s);
+        return gather_ids != nullptr;
     }
     { StageScope t(h, PROX_STAGE_RISK_SELECT, s); launch_risk_select(h, B, s); }
     // large batches: the at-risk slots and the batch itself on the tensor cores, exact recheck of the
@@ -350,6 +357,7 @@ static void enqueue_probe_and_resolve(prox_handle *h, const float *queries, int3
     }
     { StageScope t(h, PROX_STAGE_CANDIDATES, s); launch_build_candidates(h, B, splits, side ? 1 : 0, s); }
     { StageScope t(h, PROX_STAGE_RESOLVE, s); launch_resolve(h, B, out_hit, s); }
+    return false;
 }
 
 // First half of a batch: probe and replay, answers of hits on stored keys, and for every miss
@@ -363,11 +371,17 @@ static const float *enqueue_lookup_and_scan(prox_handle *h, const float *queries
         queries = h->qn;
     }
 
-    enqueue_probe_and_resolve(h, queries, B, out_hit, s);
-    {
+    const bool gathered = enqueue_probe_and_resolve(h, queries, B, out_hit, h->rho == 1 ? out_ids : nullptr,
+                                                    h->rho == 1 ? out_dists : nullptr, s);
+    if (!gathered) {
         StageScope t(h, PROX_STAGE_GATHER, s);
         if (h->rho == 1) launch_gather_hits(h, B, out_ids, out_dists, s);
         else launch_hit_rerank(h, queries, B, 1, out_ids, out_dists, s);     // before the scatter rewrites slots
+    }
+    if (small_corpus_fits(h, B) && h->scan_mode == PROX_SCAN_AUTO) {
+        StageScope t(h, PROX_STAGE_SCAN, s);
+        launch_small_exact(h, queries, s);
+        return queries;
     }
     { StageScope t(h, PROX_STAGE_PREP_MISS, s); launch_prep_miss(h, queries, B, s); }
     const int passes = (B + kScanQ - 1) / kScanQ;
@@ -499,7 +513,7 @@ extern "C" int32_t prox_probe_batch(prox_handle *h, const float *queries, int32_
         h->launches++;
         queries = h->qn;
     }
-    enqueue_probe_and_resolve(h, queries, B, out_hit, s);
+    enqueue_probe_and_resolve(h, queries, B, out_hit, nullptr, nullptr, s);
     if (out_slot || out_min_dist) launch_probe_outputs(h, B, out_slot, out_min_dist, s);
     if (out_min_dist && h->metric == PROX_METRIC_COSINE) {
         launch_scale(out_min_dist, B, 0.5f, s);

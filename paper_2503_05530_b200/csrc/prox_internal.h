@@ -37,6 +37,7 @@ struct DevState {
     int n_probe;              // queries of the current batch (read by the coarse probe's kernels)
     int n_pfail;              // queries whose coarse probe was not certified
     int n_over;               // queries whose exact pass collected more rows than it can hold
+    long long fifo_head;      // FIFO: slot of the oldest entry (the stored entries form a ring in slot order)
     int n_pairs;              // pairs listed by the tensor-core pass over the at-risk slots and the batch
     int side_overflow;        // 1 = more such pairs than the list holds: the fp64 rows are used instead
     // statistics
@@ -172,6 +173,9 @@ void launch_probe(prox_handle *h, const float *q, int B, int mode, cudaStream_t 
 void launch_build_candidates(prox_handle *h, int B, int splits, int lists_ready, cudaStream_t s);   // splits < 0: as the probe used
 void launch_resolve(prox_handle *h, int B, uint8_t *out_hit, cudaStream_t s);
 void launch_gather_hits(prox_handle *h, int B, int64_t *out_ids, float *out_dists, cudaStream_t s);
+bool small_lookup_fits(const prox_handle *h, int B);
+void launch_small_lookup(prox_handle *h, const float *q, int B, uint8_t *out_hit, int64_t *out_ids, float *out_dists,
+                         cudaStream_t s);   // small B and capacity: probe .. replay (.. gather when out_ids is given) in two launches
 void launch_hit_rerank(prox_handle *h, const float *q, int B, int kind, int64_t *out_ids, float *out_dists,
                        cudaStream_t s);   // rho > 1: hits of that kind (1 stored key, 2 key of this batch)
 void launch_scatter(prox_handle *h, const float *q, int B, int64_t *out_ids, float *out_dists,
@@ -195,6 +199,8 @@ void free_scan_tc(prox_handle *h);
 void launch_merge_select(prox_handle *h, int B, int for_probe, cudaStream_t s);   // all passes of the batch at once
 void launch_rerank(prox_handle *h, const float *q, int B, cudaStream_t s);
 void launch_fallback(prox_handle *h, const float *q, int B, cudaStream_t s);
+bool small_corpus_fits(const prox_handle *h, int B);
+void launch_small_exact(prox_handle *h, const float *q, cudaStream_t s);   // all misses of a small batch over a small corpus, fp64, one launch
 // row shards
 void launch_shard_pack(prox_handle *h, int B, void *xchg, cudaStream_t s);       // this shard's exchange record
 void launch_shard_merge(prox_handle *h, int B, const void *gathered, int G, cudaStream_t s);   // G records -> res_ids / res_dists

@@ -740,8 +740,10 @@ constexpr int kOverBuf = 4096;
 
 // Sorts the n entries of the buffer by (distance, row) and keeps the first k; returns how many stay.
 __device__ int over_compact(double *bd, int *bid, int n, int k) {
-    for (int e = n + threadIdx.x; e < kOverBuf; e += blockDim.x) { bd[e] = INFINITY; bid[e] = 0x7fffffff; }
-    block_sort_asc(bd, bid, kOverBuf);
+    int n2 = 2;
+    while (n2 < n) n2 <<= 1;                   // (n <= kOverBuf, a power of two)
+    for (int e = n + threadIdx.x; e < n2; e += blockDim.x) { bd[e] = INFINITY; bid[e] = 0x7fffffff; }
+    block_sort_asc(bd, bid, n2);
     return n < k ? n : k;
 }
 
@@ -750,7 +752,7 @@ __global__ void __launch_bounds__(1024)
 overflow_topk_kernel(DevState *st, const float *__restrict__ corpus, const float *__restrict__ queries, long long N,
                      int d, int k, const int32_t *__restrict__ miss_list, const int32_t *__restrict__ fail_list,
                      const float *__restrict__ fail_radius, const int32_t *__restrict__ over_list, double *over_d,
-                     int32_t *over_id, unsigned *over_ticket, int32_t *res_ids, double *res_dists) {
+                     int32_t *over_id, unsigned *over_ticket, int32_t *res_ids, double *res_dists, int direct) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *bd = reinterpret_cast<double *>(smem_raw);                 // kOverBuf
     int *bid = reinterpret_cast<int *>(bd + kOverBuf);                 // kOverBuf
@@ -758,8 +760,10 @@ overflow_topk_kernel(DevState *st, const float *__restrict__ corpus, const float
     __shared__ int s_cnt;
     __shared__ unsigned s_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-    int n_over = st->n_over;
+    // direct: the whole database call of a small batch over a small corpus (every miss, no radius)
+    int n_over = direct ? st->n_miss : st->n_over;
     if (n_over == 0) return;
+    if (direct && blockIdx.x == 0 && tid == 0) st->scan_batches++;
     if (n_over > kOverMax) {                   // beyond what the lists hold: those queries stay unanswered, and say so
         if (blockIdx.x == 0 && tid == 0) {
             atomicAdd((u64 *)&st->unresolved, (u64)(n_over - kOverMax));
@@ -771,12 +775,12 @@ overflow_topk_kernel(DevState *st, const float *__restrict__ corpus, const float
     const long long r0 = (long long)blockIdx.x * per, r1 = r0 + per < N ? r0 + per : N;
 
     for (int o = 0; o < n_over; ++o) {
-        const int f = over_list[o], m = fail_list[f];
+        const int f = direct ? o : over_list[o], m = direct ? o : fail_list[f];
         __syncthreads();
         for (int j = tid; j < d; j += blockDim.x) q_sm[j] = queries[(size_t)miss_list[m] * d + j];
         if (tid == 0) s_cnt = 0;
         // a row counts while (distance, row) <= (bound_d, bound_id): first the radius, then the block's k-th nearest
-        double bound_d = (double)fail_radius[f];
+        double bound_d = direct ? INFINITY : (double)fail_radius[f];
         int bound_id = 0x7fffffff;
         __syncthreads();
         for (long long base = r0; base < r1; base += nwarps) {
@@ -835,7 +839,7 @@ overflow_topk_kernel(DevState *st, const float *__restrict__ corpus, const float
             }
             if (tid == 0) {
                 over_ticket[o] = 0u;           // ready for the next batch
-                atomicAdd((u64 *)&st->fallback_rows, (u64)N);
+                if (!direct) atomicAdd((u64 *)&st->fallback_rows, (u64)N);
             }
         }
     }
@@ -907,26 +911,61 @@ prep_probe_kernel(DevState *st, const float *__restrict__ queries, int B, int d,
 __global__ void __launch_bounds__(128)
 probe_exact_kernel(DevState *st, const float *__restrict__ keys, const float *__restrict__ queries, int B, int d,
                    double tau, const int32_t *__restrict__ risk_pos, const int32_t *__restrict__ cand_id,
-                   const int32_t *__restrict__ cand_n, const float *__restrict__ cand_sk,
-                   const float *__restrict__ pqbn, const float *__restrict__ pqerr, double *safe_min,
-                   int32_t *safe_arg, int32_t *use_partial, int32_t *pfail_list) {
+                   const float *__restrict__ cand_score, const int32_t *__restrict__ cand_n,
+                   const float *__restrict__ cand_sk, const float *__restrict__ pqbn, const float *__restrict__ pqerr,
+                   double *safe_min, int32_t *safe_arg, int32_t *use_partial, int32_t *pfail_list) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *q_sm = reinterpret_cast<float *>(smem_raw);
     __shared__ double w_d[4];
     __shared__ int w_s[4];
+    __shared__ float w_f[4];
+    __shared__ int w_i[4];
+    __shared__ int s_list[kProbeKp], s_n;
     const int i = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (i >= B) return;
     for (int j = tid; j < d; j += blockDim.x) q_sm[j] = queries[(size_t)i * d + j];
+    if (tid == 0) s_n = 0;
+    const int n = cand_n[i];                                  // <= kProbeKp <= blockDim.x
+    // the safe candidate with the best coarse score first: its exact distance bounds the coarse
+    // score of anything that could be nearer, and few of the other candidates reach that bound
+    int my_slot = -1;
+    float my_score = -INFINITY;
+    if (tid < n) {
+        const int slot = cand_id[(size_t)i * kMaxKp + tid];
+        if (risk_pos[slot] < 0) { my_slot = slot; my_score = cand_score[(size_t)i * kMaxKp + tid]; }   // at-risk: measured elsewhere
+    }
+    float bf = my_score;
+    int bi = my_slot >= 0 ? tid : 0x7fffffff;
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) {
+        const float of = __shfl_xor_sync(0xffffffffu, bf, m);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, m);
+        if (of > bf || (of == bf && oi < bi)) { bf = of; bi = oi; }
+    }
+    if (lane == 0) { w_f[warp] = bf; w_i[warp] = bi; }
     __syncthreads();
-    const int n = cand_n[i];
+    for (int w = 0; w < 4; ++w)
+        if (w_f[w] > bf || (w_f[w] == bf && w_i[w] < bi)) { bf = w_f[w]; bi = w_i[w]; }
     double bd = INFINITY;
     int bs = 0x7fffffff;
-    for (int c = warp; c < n; c += 4) {
-        const int slot = cand_id[(size_t)i * kMaxKp + c];
-        if (risk_pos[slot] >= 0) continue;                        // measured as a full row by the fp64 probe
-        const double v = exact_sqdist_warp(q_sm, keys + (size_t)slot * d, d);
-        if (v < bd || (v == bd && slot < bs)) { bd = v; bs = slot; }
+    if (bi != 0x7fffffff) {                                   // (block-uniform)
+        const int first = cand_id[(size_t)i * kMaxKp + bi];
+        const double d1 = exact_sqdist_warp(q_sm, keys + (size_t)first * d, d);    // every warp computes it: no hand-over
+        bd = d1;
+        bs = first;
+        const double qn2 = (double)pqbn[i];
+        const double T = coarse_bound(d1, (double)pqerr[i], (double)st->ke_max, sqrt(qn2), (double)st->kn_max, d);
+        const float s_min = __double2float_rd(0.5 * (qn2 - T));
+        if (my_slot >= 0 && tid != bi && my_score >= s_min) s_list[atomicAdd(&s_n, 1)] = my_slot;
+        __syncthreads();
+        const int m = s_n;
+        for (int c = warp; c < m; c += 4) {
+            const int slot = s_list[c];
+            const double v = exact_sqdist_warp(q_sm, keys + (size_t)slot * d, d);
+            if (v < bd || (v == bd && slot < bs)) { bd = v; bs = slot; }
+        }
     }
+    __syncthreads();
     if (lane == 0) { w_d[warp] = bd; w_s[warp] = bs; }
     __syncthreads();
     if (tid == 0) {
@@ -1039,7 +1078,22 @@ void launch_fallback(prox_handle *h, const float *q, int B, cudaStream_t s) {
     auto over = metric_is_ip(h) ? overflow_topk_kernel<true> : overflow_topk_kernel<false>;
     over<<<h->scan_ctas, 1024, (size_t)kOverBuf * 12 + (size_t)h->d * 4, s>>>(
         h->st, h->corpus, q, (long long)h->N, h->d, h->k, h->miss_list, h->fail_list, h->fail_radius, h->over_list,
-        h->over_d, h->over_id, h->over_ticket, h->res_ids, h->res_dists);
+        h->over_d, h->over_id, h->over_ticket, h->res_ids, h->res_dists, 0);
+    h->launches++;
+}
+
+// The database call of a small batch over a small corpus in one launch: every row measured in fp64
+// for every miss, the k nearest by (distance, row id).  Exact by construction; stands in for the
+// coarse scan, its merge, the rerank and the exact pass, whose launches would cost more than the work.
+bool small_corpus_fits(const prox_handle *h, int B) {
+    return B <= 4 && (long long)h->N * h->d <= (1LL << 24) && h->N >= h->k;
+}
+
+void launch_small_exact(prox_handle *h, const float *q, cudaStream_t s) {
+    auto kern = metric_is_ip(h) ? overflow_topk_kernel<true> : overflow_topk_kernel<false>;
+    kern<<<h->scan_ctas, 1024, (size_t)kOverBuf * 12 + (size_t)h->d * 4, s>>>(
+        h->st, h->corpus, q, (long long)h->N, h->d, h->k, h->miss_list, h->fail_list, h->fail_radius, h->over_list,
+        h->over_d, h->over_id, h->over_ticket, h->res_ids, h->res_dists, 1);
     h->launches++;
 }
 
@@ -1056,7 +1110,7 @@ void launch_prep_probe(prox_handle *h, const float *q, int B, cudaStream_t s) {
 
 void launch_probe_exact(prox_handle *h, const float *q, int B, cudaStream_t s) {
     probe_exact_kernel<<<B, 128, (size_t)h->d * 4, s>>>(h->st, h->keys, q, B, h->d, (double)h->tau, h->risk_pos,
-                                                         h->cand_id, h->cand_n, h->cand_sk, h->pqbn, h->pqerr,
+                                                         h->cand_id, h->cand_score, h->cand_n, h->cand_sk, h->pqbn, h->pqerr,
                                                          h->safe_min, h->safe_arg, h->use_partial, h->pfail_list);
     h->launches++;
 }

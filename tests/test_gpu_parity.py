@@ -123,6 +123,22 @@ def test_d128_batch1024_fifo_ragged_tail():
     check(X, Q, 10, 500, 0.3, "fifo", 1024)
 
 
+@pytest.mark.parametrize("metric,policy,batch", [("l2", "lru", 1), ("l2", "fifo", 4), ("cosine", "lru", 3), ("ip", "fifo", 2)])
+def test_small_batches_over_a_small_corpus_take_the_short_route(metric, policy, batch):
+    """Up to four queries per call, a cache of a few hundred keys and a corpus of a few thousand rows:
+    the lookup is two launches and the database call one (every row measured in fp64); duplicate
+    rows, hits on keys of the same call and evictions all occur."""
+    X, Q = stream(6007, 256, 16, 700, 60, 1.0, 0.03, seed=81)
+    X = X.clone()
+    X[4000:4040] = X[100:140]                                          # equal rows: ties go to the lower id
+    tau = {"l2": 0.4, "cosine": 0.2, "ip": -0.8}[metric]
+    res, gpu = check(X, Q, 12, 25, tau, policy, batch, metric=metric)
+    assert 0.2 < res["hit_rate"] < 0.97 and gpu[3]["evictions"] > 0
+    if batch > 1:
+        assert gpu[3]["intra_batch_hits"] > 0
+    assert gpu[3]["uncertified"] == 0 and gpu[3]["scan_batches"] > 0
+
+
 # ------------------------------------------------------------------ degenerate cases
 def test_exact_duplicates_hit_at_tau_zero_in_and_across_batches():
     X, Q = stream(3000, 64, 8, 200, 200, 0.0, 0.05, seed=5)
@@ -189,7 +205,7 @@ def test_thousands_of_copies_of_one_row_are_still_answered_exactly(metric):
     Q = (Q / Q.norm(dim=1, keepdim=True)).contiguous()
     k = 10
     tau = 0.0 if metric == "l2" else -2.0
-    gpu = run_gpu(X.to(DEV), Q.to(DEV), k, 16, tau, "lru", 4, metric=metric)
+    gpu = run_gpu(X.to(DEV), Q.to(DEV), k, 16, tau, "lru", 6, metric=metric)       # (batches above four: the tensor-core route)
     ids, dists = oracle.exact_topk(X.numpy(), Q.numpy(), k, metric=parity.ORACLE_METRIC[metric])
     assert gpu[3]["unresolved"] == 0 and gpu[3]["hits"] == 0
     assert np.array_equal(gpu[0], ids)
