@@ -80,7 +80,10 @@ __device__ void publish_risk_list(DevState *st, int R, u64 *s_key, int *s_val, i
         risk_stamp[tid] = s_key[tid];
         risk_pos[s_val[tid]] = tid;
     }
-    if (tid == 0) st->n_risk = R;
+    if (tid == 0) {
+        st->n_risk = R;
+        if (R > 0) st->stamp_floor = (long long)s_key[0];  // stamps only grow: still a lower bound in later batches
+    }
 }
 
 __device__ __forceinline__ int risk_count(long long count, int B, long long C) {
@@ -118,7 +121,9 @@ risk_select_kernel(DevState *st, const u64 *__restrict__ stamp, int32_t *risk_po
 }
 
 // Large caches: the same selection spread over the whole GPU.  A 65536-bin histogram of the
-// stamps' leading bits names the bin that holds the R-th smallest; stamps in lower bins are at
+// leading bits of (stamp - floor), floor a lower bound of all stored stamps (so that the bins
+// cover the range the stamps really span, however long the handle has lived), names the bin
+// that holds the R-th smallest; stamps in lower bins are at
 // risk for certain, the stamps of that one bin (few, stamps being unique) are settled by one
 // block.  Work area: histogram, the two lists and their counters.
 constexpr int kRiskBins = 1 << 16;
@@ -148,8 +153,9 @@ risk_hist_kernel(const DevState *st, const u64 *__restrict__ stamp, int32_t *ris
     const long long count = st->count;
     const int R = risk_count(count, B, C);
     if (R == 0 || (long long)R >= count) return;
-    const int shift = risk_shift(st->clock);
-    for (long long s = gtid; s < count; s += nth) atomicAdd(&w->hist[(unsigned)(stamp[s] >> shift)], 1u);
+    const u64 floor = (u64)st->stamp_floor;
+    const int shift = risk_shift(st->clock - (long long)floor);
+    for (long long s = gtid; s < count; s += nth) atomicAdd(&w->hist[(unsigned)((stamp[s] - floor) >> shift)], 1u);
 }
 
 __global__ void __launch_bounds__(1024)
@@ -158,7 +164,7 @@ risk_pick_kernel(const DevState *st, RiskWork *w, int B, long long C) {
     const int tid = threadIdx.x;
     const long long count = st->count;
     const int R = risk_count(count, B, C);
-    if (tid == 0) { w->n_sure = 0; w->n_edge = 0; w->shift = risk_shift(st->clock); }
+    if (tid == 0) { w->n_sure = 0; w->n_edge = 0; w->shift = risk_shift(st->clock - st->stamp_floor); }
     if (R == 0 || (long long)R >= count) {
         if (tid == 0) w->bin = kRiskBins;                // every entry (or none) is at risk
         return;
@@ -204,9 +210,10 @@ risk_collect_kernel(const DevState *st, const u64 *__restrict__ stamp, RiskWork 
     const long long nth = (long long)gridDim.x * blockDim.x;
     const unsigned bin = (unsigned)w->bin;
     const int shift = w->shift;
+    const u64 floor = (u64)st->stamp_floor;
     for (long long s = gtid; s < count; s += nth) {
         const u64 v = stamp[s];
-        const unsigned bn = bin == (unsigned)kRiskBins ? 0u : (unsigned)(v >> shift);
+        const unsigned bn = bin == (unsigned)kRiskBins ? 0u : (unsigned)((v - floor) >> shift);
         if (bn < bin) {
             const int pos = atomicAdd(&w->n_sure, 1);
             if (pos < kMaxBatch) { w->sure_key[pos] = v; w->sure_val[pos] = (int32_t)s; }

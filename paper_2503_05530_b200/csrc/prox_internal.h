@@ -37,6 +37,7 @@ struct DevState {
     int n_probe;              // queries of the current batch (read by the coarse probe's kernels)
     int n_pfail;              // queries whose coarse probe was not certified
     int n_over;               // queries whose exact pass collected more rows than it can hold
+    long long stamp_floor;    // a lower bound of every stored stamp (the smallest stamp of the last at-risk selection)
     long long fifo_head;      // FIFO: slot of the oldest entry (the stored entries form a ring in slot order)
     int n_pairs;              // pairs listed by the tensor-core pass over the at-risk slots and the batch
     int side_overflow;        // 1 = more such pairs than the list holds: the fp64 rows are used instead
