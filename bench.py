@@ -53,23 +53,32 @@ def load_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons of one GPU, sampled while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+    """nvidia-smi clocks and throttle reasons of one GPU.  The sampler is started ahead of the timed region
+    (the tool needs a few hundred milliseconds before its first line) and keeps the time stamp of every sample;
+    `stop` reports the samples taken between `begin()` and `end()` (all of them if none was marked)."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
         self.index, self.samples, self.proc = index, [], None
+        self.t0 = self.t1 = None
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
             self.proc = None
         return self
+
+    def begin(self):
+        self.t0 = time.time()
+
+    def end(self):
+        self.t1 = time.time()
 
     def _read(self):
         for line in self.proc.stdout:
@@ -78,26 +87,35 @@ class ClockSampler:
     def stop(self) -> dict:
         if self.proc is None:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        if self.t1 is not None:                               # let a sample that was under way at the end come in
+            time.sleep(0.06)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        import datetime
+        rows = []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for s in self.samples:
             t = [x.strip() for x in s.split(",")]
-            if len(t) < 6:
+            if len(t) < 7:
                 continue
             try:
-                sm.append(float(t[0])); mx.append(float(t[1]))
+                ts = datetime.datetime.strptime(t[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(t[1]), float(t[2]), [n for n, v in zip(names, t[3:7]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
-            for name, v in zip(names, t[2:6]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
-                    reasons=sorted(reasons), samples=len(sm))
+        inside = rows
+        if self.t0 is not None and self.t1 is not None:
+            inside = [r for r in rows if self.t0 <= r[0] <= self.t1 + 0.05]
+            if not inside and rows:                           # a region shorter than the sampling period: the nearest sample
+                mid = 0.5 * (self.t0 + self.t1)
+                inside = [min(rows, key=lambda r: abs(r[0] - mid))]
+        sm = [r[1] for r in inside]
+        reasons = sorted({n for r in inside for n in r[3]})
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(r[2] for r in inside) if inside else None,
+                    reasons=reasons, samples=len(sm))
 
 
 def stream_seed(seed: int, rank: int) -> int:
@@ -224,11 +242,13 @@ def run_streams(prox, cfg, queries, taus, K, Wm, dev, local, barrier, make_handl
         qs = queries[:n_use] if queries.shape[0] >= n_use else queries.repeat((n_use + queries.shape[0] - 1) // queries.shape[0], 1)[:n_use]
         batches = [(qs[a:a + B], ids[a:a + B], dists[a:a + B], hit[a:a + B]) for a in range(0, n_use, B)]
         wq = queries[n_use:n_use + Wm * B] if queries.shape[0] >= n_use + Wm * B else qs[:Wm * B]
+        sampler = ClockSampler(local).start()
         for a in range(0, wq.shape[0], B):
             p.query_batch(wq[a:a + B])
         torch.cuda.synchronize()
-        sampler = ClockSampler(local).start()
+        sampler.begin()
         ms, stats, scan_ms, scan_n, launches = time_stream(p, batches, True, barrier)
+        sampler.end()
         clocks = sampler.stop()
         assert p.status() == prox.OK, prox.last_error()
         r = dict(tau=tau, ms=ms, hit_rate=float(hit.float().mean().item()), stats=stats, scan_ms=scan_ms, scan_n=scan_n,
@@ -252,7 +272,9 @@ def run_streams(prox, cfg, queries, taus, K, Wm, dev, local, barrier, make_handl
             hl = torch.empty(n_long, dtype=torch.uint8, device=dev)
             lb = [(ql[a:a + B], il, dl, hl[a:a + B]) for a in range(0, n_long, B)]
             sampler = ClockSampler(local).start()
+            sampler.begin()
             ms_l, st_l, scan_l, _, _ = time_stream(p, lb, True, barrier)
+            sampler.end()
             ck = sampler.stop()
             rf = scan_roofline(cfg, dict(stats=st_l, scan_ms=scan_l, clocks=ck), peaks)
             extra["sustained"] = dict(tau=tau, steps=n_long // B, value=round(n_long / (ms_l * 1e-3), 1), unit=UNIT,
@@ -588,6 +610,7 @@ def probe_points(prox, args, dev, local, peaks, steps, warmup, max_keys=0):
         for policy in ("lru", "fifo"):
             p = prox.Prox(keys[:64].contiguous(), 1, C, tau, policy)
             p.cache_load(keys)
+            sampler = ClockSampler(local).start()
             for q in batches[K:]:
                 p.probe_batch(q)
             torch.cuda.synchronize()
@@ -597,12 +620,13 @@ def probe_points(prox, args, dev, local, peaks, steps, warmup, max_keys=0):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             hits = []
             l0 = p.kernel_launches()
-            sampler = ClockSampler(local).start()
+            sampler.begin()
             e0.record()
             for q in batches[:K]:
                 hits.append(p.probe_batch(q)[0])
             e1.record()
             torch.cuda.synchronize()
+            sampler.end()
             clocks = sampler.stop()
             prof = p.profile_read()
             assert p.status() == prox.OK, prox.last_error()
@@ -643,17 +667,19 @@ def probe_points(prox, args, dev, local, peaks, steps, warmup, max_keys=0):
         for a in range(0, keys.shape[0], B):
             p.probe_batch(keys[a:a + B])
         batches = [W.make_probe_batch(keys, centres, B, 0.02, args.seed, b_) for b_ in range(K + warmup)]
+        sampler = ClockSampler(local).start()
         for q in batches[K:]:
             p.probe_batch(q)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         hits = []
-        sampler = ClockSampler(local).start()
+        sampler.begin()
         e0.record()
         for q in batches[:K]:
             hits.append(p.probe_batch(q)[0])
         e1.record()
         torch.cuda.synchronize()
+        sampler.end()
         clocks = sampler.stop()
         assert p.status() == prox.OK, prox.last_error()
         ms = e0.elapsed_time(e1) / K
