@@ -149,19 +149,20 @@ def pick_workload(name: str, free_bytes: int) -> W.Config:
     return cfg if free_bytes >= need else W.CONFIGS["1m"]
 
 
-# DRAM bytes per algorithmic byte of one scan launch, from an ncu capture of scan_tc_kernel on a cut of the 24 M x 768
-# workload (dram__bytes_read.sum + dram__bytes_write.sum against the bf16 rows + norms of the cut); the extra bytes
-# grow with the row tiles like the algorithmic ones, so the ratio carries over to a full launch.  Valid for d = 768
-# and 256 misses per launch only; None while the kernel has changed since the counters were taken.
-SCAN_TRAFFIC_RATIO_D768_M256 = None
+# DRAM traffic of one scan launch, from an ncu capture of scan_tc_kernel on a 1 M-row cut of the 24 M x 768 workload
+# (dram__bytes_read.sum = 1.5514 GB against 1.5400 GB of bf16 rows + norms; dram__bytes_write.sum = 0.0971 GB of
+# candidate appends while the thresholds of the first tiles are still open).  The bytes read grow with the row tiles
+# like the algorithmic ones, the appends do not, so a full launch is taken as ratio x algorithmic + appends.  Valid
+# for d = 768 and 256 misses per launch only; None once the kernel has changed since the counters were taken.
+SCAN_TRAFFIC_D768_M256 = dict(read_ratio=1.0074, append_bytes=97_125_888)
 
 
 def roofline_of_scan(cfg, mean_misses, scan_ms_per_launch, peaks, clocks=None, traffic=None):
     """The corpus scan: bytes = bf16 corpus + row norms once per launch, flops = 2 M N d.  The fraction is taken
     against the burst bf16 figure (or the copy bandwidth); the sustained figure stands beside it."""
     bytes_alg = cfg.N * cfg.d * 2 + cfg.N * 4
-    if traffic is None and cfg.d == 768 and mean_misses > 255 and SCAN_TRAFFIC_RATIO_D768_M256:
-        traffic = round(SCAN_TRAFFIC_RATIO_D768_M256 * bytes_alg)
+    if traffic is None and cfg.d == 768 and mean_misses > 255 and SCAN_TRAFFIC_D768_M256:
+        traffic = round(SCAN_TRAFFIC_D768_M256["read_ratio"] * bytes_alg + SCAN_TRAFFIC_D768_M256["append_bytes"])
     flops = 2.0 * mean_misses * cfg.N * cfg.d
     t = max(scan_ms_per_launch, 1e-9) * 1e-3
     t_hbm = bytes_alg / (peaks["hbm_gbs"] * 1e9)

@@ -576,6 +576,18 @@ struct ResolveOut {
     float *evt_dist;
 };
 
+// Position of the n-th set bit of mask (n counted from 0; mask has more than n bits set): five
+// halvings with a population count each.
+__device__ __forceinline__ int nth_set_bit(unsigned mask, int n) {
+    int pos = 0;
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) {
+        const int c = __popc(mask & (((1u << s) - 1u) << pos));
+        if (n >= c) { n -= c; pos += s; }
+    }
+    return pos;
+}
+
 // The misses list[a .. b) (query indices, ascending) take their slots in order.  Whole warp.
 __device__ void settle_misses(ResolveSmem &sm, ReplayState &rs, const int *list, int a, int b, int R, long long C,
                               long long clock0, DevState *st, const ResolveOut &o) {
@@ -597,10 +609,10 @@ __device__ void settle_misses(ResolveSmem &sm, ReplayState &rs, const int *list,
             const int avail = __popc(mask);
             const int use = avail < need - got ? avail : need - got;
             const int t = lane - n_free - got;             // this lane's turn among the evicting misses
-            if (t >= 0 && t < use) slot = sm.r_slot[rs.p + (int)__fns(mask, 0, t + 1)];
+            if (t >= 0 && t < use) slot = sm.r_slot[rs.p + nth_set_bit(mask, t)];
             if (ok && __popc(mask & ((1u << lane) - 1u)) < use) sm.r_alive[e] = 0;
             got += use;
-            rs.p = (use == avail) ? rs.p + 32 : rs.p + (int)__fns(mask, 0, use) + 1;
+            rs.p = (use == avail) ? rs.p + 32 : rs.p + nth_set_bit(mask, use - 1) + 1;
             __syncwarp();
         }
         if (rs.p > R) rs.p = R;

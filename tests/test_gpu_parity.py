@@ -171,6 +171,7 @@ def test_corpus_smaller_than_candidate_count():
     for N, k in [(10, 10), (37, 5), (64, 64), (129, 3)]:
         X, Q = stream(N, 16, 2, 40, 10, 1.0, 0.05, seed=N)
         check(X, Q, k, 8, 0.01, "lru", 16)
+        check(X, Q, k, 8, 0.01, "lru", 3)                    # the one-launch route of small batches
 
 
 def test_uncertified_queries_take_the_exact_pass():
@@ -531,7 +532,7 @@ def test_host_buffer_entry_point_equals_device_entry_point():
         assert np.array_equal(x, y)
 
 
-@pytest.mark.parametrize("d,batch", [(768, 64), (128, 256), (256, 24)])
+@pytest.mark.parametrize("d,batch", [(768, 64), (128, 256), (256, 24), (128, 600)])
 def test_the_three_scan_kernels_agree(d, batch):
     """Two-block tensor-core scan (default), one-block tensor-core scan and CUDA-core scan."""
     X, Q = stream(9001, d, 8, 520, 40, 1.1, 0.02, seed=10)
