@@ -10,7 +10,8 @@
  *
  * Conventions
  *  - Distances are squared Euclidean distances, for keys and corpus alike
- *    (Section 3.1: the cache uses the distance function of the database).
+ *    (Section 3.1: the cache uses the distance function of the database), unless the
+ *    handle was made by prox_create_metric with the cosine distance or the inner product.
  *  - Every pointer marked DEVICE is a device pointer valid on the GPU that was
  *    current when prox_create ran; HOST pointers are ordinary host memory.
  *  - Calls on one handle must be ordered on one stream at a time: the cache is
@@ -263,7 +264,9 @@ int32_t prox_set_scan_mode(prox_handle *h, int32_t mode);
 /* prox_kernel_launches -- kernels launched by this handle so far (host-side count). */
 int64_t prox_kernel_launches(const prox_handle *h);
 
-/* Stages of one batch, in launch order (indices of the arrays of prox_profile_read). */
+/* Stages of one batch, in launch order (indices of the arrays of prox_profile_read).  A batch of up to four
+ * queries against a small cache runs its whole lookup (at-risk selection to gather) under PROX_STAGE_PROBE, and
+ * over a small corpus its whole database call (scan to exact pass) under PROX_STAGE_SCAN. */
 enum {
     PROX_STAGE_RISK_SELECT = 0, PROX_STAGE_PROBE = 1, PROX_STAGE_CANDIDATES = 2, PROX_STAGE_RESOLVE = 3,
     PROX_STAGE_GATHER = 4, PROX_STAGE_PREP_MISS = 5, PROX_STAGE_SCAN = 6, PROX_STAGE_MERGE = 7,
