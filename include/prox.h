@@ -250,6 +250,7 @@ typedef struct prox_stats {
     int64_t unresolved;                 /* misses whose exact pass overflowed (result best effort) */
     int64_t count;                      /* |C| now */
     int64_t probe_uncertified;          /* queries whose coarse (tensor-core) probe fell back to the exact fp64 probe */
+    int64_t parallel_replays;           /* batches whose replay was solved as a fixed point instead of in query order */
 } prox_stats;
 
 /* prox_get_stats -- synchronises the stream, then copies the device counters to *out (HOST). */

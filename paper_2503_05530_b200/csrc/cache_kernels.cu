@@ -562,6 +562,14 @@ struct ResolveSmem {
     unsigned char kind[kMaxBatch];     // 1 settled (hits a safe key), 2 plain miss, 3 entangled
     unsigned char r_alive[kMaxBatch];
     unsigned char r_touched[kMaxBatch];
+    // the parallel replay (replay_parallel)
+    int p_tgt[kMaxBatch];              // per query: -1 miss, -2 its nearest safe key, h >= 0 the h-th entry of its list
+    int p_rank[kMaxBatch];             // per query: misses before it
+    int p_tm[kMaxBatch];               // query index of the m-th evicting miss
+    int p_E[kMaxBatch];                // per at-risk position: the query that evicts it (kNever: none)
+    int p_T[kMaxBatch];                // per at-risk position: the first query that hits it; at the end, the position the m-th eviction takes
+    unsigned char p_skip[kMaxBatch];   // per at-risk position: touched before the eviction pointer reaches it
+    int p_flag;                        // a case the parallel replay leaves to the sequential one
 };
 
 struct ReplayState {
@@ -670,6 +678,201 @@ __device__ void settle_misses(ResolveSmem &sm, ReplayState &rs, const int *list,
     }
 }
 
+// Exclusive prefix sum of x over the block's 1024 threads (wt: 32 ints of shared memory); total = the sum.
+__device__ __forceinline__ int block_excl_scan(int x, int *wt, int &total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = x;
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, inc, m);
+        if (lane >= m) inc += y;
+    }
+    if (lane == 31) wt[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        int w = wt[lane];
+#pragma unroll
+        for (int m = 1; m < 32; m <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, w, m);
+            if (lane >= m) w += y;
+        }
+        wt[lane] = w;
+    }
+    __syncthreads();
+    total = wt[31];
+    const int r = inc - x + (warp > 0 ? wt[warp - 1] : 0);
+    __syncthreads();                                       // wt is free again
+    return r;
+}
+
+// The replay of Algorithm 1 over one batch as a fixed point, for batches in which many queries
+// depend on one another (a cache about as small as the batch: every key is at risk).
+//
+// The outcome of query i (miss, or the key it hits) depends only on what the queries before it
+// did: which at-risk keys they evicted and which of them were inserted.  Write that as equations
+// over the whole batch:
+//   rank(i)  = misses before i; the misses of rank >= free slots evict, in order;
+//   T(q)     = the first query that hits at-risk position q (LRU only: a touched key moves to
+//              the young end and the eviction pointer passes over it);
+//   m(q)     = positions before q that the pointer does not pass over; position q is passed
+//              over iff T(q) is earlier than the (m(q)+1)-th evicting miss, and evicted by that
+//              miss otherwise: E(q);
+//   query i hits the first entry of its sorted list that is resident when it arrives: an at-risk
+//              position q with E(q) >= i (the miss that evicts q found it resident), or a query
+//              j < i that missed (and so was inserted); else its safe key within tau; else it misses.
+// Every right-hand side at "time" i uses only outcomes of earlier times, so the system has one
+// solution, the sequential replay, and iterating all equations in parallel from any start makes
+// at least the earliest wrong outcome right in each round.  In practice a batch of 1024 settles
+// in 5 to 13 rounds.  The iteration stops when a round changes nothing.
+//
+// Left to the sequential replay (returns false, nothing written): two listed keys, or a listed
+// and the safe key, at exactly the same distance (the lowest slot wins, and slots of inserted keys
+// are not part of the equations); more evictions than at-risk positions (capacity below the
+// batch size); no fixed point within kParallelRounds.
+constexpr int kNever = 0x7fffffff;
+constexpr int kParallelRounds = 48;
+constexpr int kParallelMinEntangled = 24;
+
+__device__ bool replay_parallel(ResolveSmem &sm, DevState *st, int B, int R, long long C, double tau, int policy,
+                                long long count0, long long clock0, const double *cand_d, const int32_t *cand_code,
+                                u64 *stamp, const ResolveOut &o) {
+    const int i = threadIdx.x;
+    const bool lru = policy == PROX_LRU;
+    const long long free_ll = C - count0;
+    const int free0 = free_ll <= 0 ? 0 : (free_ll > (long long)B ? B : (int)free_ll);
+    const int kind = i < B ? (int)sm.kind[i] : 0;
+    int n = 0, hd = 0, sa = -1;
+    double sd = INFINITY;
+    const int *lc = nullptr;
+    const double *ld = nullptr;
+    if (i < B) {
+        n = sm.ncand[i];
+        hd = sm.head[i];
+        sd = sm.safe_min[i];
+        sa = sm.safe_arg[i];
+        const int off = sm.off[i];
+        const bool in_smem = off + n <= kCsrCap;
+        lc = in_smem ? sm.csr_code + off : cand_code + (size_t)i * (2 * kMaxBatch);
+        ld = in_smem ? sm.csr_d + off : cand_d + (size_t)i * (2 * kMaxBatch);
+    }
+    const bool safe_hit = sa >= 0 && sd <= tau;
+    // start: every listed key is taken as resident
+    if (i < B) sm.p_tgt[i] = kind == 2 ? -1 : (kind == 1 ? -2 : hd);
+    if (i < kMaxBatch) { sm.p_skip[i] = 0; sm.p_E[i] = kNever; }
+    if (i == 0) sm.p_flag = 0;
+    __syncthreads();
+
+    int rank = 0, total_miss = 0, mq = 0, total_ev = 0;
+    bool is_miss = false, converged = false;
+    for (int round = 0; round < kParallelRounds; ++round) {
+        is_miss = i < B && sm.p_tgt[i] == -1;
+        rank = block_excl_scan(is_miss ? 1 : 0, sm.warp_tot[0], total_miss);
+        if (i < kMaxBatch) { sm.p_rank[i] = rank; sm.p_tm[i] = kNever; sm.p_T[i] = kNever; }
+        __syncthreads();
+        if (is_miss && rank >= free0) sm.p_tm[rank - free0] = i;
+        if (lru && kind == 3) {
+            const int t = sm.p_tgt[i];
+            if (t >= 0) {
+                const int code = lc[t];
+                if (code < kMaxBatch) atomicMin(&sm.p_T[code], i);
+            }
+        }
+        mq = block_excl_scan((i < R && !sm.p_skip[i]) ? 1 : 0, sm.warp_tot[1], total_ev);   // (its barriers order the writes above)
+        bool changed = false;
+        if (i < R) {
+            const int et = sm.p_tm[mq];                     // mq < R <= kMaxBatch
+            const bool skip = sm.p_T[i] < et;
+            const int E = skip ? kNever : et;
+            if ((skip ? 1 : 0) != (int)sm.p_skip[i] || E != sm.p_E[i]) changed = true;
+            sm.p_skip[i] = skip ? 1 : 0;
+            sm.p_E[i] = E;
+        }
+        __syncthreads();
+        if (kind == 3) {
+            int t = -1;
+            for (int h = hd; h < n; ++h) {
+                const int code = lc[h];
+                // (outcomes of other queries are read while their threads may be writing this round's:
+                // either value is a legitimate iterate, and a round that changes nothing read only final ones)
+                const bool valid = code < kMaxBatch ? sm.p_E[code] >= i
+                                                    : ((volatile int *)sm.p_tgt)[code - kMaxBatch] == -1;
+                if (valid) { t = h; break; }
+            }
+            if (t >= 0) {
+                const double bd = ld[t];
+                if (t + 1 < n && ld[t + 1] == bd) sm.p_flag = 1;
+                if (safe_hit) {
+                    if (sd < bd) t = -2;
+                    else if (sd == bd) sm.p_flag = 1;
+                }
+            } else if (safe_hit) {
+                t = -2;
+            }
+            if (t != sm.p_tgt[i]) { sm.p_tgt[i] = t; changed = true; }
+        }
+        const int any = __syncthreads_or(changed ? 1 : 0);
+        if (sm.p_flag) return false;
+        if (!any) { converged = true; break; }
+    }
+    if (!converged) return false;
+    // (rank, total_miss, mq, total_ev, p_tm, p_skip, p_E are those of the last round, which changed nothing)
+    const int n_evict = total_miss > free0 ? total_miss - free0 : 0;
+    if (n_evict > total_ev) return false;                  // the at-risk list would be used up
+    const int n_free = total_miss < free0 ? total_miss : free0;
+
+    if (i < R && !sm.p_skip[i] && mq < n_evict) { sm.p_T[mq] = i; sm.r_alive[i] = 0; }
+    __syncthreads();
+    if (is_miss) {
+        const int slot = rank < free0 ? (int)(count0 + rank) : sm.r_slot[sm.p_T[rank - free0]];
+        o.out_hit[i] = 0; o.src_kind[i] = 0; o.src[i] = -1;
+        o.evt_slot[i] = slot; o.evt_dist[i] = INFINITY;
+        sm.b_slot[i] = slot; sm.b_stamp[i] = (u64)(clock0 + i);
+        o.miss_list[rank] = i; o.miss_rank[i] = rank;
+    }
+    __syncthreads();
+    int intra = 0;
+    if (kind == 3 && !is_miss) {
+        const u64 t = (u64)(clock0 + i);
+        const int h = sm.p_tgt[i];
+        o.out_hit[i] = 1;
+        o.miss_rank[i] = -1;
+        if (h == -2) {
+            o.evt_slot[i] = sa; o.evt_dist[i] = (float)sd;
+            o.src_kind[i] = 1; o.src[i] = sa;
+            if (lru) atomicMax(&stamp[sa], t);
+        } else {
+            const int code = lc[h];
+            o.evt_dist[i] = (float)ld[h];
+            if (code < kMaxBatch) {
+                const int slot = sm.r_slot[code];
+                o.evt_slot[i] = slot;
+                o.src_kind[i] = 1; o.src[i] = slot;
+                if (lru) { atomicMax(&sm.r_stamp[code], t); sm.r_touched[code] = 1; }
+            } else {
+                const int j = code - kMaxBatch;
+                o.evt_slot[i] = sm.b_slot[j];
+                o.src_kind[i] = 2; o.src[i] = j;
+                if (lru) atomicMax(&sm.b_stamp[j], t);
+                intra = 1;
+            }
+        }
+    }
+    const int n_intra = __syncthreads_count(intra);
+    if (i == 0) {
+        st->count = count0 + n_free;
+        if (policy == PROX_FIFO) st->fifo_head = (st->fifo_head + n_evict) % C;
+        st->clock = clock0 + B;
+        st->n_miss = total_miss;
+        st->queries += B;
+        st->hits += B - total_miss;
+        st->misses += total_miss;
+        st->intra_hits += n_intra;
+        st->evictions += n_evict;
+        st->parallel_replays += 1;
+    }
+    return true;
+}
+
 // The whole replay, for a block of 1024 threads (sm: the block's ResolveSmem).
 __device__ void resolve_block(ResolveSmem &sm, DevState *st, int B, long long C, double tau, int policy, u64 *stamp,
                               const int32_t *risk_slot, const u64 *risk_stamp,
@@ -677,7 +880,7 @@ __device__ void resolve_block(ResolveSmem &sm, DevState *st, int B, long long C,
                               const double *cand_d, const int32_t *cand_code,
                               const int32_t *n_cand, uint8_t *out_hit, int32_t *src, int32_t *src_kind,
                               int32_t *ins_slot, int32_t *evt_slot, float *evt_dist, int32_t *miss_list,
-                              int32_t *miss_rank) {
+                              int32_t *miss_rank, bool allow_parallel) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int R = st->n_risk;
     const long long count0 = st->count, clock0 = st->clock;
@@ -811,8 +1014,11 @@ __device__ void resolve_block(ResolveSmem &sm, DevState *st, int B, long long C,
         __syncthreads();
     }
 
-    // ---- replay by warp 0
-    if (warp == 0) {
+    // ---- replay: all at once when many queries are entangled, else (or when that declines) in order by warp 0
+    bool replayed = false;
+    if (allow_parallel && n_ent >= kParallelMinEntangled)
+        replayed = replay_parallel(sm, st, B, R, C, tau, policy, count0, clock0, cand_d, cand_code, stamp, o);
+    if (!replayed && warp == 0) {
         ReplayState rs{count0, 0, 0, 0};
         int n_hit = n_settled, n_intra = 0, done_plain = 0;
         for (int k = 0; k < n_ent; ++k) {
@@ -943,11 +1149,11 @@ resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u64 *st
                const double *__restrict__ cand_d, const int32_t *__restrict__ cand_code,
                const int32_t *__restrict__ n_cand, uint8_t *out_hit, int32_t *src, int32_t *src_kind,
                int32_t *ins_slot, int32_t *evt_slot, float *evt_dist, int32_t *miss_list,
-               int32_t *miss_rank) {
+               int32_t *miss_rank, int allow_parallel) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     ResolveSmem &sm = *reinterpret_cast<ResolveSmem *>(smem_raw);
     resolve_block(sm, st, B, C, tau, policy, stamp, risk_slot, risk_stamp, g_safe_min, g_safe_arg, cand_d, cand_code,
-                  n_cand, out_hit, src, src_kind, ins_slot, evt_slot, evt_dist, miss_list, miss_rank);
+                  n_cand, out_hit, src, src_kind, ins_slot, evt_slot, evt_dist, miss_list, miss_rank, allow_parallel != 0);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1086,7 +1292,7 @@ small_resolve_kernel(DevState *st, int B, long long C, double tau, int policy, u
 
     // ---- replay, then the stored lists of the hits on keys that were there before the batch
     resolve_block(sm, st, B, C, tau, policy, stamp, risk_slot, risk_stamp, safe_min, safe_arg, cand_d, cand_code, n_cand,
-                  out_hit, src, src_kind, ins_slot, evt_slot, evt_dist, miss_list, miss_rank);
+                  out_hit, src, src_kind, ins_slot, evt_slot, evt_dist, miss_list, miss_rank, false);
     if (out_ids != nullptr) {
         __syncthreads();
         for (int i = 0; i < B; ++i) {
@@ -1357,7 +1563,8 @@ void launch_resolve(prox_handle *h, int B, uint8_t *out_hit, cudaStream_t s) {
     resolve_kernel<<<1, 1024, sizeof(ResolveSmem), s>>>(
         h->st, B, (long long)h->C, (double)h->tau, h->policy, h->stamp, h->risk_slot, h->risk_stamp,
         h->safe_min, h->safe_arg, h->cand_d, h->cand_code, h->n_cand, out_hit, h->src, h->src_kind,
-        h->ins_slot, h->evt_slot, h->evt_dist, h->miss_list, h->miss_rank);
+        h->ins_slot, h->evt_slot, h->evt_dist, h->miss_list, h->miss_rank,
+        h->scan_mode != PROX_SCAN_CUDA_CORE ? 1 : 0);      // the cross-check mode replays in query order
     h->launches++;
 }
 

@@ -560,6 +560,7 @@ extern "C" int32_t prox_get_stats(prox_handle *h, prox_stats *out, void *stream)
     out->scan_batches = st.scan_batches; out->uncertified = st.uncertified;
     out->fallback_rows = st.fallback_rows; out->unresolved = st.unresolved; out->count = st.count;
     out->probe_uncertified = st.probe_uncertified;
+    out->parallel_replays = st.parallel_replays;
     return PROX_OK;
 }
 

@@ -43,7 +43,7 @@ struct DevState {
     int side_overflow;        // 1 = more such pairs than the list holds: the fp64 rows are used instead
     // statistics
     long long queries, hits, misses, intra_hits, evictions, scan_batches, uncertified,
-        fallback_rows, unresolved, probe_uncertified;
+        fallback_rows, unresolved, probe_uncertified, parallel_replays;
 };
 
 struct Profiler;

@@ -361,11 +361,14 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             // loads whose latency hides behind the wait and the read-out
             const long long row_next = row + kUnitRows;
             const float hn_next = (tile + 1 < t_end && row_next < a.N) ? a.xh[row_next] : INFINITY;
+            // (the shared bounds are looked at on every tile at first and on every eighth tile once they
+            // move slowly: at 128 dimensions the read-out of a tile, not its products, sets the pace)
             uint32_t g_thr[kReadGroups];
+            const bool thr_tile = it < 16 || (it & 7u) == 1u;
 #pragma unroll
             for (int i = 0; i < kReadGroups; ++i) {
                 const int c = col_begin + lane + 32 * i;
-                g_thr[i] = (lane + 32 * i < ncol) ? __ldcg(&thr_g[c]) : 0u;
+                g_thr[i] = (thr_tile && lane + 32 * i < ncol) ? __ldcg(&thr_g[c]) : 0u;
             }
             bool ok = mbar_wait(smem_u32(&ctl.tmem_full[b]), bph, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
@@ -423,7 +426,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 }
                 if (last) break;
             }
-            if (!early) {
+            if (!early && thr_tile) {
 #pragma unroll
                 for (int i = 0; i < kReadGroups; ++i) {
                     const int lc = lane + 32 * i;
@@ -435,9 +438,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             }
             // the warp publishes the best score of its lane quarter for each of its columns, and takes
             // the smallest threshold of each of its column groups for the first level of the test
-            // (every tile at first, every fourth once the bounds move slowly; thresholds only rise,
+            // (every tile at first, every sixteenth once the bounds move slowly; thresholds only rise,
             // so an older minimum is still a lower bound)
-            if (it < 16 || (it & 3u) == 0u) {
+            if (it < 16 || (it & 15u) == 0u) {
 #pragma unroll
                 for (int i = 0; i < kReadGroups; ++i) {
                     float t = ctl.thr[col_begin + ((lane + 32 * i) < cw ? lane + 32 * i : 0)];

@@ -33,7 +33,7 @@ class ProxError(RuntimeError):
 class Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("queries", "hits", "misses", "intra_batch_hits", "evictions",
                                           "scan_batches", "uncertified", "fallback_rows", "unresolved",
-                                          "count", "probe_uncertified")]
+                                          "count", "probe_uncertified", "parallel_replays")]
 
     def as_dict(self) -> dict:
         return {n: int(getattr(self, n)) for n, _ in self._fields_}

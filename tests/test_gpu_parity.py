@@ -402,6 +402,52 @@ def test_probe_only_prefilled_cache(policy, n_keys):
 
 
 @pytest.mark.parametrize("policy", ["lru", "fifo"])
+@pytest.mark.parametrize("n_keys,batch,d", [(1024, 1024, 768), (1024, 1000, 64), (2048, 1024, 64), (700, 1024, 64), (300, 512, 64)])
+@pytest.mark.parametrize("in_order", [False, True])
+def test_probe_only_cache_as_small_as_the_batch(policy, n_keys, batch, d, in_order):
+    """A full cache of about as many keys as the batch has queries: every key is at risk, every hit
+    is on a key that an earlier miss of the same batch may have evicted, and a third of the batch
+    is near an earlier query of the batch.  The replay solves such a batch as a fixed point; with
+    the cross-check mode it runs in query order.  Both against the oracle, flag by flag and slot
+    by slot, over several batches (the state carries over).  Capacities below the batch size use
+    up the at-risk list, which the fixed-point replay leaves to the in-order one."""
+    keys, centres = W.make_probe_keys(n_keys, d, 4 * n_keys, seed=31)      # most fresh draws find no key of their component
+    tau = 0.5 if d == 768 else 0.02
+    p = prox.Prox(keys[:64].contiguous().to(DEV), 1, n_keys, tau, policy)
+    if in_order:
+        p.set_scan_mode(prox.SCAN_CUDA_CORE)
+    p.cache_load(keys.to(DEV))
+    o = oracle.Oracle(None, d, 1, n_keys, float(np.float32(tau)), oracle.LRU if policy == "lru" else oracle.FIFO)
+    o.cache_load(keys.numpy())
+    gen = torch.Generator().manual_seed(77)
+    rates = []
+    for b in range(4):
+        Q = W.make_probe_batch(keys, centres, batch, 0.02 if d == 768 else 0.01, 31, b)
+        # a third of the queries repeat, slightly moved, an earlier query of the same batch
+        idx = torch.randperm(batch, generator=gen)[: batch // 3]
+        src = (torch.rand(batch // 3, generator=gen) * idx.float()).long()
+        moved = Q[src] + 1e-3 * torch.randn(batch // 3, d, generator=gen)
+        Q[idx] = torch.where((idx > 0)[:, None], moved, Q[idx])
+        hit, slot, dist = p.probe_batch(Q.to(DEV))
+        torch.cuda.synchronize()
+        r = o.query(Q.numpy())
+        assert np.array_equal(hit.cpu().numpy(), r["hit"]), f"batch {b}: first differing flag at {np.nonzero(hit.cpu().numpy() != r['hit'])[0][:1]}"
+        assert np.array_equal(slot.cpu().numpy(), r["slot"]), f"batch {b}: first differing slot at {np.nonzero(slot.cpu().numpy() != r['slot'])[0][:1]}"
+        h = r["hit"] == 1
+        assert np.allclose(dist.cpu().numpy()[h], r["best"][h], rtol=1e-6)
+        rates.append(float(r["hit"].mean()))
+    assert 0.05 < np.mean(rates) < 0.98, rates
+    assert p.status() == prox.OK
+    st = p.stats()
+    p.close()
+    if in_order:
+        assert st["parallel_replays"] == 0
+    elif n_keys >= batch:
+        assert st["parallel_replays"] >= 3, st
+    assert st["intra_batch_hits"] > 0
+
+
+@pytest.mark.parametrize("policy", ["lru", "fifo"])
 def test_probe_only_cache_above_the_multi_block_risk_selection(policy):
     """More than 65536 keys: the at-risk entries are picked by the histogram kernels spread over
     the GPU; the slots that misses overwrite show the eviction order."""
