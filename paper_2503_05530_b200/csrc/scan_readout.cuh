@@ -114,13 +114,22 @@ __device__ __forceinline__ float max_margin32(const uint32_t (&v)[32], const flo
 
 // Largest of 32 accumulator columns of this lane's row, thresholds aside.
 __device__ __forceinline__ float raw_max32(const uint32_t (&v)[32]) {
-    float m0 = -INFINITY, m1 = -INFINITY;
-#pragma unroll
-    for (int j = 0; j < 32; j += 4) {
-        m0 = max3(m0, __uint_as_float(v[j]), __uint_as_float(v[j + 1]));
-        m1 = max3(m1, __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-    }
-    return fmaxf(m0, m1);
+    // four short chains instead of two long ones: the latency of the chain, not the issue slots, is what a tile waits for
+    float m0 = max3(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]));
+    float m1 = max3(__uint_as_float(v[3]), __uint_as_float(v[4]), __uint_as_float(v[5]));
+    float m2 = max3(__uint_as_float(v[6]), __uint_as_float(v[7]), __uint_as_float(v[8]));
+    float m3 = max3(__uint_as_float(v[9]), __uint_as_float(v[10]), __uint_as_float(v[11]));
+    m0 = max3(m0, __uint_as_float(v[12]), __uint_as_float(v[13]));
+    m1 = max3(m1, __uint_as_float(v[14]), __uint_as_float(v[15]));
+    m2 = max3(m2, __uint_as_float(v[16]), __uint_as_float(v[17]));
+    m3 = max3(m3, __uint_as_float(v[18]), __uint_as_float(v[19]));
+    m0 = max3(m0, __uint_as_float(v[20]), __uint_as_float(v[21]));
+    m1 = max3(m1, __uint_as_float(v[22]), __uint_as_float(v[23]));
+    m2 = max3(m2, __uint_as_float(v[24]), __uint_as_float(v[25]));
+    m3 = max3(m3, __uint_as_float(v[26]), __uint_as_float(v[27]));
+    m0 = max3(m0, __uint_as_float(v[28]), __uint_as_float(v[29]));
+    m1 = max3(m1, __uint_as_float(v[30]), __uint_as_float(v[31]));
+    return fmaxf(max3(m0, m1, m2), m3);
 }
 
 // Up to 64 accumulator columns (queries c0 .. c0+63; the second 32 only when `two`) of one corpus
@@ -137,11 +146,14 @@ template <int CAP>
 __device__ __forceinline__ void readout64(const uint32_t (&v0)[32], const uint32_t (&v1)[32], bool two, int c0,
                                           int lc0, float hn, float tmin0, float tmin1, int32_t row,
                                           const float *thr, int *wcnt, uint32_t *best, u64 *lists, bool &need) {
-    const bool c0p = raw_max32(v0) - tmin0 > hn;
-    const bool c1p = two && raw_max32(v1) - tmin1 > hn;
+    // (both groups unconditionally, so that their chains overlap; without a second group v1 holds
+    // nothing that matters and tmin1 rules it out)
+    const float r0 = raw_max32(v0), r1 = raw_max32(v1);
+    const bool c0p = r0 - tmin0 > hn;
+    const bool c1p = two & (r1 - tmin1 > hn);
+    if (!__any_sync(0xffffffffu, c0p | c1p)) return;
     const unsigned maybe0 = __ballot_sync(0xffffffffu, c0p);
     const unsigned maybe1 = __ballot_sync(0xffffffffu, c1p);
-    if ((maybe0 | maybe1) == 0u) return;
     if (maybe0 != 0u) {
         const float m0 = max_margin32(v0, thr, c0);
         if (__any_sync(0xffffffffu, m0 > hn)) append32<CAP>(v0, c0, lc0, hn, row, thr, wcnt, best, lists, need);

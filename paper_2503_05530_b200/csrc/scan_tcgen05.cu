@@ -74,6 +74,7 @@ struct Control {
     int abort_flag;                  // set by any thread whose wait ran out
     int done;                        // read-out warps that have finished (the bound warp stops at kReadWarps)
     int first_pub;                   // read-out warps that have published the bests of their first tile
+    uint32_t issued;                 // tiles whose products have all been issued (the MMA issuers take turns)
     long long t_begin, t_end;        // row tiles of this pair (or block)
 };
 
@@ -131,6 +132,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     const int stage_bytes = ks * (resident ? kATileBytes : kATileBytes + b_tile_bytes);
     int stages = (kTileRegion - (resident ? q_block_bytes : 0)) / stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
+    // Two MMA issuers take the tiles in turn (see there).  An issuer waits for the first stage of its
+    // tile before its turn, i.e. while the other issuer may still be consuming the tile before; an
+    // mbarrier wait tells only the parity of a phase, so the fill waited for must be the very next
+    // one of its stage: the fill before it (stages earlier) has to belong to a tile that was issued
+    // before this issuer's previous tile.  That holds when the ring has at least two tiles' worth of stages.
+    const bool dual = nst <= 2 && stages >= 2 * nst;
 
     const uint32_t tiles0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;       // 1024-byte aligned
     const uint32_t q_res0 = tiles0;
@@ -155,6 +162,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         ctl.abort_flag = 0;
         ctl.done = 0;
         ctl.first_pub = 0;
+        ctl.issued = 0u;
         // Row tiles are dealt out in contiguous runs whose lengths follow the speeds that the
         // previous launch measured (SMs differ by their place on the die: up to a quarter in
         // tiles per second), so that all pairs end together.  Every block adds the same numbers
@@ -233,22 +241,40 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0 && rank == 0) {
+    } else if (warp == 1 || warp == 3) {
+        // ------------------------------------------------------------ MMA issuers
+        // One thread issues a tile's products: every tcgen05.mma costs it about a hundred cycles,
+        // and with the waits and commits of a tile the chain of one thread is longer than the
+        // products of a tile of 128 dimensions take.  So two threads (warps 1 and 3) take the
+        // tiles in turn: while one issues, the other has already waited for its row tile and its
+        // accumulator buffer and only waits for its turn, which keeps the products in tile order.
+        const uint32_t me = warp == 1 ? 0u : 1u;
+        const uint32_t n_issuers = dual ? 2u : 1u;
+        if (lane == 0 && rank == 0 && me < n_issuers) {
             const uint32_t idesc = instr_desc_bf16(kUnitRows, n_pad);
             bool ok = true;
             if (resident) ok = mbar_wait(smem_u32(&ctl.q_full), 0, abort_flag);
-            uint32_t g = 0, it = 0;
-            for (long long tile = t_begin; ok && tile < t_end; ++tile, ++it) {
+            volatile uint32_t *issued = &ctl.issued;
+            for (uint32_t it = me; ok && t_begin + (long long)it < t_end; it += n_issuers) {
                 const uint32_t b = it & 1u, bph = (it >> 1) & 1u;
+                uint32_t g = it * (uint32_t)nst;
+                // what the tile needs first; its turn last
+                if (!mbar_wait(smem_u32(&ctl.full[g % stages]), (g / stages) & 1u, abort_flag)) { ok = false; break; }
                 if (!mbar_wait(smem_u32(&ctl.tmem_empty[b]), bph ^ 1u, abort_flag)) { ok = false; break; }
+                if (dual) {
+                    const unsigned long long t0 = global_ns();
+                    uint32_t spins = 0;
+                    while (*issued != it) {
+                        if ((++spins & 1023u) == 0u && (*abort_flag || global_ns() - t0 > kWaitLimitNs)) { *abort_flag = 1; ok = false; break; }
+                    }
+                    if (!ok) break;
+                }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + b * (uint32_t)kScanQ;
                 for (int st = 0; st < nst; ++st, ++g) {
                     const int s = g % stages;
                     const uint32_t ph = (g / stages) & 1u;
-                    if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag)) { ok = false; break; }
+                    if (st > 0 && !mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag)) { ok = false; break; }
                     const uint32_t a_addr = stage0 + s * stage_bytes;
                     const uint32_t b_addr = resident ? q_res0 + st * ks * b_tile_bytes : a_addr + ks * kATileBytes;
                     for (int ka = 0; ka < ks; ++ka) {
@@ -261,14 +287,18 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                             else tc_mma_bf16(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, acc);
                         }
                     }
+                    if (st == nst - 1 && dual) {                  // the other thread's turn
+                        __threadfence_block();
+                        *issued = it + 1u;
+                    }
                     // the stage is free (in both blocks of a pair) once these are done
                     if constexpr (PAIR) tc_commit_pair(smem_u32(&ctl.empty[s]));
                     else tc_commit(smem_u32(&ctl.empty[s]));
                 }
-                if (ok) {                                         // accumulator complete
-                    if constexpr (PAIR) tc_commit_pair(smem_u32(&ctl.tmem_full[b]));
-                    else tc_commit(smem_u32(&ctl.tmem_full[b]));
-                }
+                if (!ok) { if (dual) *abort_flag = 1; break; }
+                // accumulator complete
+                if constexpr (PAIR) tc_commit_pair(smem_u32(&ctl.tmem_full[b]));
+                else tc_commit(smem_u32(&ctl.tmem_full[b]));
             }
         }
     } else if (warp == 2) {
