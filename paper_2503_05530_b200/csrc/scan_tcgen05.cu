@@ -86,7 +86,7 @@ struct Control {
 // PAIR = true runs two blocks per MMA (a cluster of two, tcgen05 cta_group::2): a pair takes 256
 // corpus rows per tile, each block loading its own 128 rows and half of the query rows, so a
 // block ingests a third less per corpus row than alone.  Block 0 of the pair issues the MMAs.
-template <int CAP, bool PAIR>
+template <int CAP, bool PAIR, bool DUAL>
 __global__ void __launch_bounds__(kThreads, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_q16,
                const __grid_constant__ CUtensorMap tm_q32, const __grid_constant__ CUtensorMap tm_q64,
@@ -137,7 +137,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     // mbarrier wait tells only the parity of a phase, so the fill waited for must be the very next
     // one of its stage: the fill before it (stages earlier) has to belong to a tile that was issued
     // before this issuer's previous tile.  That holds when the ring has at least two tiles' worth of stages.
-    const bool dual = nst <= 2 && stages >= 2 * nst;
+    // (DUAL: the launch allows it, for few dimensions; with many, a tile's products outlast the issuer's chain anyway)
+    const bool dual = DUAL && nst <= 2 && stages >= 2 * nst;
 
     const uint32_t tiles0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;       // 1024-byte aligned
     const uint32_t q_res0 = tiles0;
@@ -599,6 +600,20 @@ __global__ void speed_init_kernel(float *speed) {
 
 }  // namespace
 
+template <int CAP, bool PAIR, bool DUAL>
+static void set_scan_smem() {
+    cudaFuncSetAttribute(scan_tc_kernel<CAP, PAIR, DUAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
+}
+template <int CAP, bool PAIR, bool DUAL>
+static cudaError_t launch_scan_kernel(const cudaLaunchConfig_t &cfg, const Maps &maps, const ScanArgs &a) {
+    return cudaLaunchKernelEx(&cfg, scan_tc_kernel<CAP, PAIR, DUAL>, maps.x, maps.q16, maps.q32, maps.q64, maps.q128, maps.q256, a);
+}
+template <int CAP>
+static cudaError_t launch_scan_kernel(bool pair, bool dual, const cudaLaunchConfig_t &cfg, const Maps &maps, const ScanArgs &a) {
+    if (pair) return dual ? launch_scan_kernel<CAP, true, true>(cfg, maps, a) : launch_scan_kernel<CAP, true, false>(cfg, maps, a);
+    return dual ? launch_scan_kernel<CAP, false, true>(cfg, maps, a) : launch_scan_kernel<CAP, false, false>(cfg, maps, a);
+}
+
 // Tensor maps and the speed table of one scanned matrix: made once, at prox_create, so that the
 // batch calls neither allocate nor copy.
 static void ensure_maps(prox_handle *h, void **state, const __nv_bfloat16 *xb, long long rows,
@@ -616,10 +631,8 @@ static void ensure_maps(prox_handle *h, void **state, const __nv_bfloat16 *xb, l
             make_map(&m->q64, qb, kMaxBatch, (uint64_t)h->d, 64, ks) &&
             make_map(&m->q128, qb, kMaxBatch, (uint64_t)h->d, 128, ks) &&
             make_map(&m->q256, qb, kMaxBatch, (uint64_t)h->d, 256, ks);
-    cudaFuncSetAttribute(scan_tc_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
-    cudaFuncSetAttribute(scan_tc_kernel<512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
-    cudaFuncSetAttribute(scan_tc_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
-    cudaFuncSetAttribute(scan_tc_kernel<512, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegion + 1024);
+    set_scan_smem<256, false, false>(); set_scan_smem<512, false, false>(); set_scan_smem<256, true, false>(); set_scan_smem<512, true, false>();
+    set_scan_smem<256, false, true>(); set_scan_smem<512, false, true>(); set_scan_smem<256, true, true>(); set_scan_smem<512, true, true>();
 }
 
 void init_scan_tc(prox_handle *h) {
@@ -664,13 +677,10 @@ static int launch_scan_generic(prox_handle *h, void **state, const __nv_bfloat16
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e;
-    if (pair)
-        e = h->tc_cap == 256 ? cudaLaunchKernelEx(&cfg, scan_tc_kernel<256, true>, maps.x, maps.q16, maps.q32, maps.q64, maps.q128, maps.q256, a)
-                             : cudaLaunchKernelEx(&cfg, scan_tc_kernel<512, true>, maps.x, maps.q16, maps.q32, maps.q64, maps.q128, maps.q256, a);
-    else
-        e = h->tc_cap == 256 ? cudaLaunchKernelEx(&cfg, scan_tc_kernel<256, false>, maps.x, maps.q16, maps.q32, maps.q64, maps.q128, maps.q256, a)
-                             : cudaLaunchKernelEx(&cfg, scan_tc_kernel<512, false>, maps.x, maps.q16, maps.q32, maps.q64, maps.q128, maps.q256, a);
+    // two MMA issuers when a row tile is one or two ring stages (up to 256 dimensions)
+    const bool dual = (h->d / kChunkK) / maps.ks <= 2;
+    const cudaError_t e = h->tc_cap == 256 ? launch_scan_kernel<256>(pair, dual, cfg, maps, a)
+                                           : launch_scan_kernel<512>(pair, dual, cfg, maps, a);
     if (e != cudaSuccess) {                               // the caller falls back: leave no error behind, keep the speeds' turn
         cudaGetLastError();
         return 1;
