@@ -150,11 +150,11 @@ def pick_workload(name: str, free_bytes: int) -> W.Config:
 
 
 # DRAM traffic of one scan launch, from an ncu capture of scan_tc_kernel on a 1 M-row cut of the 24 M x 768 workload
-# (dram__bytes_read.sum = 1.5514 GB against 1.5400 GB of bf16 rows + norms; dram__bytes_write.sum = 0.0971 GB of
+# (dram__bytes_read.sum = 1.5502 GB against 1.5400 GB of bf16 rows + norms; dram__bytes_write.sum = 0.0943 GB of
 # candidate appends while the thresholds of the first tiles are still open).  The bytes read grow with the row tiles
 # like the algorithmic ones, the appends do not, so a full launch is taken as ratio x algorithmic + appends.  Valid
 # for d = 768 and 256 misses per launch only; None once the kernel has changed since the counters were taken.
-SCAN_TRAFFIC_D768_M256 = dict(read_ratio=1.0074, append_bytes=97_125_888)
+SCAN_TRAFFIC_D768_M256 = dict(read_ratio=1.0066, append_bytes=94_348_544)
 
 
 def roofline_of_scan(cfg, mean_misses, scan_ms_per_launch, peaks, clocks=None, traffic=None):
@@ -217,6 +217,35 @@ def time_stream(p, batches, device_mode, dist_barrier, profile_scan=True):
     return ms, stats, scan_ms, scan_n, launches
 
 
+def time_stream_replayed(p, batches, dist_barrier):
+    """The same batches through one recorded batch call (prox_record_batch / prox_replay_batch): every step
+    copies its queries into the recording's fixed buffer (device to device, inside the timed region) and
+    replays.  Returns (ms, stats, hit flags of the last batch)."""
+    q0, i0, d0, h0 = batches[0]
+    dev = q0.device
+    qb, ib, db, hb = torch.empty_like(q0), torch.empty_like(i0), torch.empty_like(d0), torch.empty_like(h0)
+    torch.cuda.synchronize()
+    p.reset_cache()
+    side = torch.cuda.Stream(device=dev)             # stream capture needs a stream other than the legacy default one
+    side.wait_stream(torch.cuda.current_stream(dev))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(side):
+        rec = p.record_batch(qb, ib, db, hb, stream=side)
+        dist_barrier()
+        side.synchronize()
+        e0.record(side)
+        for q, _, _, _ in batches:
+            qb.copy_(q, non_blocking=True)
+            rec.replay(stream=side)
+        e1.record(side)
+        side.synchronize()
+    dist_barrier()
+    ms = e0.elapsed_time(e1)
+    stats = p.stats()
+    rec.close()
+    return ms, stats, hb
+
+
 def scan_roofline(cfg, r, peaks):
     """Roofline of the scan over the launches that had misses to scan (a launch takes up to 256 of them;
     launches of batches without misses return at once and only add their few microseconds)."""
@@ -227,7 +256,7 @@ def scan_roofline(cfg, r, peaks):
 
 
 def run_streams(prox, cfg, queries, taus, K, Wm, dev, local, barrier, make_handle, peaks, e2e=True, stages=False,
-                sustained_steps=0):
+                sustained_steps=0, replay=False):
     """The query stream of a workload through one handle per tolerance: W untimed batches, then K
     timed ones from an empty cache (CUDA events on the launching stream); for the first tolerance
     also the same batches through the host-buffer entry point, and the long run."""
@@ -283,6 +312,12 @@ def run_streams(prox, cfg, queries, taus, K, Wm, dev, local, barrier, make_handl
                                       scan_ms_per_launch=rf["ms_per_launch"], scan_bound=rf["bound"], scan_frac=rf["frac"],
                                       scan_frac_of_sustained_peak=rf.get("frac_of_sustained_peak"),
                                       ms_x_sm_ghz=rf.get("ms_x_sm_ghz"), clocks=ck)
+        if tau == head_tau and replay:
+            # launch-bound shapes: the batch call recorded once and replayed (same batches, same counters)
+            ms_r, st_r, _ = time_stream_replayed(p, batches, barrier)
+            same = all(st_r[kk] == stats[kk] for kk in ("queries", "hits", "misses", "evictions", "intra_batch_hits"))
+            assert same, "the replayed stream and the plain stream disagree"
+            r["ms_replayed"] = ms_r
         if stages:
             p.reset_cache()
             p.profile(None)
@@ -332,7 +367,8 @@ def run_extra_stream_workload(prox, name, args, dev, local, peaks, K, stages=Tru
     torch.cuda.synchronize()
     t_gen = time.time() - t0
     results, _ = run_streams(prox, cfg, queries, taus, K, Wm, dev, local, lambda: None,
-                             lambda tau: prox.Prox(corpus, cfg.k, cfg.capacity, tau, cfg.policy), peaks, e2e=False, stages=stages)
+                             lambda tau: prox.Prox(corpus, cfg.k, cfg.capacity, tau, cfg.policy), peaks, e2e=False, stages=stages,
+                             replay=cfg.batch <= 64)
     head = results[taus[0]]
     rf = scan_roofline(cfg, head, peaks)
     out = dict(workload=workload_text(cfg, taus[0]), steps=K, warmup=Wm, value=round(K * cfg.batch / (head["ms"] * 1e-3), 1), unit=UNIT,
@@ -340,6 +376,12 @@ def run_extra_stream_workload(prox, name, args, dev, local, peaks, K, stages=Tru
                hit_rate=round(head["hit_rate"], 4), gpu_launches=int(head["launches"]), clocks=head["clocks"],
                roofline=rf, tau_sweep=sweep_rows(cfg, results, K, peaks), gen_seconds=round(t_gen, 1),
                l2="inputs_exceed_l2" if cfg.N * cfg.d * 2 > 126e6 else "corpus_fits_l2")
+    if "ms_replayed" in head:
+        mr = head["ms_replayed"]
+        out["replayed"] = dict(value=round(K * cfg.batch / (mr * 1e-3), 1), unit=UNIT, ms_per_step=round(mr / K, 4),
+                               us_per_query=round(mr * 1e3 / (K * cfg.batch), 3),
+                               how="prox_record_batch once, then per step a device-to-device copy of the queries into "
+                                   "the recording's buffer and prox_replay_batch; same batches, same counters")
     del corpus, queries
     gc.collect()
     torch.cuda.empty_cache()
@@ -461,7 +503,8 @@ def run_ours(args):
         return prox.Prox(corpus, cfg.k, cfg.capacity, tau, cfg.policy, rho=args.rho, metric=args.metric)
 
     results, extra = run_streams(prox, cfg, queries, taus, K, Wm, dev, local, barrier, make_handle, peaks, e2e=True,
-                                 stages=bool(args.stages) and rank == 0, sustained_steps=long_steps)
+                                 stages=bool(args.stages) and rank == 0, sustained_steps=long_steps,
+                                 replay=cfg.batch <= 64 and not sharded)
 
     # max over ranks of the times, sum over ranks of the queries
     head = results[head_tau]
@@ -494,6 +537,12 @@ def run_ours(args):
             stats=head["stats"],
         )
         line.update(extra)
+        if "ms_replayed" in head:
+            mr = head["ms_replayed"]
+            line["replayed"] = dict(value=round(K * cfg.batch / (mr * 1e-3), 1), unit=UNIT, ms_per_step=round(mr / K, 4),
+                                    us_per_query=round(mr * 1e3 / (K * cfg.batch), 3),
+                                    how="prox_record_batch once, then per step a device-to-device copy of the queries "
+                                        "into the recording's buffer and prox_replay_batch; same batches, same counters")
 
     del corpus, queries, results
     gc.collect()

@@ -427,6 +427,76 @@ extern "C" int32_t prox_query_batch(prox_handle *h, const float *queries, int32_
     return check_launch("prox_query_batch");
 }
 
+// ------------------------------------------------------------------------------------------
+// A batch call recorded once and replayed: the launches of prox_query_batch with fixed buffers,
+// captured into a CUDA graph.  For small batches over small corpora the device work of a batch is
+// tens of microseconds and the chain of launches is what a call costs; a replay submits the
+// whole chain with one call.  Two recordings are kept, because consecutive scans alternate the
+// halves of the pairs' speed table: the replays alternate the same way.
+// ------------------------------------------------------------------------------------------
+struct prox_recorded_batch {
+    prox_handle *h;
+    cudaGraphExec_t exec[2];
+    int64_t launches_per_call;
+    unsigned turn;
+};
+
+extern "C" prox_recorded_batch *prox_record_batch(prox_handle *h, const float *queries, int32_t B, int64_t *out_ids,
+                                                  float *out_dists, uint8_t *out_hit, void *stream) {
+    if (check_batch_args(h, queries, B)) return nullptr;
+    if (!out_ids || !out_dists || !out_hit) { set_err("an output pointer is NULL"); return nullptr; }
+    if (h->sharded) { set_err("a shard's calls are not recorded"); return nullptr; }
+    if (h->prof) { set_err("switch prox_profile off before recording: its events would become part of the recording"); return nullptr; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    prox_recorded_batch *r = new (std::nothrow) prox_recorded_batch();
+    if (!r) { set_err("out of host memory"); return nullptr; }
+    r->h = h; r->exec[0] = r->exec[1] = nullptr; r->turn = 0;
+    const int64_t launches0 = h->launches;
+    for (int i = 0; i < 2; ++i) {
+        cudaGraph_t g = nullptr;
+        cudaError_t e = cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal);
+        if (e == cudaSuccess) {
+            const float *q = enqueue_lookup_and_scan(h, queries, B, out_ids, out_dists, out_hit, s);
+            enqueue_answers_and_inserts(h, q, B, out_ids, out_dists, s);
+            e = cudaStreamEndCapture(s, &g);
+        }
+        if (e == cudaSuccess) e = cudaGraphInstantiate(&r->exec[i], g, 0);
+        if (g) cudaGraphDestroy(g);
+        if (e != cudaSuccess) {
+            set_err("prox_record_batch: %s", cudaGetErrorString(e));
+            cudaGetLastError();
+            if (r->exec[0]) cudaGraphExecDestroy(r->exec[0]);
+            delete r;
+            h->launches = launches0;
+            return nullptr;
+        }
+    }
+    r->launches_per_call = (h->launches - launches0) / 2;
+    h->launches = launches0;                                  // nothing has run yet
+    return r;
+}
+
+extern "C" int32_t prox_replay_batch(prox_recorded_batch *r, void *stream) {
+    g_err[0] = 0;
+    if (!r) { set_err("recording is NULL"); return PROX_ERR_INVALID_ARG; }
+    const cudaError_t e = cudaGraphLaunch(r->exec[r->turn & 1u], static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+        set_err("prox_replay_batch: %s", cudaGetErrorString(e));
+        cudaGetLastError();
+        return PROX_ERR_CUDA;
+    }
+    r->turn++;
+    r->h->launches += r->launches_per_call;
+    return PROX_OK;
+}
+
+extern "C" void prox_recorded_batch_destroy(prox_recorded_batch *r) {
+    if (!r) return;
+    for (int i = 0; i < 2; ++i)
+        if (r->exec[i]) cudaGraphExecDestroy(r->exec[i]);
+    delete r;
+}
+
 extern "C" prox_handle *prox_create_shard(const float *corpus, int64_t N, int32_t d, int32_t k, int64_t capacity,
                                           float tau, int32_t policy, int32_t metric, int64_t row_offset,
                                           int64_t n_total) {

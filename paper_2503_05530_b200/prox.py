@@ -93,6 +93,12 @@ def load_library():
     L.prox_profile.argtypes = [vp, C.c_uint32]
     L.prox_profile_read.restype = i32
     L.prox_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64), vp]
+    L.prox_record_batch.restype = vp
+    L.prox_record_batch.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    L.prox_replay_batch.restype = i32
+    L.prox_replay_batch.argtypes = [vp, vp]
+    L.prox_recorded_batch_destroy.restype = None
+    L.prox_recorded_batch_destroy.argtypes = [vp]
     L.prox_nearest_key_static.restype = i32
     L.prox_nearest_key_static.argtypes = [vp, i64, i32, vp, i32, vp, vp, vp]
     _lib = L
@@ -128,6 +134,27 @@ def nearest_key_static(keys: torch.Tensor, queries: torch.Tensor, out_slot: torc
     _check(load_library().prox_nearest_key_static(keys.data_ptr(), keys.shape[0], keys.shape[1], queries.data_ptr(),
                                                   queries.shape[0], out_slot.data_ptr(), out_dist.data_ptr(),
                                                   _stream_ptr(stream)))
+
+
+class RecordedBatch:
+    """A recorded prox_query_batch call (prox_record_batch); keeps its buffers alive."""
+
+    def __init__(self, owner, ptr, buffers):
+        self._owner, self._r, self.buffers = owner, ptr, buffers
+
+    def replay(self, stream=None):
+        _check(self._owner._lib.prox_replay_batch(self._r, _stream_ptr(stream)))
+
+    def close(self):
+        if self._r:
+            self._owner._lib.prox_recorded_batch_destroy(self._r)
+            self._r = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 class Prox:
@@ -191,6 +218,23 @@ class Prox:
         _check(self._lib.prox_query_batch(self._h, q.data_ptr(), B, out_ids.data_ptr(), out_dists.data_ptr(),
                                           out_hit.data_ptr(), _stream_ptr(stream)))
         return out_ids, out_dists, out_hit
+
+    def record_batch(self, queries: torch.Tensor, out_ids: torch.Tensor, out_dists: torch.Tensor,
+                     out_hit: torch.Tensor, stream=None) -> "RecordedBatch":
+        """prox_record_batch: the batch call on these buffers as a replayable recording (nothing runs
+        yet).  `stream` (default: the current one) must not be the legacy default stream."""
+        q = _dev_f32(queries, "queries")
+        if q.shape[1] != self.d:
+            raise ProxError("queries have the wrong dimension")
+        B = q.shape[0]
+        for t, dt in ((out_ids, torch.int64), (out_dists, torch.float32), (out_hit, torch.uint8)):
+            if not (t.is_cuda and t.is_contiguous() and t.dtype == dt and t.shape[0] == B):
+                raise ProxError("record_batch takes contiguous CUDA outputs of the batch's shape")
+        r = self._lib.prox_record_batch(self._h, q.data_ptr(), B, out_ids.data_ptr(), out_dists.data_ptr(),
+                                        out_hit.data_ptr(), _stream_ptr(stream))
+        if not r:
+            raise ProxError(f"prox_record_batch failed: {last_error()}")
+        return RecordedBatch(self, r, (q, out_ids, out_dists, out_hit))
 
     def query_batch_host(self, queries: torch.Tensor, out_ids: torch.Tensor, out_dists: torch.Tensor,
                          out_hit: torch.Tensor, stream=None):

@@ -19,7 +19,7 @@ REL_DIST = 1e-4
 
 
 def run_gpu(corpus_t, queries_t, k, capacity, tau, policy, batch, scan_mode=None, host_api=False, rho=1,
-            lsh_planes=None, lsh_bucket=0, metric="l2"):
+            lsh_planes=None, lsh_bucket=0, metric="l2", recorded=False):
     """corpus_t, queries_t: CUDA float32 tensors.  Returns numpy (ids, dists, hit) and the stats."""
     planes_t = None if lsh_planes is None else torch.as_tensor(lsh_planes).to(corpus_t.device)
     p = prox.Prox(corpus_t, k, capacity, tau, policy, rho=rho, lsh_planes=planes_t, lsh_bucket=lsh_bucket, metric=metric)
@@ -37,6 +37,28 @@ def run_gpu(corpus_t, queries_t, k, capacity, tau, policy, batch, scan_mode=None
                 b = min(n, a + batch)
                 p.query_batch_host(qh[a:b], ih[a:b], dh[a:b], hh[a:b])
             ids, dists, hit = ih, dh, hh
+        elif recorded:
+            # the batch call recorded once on fixed buffers and replayed for every full batch; a ragged
+            # last batch takes the plain call on the same stream
+            dev = corpus_t.device
+            qb = torch.empty(batch, queries_t.shape[1], dtype=torch.float32, device=dev)
+            ib = torch.empty(batch, k, dtype=torch.int64, device=dev)
+            db = torch.empty(batch, k, dtype=torch.float32, device=dev)
+            hb = torch.empty(batch, dtype=torch.uint8, device=dev)
+            side = torch.cuda.Stream(device=dev)
+            side.wait_stream(torch.cuda.current_stream(dev))
+            with torch.cuda.stream(side):
+                rec = p.record_batch(qb, ib, db, hb, stream=side)
+                for a in range(0, n, batch):
+                    b = min(n, a + batch)
+                    if b - a == batch:
+                        qb.copy_(queries_t[a:b])
+                        rec.replay(stream=side)
+                        ids[a:b].copy_(ib); dists[a:b].copy_(db); hit[a:b].copy_(hb)
+                    else:
+                        p.query_batch(queries_t[a:b], ids[a:b], dists[a:b], hit[a:b], stream=side)
+                side.synchronize()
+                rec.close()
         else:
             for a in range(0, n, batch):
                 b = min(n, a + batch)

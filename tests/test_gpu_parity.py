@@ -578,6 +578,49 @@ def test_host_buffer_entry_point_equals_device_entry_point():
         assert np.array_equal(x, y)
 
 
+@pytest.mark.parametrize("policy,batch,d,kw", [("fifo", 1, 768, {}), ("lru", 64, 128, {}), ("lru", 3, 64, {"rho": 2}),
+                                               ("fifo", 200, 128, {"metric": "cosine"}), ("lru", 1, 128, {"metric": "ip"})])
+def test_recorded_batches_replay_the_plain_call(policy, batch, d, kw):
+    """prox_record_batch / prox_replay_batch: the batch call captured once on fixed buffers and
+    replayed for a stream of batches, against the oracle (the cache state carries over from replay
+    to replay) and, output for output and counter for counter, against the plain call."""
+    X, Q = stream(9001, d, 16, 900 if batch > 1 else 300, 400, 0.8, 0.02, seed=23)
+    l2 = {768: 0.7, 128: 0.13, 64: 0.08}[d]                    # about the squared distance of two noisy copies of a topic
+    tau = {"ip": l2 / 2 - 1.0, "cosine": l2 / 2}.get(kw.get("metric"), l2)
+    res, gpu = check(X, Q, 10, 50, tau, policy, batch, recorded=True, **kw)
+    assert 0.0 < res["hit_rate"] < 1.0
+    plain = run_gpu(X.to(DEV), Q.to(DEV), 10, 50, tau, policy, batch, **kw)
+    for x, y in zip(gpu[:3], plain[:3]):
+        assert np.array_equal(x, y)
+    assert gpu[3] == plain[3]
+
+
+def test_recording_argument_checks():
+    X, Q = stream(3001, 64, 8, 64, 20, 1.1, 0.02, seed=24)
+    p = prox.Prox(X.to(DEV), 5, 20, 0.5, "lru")
+    q = Q[:8].to(DEV)
+    ids = torch.empty(8, 5, dtype=torch.int64, device=DEV)
+    dist = torch.empty(8, 5, dtype=torch.float32, device=DEV)
+    hit = torch.empty(8, dtype=torch.uint8, device=DEV)
+    side = torch.cuda.Stream()
+    p.profile(None)
+    with pytest.raises(prox.ProxError, match="prox_profile"):
+        p.record_batch(q, ids, dist, hit, stream=side)
+    p.profile(())
+    with pytest.raises(prox.ProxError):
+        p.record_batch(q, ids, dist, hit.to(torch.int32), stream=side)
+    launches = p.kernel_launches()
+    rec = p.record_batch(q, ids, dist, hit, stream=side)
+    assert p.kernel_launches() == launches and p.stats()["queries"] == 0      # recording runs nothing
+    rec.replay(stream=side)
+    side.synchronize()
+    assert p.stats()["queries"] == 8 and p.kernel_launches() > launches
+    assert p.status() == prox.OK
+    rec.close()
+    rec.close()
+    p.close()
+
+
 @pytest.mark.parametrize("d,batch", [(768, 64), (128, 256), (256, 24), (128, 600)])
 def test_the_three_scan_kernels_agree(d, batch):
     """Two-block tensor-core scan (default), one-block tensor-core scan and CUDA-core scan."""
