@@ -298,7 +298,7 @@ risk_ring_kernel(DevState *st, const u64 *__restrict__ stamp, int32_t *risk_pos,
 //   mode 4  mode 1, but only if that pass listed more pairs than it can hold (else return at once).
 // ------------------------------------------------------------------------------------------
 constexpr int PQ = 32;
-constexpr int kProbeColsWide = 64, kProbeColsNarrow = 32;
+constexpr int kProbeColsWide = 64, kProbeColsNarrow = 32, kProbeColsTiny = 16;
 
 // PC = columns per block tile, PD = dimensions per step: 64 x 32, or 32 x 64 for a small cache,
 // where the wide tiles leave most SMs without a block and the time goes into the chain of steps
@@ -1461,7 +1461,10 @@ __global__ void cache_load_kernel(long long n, int d, int k, const float *__rest
 static int probe_cols(const prox_handle *h, int B) {
     const long long wide = (h->C + B + kProbeColsWide - 1) / kProbeColsWide;
     const int qtiles = (B + PQ - 1) / PQ;
-    return wide * qtiles < 2LL * h->num_sms ? kProbeColsNarrow : kProbeColsWide;
+    if (wide * qtiles >= 2LL * h->num_sms) return kProbeColsWide;
+    // fewer blocks than SMs even with narrow tiles (a small batch against a small cache): halve the tiles again
+    const long long narrow = (h->C + B + kProbeColsNarrow - 1) / kProbeColsNarrow;
+    return narrow * qtiles < h->num_sms ? kProbeColsTiny : kProbeColsNarrow;
 }
 
 static int probe_splits(const prox_handle *h, int B) {
@@ -1538,8 +1541,9 @@ void launch_probe(prox_handle *h, const float *q, int B, int mode, cudaStream_t 
         if (splits > tiles) splits = tiles;
     }
     dim3 grid((B + PQ - 1) / PQ, splits);
-    auto kern = PC == kProbeColsNarrow ? (metric_is_ip(h) ? probe_kernel<kProbeColsNarrow, 64, true> : probe_kernel<kProbeColsNarrow, 64, false>)
-                                       : (metric_is_ip(h) ? probe_kernel<kProbeColsWide, 32, true> : probe_kernel<kProbeColsWide, 32, false>);
+    auto kern = PC == kProbeColsTiny     ? (metric_is_ip(h) ? probe_kernel<kProbeColsTiny, 64, true> : probe_kernel<kProbeColsTiny, 64, false>)
+                : PC == kProbeColsNarrow ? (metric_is_ip(h) ? probe_kernel<kProbeColsNarrow, 64, true> : probe_kernel<kProbeColsNarrow, 64, false>)
+                                         : (metric_is_ip(h) ? probe_kernel<kProbeColsWide, 32, true> : probe_kernel<kProbeColsWide, 32, false>);
     kern<<<grid, 256, 0, s>>>(h->st, h->keys, q, h->risk_pos, B, h->d, h->part_min, h->part_arg, h->d_risk, h->d_intra, mode,
                               h->risk_slot, h->pfail_list);
     h->launches++;

@@ -17,7 +17,7 @@ constexpr int kTileRows = 128;               // corpus rows per scan tile (MMA M
 constexpr int kBufCap = 512;                 // entries of one (CTA, query) candidate buffer
 constexpr int kCollectCap = 2048;            // rows the exact pass may collect per query
 constexpr int kOverMax = 64;                 // queries per batch whose collection may overflow and still be answered exactly
-constexpr int kProbeSplitMax = 64;           // column splits of the probe grid
+constexpr int kProbeSplitMax = 128;          // column splits of the probe grid
 constexpr int kPairCap = 1 << 20;             // query-key pairs the tensor-core pass over at-risk slots and batch may hand on
 constexpr int kSideMinBatch = 512;            // batches from this size on take that pass instead of fp64 rows
 constexpr int kProbeKp = 64;                 // slots per query the coarse probe keeps for the exact recheck
