@@ -792,8 +792,8 @@ __device__ bool replay_parallel(ResolveSmem &sm, DevState *st, int B, int R, lon
             int t = -1;
             for (int h = hd; h < n; ++h) {
                 const int code = lc[h];
-                // (outcomes of other queries are read while their threads may be writing this round's:
-                // either value is a legitimate iterate, and a round that changes nothing read only final ones)
+                // (outcomes of other queries are read while their threads may be writing this sweep's:
+                // either value is a legitimate iterate, and a sweep that changes nothing read only final ones)
                 const bool valid = code < kMaxBatch ? sm.p_E[code] >= i
                                                     : ((volatile int *)sm.p_tgt)[code - kMaxBatch] == -1;
                 if (valid) { t = h; break; }
@@ -815,7 +815,7 @@ __device__ bool replay_parallel(ResolveSmem &sm, DevState *st, int B, int R, lon
         if (!any) { converged = true; break; }
     }
     if (!converged) return false;
-    // (rank, total_miss, mq, total_ev, p_tm, p_skip, p_E are those of the last round, which changed nothing)
+    // (rank, total_miss, mq, total_ev, p_tm, p_skip, p_E are those of the last sweep, which changed nothing)
     const int n_evict = total_miss > free0 ? total_miss - free0 : 0;
     if (n_evict > total_ev) return false;                  // the at-risk list would be used up
     const int n_free = total_miss < free0 ? total_miss : free0;
@@ -967,7 +967,7 @@ __device__ void resolve_block(ResolveSmem &sm, DevState *st, int B, long long C,
                 if (hd == n) { kind = safe_hit ? 1 : 2; changed = true; }
                 else if (safe_hit && sd < ld[hd]) { kind = 1; changed = true; }
             }
-            __syncthreads();                               // everyone has read the kinds of this round
+            __syncthreads();                               // everyone has read the kinds of this pass
             if (changed) sm.kind[i] = (unsigned char)kind;
             if (!__syncthreads_or(changed ? 1 : 0)) break;
         }
