@@ -16,8 +16,10 @@ namespace prox {
 namespace {
 
 constexpr int kSideTile = 128;            // queries x columns of one block
-constexpr int kSideK = 32;                // dimensions per pipeline step
+constexpr int kSideK = 64;                // dimensions per pipeline step
 constexpr int kSideLd = kSideK + 8;       // row pitch in shared memory (bf16): fragment loads without bank conflicts
+constexpr int kSideStages = 3;            // steps in flight: the operands come from L2, a microsecond away
+constexpr int kSideSmem = kSideStages * 2 * kSideTile * kSideLd * 2;   // bytes of dynamic shared memory
 
 __device__ __forceinline__ void cp_async16(void *dst, const void *src, bool pred) {
     const unsigned d = (unsigned)__cvta_generic_to_shared(dst);
@@ -52,9 +54,12 @@ probe_side_kernel(DevState *st, const __nv_bfloat16 *__restrict__ pqb, const flo
                   const float *__restrict__ pqerr, const __nv_bfloat16 *__restrict__ keys_b,
                   const float *__restrict__ kh, const int32_t *__restrict__ risk_slot, int B, int d, double tau,
                   uint32_t *pairs) {
-    __shared__ __align__(16) __nv_bfloat16 As[2][kSideTile][kSideLd];
-    __shared__ __align__(16) __nv_bfloat16 Bs[2][kSideTile][kSideLd];
+    extern __shared__ __align__(16) unsigned char side_smem[];
+    typedef __nv_bfloat16 (*Tile)[kSideTile][kSideLd];
+    Tile As = reinterpret_cast<Tile>(side_smem);                                   // [kSideStages][kSideTile][kSideLd]
+    Tile Bs = reinterpret_cast<Tile>(side_smem + (size_t)kSideStages * kSideTile * kSideLd * 2);
     __shared__ float col_n2[kSideTile], col_err[kSideTile];
+    __shared__ double col_n[kSideTile];                       // |bf16 column|, one square root per column instead of one per pair
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int R = st->n_risk;
     const int i0 = blockIdx.x * kSideTile;
@@ -64,12 +69,12 @@ probe_side_kernel(DevState *st, const __nv_bfloat16 *__restrict__ pqb, const flo
     if (c0 >= n_cols) return;
     if (batch_cols && c0 >= i0 + kSideTile - 1) return;       // no column of the tile precedes a query of the tile
 
-    // rows this thread copies: two of A (queries) and two of B (columns), 16 bytes of each per step
-    const int lr = tid >> 2, part = tid & 3;
-    const __nv_bfloat16 *a_src[2], *b_src[2];
+    // rows this thread copies: four of A (queries) and four of B (columns), 16 bytes of each per step
+    const int lr = tid >> 3, part = tid & 7;
+    const __nv_bfloat16 *a_src[4], *b_src[4];
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
-        const int r = lr + 64 * u;
+    for (int u = 0; u < 4; ++u) {
+        const int r = lr + 32 * u;
         a_src[u] = (i0 + r < B) ? pqb + (size_t)(i0 + r) * d + part * 8 : nullptr;
         const int c = c0 + r;
         b_src[u] = nullptr;
@@ -84,12 +89,13 @@ probe_side_kernel(DevState *st, const __nv_bfloat16 *__restrict__ pqb, const flo
         }
         col_n2[tid] = n2;
         col_err[tid] = er;
+        col_n[tid] = sqrt((double)n2);
     }
     auto load_stage = [&](int stage, int k0) {
         const bool in_row = k0 + part * 8 < d;                // d is a multiple of 16: the last step may be half empty
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int r = lr + 64 * u;
+        for (int u = 0; u < 4; ++u) {
+            const int r = lr + 32 * u;
             const bool pa = in_row && a_src[u] != nullptr, pb = in_row && b_src[u] != nullptr;
             cp_async16(&As[stage][r][part * 8], pa ? a_src[u] + k0 : pqb, pa);
             cp_async16(&Bs[stage][r][part * 8], pb ? b_src[u] + k0 : pqb, pb);
@@ -108,16 +114,14 @@ probe_side_kernel(DevState *st, const __nv_bfloat16 *__restrict__ pqb, const flo
     const int g = lane >> 2, t = lane & 3;
     const int steps = (d + kSideK - 1) / kSideK;
 
+    // (one commit group per step, empty past the last step, so that "all but the newest two" is always step s)
     load_stage(0, 0);
+    if (steps > 1) load_stage(1, kSideK); else cp_async_commit();
     for (int s = 0; s < steps; ++s) {
-        if (s + 1 < steps) {
-            load_stage((s + 1) & 1, (s + 1) * kSideK);
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
-        }
+        if (s + 2 < steps) load_stage((s + 2) % kSideStages, (s + 2) * kSideK); else cp_async_commit();
+        cp_async_wait<2>();
         __syncthreads();
-        const int st_ = s & 1;
+        const int st_ = s % kSideStages;
 #pragma unroll
         for (int kk = 0; kk < kSideK / 16; ++kk) {
             uint32_t af[2][4];
@@ -160,7 +164,7 @@ probe_side_kernel(DevState *st, const __nv_bfloat16 *__restrict__ pqb, const flo
                     if (c >= n_cols || (batch_cols && c >= i)) continue;
                     const double n2 = (double)col_n2[lc];
                     const double coarse = qn2 + n2 - 2.0 * (double)acc[mi][ni][2 * half + cc];
-                    if (coarse <= side_coarse_bound(root_tau, qa, (double)col_err[lc], qn, sqrt(n2), d)) {
+                    if (coarse <= side_coarse_bound(root_tau, qa, (double)col_err[lc], qn, col_n[lc], d)) {
                         const int pos = atomicAdd(&st->n_pairs, 1);
                         if (pos < kPairCap) pairs[pos] = ((uint32_t)i << 16) | (uint32_t)(batch_cols ? kMaxBatch + c : c);
                         else st->side_overflow = 1;
@@ -201,9 +205,14 @@ probe_pairs_exact_kernel(const DevState *__restrict__ st, const float *__restric
     }
 }
 
+// Kernel attributes belong to a device: set when a handle is created there.
+void set_probe_side_attributes() {
+    cudaFuncSetAttribute(probe_side_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSideSmem);
+}
+
 void launch_probe_side(prox_handle *h, const float *q, int B, cudaStream_t s) {
     dim3 grid((B + kSideTile - 1) / kSideTile, 2 * kMaxBatch / kSideTile);
-    probe_side_kernel<<<grid, 256, 0, s>>>(h->st, h->pqb, h->pqbn, h->pqerr, h->keys_b, h->kh, h->risk_slot, B, h->d,
+    probe_side_kernel<<<grid, 256, kSideSmem, s>>>(h->st, h->pqb, h->pqbn, h->pqerr, h->keys_b, h->kh, h->risk_slot, B, h->d,
                                            (double)h->tau, h->side_pairs);
     probe_pairs_exact_kernel<<<h->num_sms * 4, 256, 0, s>>>(h->st, h->keys, q, h->risk_slot, h->d, (double)h->tau,
                                                            h->side_pairs, h->cand_d, h->cand_code, h->n_cand);

@@ -162,6 +162,7 @@ static prox_handle *create_handle(const float *corpus, int64_t N, int32_t d, int
     h->num_sms = prop.multiProcessorCount;
     h->scan_ctas = h->num_sms;
     set_cache_kernel_attributes();
+    set_probe_side_attributes();
     set_scan_kernel_attributes();
 
     const size_t MB = kMaxBatch, C = (size_t)capacity, P = (size_t)h->scan_ctas;

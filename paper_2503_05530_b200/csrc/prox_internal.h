@@ -164,6 +164,7 @@ struct prox_handle {
 namespace prox {
 // per-device kernel attributes (dynamic shared memory limits), set at prox_create
 void set_cache_kernel_attributes();
+void set_probe_side_attributes();
 void set_scan_kernel_attributes();
 // create-time kernels
 void launch_convert_corpus(prox_handle *h, cudaStream_t s);
