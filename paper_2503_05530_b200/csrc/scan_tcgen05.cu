@@ -631,6 +631,13 @@ static void ensure_maps(prox_handle *h, void **state, const __nv_bfloat16 *xb, l
             make_map(&m->q64, qb, kMaxBatch, (uint64_t)h->d, 64, ks) &&
             make_map(&m->q128, qb, kMaxBatch, (uint64_t)h->d, 128, ks) &&
             make_map(&m->q256, qb, kMaxBatch, (uint64_t)h->d, 256, ks);
+    if (m->speed) {
+        // equal speeds from the start, for the launch shape the handle takes by default: the first scan of a
+        // handle may be recorded (prox_record_batch), and a recording must not carry the table's reset
+        speed_init_kernel<<<1, 256>>>(m->speed);
+        const bool pair = h->scan_ctas >= 2 && rows >= 2 * kTileRows;
+        m->units = pair ? (h->scan_ctas & ~1) / 2 : h->scan_ctas;
+    }
     set_scan_smem<256, false, false>(); set_scan_smem<512, false, false>(); set_scan_smem<256, true, false>(); set_scan_smem<512, true, false>();
     set_scan_smem<256, false, true>(); set_scan_smem<512, false, true>(); set_scan_smem<256, true, true>(); set_scan_smem<512, true, true>();
 }
