@@ -42,12 +42,14 @@ __device__ int select_smallest(const u64 *__restrict__ keys, const int32_t *__re
                 if ((v & mask) == prefix) atomicAdd(&hist[(unsigned)(v >> (8 * p)) & 255u], 1u);
             }
             __syncthreads();
-            if (tid == 0) {
-                int rem = *s_remaining, b = 0;
-                while (b < 255 && (int)hist[b] < rem) { rem -= (int)hist[b]; ++b; }
-                *s_remaining = rem;
-                *s_prefix = prefix | ((u64)b << (8 * p));
-                *s_mask = mask | (0xffull << (8 * p));
+            if (tid < 32) {
+                int rem = *s_remaining;
+                const int b = radix_digit_walk(hist, rem, false);
+                if (tid == 0) {
+                    *s_remaining = rem;
+                    *s_prefix = prefix | ((u64)b << (8 * p));
+                    *s_mask = mask | (0xffull << (8 * p));
+                }
             }
             __syncthreads();
         }
@@ -564,7 +566,6 @@ struct ResolveSmem {
     unsigned char r_touched[kMaxBatch];
     // the parallel replay (replay_parallel)
     int p_tgt[kMaxBatch];              // per query: -1 miss, -2 its nearest safe key, h >= 0 the h-th entry of its list
-    int p_rank[kMaxBatch];             // per query: misses before it
     int p_tm[kMaxBatch];               // query index of the m-th evicting miss
     int p_E[kMaxBatch];                // per at-risk position: the query that evicts it (kNever: none)
     int p_T[kMaxBatch];                // per at-risk position: the first query that hits it; at the end, the position the m-th eviction takes
@@ -767,7 +768,7 @@ __device__ bool replay_parallel(ResolveSmem &sm, DevState *st, int B, int R, lon
     for (int round = 0; round < kParallelRounds; ++round) {
         is_miss = i < B && sm.p_tgt[i] == -1;
         rank = block_excl_scan(is_miss ? 1 : 0, sm.warp_tot[0], total_miss);
-        if (i < kMaxBatch) { sm.p_rank[i] = rank; sm.p_tm[i] = kNever; sm.p_T[i] = kNever; }
+        if (i < kMaxBatch) { sm.p_tm[i] = kNever; sm.p_T[i] = kNever; }
         __syncthreads();
         if (is_miss && rank >= free0) sm.p_tm[rank - free0] = i;
         if (lru && kind == 3) {

@@ -324,12 +324,14 @@ merge_select_kernel(const int *__restrict__ n_active, int n_lists, int stride, i
                 }
             }
             __syncthreads();
-            if (tid == 0) {                        // walk the digits from the top: largest scores first
-                int rem = s_remaining, b = 255;
-                while (b > 0 && (int)hist[b] < rem) { rem -= (int)hist[b]; --b; }
-                s_remaining = rem;
-                s_prefix = prefix | ((uint32_t)b << (8 * dg));
-                s_mask = mask | (0xffu << (8 * dg));
+            if (warp == 0) {                       // walk the digits from the top: largest scores first
+                int rem = s_remaining;
+                const int b = radix_digit_walk(hist, rem, true);
+                if (lane == 0) {
+                    s_remaining = rem;
+                    s_prefix = prefix | ((uint32_t)b << (8 * dg));
+                    s_mask = mask | (0xffu << (8 * dg));
+                }
             }
             __syncthreads();
         }

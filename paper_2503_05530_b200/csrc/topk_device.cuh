@@ -24,6 +24,35 @@ __device__ __forceinline__ u64 pack_entry(float score, int32_t row) {
 __device__ __forceinline__ float entry_score(u64 e) { return o2f((uint32_t)(e >> 32)); }
 __device__ __forceinline__ int32_t entry_row(u64 e) { return (int32_t)(uint32_t)e; }
 
+// One digit of a radix select, for one whole warp: the 256 bins of hist are walked from the top
+// (descending) or from the bottom until the bin that holds the rem-th entry (rem >= 1); returns
+// that bin and leaves in rem the rank inside it.  If all bins together hold fewer than rem entries
+// the walk ends at its last bin, with the counts of all others taken off rem.  Lane l sums the
+// eight bins 8 l .. 8 l + 7 of the walk; a prefix sum over the lanes finds the lane of the answer.
+__device__ __forceinline__ int radix_digit_walk(const unsigned *hist, int &rem, bool descending) {
+    const int lane = threadIdx.x & 31;
+    int c[8], tot = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int w = 8 * lane + j;
+        c[j] = (int)hist[descending ? 255 - w : w];
+        tot += c[j];
+    }
+    int incl = tot;
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, incl, m);
+        if (lane >= m) incl += y;
+    }
+    const unsigned reach = __ballot_sync(0xffffffffu, incl >= rem);
+    const int owner = reach ? __ffs(reach) - 1 : 31;
+    int r = rem - (incl - tot), j = 0;
+    while (j < 7 && c[j] < r) { r -= c[j]; ++j; }
+    const int w = 8 * owner + __shfl_sync(0xffffffffu, j, owner);
+    rem = __shfl_sync(0xffffffffu, r, owner);
+    return descending ? 255 - w : w;
+}
+
 __device__ __forceinline__ u64 shfl_xor_u64(u64 v, int m) {
     uint32_t lo = __shfl_xor_sync(0xffffffffu, (uint32_t)v, m);
     uint32_t hi = __shfl_xor_sync(0xffffffffu, (uint32_t)(v >> 32), m);
