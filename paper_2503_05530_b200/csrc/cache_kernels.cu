@@ -175,7 +175,6 @@ risk_pick_kernel(const DevState *st, RiskWork *w, int B, long long C) {
     // bin inside it where the running count reaches R
     constexpr int per = kRiskBins / 1024;
     static_assert(per == 64, "two coalesced loads per lane cover one group");
-    __shared__ unsigned fine[per];
     __shared__ unsigned s_acc;
     __shared__ int s_group;
     const int lane = tid & 31, warp = tid >> 5;
@@ -186,21 +185,48 @@ risk_pick_kernel(const DevState *st, RiskWork *w, int B, long long C) {
         if (lane == 0) part[g] = v;
     }
     __syncthreads();
-    if (tid == 0) {
-        unsigned acc = 0;
-        int t = 0;
-        while (t < 1023 && acc + part[t] < (unsigned)R) { acc += part[t]; ++t; }
-        s_acc = acc;
-        s_group = t;
+    // the first group whose running count reaches R (the last group if none does): running counts by a
+    // block-wide prefix sum; they only grow, so the group is the number of groups that stay below R
+    __shared__ unsigned wt[32];
+    unsigned incl = part[tid];
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const unsigned y = __shfl_up_sync(0xffffffffu, incl, m);
+        if (lane >= m) incl += y;
+    }
+    if (lane == 31) wt[warp] = incl;
+    if (tid == 0) s_acc = 0;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned v = wt[lane];
+#pragma unroll
+        for (int m = 1; m < 32; m <<= 1) {
+            const unsigned y = __shfl_up_sync(0xffffffffu, v, m);
+            if (lane >= m) v += y;
+        }
+        wt[lane] = v;
     }
     __syncthreads();
-    if (tid < per) fine[tid] = w->hist[s_group * per + tid];
+    if (warp > 0) incl += wt[warp - 1];
+    int t = __syncthreads_count(incl < (unsigned)R);
+    if (t > 1023) t = 1023;
+    if (tid == t - 1) s_acc = incl;                      // the count before group t
+    if (tid == 0) s_group = t;
     __syncthreads();
-    if (tid == 0) {
-        unsigned acc = s_acc;
-        int i = 0;
-        while (i < per - 1 && acc + fine[i] < (unsigned)R) { acc += fine[i]; ++i; }
-        w->bin = s_group * per + i;
+    // the same inside the group's 64 bins, by one warp (two bins a lane)
+    if (warp == 0) {
+        const unsigned f0 = w->hist[t * per + 2 * lane], f1 = w->hist[t * per + 2 * lane + 1];
+        unsigned in2 = f0 + f1;
+#pragma unroll
+        for (int m = 1; m < 32; m <<= 1) {
+            const unsigned y = __shfl_up_sync(0xffffffffu, in2, m);
+            if (lane >= m) in2 += y;
+        }
+        const unsigned before = s_acc + in2 - f0 - f1;
+        int i = __popc(__ballot_sync(0xffffffffu, before + f0 < (unsigned)R)) +
+                __popc(__ballot_sync(0xffffffffu, before + f0 + f1 < (unsigned)R));
+        if (i > per - 1) i = per - 1;
+        if (lane == 0) w->bin = t * per + i;
     }
 }
 
