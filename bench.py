@@ -53,11 +53,11 @@ def load_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons of one GPU.  The sampler is started ahead of the timed region
+    """nvidia-smi clocks, throttle reasons and power draw of one GPU (read only).  The sampler is started ahead of the timed region
     (the tool needs a few hundred milliseconds before its first line) and keeps the time stamp of every sample;
     `stop` reports the samples taken between `begin()` and `end()` (all of them if none was marked)."""
     FIELDS = ("timestamp,clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,power.draw")
 
     def __init__(self, index: int):
         self.index, self.samples, self.proc = index, [], None
@@ -103,7 +103,11 @@ class ClockSampler:
                 continue
             try:
                 ts = datetime.datetime.strptime(t[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
-                rows.append((ts, float(t[1]), float(t[2]), [n for n, v in zip(names, t[3:7]) if v.lower().startswith("active")]))
+                try:
+                    watts = float(t[7]) if len(t) > 7 else None
+                except ValueError:
+                    watts = None
+                rows.append((ts, float(t[1]), float(t[2]), [n for n, v in zip(names, t[3:7]) if v.lower().startswith("active")], watts))
             except ValueError:
                 continue
         inside = rows
@@ -114,8 +118,9 @@ class ClockSampler:
                 inside = [min(rows, key=lambda r: abs(r[0] - mid))]
         sm = [r[1] for r in inside]
         reasons = sorted({n for r in inside for n in r[3]})
+        watts = [r[4] for r in inside if r[4] is not None]
         return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(r[2] for r in inside) if inside else None,
-                    reasons=reasons, samples=len(sm))
+                    reasons=reasons, samples=len(sm), power_w=round(statistics.median(watts), 1) if watts else None)
 
 
 def stream_seed(seed: int, rank: int) -> int:
