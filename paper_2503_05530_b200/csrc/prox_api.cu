@@ -336,7 +336,7 @@ static bool enqueue_probe_and_resolve(prox_handle *h, const float *queries, int3
             // safe slots: coarse scores on the tensor cores, exact recheck of the best few;
             // at-risk slots and the batch itself: full fp64 rows (or the pass above); uncertified
             // queries: fp64 over all slots
-            if (launch_probe_scan_tc(h, s) != 0) coarse = false;
+            if (launch_probe_scan_tc(h, B, s) != 0) coarse = false;
             if (coarse) launch_merge_select(h, B, 1, s);
         }
         if (side) launch_probe_side(h, queries, B, s);
@@ -389,7 +389,7 @@ static const float *enqueue_lookup_and_scan(prox_handle *h, const float *queries
     {
         StageScope t(h, PROX_STAGE_SCAN, s);
         // the tensor-core scan takes all passes of the batch in one launch, its CUDA-core twin one by one
-        if (h->scan_mode == PROX_SCAN_CUDA_CORE || launch_scan_tc(h, s) != 0)
+        if (h->scan_mode == PROX_SCAN_CUDA_CORE || launch_scan_tc(h, B, s) != 0)
             for (int p = 0; p < passes; ++p) launch_scan_pass(h, p, s);
     }
     { StageScope t(h, PROX_STAGE_MERGE, s); launch_merge_select(h, B, 0, s); }

@@ -191,11 +191,11 @@ void launch_reset(prox_handle *h, cudaStream_t s);
 // scan kernels
 void launch_prep_miss(prox_handle *h, const float *q, int B, cudaStream_t s);
 void launch_prep_probe(prox_handle *h, const float *q, int B, cudaStream_t s);
-int launch_probe_scan_tc(prox_handle *h, cudaStream_t s);              // coarse probe over the bf16 keys, all passes; nonzero = not available
+int launch_probe_scan_tc(prox_handle *h, int B, cudaStream_t s);              // coarse probe over the bf16 keys, all passes; nonzero = not available
 void launch_probe_exact(prox_handle *h, const float *q, int B, cudaStream_t s);
 void launch_probe_side(prox_handle *h, const float *q, int B, cudaStream_t s);   // at-risk slots and batch on the tensor cores -> candidate lists
 void launch_scan_pass(prox_handle *h, int pass, cudaStream_t s);       // CUDA-core scan
-int launch_scan_tc(prox_handle *h, cudaStream_t s);                    // tcgen05 scan, all passes of the batch; nonzero = not available
+int launch_scan_tc(prox_handle *h, int B, cudaStream_t s);                  // tcgen05 scan, all passes of the batch; nonzero = not available
 void init_scan_tc(prox_handle *h);                                      // tensor maps, at prox_create
 void free_scan_tc(prox_handle *h);
 void launch_merge_select(prox_handle *h, int B, int for_probe, cudaStream_t s);   // all passes of the batch at once

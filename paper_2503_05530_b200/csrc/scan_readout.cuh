@@ -28,7 +28,8 @@ __device__ __forceinline__ uint32_t select32(const uint32_t (&v)[32], int j) {
 // the instruction cache.
 template <int CAP>
 __device__ __forceinline__ void append32(const uint32_t (&v)[32], int c0, int lc0, float hn, int32_t row,
-                                         const float *thr, int *wcnt, uint32_t *best, u64 *lists, bool &need) {
+                                         const float *thr, int *wcnt, uint32_t *best, u64 *lists, bool &need,
+                                         int best_stride = 1) {
     uint32_t pass = 0;
 #pragma unroll
     for (int j4 = 0; j4 < 8; ++j4) {
@@ -61,7 +62,8 @@ __device__ __forceinline__ void append32(const uint32_t (&v)[32], int c0, int lc
         }
         if (mine) {                                              // the warp's columns are its own: plain updates
             wcnt[lc0 + lane] = base_mine + 32;
-            if (top_mine > best[c0 + lane]) best[c0 + lane] = top_mine;
+            uint32_t *bp = best + (size_t)(c0 + lane) * best_stride;      // (stride 1: the block's table; else the shared one)
+            if (top_mine > *bp) *bp = top_mine;
         }
         __syncwarp();
         if (__any_sync(0xffffffffu, mine && base_mine + 32 > CAP - 33)) need = true;
@@ -74,7 +76,7 @@ __device__ __forceinline__ void append32(const uint32_t (&v)[32], int c0, int lc
         const u64 ent = pack_entry(__uint_as_float(select32(v, j)) - hn, row);
         const int pos = atomicAdd(&wcnt[lc0 + j], 1);
         if (pos < CAP) lists[(size_t)(c0 + j) * CAP + pos] = ent;
-        atomicMax(&best[c0 + j], (uint32_t)(ent >> 32));
+        atomicMax(&best[(size_t)(c0 + j) * best_stride], (uint32_t)(ent >> 32));
         full |= pos + 1 > CAP - 33;                              // this list must be cut before the next tile
     }
     if (__any_sync(0xffffffffu, full)) need = true;
@@ -145,7 +147,8 @@ __device__ __forceinline__ float raw_max32(const uint32_t (&v)[32]) {
 template <int CAP>
 __device__ __forceinline__ void readout64(const uint32_t (&v0)[32], const uint32_t (&v1)[32], bool two, int c0,
                                           int lc0, float hn, float tmin0, float tmin1, int32_t row,
-                                          const float *thr, int *wcnt, uint32_t *best, u64 *lists, bool &need) {
+                                          const float *thr, int *wcnt, uint32_t *best, u64 *lists, bool &need,
+                                          int best_stride = 1) {
     // (both groups unconditionally, so that their chains overlap; without a second group v1 holds
     // nothing that matters and tmin1 rules it out)
     const float r0 = raw_max32(v0), r1 = raw_max32(v1);
@@ -156,12 +159,12 @@ __device__ __forceinline__ void readout64(const uint32_t (&v0)[32], const uint32
     const unsigned maybe1 = __ballot_sync(0xffffffffu, c1p);
     if (maybe0 != 0u) {
         const float m0 = max_margin32(v0, thr, c0);
-        if (__any_sync(0xffffffffu, m0 > hn)) append32<CAP>(v0, c0, lc0, hn, row, thr, wcnt, best, lists, need);
+        if (__any_sync(0xffffffffu, m0 > hn)) append32<CAP>(v0, c0, lc0, hn, row, thr, wcnt, best, lists, need, best_stride);
     }
     if (maybe1 != 0u) {
         const float m1 = max_margin32(v1, thr, c0 + 32);
         if (__any_sync(0xffffffffu, m1 > hn))
-            append32<CAP>(v1, c0 + 32, lc0 + 32, hn, row, thr, wcnt, best, lists, need);
+            append32<CAP>(v1, c0 + 32, lc0 + 32, hn, row, thr, wcnt, best, lists, need, best_stride);
     }
 }
 

@@ -547,6 +547,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     }
 }
 
+#include "scan_tc_multi.cuh"
+
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
@@ -640,6 +642,8 @@ static void ensure_maps(prox_handle *h, void **state, const __nv_bfloat16 *xb, l
     }
     set_scan_smem<256, false, false>(); set_scan_smem<512, false, false>(); set_scan_smem<256, true, false>(); set_scan_smem<512, true, false>();
     set_scan_smem<256, false, true>(); set_scan_smem<512, false, true>(); set_scan_smem<256, true, true>(); set_scan_smem<512, true, true>();
+    cudaFuncSetAttribute(scan_tc_multi_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegionM + 1024);
+    cudaFuncSetAttribute(scan_tc_multi_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileRegionM + 1024);
 }
 
 void init_scan_tc(prox_handle *h) {
@@ -652,7 +656,7 @@ void init_scan_tc(prox_handle *h) {
 // block qb.  Returns nonzero when the tensor-core path cannot run (no tensor-map encoder in the
 // driver, out of memory for the maps); the caller then falls back.
 static int launch_scan_generic(prox_handle *h, void **state, const __nv_bfloat16 *xb, const float *xh, long long rows,
-                               const __nv_bfloat16 *qb, const int *n_active, int kp, cudaStream_t s) {
+                               const __nv_bfloat16 *qb, const int *n_active, int n_max, int kp, cudaStream_t s) {
     if (!*state) return 1;
     Maps &maps = *static_cast<Maps *>(*state);
     if (!maps.ok) return 1;
@@ -686,8 +690,17 @@ static int launch_scan_generic(prox_handle *h, void **state, const __nv_bfloat16
     cfg.numAttrs = 1;
     // two MMA issuers when a row tile is one or two ring stages (up to 256 dimensions)
     const bool dual = (h->d / kChunkK) / maps.ks <= 2;
-    const cudaError_t e = h->tc_cap == 256 ? launch_scan_kernel<256>(pair, dual, cfg, maps, a)
-                                           : launch_scan_kernel<512>(pair, dual, cfg, maps, a);
+    // up to 128 dimensions and more queries than one pass takes: every pair serves all passes (the row tiles
+    // are read once instead of once per pass)
+    const bool multi = pair && (h->d / kChunkK) / maps.ks == 1 && n_max > kScanQ && h->scan_mode == PROX_SCAN_AUTO;
+    cudaError_t e;
+    if (multi) {
+        cfg.dynamicSmemBytes = kTileRegionM + 1024;
+        e = h->tc_cap == 256 ? cudaLaunchKernelEx(&cfg, scan_tc_multi_kernel<256>, maps.x, maps.q128, a)
+                             : cudaLaunchKernelEx(&cfg, scan_tc_multi_kernel<512>, maps.x, maps.q128, a);
+    } else {
+        e = h->tc_cap == 256 ? launch_scan_kernel<256>(pair, dual, cfg, maps, a) : launch_scan_kernel<512>(pair, dual, cfg, maps, a);
+    }
     if (e != cudaSuccess) {                               // the caller falls back: leave no error behind, keep the speeds' turn
         cudaGetLastError();
         return 1;
@@ -700,15 +713,15 @@ static int launch_scan_generic(prox_handle *h, void **state, const __nv_bfloat16
 // The corpus scan of the misses, all passes of the batch in one launch.  Nonzero: the handle cannot
 // take the tensor-core path (d not a multiple of 64, fewer corpus rows than one tile); the caller
 // then runs the CUDA-core scan.
-int launch_scan_tc(prox_handle *h, cudaStream_t s) {
+int launch_scan_tc(prox_handle *h, int B, cudaStream_t s) {
     if (h->d % kChunkK || h->N < kTileRows) return 1;
-    return launch_scan_generic(h, &h->tc_state, h->xb, h->xh, (long long)h->N, h->qb, &h->st->n_miss, h->kp, s);
+    return launch_scan_generic(h, &h->tc_state, h->xb, h->xh, (long long)h->N, h->qb, &h->st->n_miss, B, h->kp, s);
 }
 
 // The coarse probe: the same scan over the bf16 copies of the cached keys, all batch queries,
 // keeping the kProbeKp best slots per query.
-int launch_probe_scan_tc(prox_handle *h, cudaStream_t s) {
-    return launch_scan_generic(h, &h->tc_state_keys, h->keys_b, h->kh, (long long)h->C, h->pqb, &h->st->n_probe,
+int launch_probe_scan_tc(prox_handle *h, int B, cudaStream_t s) {
+    return launch_scan_generic(h, &h->tc_state_keys, h->keys_b, h->kh, (long long)h->C, h->pqb, &h->st->n_probe, B,
                                kProbeKp, s);
 }
 
