@@ -621,7 +621,7 @@ def test_recording_argument_checks():
     p.close()
 
 
-@pytest.mark.parametrize("d,batch", [(768, 64), (128, 256), (256, 24), (128, 600)])
+@pytest.mark.parametrize("d,batch", [(768, 64), (128, 256), (256, 24), (128, 600), (128, 300), (64, 1000)])
 def test_the_three_scan_kernels_agree(d, batch):
     """Two-block tensor-core scan (default), one-block tensor-core scan and CUDA-core scan."""
     X, Q = stream(9001, d, 8, 520, 40, 1.1, 0.02, seed=10)
