@@ -180,7 +180,8 @@ def roofline_of_scan(cfg, mean_misses, scan_ms_per_launch, peaks, clocks=None, t
     else:
         ach, peak, unit, bound = bytes_alg / t / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
     out = dict(bound=bound, achieved=round(ach, 2), peak=peak, unit=unit, frac=round(ach / peak, 4),
-               traffic=traffic, kernel="scan_tc_kernel", peak_source=peaks["source"],
+               traffic=traffic, kernel="scan_tc_multi_kernel" if (cfg.d <= 128 and cfg.batch > 256) else "scan_tc_kernel",
+               peak_source=peaks["source"],
                peak_kind="burst bf16 GEMM" if bound == "tensor" else "copy bandwidth", **more,
                hbm_gbs=round(bytes_alg / t / 1e9, 1), tflops=round(flops / t / 1e12, 1),
                mean_misses_per_launch=round(mean_misses, 2), ms_per_launch=round(scan_ms_per_launch, 4),
